@@ -1,0 +1,289 @@
+/*
+ * qtale.h -- C ABI of libqtale: forward pass of a token-adaptive transformer
+ * layer with low-bit group-quantised weights (QTALE, arXiv 2602.10431) on one
+ * NVIDIA B200 (sm_100a).
+ *
+ * Per layer the path is: router score per token and execute / bypass decision
+ * (Eq. 2, Eq. 9), gathering of the executed tokens into a dense tensor
+ * (App. B.2), the layer function f_l on the executed tokens only with every
+ * linear a b-bit group-quantised matmul (Eq. 1; Sec. 4.1 implementation
+ * details), and the residual write-back x + f_l(x) for executed tokens while
+ * bypassed tokens keep x (Eq. 3).
+ *
+ * Conventions
+ *  - Every function returns an int status: QTALE_OK (0) or a negative
+ *    QTALE_ERR_* code; qtale_strerror() names it.  Arguments are validated on
+ *    the host; on error nothing is launched and no output is touched.
+ *  - Unless a parameter says "host", every pointer is a DEVICE pointer owned
+ *    by the caller, 16-byte aligned.  The library never allocates or frees
+ *    device memory; scratch comes from a caller workspace whose size the
+ *    matching *_workspace_bytes() query returns.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *    Calls enqueue work and return without synchronising.  The number of
+ *    executed tokens stays on the device (int32) and is never read back by
+ *    the library.
+ *  - Activations are bf16, row-major, innermost dimension contiguous.
+ *    Tokens of all sequences are flattened: token t of the call belongs to
+ *    sequence b with cu_seqlens[b] <= t < cu_seqlens[b+1].
+ *  - A device-side wait that exceeds its iteration limit ends the kernel
+ *    normally and records QTALE_ERR_TIMEOUT in a device status word that
+ *    qtale_device_status() reads.
+ */
+#ifndef QTALE_H_
+#define QTALE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define QTALE_OK 0
+#define QTALE_ERR_NULL (-1)      /* a required pointer is NULL */
+#define QTALE_ERR_ALIGN (-2)     /* pointer or pitch not 16-byte aligned */
+#define QTALE_ERR_SHAPE (-3)     /* unsupported or inconsistent sizes */
+#define QTALE_ERR_BITS (-4)      /* bits not in {3, 4} */
+#define QTALE_ERR_GROUP (-5)     /* group not in {64, 128} */
+#define QTALE_ERR_WORKSPACE (-6) /* workspace too small */
+#define QTALE_ERR_CAPACITY (-7)  /* a count exceeds the capacity of its buffer */
+#define QTALE_ERR_TIMEOUT (-8)   /* a bounded device-side wait gave up */
+#define QTALE_ERR_CUDA (-9)      /* a CUDA runtime / driver call failed */
+#define QTALE_ERR_MODE (-10)     /* unknown mode / epilogue / phase */
+
+const char* qtale_strerror(int status);
+
+/* Reads (synchronously, after cudaStreamSynchronize of `stream`) and clears
+ * the device status word of the current device.  Returns QTALE_OK or the
+ * first device-side error recorded since the last call. */
+int qtale_device_status(void* stream);
+
+/* ------------------------------------------------------------------------- */
+/* Selection (Eq. 2, Eq. 9)                                                   */
+/* ------------------------------------------------------------------------- */
+
+#define QTALE_SELECT_THRESHOLD 0 /* execute iff p0 >= theta            (Eq. 9) */
+#define QTALE_SELECT_TOPK 1      /* the k highest scores (extension, see below) */
+#define QTALE_SELECT_FORCED 2    /* caller supplies the index list              */
+
+/* k of top-k selection for a requested execution ratio: floor(ratio*n + 0.5),
+ * clamped to [0, n].  Host function. */
+int qtale_topk_count(double ratio, int n_valid);
+
+size_t qtale_router_select_workspace_bytes(int T);
+
+/*
+ * Router score, execute decision and ordered compaction in one launch.
+ *
+ * Score (Eq. 9 specialised to a linear two-class router): the router emits
+ * two class logits (g0 execute, g1 bypass); with a linear router their
+ * difference is z_t = w_router . x_t + bias and softmax([g0,g1])[0] =
+ * 1 / (1 + exp(-z_t)).  The dot product accumulates in fp64; the score is
+ * stored as fp32.  If scores_override != NULL the router is skipped and those
+ * scores are used (and copied to scores_out).
+ *
+ * Decision: THRESHOLD: execute iff score >= theta (fp32 compare, ties
+ * execute), one theta for all layers.  TOPK (not in the paper, which controls
+ * the ratio through theta only): the k valid tokens of the call with the
+ * highest scores, equal scores ordered by lower token index.  Tokens with
+ * valid[t] == 0 (padding, App. B.2) never execute.
+ *
+ * Outputs: scores_out[T]; idx_out[T]: ascending token indices of executed
+ * tokens in its first *n_exec_out entries (rest untouched); n_exec_out[1];
+ * cu_exec_out[B+1]: offsets of each sequence's executed tokens inside idx_out;
+ * pos_out[T]: for executed token i its position inside its sequence,
+ * idx - cu_seqlens[b] + (pos0 ? pos0[b] : 0).
+ *
+ *   x          [T, d] bf16              w_router  [d] fp32
+ *   valid      [T] uint8 or NULL        cu_seqlens [B+1] int32, pos0 [B] or NULL
+ * Limits: d % 8 == 0, 1 <= T <= 2^24, 1 <= B <= T.
+ */
+int qtale_router_select(const void* x, int T, int d, const float* w_router, float bias,
+                        const float* scores_override, const uint8_t* valid,
+                        const int32_t* cu_seqlens, int B, const int32_t* pos0, int mode,
+                        float theta, int k, float* scores_out, int32_t* idx_out,
+                        int32_t* n_exec_out, int32_t* cu_exec_out, int32_t* pos_out, void* ws,
+                        size_t ws_bytes, void* stream);
+
+/* Bookkeeping for a caller-supplied ascending index list (QTALE_SELECT_FORCED):
+ * fills n_exec_out, cu_exec_out and pos_out as qtale_router_select does.
+ * idx [n] int32 device, 0 <= n <= T. */
+int qtale_index_bookkeeping(const int32_t* idx, int n, int T, const int32_t* cu_seqlens, int B,
+                            const int32_t* pos0, int32_t* n_exec_out, int32_t* cu_exec_out,
+                            int32_t* pos_out, void* stream);
+
+/* ------------------------------------------------------------------------- */
+/* Gather / scatter (App. B.2; Eq. 3)                                          */
+/* ------------------------------------------------------------------------- */
+
+/*
+ * Gather of the executed rows: xc[i,:] = x[idx[i],:] for i < *n_exec.
+ * If rms_gamma != NULL also hn[i,:] = x[idx[i],:] / sqrt(mean(x^2) + eps) * gamma
+ * (fp32 arithmetic, one bf16 rounding).  xc_out or hn_out may be NULL (not
+ * both).  Rows i >= *n_exec of the outputs are left untouched.
+ *   x [T, d] bf16; idx [T] int32; n_exec [1] int32; rms_gamma [d] fp32;
+ *   xc_out, hn_out [T, d] bf16 (capacity T rows).  d % 8 == 0.
+ */
+int qtale_compact(const void* x, const int32_t* idx, const int32_t* n_exec, int T, int d,
+                  const float* rms_gamma, float eps, void* xc_out, void* hn_out, void* stream);
+
+/*
+ * Residual scatter (Eq. 3, execute branch), in place:
+ * x[idx[i],:] = bf16(float(xc[i,:]) + f[i,:]) for i < *n_exec; every other row
+ * of x is left untouched (bypass branch).  xc bf16 [T, d]; f fp32 [T, d].
+ */
+int qtale_scatter_add(void* x_inout, const void* xc, const float* f, const int32_t* idx,
+                      const int32_t* n_exec, int T, int d, void* stream);
+
+/* ------------------------------------------------------------------------- */
+/* Weight-only quantised GEMM (Sec. 4.1: 4-bit / 3-bit, per-group parameters) */
+/* ------------------------------------------------------------------------- */
+
+/* A quantised linear W[N, K] (y = x W^T) in the kernel-native layout written
+ * by qtale_wq_repack.  Dequantisation: w = (code - zero) * scale with one
+ * fp16 scale and one integer-valued fp16 zero-point per `group` consecutive
+ * input features of a row. */
+typedef struct {
+  const void* packed; /* device copy of the repacked blob */
+  int N, K;           /* logical shape */
+  int bits;           /* 3 or 4 */
+  int group;          /* 64 or 128 */
+  int row_mode;       /* QTALE_WQ_ROWS_* the blob was repacked with */
+} qtale_wq_weight;
+
+#define QTALE_WQ_ROWS_PLAIN 0  /* output feature n sits in tile n / 128, lane n % 128       */
+#define QTALE_WQ_ROWS_SWIGLU 1 /* W = [gate; up] (N = 2F): each 128-row tile holds 64 gate
+                                  rows and the matching 64 up rows, needed by EPI_SWIGLU   */
+
+/*
+ * Offline repack, HOST pointers.  Input is the interface layout: codes
+ * row-major [N, row_bytes]; 4-bit: two codes per byte, even k in the low
+ * nibble, row_bytes = ceil(K/2); 3-bit: little-endian bit stream along K,
+ * row_bytes = ceil(3K/8); scales / zeros fp16 [N, ceil(K/group)].
+ * Call with packed_out == NULL to get the blob size in *bytes; then with a
+ * buffer of that size.  Rows are padded to a multiple of 128 and K to a
+ * multiple of `group` with codes equal to the zero-point (weight 0).
+ */
+int qtale_wq_repack(const uint8_t* codes, const uint16_t* scales, const uint16_t* zeros, int N,
+                    int K, int bits, int group, int row_mode, void* packed_out, size_t* bytes);
+
+#define QTALE_EPI_STORE_BF16 0    /* y[m,n] = bf16(acc)                                  */
+#define QTALE_EPI_STORE_F32 1     /* y[m,n] = acc                                  (fp32) */
+#define QTALE_EPI_RESID_F32 2     /* y[m,n] = float(resid[idx[m],n]) + acc         (fp32) */
+#define QTALE_EPI_RESID_SCATTER 3 /* dst[idx[m],n] = bf16(resid_f32[m,n] + acc)    (Eq. 3) */
+#define QTALE_EPI_SWIGLU 4        /* y[m,j] = bf16(silu(acc[m,j]) * acc[m,F+j]), N = 2F;
+                                     needs QTALE_WQ_ROWS_SWIGLU weights                   */
+
+typedef struct {
+  const int32_t* idx;    /* [M_cap] row indices (RESID_F32, RESID_SCATTER) */
+  const void* resid;     /* RESID_F32: bf16 [T, ld_resid] gathered by idx;
+                            RESID_SCATTER: fp32 [M_cap, ld_resid] dense          */
+  int ld_resid;          /* elements */
+  void* dst;             /* RESID_SCATTER: bf16 [T, ld_dst], rows idx[m] written */
+  int ld_dst;
+} qtale_epilogue_args;
+
+/*
+ * y = epilogue(a W^T) on the tensor cores; rows m >= *m_dev (or >= M_cap when
+ * m_dev == NULL) are neither computed nor written.
+ *   a  bf16 [M_cap, lda]  (lda >= K elements, lda * 2 bytes % 16 == 0)
+ *   y  [M_cap, ldy]; element type set by the epilogue
+ * The packed weights are dequantised to bf16 inside the kernel (exact
+ * (code - zero) * scale in fp32, one rounding) and accumulated in fp32.
+ */
+int qtale_wq_gemm(const void* a, int lda, const int32_t* m_dev, int M_cap, const qtale_wq_weight* w,
+                  int epilogue, const qtale_epilogue_args* epi, void* y, int ldy, void* stream);
+
+/* ------------------------------------------------------------------------- */
+/* Layer and model                                                             */
+/* ------------------------------------------------------------------------- */
+
+typedef struct {
+  int d, n_heads, n_kv_heads, head_dim, ffn; /* Llama-style decoder layer shape          */
+  int bits, group;                          /* quantisation of the four linears          */
+  float rms_eps, rope_theta;                /* RMSNorm epsilon, rotary base               */
+  int select_mode;                          /* QTALE_SELECT_*                             */
+  float theta;                              /* threshold of Eq. 9 (THRESHOLD)             */
+  float ratio;                              /* execution ratio in [0,1] (TOPK)            */
+} qtale_layer_config;
+
+typedef struct {
+  qtale_wq_weight qkv;     /* [(H + 2 Hkv) hd, d]: Wq rows, then Wk, then Wv   */
+  qtale_wq_weight o;       /* [d, H hd]                                        */
+  qtale_wq_weight gate_up; /* [2 F, d]: gate rows then up rows                 */
+  qtale_wq_weight down;    /* [d, F]                                           */
+  const float* gamma1;     /* [d] fp32, pre-attention RMSNorm gain             */
+  const float* gamma2;     /* [d] fp32, pre-MLP RMSNorm gain                   */
+  const float* router_w;   /* [d] fp32, execute-minus-bypass logit weights     */
+  float router_b;
+} qtale_layer_weights;
+
+/* Per-layer KV cache.  Only executed tokens enter it: a bypassed token does not
+ * evaluate f_l (Eq. 3) and therefore produces no key or value at that layer. */
+typedef struct {
+  void* k;         /* bf16 [B, cap, n_kv_heads * head_dim], rotary already applied */
+  void* v;         /* bf16 [B, cap, n_kv_heads * head_dim]                         */
+  int32_t* kv_len; /* int32 [B], entries in use per sequence (updated)             */
+  int cap;
+} qtale_kv_cache;
+
+#define QTALE_PHASE_PREFILL 0 /* any sequence lengths; cache (if given) must be empty */
+#define QTALE_PHASE_DECODE 1  /* exactly one new token per sequence, cache required   */
+
+size_t qtale_layer_workspace_bytes(const qtale_layer_config* cfg, int T_cap, int B_cap);
+
+/*
+ * One token-adaptive layer, in place on x (Eq. 1, 3, 9; App. B.2).
+ * Executed tokens: x <- x + f_l(x) with f_l = attention branch + MLP branch on
+ * the gathered executed tokens; attention is causal among the executed tokens
+ * of the same sequence (plus that sequence's cache entries in DECODE), RoPE
+ * uses each token's original position.  Bypassed tokens: x unchanged.
+ *
+ *   x_inout [T, d] bf16; cu_seqlens [B+1]; pos0 [B] or NULL (position of each
+ *   sequence's first token in this call); valid [T] or NULL;
+ *   scores_override [T] or NULL; forced_idx [forced_n] (FORCED mode);
+ *   kv NULL or the layer's cache; n_exec_out [1] device int32;
+ *   scores_out [T] fp32 or NULL.
+ * `cfg`, `w`, `kv` are host structs holding device pointers.
+ */
+int qtale_layer_forward(const qtale_layer_config* cfg, const qtale_layer_weights* w, void* x_inout,
+                        int T, const int32_t* cu_seqlens, int B, const int32_t* pos0,
+                        const uint8_t* valid, const float* scores_override,
+                        const int32_t* forced_idx, int forced_n, const qtale_kv_cache* kv,
+                        int phase, int32_t* n_exec_out, float* scores_out, void* ws,
+                        size_t ws_bytes, void* stream);
+
+typedef struct {
+  int n_layers, vocab;
+  qtale_layer_config layer; /* shared by all layers; theta is the single global threshold */
+} qtale_model_config;
+
+typedef struct {
+  const void* embed;                 /* bf16 [vocab, d]                         */
+  const qtale_layer_weights* layers; /* HOST array [n_layers]                   */
+  const float* final_gamma;          /* [d] fp32                                */
+  const void* lm_head;               /* bf16 [vocab, d] or NULL                 */
+} qtale_model_weights;
+
+size_t qtale_model_workspace_bytes(const qtale_model_config* cfg, int T_cap, int B_cap,
+                                   int n_logit_rows);
+
+/*
+ * Prefill of a stack of token-adaptive layers: embedding gather, n_layers x
+ * qtale_layer_forward sharing one theta (Sec. 3.4) or, when per_layer_ratio
+ * (HOST float [n_layers]) is given, per-layer top-k at those ratios; final
+ * RMSNorm and LM head on the requested rows.
+ *   ids [T] int32; hidden_out [T, d] bf16 (final residual stream);
+ *   logits_out fp32 [n_logit_rows, vocab] or NULL; logit_rows [n_logit_rows]
+ *   int32 device; per_layer_n_exec [n_layers] int32 device.
+ */
+int qtale_model_prefill(const qtale_model_config* cfg, const qtale_model_weights* w,
+                        const int32_t* ids, int T, const int32_t* cu_seqlens, int B,
+                        const float* per_layer_ratio, void* hidden_out, float* logits_out,
+                        const int32_t* logit_rows, int n_logit_rows, int32_t* per_layer_n_exec,
+                        void* ws, size_t ws_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QTALE_H_ */

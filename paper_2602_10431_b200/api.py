@@ -1,0 +1,353 @@
+"""Thin Python binding over libqtale's C ABI (argument marshalling only).
+
+Every function here forwards to the `extern "C"` entry point of the same name
+declared in include/qtale.h; all arithmetic of the path runs in the library's
+CUDA kernels.  PyTorch supplies device memory and the current stream.  There
+is no fallback: importing this module without the built library, or calling
+it without a CUDA device, raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libqtale.so")
+
+SELECT_THRESHOLD, SELECT_TOPK, SELECT_FORCED = 0, 1, 2
+EPI_STORE_BF16, EPI_STORE_F32, EPI_RESID_F32, EPI_RESID_SCATTER, EPI_SWIGLU = 0, 1, 2, 3, 4
+ROWS_PLAIN, ROWS_SWIGLU = 0, 1
+PHASE_PREFILL, PHASE_DECODE = 0, 1
+
+EXPORTS = [
+    "qtale_strerror", "qtale_device_status", "qtale_topk_count",
+    "qtale_router_select_workspace_bytes", "qtale_router_select", "qtale_index_bookkeeping",
+    "qtale_compact", "qtale_scatter_add", "qtale_wq_repack", "qtale_wq_gemm",
+    "qtale_layer_workspace_bytes", "qtale_layer_forward", "qtale_model_workspace_bytes",
+    "qtale_model_prefill",
+]
+
+
+class QtaleError(RuntimeError):
+    pass
+
+
+class WqWeight(C.Structure):
+    _fields_ = [("packed", C.c_void_p), ("N", C.c_int), ("K", C.c_int), ("bits", C.c_int),
+                ("group", C.c_int), ("row_mode", C.c_int)]
+
+
+class EpilogueArgs(C.Structure):
+    _fields_ = [("idx", C.c_void_p), ("resid", C.c_void_p), ("ld_resid", C.c_int),
+                ("dst", C.c_void_p), ("ld_dst", C.c_int)]
+
+
+class LayerConfig(C.Structure):
+    _fields_ = [("d", C.c_int), ("n_heads", C.c_int), ("n_kv_heads", C.c_int),
+                ("head_dim", C.c_int), ("ffn", C.c_int), ("bits", C.c_int), ("group", C.c_int),
+                ("rms_eps", C.c_float), ("rope_theta", C.c_float), ("select_mode", C.c_int),
+                ("theta", C.c_float), ("ratio", C.c_float)]
+
+
+class LayerWeightsC(C.Structure):
+    _fields_ = [("qkv", WqWeight), ("o", WqWeight), ("gate_up", WqWeight), ("down", WqWeight),
+                ("gamma1", C.c_void_p), ("gamma2", C.c_void_p), ("router_w", C.c_void_p),
+                ("router_b", C.c_float)]
+
+
+class KvCacheC(C.Structure):
+    _fields_ = [("k", C.c_void_p), ("v", C.c_void_p), ("kv_len", C.c_void_p), ("cap", C.c_int)]
+
+
+class ModelConfig(C.Structure):
+    _fields_ = [("n_layers", C.c_int), ("vocab", C.c_int), ("layer", LayerConfig)]
+
+
+class ModelWeightsC(C.Structure):
+    _fields_ = [("embed", C.c_void_p), ("layers", C.POINTER(LayerWeightsC)),
+                ("final_gamma", C.c_void_p), ("lm_head", C.c_void_p)]
+
+
+_lib = None
+
+
+def lib():
+    """Loads libqtale.so; raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise QtaleError("libqtale.so is missing: run `python -m paper_2602_10431_b200.build`")
+        L = C.CDLL(LIB_PATH)
+        L.qtale_strerror.restype = C.c_char_p
+        L.qtale_strerror.argtypes = [C.c_int]
+        L.qtale_device_status.argtypes = [C.c_void_p]
+        L.qtale_topk_count.argtypes = [C.c_double, C.c_int]
+        L.qtale_router_select_workspace_bytes.restype = C.c_size_t
+        L.qtale_router_select_workspace_bytes.argtypes = [C.c_int]
+        L.qtale_router_select.argtypes = [
+            C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_float, C.c_void_p, C.c_void_p,
+            C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_float, C.c_int, C.c_void_p, C.c_void_p,
+            C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+        L.qtale_index_bookkeeping.argtypes = [
+            C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p,
+            C.c_void_p, C.c_void_p]
+        L.qtale_compact.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int,
+                                    C.c_void_p, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.qtale_scatter_add.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                        C.c_int, C.c_int, C.c_void_p]
+        L.qtale_wq_repack.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
+                                      C.c_int, C.c_int, C.c_void_p, C.POINTER(C.c_size_t)]
+        L.qtale_wq_gemm.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.POINTER(WqWeight),
+                                    C.c_int, C.POINTER(EpilogueArgs), C.c_void_p, C.c_int,
+                                    C.c_void_p]
+        L.qtale_layer_workspace_bytes.restype = C.c_size_t
+        L.qtale_layer_workspace_bytes.argtypes = [C.POINTER(LayerConfig), C.c_int, C.c_int]
+        L.qtale_layer_forward.argtypes = [
+            C.POINTER(LayerConfig), C.POINTER(LayerWeightsC), C.c_void_p, C.c_int, C.c_void_p,
+            C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.POINTER(KvCacheC),
+            C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+        L.qtale_model_workspace_bytes.restype = C.c_size_t
+        L.qtale_model_workspace_bytes.argtypes = [C.POINTER(ModelConfig), C.c_int, C.c_int, C.c_int]
+        L.qtale_model_prefill.argtypes = [
+            C.POINTER(ModelConfig), C.POINTER(ModelWeightsC), C.c_void_p, C.c_int, C.c_void_p,
+            C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p,
+            C.c_void_p, C.c_size_t, C.c_void_p]
+        _lib = L
+    return _lib
+
+
+def strerror(rc: int) -> str:
+    return lib().qtale_strerror(int(rc)).decode()
+
+
+def check(rc: int, what: str = "") -> None:
+    if rc != 0:
+        raise QtaleError("%s failed: %s (%d)" % (what or "libqtale call", strerror(rc), rc))
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def device_status() -> int:
+    return int(lib().qtale_device_status(_stream()))
+
+
+def topk_count(ratio: float, n_valid: int) -> int:
+    return int(lib().qtale_topk_count(float(ratio), int(n_valid)))
+
+
+# ---------------------------------------------------------------------------------
+# selection
+# ---------------------------------------------------------------------------------
+
+def router_select(x, w_router, bias, cu_seqlens, mode, theta=0.5, k=0, scores_override=None,
+                  valid=None, pos0=None, out=None):
+    """qtale_router_select.  x bf16 [T, d]; w_router fp32 [d]; cu_seqlens int32 [B+1].
+    Returns dict(scores, idx, n_exec, cu_exec, pos) of device tensors."""
+    T = int(x.shape[0]) if x is not None else int(scores_override.shape[0])
+    d = int(x.shape[1]) if x is not None else 0
+    dev = (x if x is not None else scores_override).device
+    B = int(cu_seqlens.shape[0]) - 1
+    o = out or {}
+    scores = o.get("scores", None)
+    if scores is None:
+        scores = torch.empty(T, dtype=torch.float32, device=dev)
+    idx = o.get("idx") if "idx" in o else torch.full((T,), -1, dtype=torch.int32, device=dev)
+    pos = o.get("pos") if "pos" in o else torch.full((T,), -1, dtype=torch.int32, device=dev)
+    n_exec = o.get("n_exec") if "n_exec" in o else torch.zeros(1, dtype=torch.int32, device=dev)
+    cu_exec = o.get("cu_exec") if "cu_exec" in o else torch.zeros(B + 1, dtype=torch.int32, device=dev)
+    ws = o.get("ws") if "ws" in o else torch.zeros(256, dtype=torch.uint8, device=dev)
+    check(lib().qtale_router_select(
+        _ptr(x), T, d, _ptr(w_router), float(bias), _ptr(scores_override), _ptr(valid),
+        _ptr(cu_seqlens), B, _ptr(pos0), int(mode), float(theta), int(k), _ptr(scores), _ptr(idx),
+        _ptr(n_exec), _ptr(cu_exec), _ptr(pos), _ptr(ws), ws.numel(), _stream()),
+        "qtale_router_select")
+    return dict(scores=scores, idx=idx, n_exec=n_exec, cu_exec=cu_exec, pos=pos, ws=ws)
+
+
+def index_bookkeeping(idx, n, T, cu_seqlens, pos0=None):
+    dev = cu_seqlens.device
+    B = int(cu_seqlens.shape[0]) - 1
+    n_exec = torch.zeros(1, dtype=torch.int32, device=dev)
+    cu_exec = torch.zeros(B + 1, dtype=torch.int32, device=dev)
+    pos = torch.full((max(T, 1),), -1, dtype=torch.int32, device=dev)
+    check(lib().qtale_index_bookkeeping(_ptr(idx), int(n), int(T), _ptr(cu_seqlens), B, _ptr(pos0),
+                                        _ptr(n_exec), _ptr(cu_exec), _ptr(pos), _stream()),
+          "qtale_index_bookkeeping")
+    return dict(n_exec=n_exec, cu_exec=cu_exec, pos=pos)
+
+
+# ---------------------------------------------------------------------------------
+# gather / scatter
+# ---------------------------------------------------------------------------------
+
+def compact(x, idx, n_exec, rms_gamma=None, eps=1e-5, want_xc=True, xc_out=None, hn_out=None):
+    """qtale_compact.  Returns (xc, hn); either may be None."""
+    T, d = int(x.shape[0]), int(x.shape[1])
+    xc = xc_out if xc_out is not None else (torch.zeros_like(x) if want_xc else None)
+    hn = hn_out if hn_out is not None else (torch.zeros_like(x) if rms_gamma is not None else None)
+    check(lib().qtale_compact(_ptr(x), _ptr(idx), _ptr(n_exec), T, d, _ptr(rms_gamma), float(eps),
+                              _ptr(xc), _ptr(hn), _stream()), "qtale_compact")
+    return xc, hn
+
+
+def scatter_add(x_inout, xc, f, idx, n_exec):
+    T, d = int(x_inout.shape[0]), int(x_inout.shape[1])
+    check(lib().qtale_scatter_add(_ptr(x_inout), _ptr(xc), _ptr(f), _ptr(idx), _ptr(n_exec), T, d,
+                                  _stream()), "qtale_scatter_add")
+    return x_inout
+
+
+# ---------------------------------------------------------------------------------
+# quantised weights
+# ---------------------------------------------------------------------------------
+
+def wq_repack(packed_codes: np.ndarray, scales: np.ndarray, zeros: np.ndarray, N, K, bits, group,
+              row_mode=ROWS_PLAIN) -> np.ndarray:
+    """qtale_wq_repack on host arrays; returns the native blob as a uint8 numpy array."""
+    codes = np.ascontiguousarray(packed_codes, dtype=np.uint8)
+    s = np.ascontiguousarray(scales).view(np.uint16)
+    z = np.ascontiguousarray(zeros).view(np.uint16)
+    nbytes = C.c_size_t(0)
+    check(lib().qtale_wq_repack(None, None, None, N, K, bits, group, row_mode, None,
+                                C.byref(nbytes)), "qtale_wq_repack(size)")
+    out = np.empty(nbytes.value, dtype=np.uint8)
+    check(lib().qtale_wq_repack(codes.ctypes.data, s.ctypes.data, z.ctypes.data, N, K, bits, group,
+                                row_mode, out.ctypes.data, C.byref(nbytes)), "qtale_wq_repack")
+    return out
+
+
+class QuantWeight:
+    """Device copy of a repacked quantised linear plus its C descriptor."""
+
+    def __init__(self, wq: dict, device="cuda", row_mode=ROWS_PLAIN):
+        blob = wq_repack(wq["packed"], wq["scales"], wq["zeros"], wq["N"], wq["K"], wq["bits"],
+                         wq["group"], row_mode)
+        self.blob = torch.from_numpy(blob).to(device)
+        self.N, self.K, self.bits, self.group, self.row_mode = (wq["N"], wq["K"], wq["bits"],
+                                                                 wq["group"], row_mode)
+        self.c = WqWeight(self.blob.data_ptr(), self.N, self.K, self.bits, self.group, row_mode)
+
+
+def wq_gemm(a, w: QuantWeight, m_dev=None, epilogue=EPI_STORE_BF16, y=None, idx=None, resid=None,
+            dst=None):
+    """qtale_wq_gemm.  a bf16 [M_cap, K]; returns y (or dst for RESID_SCATTER)."""
+    M_cap, lda = int(a.shape[0]), int(a.stride(0))
+    epi = None
+    if epilogue in (EPI_RESID_F32, EPI_RESID_SCATTER):
+        epi = EpilogueArgs(idx.data_ptr(), resid.data_ptr(), int(resid.stride(0)),
+                           dst.data_ptr() if dst is not None else None,
+                           int(dst.stride(0)) if dst is not None else 0)
+    if y is None and epilogue != EPI_RESID_SCATTER:
+        n_out = w.N // 2 if epilogue == EPI_SWIGLU else w.N
+        dt = torch.bfloat16 if epilogue in (EPI_STORE_BF16, EPI_SWIGLU) else torch.float32
+        y = torch.zeros(M_cap, n_out, dtype=dt, device=a.device)
+    check(lib().qtale_wq_gemm(_ptr(a), lda, _ptr(m_dev), M_cap, C.byref(w.c), int(epilogue),
+                              C.byref(epi) if epi is not None else None, _ptr(y),
+                              int(y.stride(0)) if y is not None else 0, _stream()), "qtale_wq_gemm")
+    return dst if epilogue == EPI_RESID_SCATTER else y
+
+
+# ---------------------------------------------------------------------------------
+# layer / model
+# ---------------------------------------------------------------------------------
+
+def layer_config(sh, select_mode=SELECT_THRESHOLD, theta=0.5, ratio=1.0) -> LayerConfig:
+    return LayerConfig(sh.d, sh.n_heads, sh.n_kv_heads, sh.head_dim, sh.ffn, sh.bits, sh.group,
+                       sh.rms_eps, sh.rope_theta, int(select_mode), float(theta), float(ratio))
+
+
+class LayerWeights:
+    """Device-resident weights of one layer (from inputs.layer_weights)."""
+
+    def __init__(self, w: dict, device="cuda", fuse_swiglu=True):
+        self.qkv = QuantWeight(w["qkv"], device)
+        self.o = QuantWeight(w["o"], device)
+        self.gate_up = QuantWeight(w["gate_up"], device, ROWS_SWIGLU if fuse_swiglu else ROWS_PLAIN)
+        self.down = QuantWeight(w["down"], device)
+        self.gamma1 = torch.from_numpy(np.ascontiguousarray(w["gamma1"], np.float32)).to(device)
+        self.gamma2 = torch.from_numpy(np.ascontiguousarray(w["gamma2"], np.float32)).to(device)
+        self.router_w = torch.from_numpy(np.ascontiguousarray(w["router_w"], np.float32)).to(device)
+        self.router_b = float(w["router_b"])
+        self.c = LayerWeightsC(self.qkv.c, self.o.c, self.gate_up.c, self.down.c,
+                               self.gamma1.data_ptr(), self.gamma2.data_ptr(),
+                               self.router_w.data_ptr(), self.router_b)
+
+    def set_router_bias(self, b: float):
+        self.router_b = float(b)
+        self.c.router_b = float(b)
+
+
+class KvCache:
+    def __init__(self, B, cap, kv_dim, device="cuda"):
+        self.k = torch.zeros(B, cap, kv_dim, dtype=torch.bfloat16, device=device)
+        self.v = torch.zeros(B, cap, kv_dim, dtype=torch.bfloat16, device=device)
+        self.kv_len = torch.zeros(B, dtype=torch.int32, device=device)
+        self.cap = cap
+        self.c = KvCacheC(self.k.data_ptr(), self.v.data_ptr(), self.kv_len.data_ptr(), cap)
+
+
+def layer_workspace_bytes(cfg: LayerConfig, T_cap: int, B_cap: int) -> int:
+    return int(lib().qtale_layer_workspace_bytes(C.byref(cfg), int(T_cap), int(B_cap)))
+
+
+def layer_forward(cfg: LayerConfig, w: LayerWeights, x_inout, cu_seqlens, ws, n_exec_out=None,
+                  scores_out=None, pos0=None, valid=None, scores_override=None, forced_idx=None,
+                  forced_n=0, kv: KvCache | None = None, phase=PHASE_PREFILL):
+    """qtale_layer_forward, in place on x_inout (bf16 [T, d])."""
+    T = int(x_inout.shape[0])
+    B = int(cu_seqlens.shape[0]) - 1
+    check(lib().qtale_layer_forward(
+        C.byref(cfg), C.byref(w.c), _ptr(x_inout), T, _ptr(cu_seqlens), B, _ptr(pos0), _ptr(valid),
+        _ptr(scores_override), _ptr(forced_idx), int(forced_n),
+        C.byref(kv.c) if kv is not None else None, int(phase), _ptr(n_exec_out), _ptr(scores_out),
+        _ptr(ws), ws.numel() * ws.element_size(), _stream()), "qtale_layer_forward")
+    return x_inout
+
+
+def model_workspace_bytes(cfg: ModelConfig, T_cap, B_cap, n_logit_rows) -> int:
+    return int(lib().qtale_model_workspace_bytes(C.byref(cfg), int(T_cap), int(B_cap),
+                                                 int(n_logit_rows)))
+
+
+def model_prefill(cfg: ModelConfig, layers, embed, ids, cu_seqlens, ws, hidden_out,
+                  per_layer_ratio=None, final_gamma=None, lm_head=None, logit_rows=None,
+                  logits_out=None, per_layer_n_exec=None):
+    """qtale_model_prefill.  layers: list of LayerWeights."""
+    T = int(ids.shape[0])
+    B = int(cu_seqlens.shape[0]) - 1
+    arr = (LayerWeightsC * len(layers))(*[l.c for l in layers])
+    mw = ModelWeightsC(embed.data_ptr(), arr,
+                       final_gamma.data_ptr() if final_gamma is not None else None,
+                       lm_head.data_ptr() if lm_head is not None else None)
+    ratios = None
+    if per_layer_ratio is not None:
+        ratios = (C.c_float * len(layers))(*[float(r) for r in per_layer_ratio])
+    n_rows = int(logit_rows.shape[0]) if logit_rows is not None else 0
+    check(lib().qtale_model_prefill(
+        C.byref(cfg), C.byref(mw), _ptr(ids), T, _ptr(cu_seqlens), B,
+        C.cast(ratios, C.c_void_p) if ratios is not None else None, _ptr(hidden_out),
+        _ptr(logits_out), _ptr(logit_rows), n_rows, _ptr(per_layer_n_exec), _ptr(ws),
+        ws.numel() * ws.element_size(), _stream()), "qtale_model_prefill")
+    return hidden_out
+
+
+# ---------------------------------------------------------------------------------
+# host <-> device helpers for bf16 held as float32 numpy arrays
+# ---------------------------------------------------------------------------------
+
+def to_device_bf16(a: np.ndarray, device="cuda") -> torch.Tensor:
+    """float32 numpy array of bf16-representable values -> bf16 device tensor (exact)."""
+    return torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).to(device).to(torch.bfloat16)
+
+
+def to_host_f32(t: torch.Tensor) -> np.ndarray:
+    return t.detach().to(torch.float32).cpu().numpy()

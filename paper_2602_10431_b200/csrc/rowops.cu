@@ -1,0 +1,383 @@
+// Bandwidth-bound row kernels: gather (+RMSNorm) of executed tokens (App. B.2),
+// residual scatter (Eq. 3), fp32 RMSNorm, rotary embedding, SwiGLU, KV-cache
+// append, embedding gather.  All move 16 bytes per thread per access, keep a
+// row's data in registers between the reduction and the write, and read the
+// executed-token count from device memory.
+#include "rowops.cuh"
+
+namespace qtale {
+
+constexpr int kRowThreads = 256;
+
+// ---- gather (+ RMSNorm) ------------------------------------------------------
+// One warp per executed row; the row (d <= 32*8*MAXC bf16) stays in registers.
+template <int MAXC>
+__global__ void __launch_bounds__(kRowThreads)
+    compact_kernel(const uint4* __restrict__ x, const int32_t* __restrict__ idx,
+                   const int32_t* __restrict__ n_exec, int cap, int d,
+                   const float* __restrict__ gamma, float eps, uint4* __restrict__ xc,
+                   uint4* __restrict__ hn) {
+  const int lane = threadIdx.x & 31;
+  const int warps = (gridDim.x * blockDim.x) >> 5;
+  const int n = n_exec ? min(*n_exec, cap) : cap;
+  const int chunks = d >> 3;  // 16-byte chunks per row
+  for (int i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < n; i += warps) {
+    const uint4* src = x + (size_t)idx[i] * chunks;
+    uint4 v[MAXC];
+#pragma unroll
+    for (int c = 0; c < MAXC; ++c) {
+      const int cc = c * 32 + lane;
+      if (cc < chunks) v[c] = ld_nc_16(src + cc);
+    }
+    if (xc) {
+#pragma unroll
+      for (int c = 0; c < MAXC; ++c) {
+        const int cc = c * 32 + lane;
+        if (cc < chunks) st_16(xc + (size_t)i * chunks + cc, v[c]);
+      }
+    }
+    if (hn) {
+      float ss = 0.f;
+#pragma unroll
+      for (int c = 0; c < MAXC; ++c) {
+        const int cc = c * 32 + lane;
+        if (cc < chunks) {
+          const uint32_t u[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const float a = bf16_lo(u[q]), b = bf16_hi(u[q]);
+            ss = fmaf(a, a, ss);
+            ss = fmaf(b, b, ss);
+          }
+        }
+      }
+      ss = warp_sum(ss);
+      const float inv = rsqrtf(ss / (float)d + eps);
+#pragma unroll
+      for (int c = 0; c < MAXC; ++c) {
+        const int cc = c * 32 + lane;
+        if (cc < chunks) {
+          const float4 g0 = *reinterpret_cast<const float4*>(gamma + cc * 8);
+          const float4 g1 = *reinterpret_cast<const float4*>(gamma + cc * 8 + 4);
+          uint4 o;
+          o.x = pack_bf16x2(bf16_lo(v[c].x) * inv * g0.x, bf16_hi(v[c].x) * inv * g0.y);
+          o.y = pack_bf16x2(bf16_lo(v[c].y) * inv * g0.z, bf16_hi(v[c].y) * inv * g0.w);
+          o.z = pack_bf16x2(bf16_lo(v[c].z) * inv * g1.x, bf16_hi(v[c].z) * inv * g1.y);
+          o.w = pack_bf16x2(bf16_lo(v[c].w) * inv * g1.z, bf16_hi(v[c].w) * inv * g1.w);
+          st_16(hn + (size_t)i * chunks + cc, o);
+        }
+      }
+    }
+  }
+}
+
+// ---- residual scatter: x[idx[i]] = bf16(float(xc[i]) + f[i]) -------------------
+__global__ void __launch_bounds__(kRowThreads)
+    scatter_add_kernel(uint4* __restrict__ x, const uint4* __restrict__ xc,
+                       const float4* __restrict__ f, const int32_t* __restrict__ idx,
+                       const int32_t* __restrict__ n_exec, int cap, int d) {
+  const int lane = threadIdx.x & 31;
+  const int warps = (gridDim.x * blockDim.x) >> 5;
+  const int n = min(*n_exec, cap);
+  const int chunks = d >> 3;
+  for (int i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < n; i += warps) {
+    uint4* dst = x + (size_t)idx[i] * chunks;
+    for (int cc = lane; cc < chunks; cc += 32) {
+      const uint4 a = ld_nc_16(xc + (size_t)i * chunks + cc);
+      const float4 f0 = f[((size_t)i * chunks + cc) * 2];
+      const float4 f1 = f[((size_t)i * chunks + cc) * 2 + 1];
+      uint4 o;
+      o.x = pack_bf16x2(bf16_lo(a.x) + f0.x, bf16_hi(a.x) + f0.y);
+      o.y = pack_bf16x2(bf16_lo(a.y) + f0.z, bf16_hi(a.y) + f0.w);
+      o.z = pack_bf16x2(bf16_lo(a.z) + f1.x, bf16_hi(a.z) + f1.y);
+      o.w = pack_bf16x2(bf16_lo(a.w) + f1.z, bf16_hi(a.w) + f1.w);
+      st_16(dst + cc, o);
+    }
+  }
+}
+
+// ---- RMSNorm of an fp32 tensor into bf16: one CTA per row ---------------------
+template <int MAXC>
+__global__ void __launch_bounds__(kRowThreads)
+    rmsnorm_f32_kernel(const float4* __restrict__ u, const int32_t* __restrict__ n_rows, int cap,
+                       int d, const float* __restrict__ gamma, float eps, uint2* __restrict__ out) {
+  __shared__ float s_part[kRowThreads / 32];
+  __shared__ float s_inv;
+  const int n = n_rows ? min(*n_rows, cap) : cap;
+  const int chunks = d >> 2;  // float4 chunks per row
+  for (int i = blockIdx.x; i < n; i += gridDim.x) {
+    float4 v[MAXC];
+    float ss = 0.f;
+#pragma unroll
+    for (int c = 0; c < MAXC; ++c) {
+      const int cc = c * kRowThreads + threadIdx.x;
+      if (cc < chunks) {
+        v[c] = u[(size_t)i * chunks + cc];
+        ss = fmaf(v[c].x, v[c].x, ss);
+        ss = fmaf(v[c].y, v[c].y, ss);
+        ss = fmaf(v[c].z, v[c].z, ss);
+        ss = fmaf(v[c].w, v[c].w, ss);
+      }
+    }
+    ss = warp_sum(ss);
+    if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+      float t = threadIdx.x < kRowThreads / 32 ? s_part[threadIdx.x] : 0.f;
+      t = warp_sum(t);
+      if (threadIdx.x == 0) s_inv = rsqrtf(t / (float)d + eps);
+    }
+    __syncthreads();
+    const float inv = s_inv;
+#pragma unroll
+    for (int c = 0; c < MAXC; ++c) {
+      const int cc = c * kRowThreads + threadIdx.x;
+      if (cc < chunks) {
+        const float4 g = *reinterpret_cast<const float4*>(gamma + cc * 4);
+        uint2 o;
+        o.x = pack_bf16x2(v[c].x * inv * g.x, v[c].y * inv * g.y);
+        o.y = pack_bf16x2(v[c].z * inv * g.z, v[c].w * inv * g.w);
+        out[(size_t)i * chunks + cc] = o;
+      }
+    }
+    __syncthreads();
+  }
+}
+
+// ---- rotary table: cs[i][j] = (cos, sin)(pos[i] * base^(-2j/hd)), fp64 math ----
+__global__ void rope_table_kernel(const int32_t* __restrict__ pos,
+                                  const int32_t* __restrict__ n_exec, int cap, int half,
+                                  float base, float2* __restrict__ cs) {
+  const int n = min(*n_exec, cap);
+  const size_t total = (size_t)n * half;
+  for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < total;
+       e += (size_t)gridDim.x * blockDim.x) {
+    const int i = (int)(e / half), j = (int)(e % half);
+    const double inv_freq = pow((double)base, -(double)j / (double)half);
+    double s, c;
+    sincos((double)pos[i] * inv_freq, &s, &c);
+    cs[e] = make_float2((float)c, (float)s);
+  }
+}
+
+// ---- rotary embedding on the q and k heads of the fused qkv tensor -------------
+// qkv: [n, ld] bf16; heads 0 .. n_rot-1 (q heads then k heads) are rotated in place,
+// pairing element j with j + hd/2.
+__global__ void __launch_bounds__(kRowThreads)
+    rope_kernel(uint4* __restrict__ qkv, const int32_t* __restrict__ n_exec, int cap, int ld,
+                int n_rot, int hd, const float2* __restrict__ cs) {
+  const int n = min(*n_exec, cap);
+  const int half = hd >> 1;
+  const int cpr = half >> 3;  // 16-byte chunks per half head
+  const size_t per_row = (size_t)n_rot * cpr;
+  const size_t total = (size_t)n * per_row;
+  const int ldc = ld >> 3;
+  for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < total;
+       e += (size_t)gridDim.x * blockDim.x) {
+    const int i = (int)(e / per_row);
+    const int r = (int)(e % per_row);
+    const int h = r / cpr, c = r % cpr;
+    uint4* p0 = qkv + (size_t)i * ldc + (size_t)h * (hd >> 3) + c;
+    uint4* p1 = p0 + cpr;
+    const uint4 a = *p0, b = *p1;
+    const float4* t = reinterpret_cast<const float4*>(cs + (size_t)i * half + c * 8);
+    const float4 t0 = t[0], t1 = t[1], t2 = t[2], t3 = t[3];  // (c,s) x 8
+    const uint32_t au[4] = {a.x, a.y, a.z, a.w}, bu[4] = {b.x, b.y, b.z, b.w};
+    const float cv[8] = {t0.x, t0.z, t1.x, t1.z, t2.x, t2.z, t3.x, t3.z};
+    const float sv[8] = {t0.y, t0.w, t1.y, t1.w, t2.y, t2.w, t3.y, t3.w};
+    uint32_t ao[4], bo[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const float a0 = bf16_lo(au[q]), a1 = bf16_hi(au[q]);
+      const float b0 = bf16_lo(bu[q]), b1 = bf16_hi(bu[q]);
+      ao[q] = pack_bf16x2(a0 * cv[2 * q] - b0 * sv[2 * q], a1 * cv[2 * q + 1] - b1 * sv[2 * q + 1]);
+      bo[q] = pack_bf16x2(b0 * cv[2 * q] + a0 * sv[2 * q], b1 * cv[2 * q + 1] + a1 * sv[2 * q + 1]);
+    }
+    *p0 = make_uint4(ao[0], ao[1], ao[2], ao[3]);
+    *p1 = make_uint4(bo[0], bo[1], bo[2], bo[3]);
+  }
+}
+
+// ---- SwiGLU: act[i, j] = silu(gu[i, j]) * gu[i, F + j] --------------------------
+__global__ void __launch_bounds__(kRowThreads)
+    swiglu_kernel(const uint4* __restrict__ gu, const int32_t* __restrict__ n_exec, int cap, int F,
+                  uint4* __restrict__ act) {
+  const int n = min(*n_exec, cap);
+  const int fc = F >> 3;
+  const size_t total = (size_t)n * fc;
+  for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < total;
+       e += (size_t)gridDim.x * blockDim.x) {
+    const size_t i = e / fc, c = e % fc;
+    const uint4 g = ld_nc_16(gu + i * 2 * fc + c);
+    const uint4 u = ld_nc_16(gu + i * 2 * fc + fc + c);
+    const uint32_t gg[4] = {g.x, g.y, g.z, g.w}, uu[4] = {u.x, u.y, u.z, u.w};
+    uint32_t o[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const float g0 = bf16_lo(gg[q]), g1 = bf16_hi(gg[q]);
+      o[q] = pack_bf16x2(g0 / (1.f + __expf(-g0)) * bf16_lo(uu[q]),
+                         g1 / (1.f + __expf(-g1)) * bf16_hi(uu[q]));
+    }
+    st_16(act + e, make_uint4(o[0], o[1], o[2], o[3]));
+  }
+}
+
+// ---- KV-cache append of the executed tokens' K (rotated) and V ------------------
+__global__ void __launch_bounds__(kRowThreads)
+    kv_append_kernel(const uint4* __restrict__ qkv, const int32_t* __restrict__ n_exec, int cap_rows,
+                     int ld, int q_dim, int kv_dim, const int32_t* __restrict__ cu_exec, int B,
+                     uint4* __restrict__ cache_k, uint4* __restrict__ cache_v,
+                     const int32_t* __restrict__ kv_len, int cap) {
+  const int n = min(*n_exec, cap_rows);
+  const int kc = kv_dim >> 3;
+  const int ldc = ld >> 3;
+  const size_t total = (size_t)n * kc;
+  for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < total;
+       e += (size_t)gridDim.x * blockDim.x) {
+    const int i = (int)(e / kc), c = (int)(e % kc);
+    int lo = 0, hi = B;  // sequence of executed token i: cu_exec[lo] <= i < cu_exec[hi]
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (cu_exec[mid] <= i) lo = mid; else hi = mid;
+    }
+    const int slot = kv_len[lo] + (i - cu_exec[lo]);
+    if (slot >= cap) continue;  // capacity is validated on the host for the worst case
+    const size_t dst = ((size_t)lo * cap + slot) * kc + c;
+    cache_k[dst] = qkv[(size_t)i * ldc + (q_dim >> 3) + c];
+    cache_v[dst] = qkv[(size_t)i * ldc + ((q_dim + kv_dim) >> 3) + c];
+  }
+}
+
+__global__ void kv_len_update_kernel(int32_t* kv_len, const int32_t* cu_exec, int B, int cap) {
+  for (int b = blockIdx.x * blockDim.x + threadIdx.x; b < B; b += gridDim.x * blockDim.x)
+    kv_len[b] = min(cap, kv_len[b] + cu_exec[b + 1] - cu_exec[b]);
+}
+
+// ---- embedding gather ------------------------------------------------------------
+__global__ void __launch_bounds__(kRowThreads)
+    embed_kernel(const uint4* __restrict__ embed, const int32_t* __restrict__ ids, int T, int d,
+                 int vocab, uint4* __restrict__ out) {
+  const int lane = threadIdx.x & 31;
+  const int warps = (gridDim.x * blockDim.x) >> 5;
+  const int chunks = d >> 3;
+  for (int t = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; t < T; t += warps) {
+    int id = ids[t];
+    id = id < 0 ? 0 : (id >= vocab ? vocab - 1 : id);
+    for (int cc = lane; cc < chunks; cc += 32)
+      st_16(out + (size_t)t * chunks + cc, ld_nc_16(embed + (size_t)id * chunks + cc));
+  }
+}
+
+// ---- host launchers ----------------------------------------------------------------
+
+static int row_grid(int per_sm) { return sm_count() * per_sm; }
+
+int launch_compact(const void* x, const int32_t* idx, const int32_t* n_exec, int cap, int d,
+                   const float* gamma, float eps, void* xc, void* hn, cudaStream_t s) {
+  const int chunks = d / 8;
+  const int grid = row_grid(8);
+  auto X = static_cast<const uint4*>(x);
+  auto XC = static_cast<uint4*>(xc);
+  auto HN = static_cast<uint4*>(hn);
+  if (chunks <= 32 * 4)
+    compact_kernel<4><<<grid, kRowThreads, 0, s>>>(X, idx, n_exec, cap, d, gamma, eps, XC, HN);
+  else if (chunks <= 32 * 16)
+    compact_kernel<16><<<grid, kRowThreads, 0, s>>>(X, idx, n_exec, cap, d, gamma, eps, XC, HN);
+  else if (chunks <= 32 * 32)
+    compact_kernel<32><<<grid, kRowThreads, 0, s>>>(X, idx, n_exec, cap, d, gamma, eps, XC, HN);
+  else
+    return QTALE_ERR_SHAPE;
+  return launch_status(cudaGetLastError());
+}
+
+int launch_scatter_add(void* x, const void* xc, const float* f, const int32_t* idx,
+                       const int32_t* n_exec, int cap, int d, cudaStream_t s) {
+  scatter_add_kernel<<<row_grid(8), kRowThreads, 0, s>>>(
+      static_cast<uint4*>(x), static_cast<const uint4*>(xc), reinterpret_cast<const float4*>(f),
+      idx, n_exec, cap, d);
+  return launch_status(cudaGetLastError());
+}
+
+int launch_rmsnorm_f32(const float* u, const int32_t* n_rows, int cap, int d, const float* gamma,
+                       float eps, void* out, cudaStream_t s) {
+  const int chunks = d / 4;
+  const int grid = min(cap, row_grid(8));
+  auto U = reinterpret_cast<const float4*>(u);
+  auto O = static_cast<uint2*>(out);
+  if (chunks <= kRowThreads * 1)
+    rmsnorm_f32_kernel<1><<<grid, kRowThreads, 0, s>>>(U, n_rows, cap, d, gamma, eps, O);
+  else if (chunks <= kRowThreads * 4)
+    rmsnorm_f32_kernel<4><<<grid, kRowThreads, 0, s>>>(U, n_rows, cap, d, gamma, eps, O);
+  else if (chunks <= kRowThreads * 8)
+    rmsnorm_f32_kernel<8><<<grid, kRowThreads, 0, s>>>(U, n_rows, cap, d, gamma, eps, O);
+  else
+    return QTALE_ERR_SHAPE;
+  return launch_status(cudaGetLastError());
+}
+
+int launch_rope_table(const int32_t* pos, const int32_t* n_exec, int cap, int hd, float base,
+                      float* cs, cudaStream_t s) {
+  rope_table_kernel<<<row_grid(4), 256, 0, s>>>(pos, n_exec, cap, hd / 2, base,
+                                                reinterpret_cast<float2*>(cs));
+  return launch_status(cudaGetLastError());
+}
+
+int launch_rope(void* qkv, const int32_t* n_exec, int cap, int ld, int n_rot, int hd,
+                const float* cs, cudaStream_t s) {
+  rope_kernel<<<row_grid(8), kRowThreads, 0, s>>>(static_cast<uint4*>(qkv), n_exec, cap, ld, n_rot,
+                                                  hd, reinterpret_cast<const float2*>(cs));
+  return launch_status(cudaGetLastError());
+}
+
+int launch_swiglu(const void* gu, const int32_t* n_exec, int cap, int F, void* act,
+                  cudaStream_t s) {
+  swiglu_kernel<<<row_grid(8), kRowThreads, 0, s>>>(static_cast<const uint4*>(gu), n_exec, cap, F,
+                                                    static_cast<uint4*>(act));
+  return launch_status(cudaGetLastError());
+}
+
+int launch_kv_append(const void* qkv, const int32_t* n_exec, int cap_rows, int ld, int q_dim,
+                     int kv_dim, const int32_t* cu_exec, int B, void* cache_k, void* cache_v,
+                     int32_t* kv_len, int cap, cudaStream_t s) {
+  kv_append_kernel<<<row_grid(4), kRowThreads, 0, s>>>(
+      static_cast<const uint4*>(qkv), n_exec, cap_rows, ld, q_dim, kv_dim, cu_exec, B,
+      static_cast<uint4*>(cache_k), static_cast<uint4*>(cache_v), kv_len, cap);
+  if (cudaGetLastError() != cudaSuccess) return QTALE_ERR_CUDA;
+  kv_len_update_kernel<<<(B + 255) / 256, 256, 0, s>>>(kv_len, cu_exec, B, cap);
+  return launch_status(cudaGetLastError());
+}
+
+int launch_embed(const void* embed, const int32_t* ids, int T, int d, int vocab, void* out,
+                 cudaStream_t s) {
+  embed_kernel<<<row_grid(8), kRowThreads, 0, s>>>(static_cast<const uint4*>(embed), ids, T, d,
+                                                   vocab, static_cast<uint4*>(out));
+  return launch_status(cudaGetLastError());
+}
+
+}  // namespace qtale
+
+using namespace qtale;
+
+extern "C" {
+
+int qtale_compact(const void* x, const int32_t* idx, const int32_t* n_exec, int T, int d,
+                  const float* rms_gamma, float eps, void* xc_out, void* hn_out, void* stream) {
+  if (!x || !idx || !n_exec) return QTALE_ERR_NULL;
+  if (!xc_out && !hn_out) return QTALE_ERR_NULL;
+  if (hn_out && !rms_gamma) return QTALE_ERR_NULL;
+  if (T < 1 || d < 8 || d % 8 != 0) return QTALE_ERR_SHAPE;
+  if (!aligned16(x) || !aligned16(xc_out) || !aligned16(hn_out) || !aligned16(rms_gamma))
+    return QTALE_ERR_ALIGN;
+  return launch_compact(x, idx, n_exec, T, d, rms_gamma, eps, xc_out, hn_out,
+                        static_cast<cudaStream_t>(stream));
+}
+
+int qtale_scatter_add(void* x_inout, const void* xc, const float* f, const int32_t* idx,
+                      const int32_t* n_exec, int T, int d, void* stream) {
+  if (!x_inout || !xc || !f || !idx || !n_exec) return QTALE_ERR_NULL;
+  if (T < 1 || d < 8 || d % 8 != 0) return QTALE_ERR_SHAPE;
+  if (!aligned16(x_inout) || !aligned16(xc) || !aligned16(f)) return QTALE_ERR_ALIGN;
+  return launch_scatter_add(x_inout, xc, f, idx, n_exec, T, d, static_cast<cudaStream_t>(stream));
+}
+
+}  // extern "C"
