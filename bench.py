@@ -247,18 +247,19 @@ def run_ours(args):
     k = api.topk_count(ratio, T)
     m_dev = torch.tensor([k], dtype=torch.int32, device=dev)
     qd = sh.n_heads * sh.head_dim
-    a_d = torch.randn(T, sh.d, device=dev).to(torch.bfloat16)
-    a_q = torch.randn(T, qd, device=dev).to(torch.bfloat16)
-    a_f = torch.randn(T, sh.ffn, device=dev).to(torch.bfloat16)
-    y_qkv = torch.empty(T, lw.qkv.N, dtype=torch.bfloat16, device=dev)
-    y_o = torch.empty(T, sh.d, dtype=torch.bfloat16, device=dev)
-    y_act = torch.empty(T, sh.ffn, dtype=torch.bfloat16, device=dev)
+    adt = api.act_torch_dtype(cfg.act_dtype)
+    a_d = torch.randn(T, sh.d, device=dev).to(adt)
+    a_q = torch.randn(T, qd, device=dev).to(adt)
+    a_f = torch.randn(T, sh.ffn, device=dev).to(adt)
+    y_qkv = torch.empty(T, lw.qkv.N, dtype=adt, device=dev)
+    y_o = torch.empty(T, sh.d, dtype=adt, device=dev)
+    y_act = torch.empty(T, sh.ffn, dtype=adt, device=dev)
 
     def gemms(i):
-        api.wq_gemm(a_d, lw.qkv, m_dev, api.EPI_STORE_BF16, y=y_qkv)
-        api.wq_gemm(a_q, lw.o, m_dev, api.EPI_STORE_BF16, y=y_o)
+        api.wq_gemm(a_d, lw.qkv, m_dev, api.EPI_STORE_16, y=y_qkv)
+        api.wq_gemm(a_q, lw.o, m_dev, api.EPI_STORE_16, y=y_o)
         api.wq_gemm(a_d, lw.gate_up, m_dev, api.EPI_SWIGLU, y=y_act)
-        api.wq_gemm(a_f, lw.down, m_dev, api.EPI_STORE_BF16, y=y_o)
+        api.wq_gemm(a_f, lw.down, m_dev, api.EPI_STORE_16, y=y_o)
 
     g_steps = max(3, args.steps // 2)
     g_ms = timed(gemms, g_steps, 3) / g_steps
@@ -285,8 +286,10 @@ def run_ours(args):
 
     line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps,
                 warmup=args.warmup, ms_per_step=ms_per_step, higher_is_better=True, scaling="weak",
-                vs_baseline=None, dtype="bf16", data="synthetic",
+                vs_baseline=None, dtype="f16", data="synthetic",
                 config=dict(workload=WORKLOAD, ratio=ratio, select="topk", executed_tokens=n_exec,
+                            precision="bf16 residual stream in/out; fp16 internal activations and "
+                                      "dequantised weights, fp32 accumulation",
                             tokens=T,
                             l2="inputs larger than L2 (packed weights 107 MB + more than 1 GB of "
                                "activations per step, %d rotating input buffers)" % n_buf,

@@ -22,7 +22,13 @@
  *    Calls enqueue work and return without synchronising.  The number of
  *    executed tokens stays on the device (int32) and is never read back by
  *    the library.
- *  - Activations are bf16, row-major, innermost dimension contiguous.
+ *  - The residual stream (layer input / output) is bf16, row-major, innermost
+ *    dimension contiguous.  Tensors the layer keeps between its kernels
+ *    (normed activations, q/k/v, attention output, SwiGLU activation, KV cache)
+ *    are 16-bit in the format `act_dtype` selects: QTALE_ACT_BF16, or
+ *    QTALE_ACT_F16 whose three extra significand bits keep the accumulated
+ *    rounding error of a 4096-wide layer inside the max-abs 2e-2 bound (fp16's
+ *    range, 65504, must then cover those tensors).  Accumulation is fp32.
  *    Tokens of all sequences are flattened: token t of the call belongs to
  *    sequence b with cu_seqlens[b] <= t < cu_seqlens[b+1].
  *  - A device-side wait that exceeds its iteration limit ends the kernel
@@ -49,7 +55,10 @@ extern "C" {
 #define QTALE_ERR_CAPACITY (-7)  /* a count exceeds the capacity of its buffer */
 #define QTALE_ERR_TIMEOUT (-8)   /* a bounded device-side wait gave up */
 #define QTALE_ERR_CUDA (-9)      /* a CUDA runtime / driver call failed */
-#define QTALE_ERR_MODE (-10)     /* unknown mode / epilogue / phase */
+#define QTALE_ERR_MODE (-10)     /* unknown mode / epilogue / phase / dtype */
+
+#define QTALE_ACT_BF16 0
+#define QTALE_ACT_F16 1
 
 const char* qtale_strerror(int status);
 
@@ -119,13 +128,15 @@ int qtale_index_bookkeeping(const int32_t* idx, int n, int T, const int32_t* cu_
 /*
  * Gather of the executed rows: xc[i,:] = x[idx[i],:] for i < *n_exec.
  * If rms_gamma != NULL also hn[i,:] = x[idx[i],:] / sqrt(mean(x^2) + eps) * gamma
- * (fp32 arithmetic, one bf16 rounding).  xc_out or hn_out may be NULL (not
- * both).  Rows i >= *n_exec of the outputs are left untouched.
+ * (fp32 arithmetic, one rounding to act_dtype).  xc_out or hn_out may be NULL
+ * (not both).  Rows i >= *n_exec of the outputs are left untouched.
  *   x [T, d] bf16; idx [T] int32; n_exec [1] int32; rms_gamma [d] fp32;
- *   xc_out, hn_out [T, d] bf16 (capacity T rows).  d % 8 == 0.
+ *   xc_out [T, d] bf16 (byte copy), hn_out [T, d] act_dtype (capacity T rows).
+ *   d % 8 == 0.
  */
 int qtale_compact(const void* x, const int32_t* idx, const int32_t* n_exec, int T, int d,
-                  const float* rms_gamma, float eps, void* xc_out, void* hn_out, void* stream);
+                  const float* rms_gamma, float eps, int act_dtype, void* xc_out, void* hn_out,
+                  void* stream);
 
 /*
  * Residual scatter (Eq. 3, execute branch), in place:
@@ -167,11 +178,11 @@ typedef struct {
 int qtale_wq_repack(const uint8_t* codes, const uint16_t* scales, const uint16_t* zeros, int N,
                     int K, int bits, int group, int row_mode, void* packed_out, size_t* bytes);
 
-#define QTALE_EPI_STORE_BF16 0    /* y[m,n] = bf16(acc)                                  */
+#define QTALE_EPI_STORE_16 0      /* y[m,n] = act_dtype(acc)                             */
 #define QTALE_EPI_STORE_F32 1     /* y[m,n] = acc                                  (fp32) */
 #define QTALE_EPI_RESID_F32 2     /* y[m,n] = float(resid[idx[m],n]) + acc         (fp32) */
 #define QTALE_EPI_RESID_SCATTER 3 /* dst[idx[m],n] = bf16(resid_f32[m,n] + acc)    (Eq. 3) */
-#define QTALE_EPI_SWIGLU 4        /* y[m,j] = bf16(silu(acc[m,j]) * acc[m,F+j]), N = 2F;
+#define QTALE_EPI_SWIGLU 4        /* y[m,j] = act_dtype(silu(acc[m,j]) * acc[m,F+j]), N = 2F;
                                      needs QTALE_WQ_ROWS_SWIGLU weights                   */
 
 typedef struct {
@@ -186,13 +197,15 @@ typedef struct {
 /*
  * y = epilogue(a W^T) on the tensor cores; rows m >= *m_dev (or >= M_cap when
  * m_dev == NULL) are neither computed nor written.
- *   a  bf16 [M_cap, lda]  (lda >= K elements, lda * 2 bytes % 16 == 0)
+ *   a  act_dtype [M_cap, lda]  (lda >= K elements, lda * 2 bytes % 16 == 0)
  *   y  [M_cap, ldy]; element type set by the epilogue
- * The packed weights are dequantised to bf16 inside the kernel (exact
- * (code - zero) * scale in fp32, one rounding) and accumulated in fp32.
+ * The packed weights are dequantised inside the kernel to the 16-bit format of
+ * `a` (exact (code - zero) * scale in fp32, one rounding) and accumulated in
+ * fp32.
  */
 int qtale_wq_gemm(const void* a, int lda, const int32_t* m_dev, int M_cap, const qtale_wq_weight* w,
-                  int epilogue, const qtale_epilogue_args* epi, void* y, int ldy, void* stream);
+                  int act_dtype, int epilogue, const qtale_epilogue_args* epi, void* y, int ldy,
+                  void* stream);
 
 /* ------------------------------------------------------------------------- */
 /* Layer and model                                                             */
@@ -204,7 +217,11 @@ typedef struct {
   float rms_eps, rope_theta;                /* RMSNorm epsilon, rotary base               */
   int select_mode;                          /* QTALE_SELECT_*                             */
   float theta;                              /* threshold of Eq. 9 (THRESHOLD)             */
-  float ratio;                              /* execution ratio in [0,1] (TOPK)            */
+  float ratio;                              /* execution ratio in [0,1] (TOPK): k =
+                                               qtale_topk_count(ratio, T), capped by the
+                                               number of valid tokens                      */
+  int act_dtype;                            /* QTALE_ACT_*: format of the layer's internal
+                                               16-bit tensors and of its KV cache          */
 } qtale_layer_config;
 
 typedef struct {
@@ -221,8 +238,8 @@ typedef struct {
 /* Per-layer KV cache.  Only executed tokens enter it: a bypassed token does not
  * evaluate f_l (Eq. 3) and therefore produces no key or value at that layer. */
 typedef struct {
-  void* k;         /* bf16 [B, cap, n_kv_heads * head_dim], rotary already applied */
-  void* v;         /* bf16 [B, cap, n_kv_heads * head_dim]                         */
+  void* k;         /* act_dtype [B, cap, n_kv_heads * head_dim], rotary already applied */
+  void* v;         /* act_dtype [B, cap, n_kv_heads * head_dim]                         */
   int32_t* kv_len; /* int32 [B], entries in use per sequence (updated)             */
   int cap;
 } qtale_kv_cache;

@@ -18,7 +18,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libqtale.so")
 
 SELECT_THRESHOLD, SELECT_TOPK, SELECT_FORCED = 0, 1, 2
-EPI_STORE_BF16, EPI_STORE_F32, EPI_RESID_F32, EPI_RESID_SCATTER, EPI_SWIGLU = 0, 1, 2, 3, 4
+EPI_STORE_16, EPI_STORE_F32, EPI_RESID_F32, EPI_RESID_SCATTER, EPI_SWIGLU = 0, 1, 2, 3, 4
+ACT_BF16, ACT_F16 = 0, 1
 ROWS_PLAIN, ROWS_SWIGLU = 0, 1
 PHASE_PREFILL, PHASE_DECODE = 0, 1
 
@@ -49,7 +50,7 @@ class LayerConfig(C.Structure):
     _fields_ = [("d", C.c_int), ("n_heads", C.c_int), ("n_kv_heads", C.c_int),
                 ("head_dim", C.c_int), ("ffn", C.c_int), ("bits", C.c_int), ("group", C.c_int),
                 ("rms_eps", C.c_float), ("rope_theta", C.c_float), ("select_mode", C.c_int),
-                ("theta", C.c_float), ("ratio", C.c_float)]
+                ("theta", C.c_float), ("ratio", C.c_float), ("act_dtype", C.c_int)]
 
 
 class LayerWeightsC(C.Structure):
@@ -95,13 +96,14 @@ def lib():
             C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p,
             C.c_void_p, C.c_void_p]
         L.qtale_compact.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int,
-                                    C.c_void_p, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p]
+                                    C.c_void_p, C.c_float, C.c_int, C.c_void_p, C.c_void_p,
+                                    C.c_void_p]
         L.qtale_scatter_add.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                         C.c_int, C.c_int, C.c_void_p]
         L.qtale_wq_repack.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
                                       C.c_int, C.c_int, C.c_void_p, C.POINTER(C.c_size_t)]
         L.qtale_wq_gemm.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.POINTER(WqWeight),
-                                    C.c_int, C.POINTER(EpilogueArgs), C.c_void_p, C.c_int,
+                                    C.c_int, C.c_int, C.POINTER(EpilogueArgs), C.c_void_p, C.c_int,
                                     C.c_void_p]
         L.qtale_layer_workspace_bytes.restype = C.c_size_t
         L.qtale_layer_workspace_bytes.argtypes = [C.POINTER(LayerConfig), C.c_int, C.c_int]
@@ -189,13 +191,20 @@ def index_bookkeeping(idx, n, T, cu_seqlens, pos0=None):
 # gather / scatter
 # ---------------------------------------------------------------------------------
 
-def compact(x, idx, n_exec, rms_gamma=None, eps=1e-5, want_xc=True, xc_out=None, hn_out=None):
-    """qtale_compact.  Returns (xc, hn); either may be None."""
+def act_torch_dtype(act_dtype):
+    return torch.float16 if act_dtype == ACT_F16 else torch.bfloat16
+
+
+def compact(x, idx, n_exec, rms_gamma=None, eps=1e-5, want_xc=True, xc_out=None, hn_out=None,
+            act_dtype=ACT_BF16):
+    """qtale_compact.  Returns (xc, hn); either may be None.  hn is in act_dtype."""
     T, d = int(x.shape[0]), int(x.shape[1])
     xc = xc_out if xc_out is not None else (torch.zeros_like(x) if want_xc else None)
-    hn = hn_out if hn_out is not None else (torch.zeros_like(x) if rms_gamma is not None else None)
+    hn = hn_out
+    if hn is None and rms_gamma is not None:
+        hn = torch.zeros(T, d, dtype=act_torch_dtype(act_dtype), device=x.device)
     check(lib().qtale_compact(_ptr(x), _ptr(idx), _ptr(n_exec), T, d, _ptr(rms_gamma), float(eps),
-                              _ptr(xc), _ptr(hn), _stream()), "qtale_compact")
+                              int(act_dtype), _ptr(xc), _ptr(hn), _stream()), "qtale_compact")
     return xc, hn
 
 
@@ -237,10 +246,12 @@ class QuantWeight:
         self.c = WqWeight(self.blob.data_ptr(), self.N, self.K, self.bits, self.group, row_mode)
 
 
-def wq_gemm(a, w: QuantWeight, m_dev=None, epilogue=EPI_STORE_BF16, y=None, idx=None, resid=None,
+def wq_gemm(a, w: QuantWeight, m_dev=None, epilogue=EPI_STORE_16, y=None, idx=None, resid=None,
             dst=None):
-    """qtale_wq_gemm.  a bf16 [M_cap, K]; returns y (or dst for RESID_SCATTER)."""
+    """qtale_wq_gemm.  a bf16 or fp16 [M_cap, K] (its dtype is the act_dtype); returns y
+    (or dst for RESID_SCATTER)."""
     M_cap, lda = int(a.shape[0]), int(a.stride(0))
+    act_dtype = ACT_F16 if a.dtype == torch.float16 else ACT_BF16
     epi = None
     if epilogue in (EPI_RESID_F32, EPI_RESID_SCATTER):
         epi = EpilogueArgs(idx.data_ptr(), resid.data_ptr(), int(resid.stride(0)),
@@ -248,9 +259,9 @@ def wq_gemm(a, w: QuantWeight, m_dev=None, epilogue=EPI_STORE_BF16, y=None, idx=
                            int(dst.stride(0)) if dst is not None else 0)
     if y is None and epilogue != EPI_RESID_SCATTER:
         n_out = w.N // 2 if epilogue == EPI_SWIGLU else w.N
-        dt = torch.bfloat16 if epilogue in (EPI_STORE_BF16, EPI_SWIGLU) else torch.float32
+        dt = a.dtype if epilogue in (EPI_STORE_16, EPI_SWIGLU) else torch.float32
         y = torch.zeros(M_cap, n_out, dtype=dt, device=a.device)
-    check(lib().qtale_wq_gemm(_ptr(a), lda, _ptr(m_dev), M_cap, C.byref(w.c), int(epilogue),
+    check(lib().qtale_wq_gemm(_ptr(a), lda, _ptr(m_dev), M_cap, C.byref(w.c), act_dtype, int(epilogue),
                               C.byref(epi) if epi is not None else None, _ptr(y),
                               int(y.stride(0)) if y is not None else 0, _stream()), "qtale_wq_gemm")
     return dst if epilogue == EPI_RESID_SCATTER else y
@@ -260,9 +271,11 @@ def wq_gemm(a, w: QuantWeight, m_dev=None, epilogue=EPI_STORE_BF16, y=None, idx=
 # layer / model
 # ---------------------------------------------------------------------------------
 
-def layer_config(sh, select_mode=SELECT_THRESHOLD, theta=0.5, ratio=1.0) -> LayerConfig:
+def layer_config(sh, select_mode=SELECT_THRESHOLD, theta=0.5, ratio=1.0,
+                 act_dtype=ACT_F16) -> LayerConfig:
     return LayerConfig(sh.d, sh.n_heads, sh.n_kv_heads, sh.head_dim, sh.ffn, sh.bits, sh.group,
-                       sh.rms_eps, sh.rope_theta, int(select_mode), float(theta), float(ratio))
+                       sh.rms_eps, sh.rope_theta, int(select_mode), float(theta), float(ratio),
+                       int(act_dtype))
 
 
 class LayerWeights:
@@ -287,9 +300,10 @@ class LayerWeights:
 
 
 class KvCache:
-    def __init__(self, B, cap, kv_dim, device="cuda"):
-        self.k = torch.zeros(B, cap, kv_dim, dtype=torch.bfloat16, device=device)
-        self.v = torch.zeros(B, cap, kv_dim, dtype=torch.bfloat16, device=device)
+    def __init__(self, B, cap, kv_dim, device="cuda", act_dtype=ACT_F16):
+        dt = act_torch_dtype(act_dtype)
+        self.k = torch.zeros(B, cap, kv_dim, dtype=dt, device=device)
+        self.v = torch.zeros(B, cap, kv_dim, dtype=dt, device=device)
         self.kv_len = torch.zeros(B, dtype=torch.int32, device=device)
         self.cap = cap
         self.c = KvCacheC(self.k.data_ptr(), self.v.data_ptr(), self.kv_len.data_ptr(), cap)
@@ -347,6 +361,12 @@ def model_prefill(cfg: ModelConfig, layers, embed, ids, cu_seqlens, ws, hidden_o
 def to_device_bf16(a: np.ndarray, device="cuda") -> torch.Tensor:
     """float32 numpy array of bf16-representable values -> bf16 device tensor (exact)."""
     return torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).to(device).to(torch.bfloat16)
+
+
+def to_device_act(a: np.ndarray, act_dtype, device="cuda") -> torch.Tensor:
+    """float32 numpy array -> device tensor in the given 16-bit activation format (rounds)."""
+    return torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).to(device).to(
+        act_torch_dtype(act_dtype))
 
 
 def to_host_f32(t: torch.Tensor) -> np.ndarray:

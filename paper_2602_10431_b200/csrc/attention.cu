@@ -39,13 +39,22 @@ __device__ __forceinline__ void ldsm_x4_trans(uint32_t (&r)[4], const void* smem
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
                : "r"(s));
 }
-__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0,
-                                               uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
-      "{%0,%1,%2,%3};"
-      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+template <int ACT>
+__device__ __forceinline__ void mma_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0,
+                                          uint32_t b1) {
+  if (ACT == 1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+        "{%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+  } else {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+        "{%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+  }
 }
 
 // ---------------------------------------------------------------------------
@@ -73,7 +82,7 @@ __device__ __forceinline__ void load_tile(unsigned char* smem, const __nv_bfloat
   }
 }
 
-template <int HD>
+template <int HD, int ACT>
 __global__ void __launch_bounds__(kAttnThreads)
     attn_prefill_kernel(const __nv_bfloat16* __restrict__ qkv, int ld, int k_off, int v_off,
                         const int32_t* __restrict__ cu_exec, int B, int rep,
@@ -161,8 +170,8 @@ __global__ void __launch_bounds__(kAttnThreads)
         const int r = np * 16 + (mat >> 1) * 8 + (lane & 7);
         const int c = ks * 2 + (mat & 1);
         ldsm_x4(kf, k_s + sw_off<HD>(r, c));
-        mma_bf16_16816(s[2 * np], qf[ks], kf[0], kf[1]);
-        mma_bf16_16816(s[2 * np + 1], qf[ks], kf[2], kf[3]);
+        mma_16816<ACT>(s[2 * np], qf[ks], kf[0], kf[1]);
+        mma_16816<ACT>(s[2 * np + 1], qf[ks], kf[2], kf[3]);
       }
     }
     // scale, causal / length mask (only the diagonal tile needs it)
@@ -212,8 +221,8 @@ __global__ void __launch_bounds__(kAttnThreads)
       const float p2 = exp2f(s[i][2] - msafe[1]), p3 = exp2f(s[i][3] - msafe[1]);
       l_run[0] += p0 + p1;
       l_run[1] += p2 + p3;
-      pf[i >> 1][(i & 1) * 2 + 0] = pack_bf16x2(p0, p1);
-      pf[i >> 1][(i & 1) * 2 + 1] = pack_bf16x2(p2, p3);
+      pf[i >> 1][(i & 1) * 2 + 0] = Act16<ACT>::pack(p0, p1);
+      pf[i >> 1][(i & 1) * 2 + 1] = Act16<ACT>::pack(p2, p3);
     }
     // O += P V
 #pragma unroll
@@ -225,8 +234,8 @@ __global__ void __launch_bounds__(kAttnThreads)
         const int r = kk * 16 + (mat & 1) * 8 + (lane & 7);
         const int c = np * 2 + (mat >> 1);
         ldsm_x4_trans(vf, v_s + sw_off<HD>(r, c));
-        mma_bf16_16816(o[2 * np], pf[kk], vf[0], vf[1]);
-        mma_bf16_16816(o[2 * np + 1], pf[kk], vf[2], vf[3]);
+        mma_16816<ACT>(o[2 * np], pf[kk], vf[0], vf[1]);
+        mma_16816<ACT>(o[2 * np + 1], pf[kk], vf[2], vf[3]);
       }
     }
     __syncthreads();  // all warps done with this buffer before it is refilled
@@ -246,10 +255,10 @@ __global__ void __launch_bounds__(kAttnThreads)
     const int col = h * HD + i * 8 + 2 * t;
     if (ra < len)
       *reinterpret_cast<uint32_t*>(out + (size_t)(seq0 + ra) * ldo + col) =
-          pack_bf16x2(o[i][0] * inv0, o[i][1] * inv0);
+          Act16<ACT>::pack(o[i][0] * inv0, o[i][1] * inv0);
     if (rb < len)
       *reinterpret_cast<uint32_t*>(out + (size_t)(seq0 + rb) * ldo + col) =
-          pack_bf16x2(o[i][2] * inv1, o[i][3] * inv1);
+          Act16<ACT>::pack(o[i][2] * inv1, o[i][3] * inv1);
   }
 }
 
@@ -258,7 +267,7 @@ __global__ void __launch_bounds__(kAttnThreads)
 // ---------------------------------------------------------------------------
 constexpr int kDecThreads = 128;
 
-template <int HD, int REP>
+template <int HD, int REP, int ACT>
 __global__ void __launch_bounds__(kDecThreads)
     attn_decode_kernel(const __nv_bfloat16* __restrict__ qkv, int ld,
                        const int32_t* __restrict__ idx, const int32_t* __restrict__ n_exec,
@@ -288,8 +297,8 @@ __global__ void __launch_bounds__(kDecThreads)
     const uint32_t u[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
-      q[r][2 * e] = bf16_lo(u[e]) * scale_log2;
-      q[r][2 * e + 1] = bf16_hi(u[e]) * scale_log2;
+      q[r][2 * e] = Act16<ACT>::lo(u[e]) * scale_log2;
+      q[r][2 * e + 1] = Act16<ACT>::hi(u[e]) * scale_log2;
     }
   }
   float m[REP], l[REP], acc[REP][8];
@@ -322,8 +331,8 @@ __global__ void __launch_bounds__(kDecThreads)
       float kf[8], vf[8];
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
-        kf[2 * e] = ok ? bf16_lo(ku[e]) : 0.f; kf[2 * e + 1] = ok ? bf16_hi(ku[e]) : 0.f;
-        vf[2 * e] = ok ? bf16_lo(vu[e]) : 0.f; vf[2 * e + 1] = ok ? bf16_hi(vu[e]) : 0.f;
+        kf[2 * e] = ok ? Act16<ACT>::lo(ku[e]) : 0.f; kf[2 * e + 1] = ok ? Act16<ACT>::hi(ku[e]) : 0.f;
+        vf[2 * e] = ok ? Act16<ACT>::lo(vu[e]) : 0.f; vf[2 * e + 1] = ok ? Act16<ACT>::hi(vu[e]) : 0.f;
       }
 #pragma unroll
       for (int r = 0; r < REP; ++r) {
@@ -361,15 +370,15 @@ __global__ void __launch_bounds__(kDecThreads)
       num += w * s_acc[gI][r][c];
       den += w * s_l[gI][r];
     }
-    out[(size_t)i * ldo + (size_t)(hk * REP + r) * HD + c] =
-        __float2bfloat16_rn(den > 0.f ? num / den : 0.f);
+    reinterpret_cast<unsigned short*>(out)[(size_t)i * ldo + (size_t)(hk * REP + r) * HD + c] =
+        Act16<ACT>::one(den > 0.f ? num / den : 0.f);
   }
 }
 
 // ---------------------------------------------------------------------------
 // host launchers
 // ---------------------------------------------------------------------------
-template <int HD>
+template <int HD, int ACT>
 static int launch_prefill_hd(const void* qkv, int ld, int k_off, int v_off, const int32_t* cu_exec,
                              int B, int H, int Hkv, int T_cap, void* out, int ldo, cudaStream_t s) {
   const size_t smem = (size_t)5 * kBK * HD * 2;
@@ -377,7 +386,7 @@ static int launch_prefill_hd(const void* qkv, int ld, int k_off, int v_off, cons
   int dev = 0;
   cudaGetDevice(&dev);
   if (dev >= 0 && dev < 64 && !configured[dev]) {
-    if (cudaFuncSetAttribute(attn_prefill_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    if (cudaFuncSetAttribute(attn_prefill_kernel<HD, ACT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)smem) != cudaSuccess)
       return QTALE_ERR_CUDA;
     configured[dev] = true;
@@ -385,21 +394,25 @@ static int launch_prefill_hd(const void* qkv, int ld, int k_off, int v_off, cons
   const int max_tiles = (T_cap + kBQ - 1) / kBQ + B;
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)HD);
   dim3 grid(max_tiles, H);
-  attn_prefill_kernel<HD><<<grid, kAttnThreads, smem, s>>>(
+  attn_prefill_kernel<HD, ACT><<<grid, kAttnThreads, smem, s>>>(
       static_cast<const __nv_bfloat16*>(qkv), ld, k_off, v_off, cu_exec, B, H / Hkv,
       static_cast<__nv_bfloat16*>(out), ldo, scale_log2);
   return launch_status(cudaGetLastError());
 }
 
-int launch_attn_prefill(const void* qkv, int ld, int H, int Hkv, int hd, const int32_t* cu_exec,
-                        int B, int T_cap, void* out, int ldo, cudaStream_t s) {
+int launch_attn_prefill(const void* qkv, int ld, int H, int Hkv, int hd, int act,
+                        const int32_t* cu_exec, int B, int T_cap, void* out, int ldo,
+                        cudaStream_t s) {
   const int k_off = H * hd, v_off = (H + Hkv) * hd;
-  if (hd == 128) return launch_prefill_hd<128>(qkv, ld, k_off, v_off, cu_exec, B, H, Hkv, T_cap, out, ldo, s);
-  if (hd == 64) return launch_prefill_hd<64>(qkv, ld, k_off, v_off, cu_exec, B, H, Hkv, T_cap, out, ldo, s);
+#define QTALE_PF(HD_, ACT_) \
+  launch_prefill_hd<HD_, ACT_>(qkv, ld, k_off, v_off, cu_exec, B, H, Hkv, T_cap, out, ldo, s)
+  if (hd == 128) return act == QTALE_ACT_F16 ? QTALE_PF(128, 1) : QTALE_PF(128, 0);
+  if (hd == 64) return act == QTALE_ACT_F16 ? QTALE_PF(64, 1) : QTALE_PF(64, 0);
+#undef QTALE_PF
   return QTALE_ERR_SHAPE;
 }
 
-template <int HD>
+template <int HD, int ACT>
 static int launch_decode_hd(const void* qkv, int ld, int H, int Hkv, const int32_t* idx,
                             const int32_t* n_exec, int B_cap, const void* ck, const void* cv,
                             const int32_t* kv_len, int cap, void* out, int ldo, cudaStream_t s) {
@@ -411,7 +424,7 @@ static int launch_decode_hd(const void* qkv, int ld, int H, int Hkv, const int32
   auto O = static_cast<__nv_bfloat16*>(out);
   const int rep = H / Hkv;
 #define QTALE_DEC(R)                                                                              \
-  attn_decode_kernel<HD, R><<<grid, kDecThreads, 0, s>>>(Q, ld, idx, n_exec, K, V, kv_len, cap,   \
+  attn_decode_kernel<HD, R, ACT><<<grid, kDecThreads, 0, s>>>(Q, ld, idx, n_exec, K, V, kv_len, cap,   \
                                                          Hkv, O, ldo, scale_log2)
   if (rep == 1) QTALE_DEC(1);
   else if (rep == 2) QTALE_DEC(2);
@@ -422,13 +435,15 @@ static int launch_decode_hd(const void* qkv, int ld, int H, int Hkv, const int32
   return launch_status(cudaGetLastError());
 }
 
-int launch_attn_decode(const void* qkv, int ld, int H, int Hkv, int hd, const int32_t* idx,
+int launch_attn_decode(const void* qkv, int ld, int H, int Hkv, int hd, int act, const int32_t* idx,
                        const int32_t* n_exec, int B_cap, const void* cache_k, const void* cache_v,
                        const int32_t* kv_len, int cap, void* out, int ldo, cudaStream_t s) {
-  if (hd == 128)
-    return launch_decode_hd<128>(qkv, ld, H, Hkv, idx, n_exec, B_cap, cache_k, cache_v, kv_len, cap, out, ldo, s);
-  if (hd == 64)
-    return launch_decode_hd<64>(qkv, ld, H, Hkv, idx, n_exec, B_cap, cache_k, cache_v, kv_len, cap, out, ldo, s);
+#define QTALE_DC(HD_, ACT_)                                                                       \
+  launch_decode_hd<HD_, ACT_>(qkv, ld, H, Hkv, idx, n_exec, B_cap, cache_k, cache_v, kv_len, cap, \
+                              out, ldo, s)
+  if (hd == 128) return act == QTALE_ACT_F16 ? QTALE_DC(128, 1) : QTALE_DC(128, 0);
+  if (hd == 64) return act == QTALE_ACT_F16 ? QTALE_DC(64, 1) : QTALE_DC(64, 0);
+#undef QTALE_DC
   return QTALE_ERR_SHAPE;
 }
 

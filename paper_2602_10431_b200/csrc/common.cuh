@@ -47,6 +47,38 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return r;
 }
 
+// 16-bit activation formats of the tensors the layer keeps between its kernels.
+// ACT = QTALE_ACT_BF16 (0) or QTALE_ACT_F16 (1).  Both are read as two values per
+// 32-bit word (element 0 in the low half) and written with one rounding.
+template <int ACT>
+struct Act16;
+template <>
+struct Act16<0> {
+  static __device__ __forceinline__ float lo(uint32_t p) { return bf16_lo(p); }
+  static __device__ __forceinline__ float hi(uint32_t p) { return bf16_hi(p); }
+  static __device__ __forceinline__ uint32_t pack(float l, float h) { return pack_bf16x2(l, h); }
+  static __device__ __forceinline__ unsigned short one(float v) {
+    return __bfloat16_as_ushort(__float2bfloat16_rn(v));
+  }
+};
+template <>
+struct Act16<1> {
+  static __device__ __forceinline__ float lo(uint32_t p) {
+    return __half2float(__ushort_as_half((unsigned short)(p & 0xFFFFu)));
+  }
+  static __device__ __forceinline__ float hi(uint32_t p) {
+    return __half2float(__ushort_as_half((unsigned short)(p >> 16)));
+  }
+  static __device__ __forceinline__ uint32_t pack(float l, float h) {
+    uint32_t r;
+    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(h), "f"(l));
+    return r;
+  }
+  static __device__ __forceinline__ unsigned short one(float v) {
+    return __half_as_ushort(__float2half_rn(v));
+  }
+};
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);

@@ -65,6 +65,7 @@ static int check_config(const qtale_layer_config* c) {
     return QTALE_ERR_SHAPE;
   if (c->select_mode < QTALE_SELECT_THRESHOLD || c->select_mode > QTALE_SELECT_FORCED)
     return QTALE_ERR_MODE;
+  if (c->act_dtype != QTALE_ACT_BF16 && c->act_dtype != QTALE_ACT_F16) return QTALE_ERR_MODE;
   return QTALE_OK;
 }
 
@@ -82,6 +83,7 @@ static int layer_forward_impl(const qtale_layer_config* c, const qtale_layer_wei
                               cudaStream_t s) {
   const int d = c->d, H = c->n_heads, Hkv = c->n_kv_heads, hd = c->head_dim, F = c->ffn;
   const int qd = H * hd, kvd = Hkv * hd, nqkv = qd + 2 * kvd;
+  const int act = c->act_dtype;
 
   // 1. execute / bypass decision and index lists
   const int32_t* idx = ws.idx;
@@ -103,23 +105,23 @@ static int layer_forward_impl(const qtale_layer_config* c, const qtale_layer_wei
     return QTALE_ERR_CUDA;
 
   // 2. gather the executed tokens and apply the first RMSNorm
-  QTALE_TRY(launch_compact(x, idx, ws.n_exec, T, d, w->gamma1, c->rms_eps, nullptr, ws.hn, s));
+  QTALE_TRY(launch_compact(x, idx, ws.n_exec, T, d, w->gamma1, c->rms_eps, act, nullptr, ws.hn, s));
   // 3. q, k, v projections
-  QTALE_TRY(wq_gemm_launch(ws.hn, d, ws.n_exec, T, &w->qkv, QTALE_EPI_STORE_BF16, nullptr, ws.qkv,
+  QTALE_TRY(wq_gemm_launch(ws.hn, d, ws.n_exec, T, &w->qkv, act, QTALE_EPI_STORE_16, nullptr, ws.qkv,
                            nqkv, s));
   // 4. rotary embedding at the original positions
   QTALE_TRY(launch_rope_table(ws.pos, ws.n_exec, T, hd, c->rope_theta, ws.cs, s));
-  QTALE_TRY(launch_rope(ws.qkv, ws.n_exec, T, nqkv, H + Hkv, hd, ws.cs, s));
+  QTALE_TRY(launch_rope(ws.qkv, ws.n_exec, T, nqkv, H + Hkv, hd, ws.cs, act, s));
   // 5. attention among executed tokens (+ cache)
   if (kv) {
     QTALE_TRY(launch_kv_append(ws.qkv, ws.n_exec, T, nqkv, qd, kvd, ws.cu_exec, B, kv->k, kv->v,
                                kv->kv_len, kv->cap, s));
   }
   if (phase == QTALE_PHASE_DECODE) {
-    QTALE_TRY(launch_attn_decode(ws.qkv, nqkv, H, Hkv, hd, idx, ws.n_exec, T, kv->k, kv->v,
+    QTALE_TRY(launch_attn_decode(ws.qkv, nqkv, H, Hkv, hd, act, idx, ws.n_exec, T, kv->k, kv->v,
                                  kv->kv_len, kv->cap, ws.ao, qd, s));
   } else {
-    QTALE_TRY(launch_attn_prefill(ws.qkv, nqkv, H, Hkv, hd, ws.cu_exec, B, T, ws.ao, qd, s));
+    QTALE_TRY(launch_attn_prefill(ws.qkv, nqkv, H, Hkv, hd, act, ws.cu_exec, B, T, ws.ao, qd, s));
   }
   // 6. output projection + residual: u = x[idx] + attention branch (fp32)
   qtale_epilogue_args e;
@@ -128,24 +130,24 @@ static int layer_forward_impl(const qtale_layer_config* c, const qtale_layer_wei
   e.ld_resid = d;
   e.dst = nullptr;
   e.ld_dst = 0;
-  QTALE_TRY(wq_gemm_launch(ws.ao, qd, ws.n_exec, T, &w->o, QTALE_EPI_RESID_F32, &e, ws.u, d, s));
+  QTALE_TRY(wq_gemm_launch(ws.ao, qd, ws.n_exec, T, &w->o, act, QTALE_EPI_RESID_F32, &e, ws.u, d, s));
   // 7. second RMSNorm
-  QTALE_TRY(launch_rmsnorm_f32(ws.u, ws.n_exec, T, d, w->gamma2, c->rms_eps, ws.hn, s));
+  QTALE_TRY(launch_rmsnorm_f32(ws.u, ws.n_exec, T, d, w->gamma2, c->rms_eps, act, ws.hn, s));
   // 8. gate / up projections and SwiGLU
   if (w->gate_up.row_mode == QTALE_WQ_ROWS_SWIGLU) {
-    QTALE_TRY(wq_gemm_launch(ws.hn, d, ws.n_exec, T, &w->gate_up, QTALE_EPI_SWIGLU, nullptr, ws.act,
+    QTALE_TRY(wq_gemm_launch(ws.hn, d, ws.n_exec, T, &w->gate_up, act, QTALE_EPI_SWIGLU, nullptr, ws.act,
                              F, s));
   } else {
-    QTALE_TRY(wq_gemm_launch(ws.hn, d, ws.n_exec, T, &w->gate_up, QTALE_EPI_STORE_BF16, nullptr,
+    QTALE_TRY(wq_gemm_launch(ws.hn, d, ws.n_exec, T, &w->gate_up, act, QTALE_EPI_STORE_16, nullptr,
                              ws.gu, 2 * F, s));
-    QTALE_TRY(launch_swiglu(ws.gu, ws.n_exec, T, F, ws.act, s));
+    QTALE_TRY(launch_swiglu(ws.gu, ws.n_exec, T, F, ws.act, act, s));
   }
   // 9. down projection + residual scatter: x[idx] = bf16(u + MLP branch)   (Eq. 3)
   e.resid = ws.u;
   e.ld_resid = d;
   e.dst = x;
   e.ld_dst = d;
-  QTALE_TRY(wq_gemm_launch(ws.act, F, ws.n_exec, T, &w->down, QTALE_EPI_RESID_SCATTER, &e, nullptr,
+  QTALE_TRY(wq_gemm_launch(ws.act, F, ws.n_exec, T, &w->down, act, QTALE_EPI_RESID_SCATTER, &e, nullptr,
                            0, s));
   return QTALE_OK;
 }
@@ -255,7 +257,7 @@ int qtale_model_prefill(const qtale_model_config* cfg, const qtale_model_weights
   }
   if (logits_out) {
     QTALE_TRY(launch_compact(hidden_out, logit_rows, nullptr, n_logit_rows, d, w->final_gamma,
-                             cfg->layer.rms_eps, nullptr, hrows, s));
+                             cfg->layer.rms_eps, QTALE_ACT_BF16, nullptr, hrows, s));
     QTALE_TRY(bf16_gemm_launch(hrows, d, nullptr, n_logit_rows, w->lm_head, cfg->vocab, d, d,
                                logits_out, cfg->vocab, s));
   }

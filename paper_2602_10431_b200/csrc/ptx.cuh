@@ -162,11 +162,12 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t smem_addr) {
   return d;
 }
 
-// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M x N tile.
-__host__ __device__ constexpr uint32_t idesc_bf16_f32(int M, int N) {
+// Instruction descriptor: bf16 x bf16 (or fp16 x fp16) -> fp32, both operands
+// K-major, M x N tile.  A and B always share one 16-bit format.
+__host__ __device__ constexpr uint32_t idesc_16bit_f32(int M, int N, bool f16) {
   return (1u << 4)                      // D format fp32
-         | (1u << 7)                    // A format bf16
-         | (1u << 10)                   // B format bf16
+         | ((f16 ? 0u : 1u) << 7)       // A format: 0 fp16, 1 bf16
+         | ((f16 ? 0u : 1u) << 10)      // B format: same as A
          | ((uint32_t)(N >> 3) << 17)   // N / 8
          | ((uint32_t)(M >> 4) << 24);  // M / 16
 }

@@ -9,9 +9,9 @@
 
 namespace qtale {
 
-constexpr int kRouterThreads = 256;  // 8 warps
-constexpr int kRowsPerWarp = 4;
-constexpr int kSelectThreads = 1024;
+constexpr int kRouterThreads = 512;  // 16 warps
+constexpr int kRowsPerWarp = 2;
+constexpr int kSelectThreads = 1024;  // upper bound of the CTA size the selection code supports
 
 struct RouterParams {
   const __nv_bfloat16* x;
@@ -62,7 +62,12 @@ __device__ void select_and_compact(const RouterParams& p, uint32_t* sh_hist, int
       for (int t = tid; t < T; t += nthr) {
         if (p.valid && !p.valid[t]) continue;
         uint32_t key = score_key(__ldcg(p.scores + t));
-        if ((key & mask) == prefix) atomicAdd(&sh_hist[(key >> shift) & 0xFF], 1u);
+        if ((key & mask) == prefix) {
+          // scores cluster in a few buckets: one atomic per distinct bucket per warp
+          const uint32_t bucket = (key >> shift) & 0xFF;
+          const uint32_t peers = __match_any_sync(__activemask(), bucket);
+          if ((int)(__ffs(peers) - 1) == (threadIdx.x & 31)) atomicAdd(&sh_hist[bucket], __popc(peers));
+        }
       }
       __syncthreads();
       if (tid == 0) {
@@ -183,7 +188,7 @@ __device__ void select_and_compact(const RouterParams& p, uint32_t* sh_hist, int
 }
 
 // ---- the fused kernel -------------------------------------------------------
-__global__ void __launch_bounds__(kSelectThreads)
+__global__ void __launch_bounds__(kRouterThreads)
     router_select_kernel(const RouterParams p) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   __shared__ uint32_t sh_hist[256];
@@ -337,7 +342,7 @@ int qtale_router_select(const void* x, int T, int d, const float* w_router, floa
   } else {
     const int n_it = (d + 255) / 256;
     smem = (size_t)n_it * 256 * sizeof(double);
-    const int warps = kSelectThreads / 32;
+    const int warps = kRouterThreads / 32;
     const int n_groups = (T + kRowsPerWarp - 1) / kRowsPerWarp;
     grid = (n_groups + warps - 1) / warps;
     const int cap = sm_count() * 2;
@@ -349,7 +354,7 @@ int qtale_router_select(const void* x, int T, int d, const float* w_router, floa
         return QTALE_ERR_CUDA;
     }
   }
-  router_select_kernel<<<grid, kSelectThreads, smem, s>>>(p);
+  router_select_kernel<<<grid, kRouterThreads, smem, s>>>(p);
   return launch_status(cudaGetLastError());
 }
 

@@ -11,7 +11,7 @@ constexpr int kRowThreads = 256;
 
 // ---- gather (+ RMSNorm) ------------------------------------------------------
 // One warp per executed row; the row (d <= 32*8*MAXC bf16) stays in registers.
-template <int MAXC>
+template <int MAXC, int ACT>
 __global__ void __launch_bounds__(kRowThreads)
     compact_kernel(const uint4* __restrict__ x, const int32_t* __restrict__ idx,
                    const int32_t* __restrict__ n_exec, int cap, int d,
@@ -60,10 +60,10 @@ __global__ void __launch_bounds__(kRowThreads)
           const float4 g0 = *reinterpret_cast<const float4*>(gamma + cc * 8);
           const float4 g1 = *reinterpret_cast<const float4*>(gamma + cc * 8 + 4);
           uint4 o;
-          o.x = pack_bf16x2(bf16_lo(v[c].x) * inv * g0.x, bf16_hi(v[c].x) * inv * g0.y);
-          o.y = pack_bf16x2(bf16_lo(v[c].y) * inv * g0.z, bf16_hi(v[c].y) * inv * g0.w);
-          o.z = pack_bf16x2(bf16_lo(v[c].z) * inv * g1.x, bf16_hi(v[c].z) * inv * g1.y);
-          o.w = pack_bf16x2(bf16_lo(v[c].w) * inv * g1.z, bf16_hi(v[c].w) * inv * g1.w);
+          o.x = Act16<ACT>::pack(bf16_lo(v[c].x) * inv * g0.x, bf16_hi(v[c].x) * inv * g0.y);
+          o.y = Act16<ACT>::pack(bf16_lo(v[c].y) * inv * g0.z, bf16_hi(v[c].y) * inv * g0.w);
+          o.z = Act16<ACT>::pack(bf16_lo(v[c].z) * inv * g1.x, bf16_hi(v[c].z) * inv * g1.y);
+          o.w = Act16<ACT>::pack(bf16_lo(v[c].w) * inv * g1.z, bf16_hi(v[c].w) * inv * g1.w);
           st_16(hn + (size_t)i * chunks + cc, o);
         }
       }
@@ -97,7 +97,7 @@ __global__ void __launch_bounds__(kRowThreads)
 }
 
 // ---- RMSNorm of an fp32 tensor into bf16: one CTA per row ---------------------
-template <int MAXC>
+template <int MAXC, int ACT>
 __global__ void __launch_bounds__(kRowThreads)
     rmsnorm_f32_kernel(const float4* __restrict__ u, const int32_t* __restrict__ n_rows, int cap,
                        int d, const float* __restrict__ gamma, float eps, uint2* __restrict__ out) {
@@ -135,8 +135,8 @@ __global__ void __launch_bounds__(kRowThreads)
       if (cc < chunks) {
         const float4 g = *reinterpret_cast<const float4*>(gamma + cc * 4);
         uint2 o;
-        o.x = pack_bf16x2(v[c].x * inv * g.x, v[c].y * inv * g.y);
-        o.y = pack_bf16x2(v[c].z * inv * g.z, v[c].w * inv * g.w);
+        o.x = Act16<ACT>::pack(v[c].x * inv * g.x, v[c].y * inv * g.y);
+        o.y = Act16<ACT>::pack(v[c].z * inv * g.z, v[c].w * inv * g.w);
         out[(size_t)i * chunks + cc] = o;
       }
     }
@@ -163,6 +163,7 @@ __global__ void rope_table_kernel(const int32_t* __restrict__ pos,
 // ---- rotary embedding on the q and k heads of the fused qkv tensor -------------
 // qkv: [n, ld] bf16; heads 0 .. n_rot-1 (q heads then k heads) are rotated in place,
 // pairing element j with j + hd/2.
+template <int ACT>
 __global__ void __launch_bounds__(kRowThreads)
     rope_kernel(uint4* __restrict__ qkv, const int32_t* __restrict__ n_exec, int cap, int ld,
                 int n_rot, int hd, const float2* __restrict__ cs) {
@@ -188,10 +189,10 @@ __global__ void __launch_bounds__(kRowThreads)
     uint32_t ao[4], bo[4];
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
-      const float a0 = bf16_lo(au[q]), a1 = bf16_hi(au[q]);
-      const float b0 = bf16_lo(bu[q]), b1 = bf16_hi(bu[q]);
-      ao[q] = pack_bf16x2(a0 * cv[2 * q] - b0 * sv[2 * q], a1 * cv[2 * q + 1] - b1 * sv[2 * q + 1]);
-      bo[q] = pack_bf16x2(b0 * cv[2 * q] + a0 * sv[2 * q], b1 * cv[2 * q + 1] + a1 * sv[2 * q + 1]);
+      const float a0 = Act16<ACT>::lo(au[q]), a1 = Act16<ACT>::hi(au[q]);
+      const float b0 = Act16<ACT>::lo(bu[q]), b1 = Act16<ACT>::hi(bu[q]);
+      ao[q] = Act16<ACT>::pack(a0 * cv[2 * q] - b0 * sv[2 * q], a1 * cv[2 * q + 1] - b1 * sv[2 * q + 1]);
+      bo[q] = Act16<ACT>::pack(b0 * cv[2 * q] + a0 * sv[2 * q], b1 * cv[2 * q + 1] + a1 * sv[2 * q + 1]);
     }
     *p0 = make_uint4(ao[0], ao[1], ao[2], ao[3]);
     *p1 = make_uint4(bo[0], bo[1], bo[2], bo[3]);
@@ -199,6 +200,7 @@ __global__ void __launch_bounds__(kRowThreads)
 }
 
 // ---- SwiGLU: act[i, j] = silu(gu[i, j]) * gu[i, F + j] --------------------------
+template <int ACT>
 __global__ void __launch_bounds__(kRowThreads)
     swiglu_kernel(const uint4* __restrict__ gu, const int32_t* __restrict__ n_exec, int cap, int F,
                   uint4* __restrict__ act) {
@@ -214,9 +216,9 @@ __global__ void __launch_bounds__(kRowThreads)
     uint32_t o[4];
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
-      const float g0 = bf16_lo(gg[q]), g1 = bf16_hi(gg[q]);
-      o[q] = pack_bf16x2(g0 / (1.f + __expf(-g0)) * bf16_lo(uu[q]),
-                         g1 / (1.f + __expf(-g1)) * bf16_hi(uu[q]));
+      const float g0 = Act16<ACT>::lo(gg[q]), g1 = Act16<ACT>::hi(gg[q]);
+      o[q] = Act16<ACT>::pack(g0 / (1.f + __expf(-g0)) * Act16<ACT>::lo(uu[q]),
+                              g1 / (1.f + __expf(-g1)) * Act16<ACT>::hi(uu[q]));
     }
     st_16(act + e, make_uint4(o[0], o[1], o[2], o[3]));
   }
@@ -272,22 +274,30 @@ __global__ void __launch_bounds__(kRowThreads)
 
 static int row_grid(int per_sm) { return sm_count() * per_sm; }
 
-int launch_compact(const void* x, const int32_t* idx, const int32_t* n_exec, int cap, int d,
-                   const float* gamma, float eps, void* xc, void* hn, cudaStream_t s) {
+template <int ACT>
+static int launch_compact_t(const void* x, const int32_t* idx, const int32_t* n_exec, int cap,
+                            int d, const float* gamma, float eps, void* xc, void* hn,
+                            cudaStream_t s) {
   const int chunks = d / 8;
   const int grid = row_grid(8);
   auto X = static_cast<const uint4*>(x);
   auto XC = static_cast<uint4*>(xc);
   auto HN = static_cast<uint4*>(hn);
   if (chunks <= 32 * 4)
-    compact_kernel<4><<<grid, kRowThreads, 0, s>>>(X, idx, n_exec, cap, d, gamma, eps, XC, HN);
+    compact_kernel<4, ACT><<<grid, kRowThreads, 0, s>>>(X, idx, n_exec, cap, d, gamma, eps, XC, HN);
   else if (chunks <= 32 * 16)
-    compact_kernel<16><<<grid, kRowThreads, 0, s>>>(X, idx, n_exec, cap, d, gamma, eps, XC, HN);
+    compact_kernel<16, ACT><<<grid, kRowThreads, 0, s>>>(X, idx, n_exec, cap, d, gamma, eps, XC, HN);
   else if (chunks <= 32 * 32)
-    compact_kernel<32><<<grid, kRowThreads, 0, s>>>(X, idx, n_exec, cap, d, gamma, eps, XC, HN);
+    compact_kernel<32, ACT><<<grid, kRowThreads, 0, s>>>(X, idx, n_exec, cap, d, gamma, eps, XC, HN);
   else
     return QTALE_ERR_SHAPE;
   return launch_status(cudaGetLastError());
+}
+
+int launch_compact(const void* x, const int32_t* idx, const int32_t* n_exec, int cap, int d,
+                   const float* gamma, float eps, int act, void* xc, void* hn, cudaStream_t s) {
+  return act == QTALE_ACT_F16 ? launch_compact_t<1>(x, idx, n_exec, cap, d, gamma, eps, xc, hn, s)
+                              : launch_compact_t<0>(x, idx, n_exec, cap, d, gamma, eps, xc, hn, s);
 }
 
 int launch_scatter_add(void* x, const void* xc, const float* f, const int32_t* idx,
@@ -298,21 +308,28 @@ int launch_scatter_add(void* x, const void* xc, const float* f, const int32_t* i
   return launch_status(cudaGetLastError());
 }
 
-int launch_rmsnorm_f32(const float* u, const int32_t* n_rows, int cap, int d, const float* gamma,
-                       float eps, void* out, cudaStream_t s) {
+template <int ACT>
+static int launch_rmsnorm_f32_t(const float* u, const int32_t* n_rows, int cap, int d,
+                                const float* gamma, float eps, void* out, cudaStream_t s) {
   const int chunks = d / 4;
   const int grid = min(cap, row_grid(8));
   auto U = reinterpret_cast<const float4*>(u);
   auto O = static_cast<uint2*>(out);
   if (chunks <= kRowThreads * 1)
-    rmsnorm_f32_kernel<1><<<grid, kRowThreads, 0, s>>>(U, n_rows, cap, d, gamma, eps, O);
+    rmsnorm_f32_kernel<1, ACT><<<grid, kRowThreads, 0, s>>>(U, n_rows, cap, d, gamma, eps, O);
   else if (chunks <= kRowThreads * 4)
-    rmsnorm_f32_kernel<4><<<grid, kRowThreads, 0, s>>>(U, n_rows, cap, d, gamma, eps, O);
+    rmsnorm_f32_kernel<4, ACT><<<grid, kRowThreads, 0, s>>>(U, n_rows, cap, d, gamma, eps, O);
   else if (chunks <= kRowThreads * 8)
-    rmsnorm_f32_kernel<8><<<grid, kRowThreads, 0, s>>>(U, n_rows, cap, d, gamma, eps, O);
+    rmsnorm_f32_kernel<8, ACT><<<grid, kRowThreads, 0, s>>>(U, n_rows, cap, d, gamma, eps, O);
   else
     return QTALE_ERR_SHAPE;
   return launch_status(cudaGetLastError());
+}
+
+int launch_rmsnorm_f32(const float* u, const int32_t* n_rows, int cap, int d, const float* gamma,
+                       float eps, int act, void* out, cudaStream_t s) {
+  return act == QTALE_ACT_F16 ? launch_rmsnorm_f32_t<1>(u, n_rows, cap, d, gamma, eps, out, s)
+                              : launch_rmsnorm_f32_t<0>(u, n_rows, cap, d, gamma, eps, out, s);
 }
 
 int launch_rope_table(const int32_t* pos, const int32_t* n_exec, int cap, int hd, float base,
@@ -323,16 +340,24 @@ int launch_rope_table(const int32_t* pos, const int32_t* n_exec, int cap, int hd
 }
 
 int launch_rope(void* qkv, const int32_t* n_exec, int cap, int ld, int n_rot, int hd,
-                const float* cs, cudaStream_t s) {
-  rope_kernel<<<row_grid(8), kRowThreads, 0, s>>>(static_cast<uint4*>(qkv), n_exec, cap, ld, n_rot,
-                                                  hd, reinterpret_cast<const float2*>(cs));
+                const float* cs, int act, cudaStream_t s) {
+  if (act == QTALE_ACT_F16)
+    rope_kernel<1><<<row_grid(8), kRowThreads, 0, s>>>(static_cast<uint4*>(qkv), n_exec, cap, ld,
+                                                       n_rot, hd, reinterpret_cast<const float2*>(cs));
+  else
+    rope_kernel<0><<<row_grid(8), kRowThreads, 0, s>>>(static_cast<uint4*>(qkv), n_exec, cap, ld,
+                                                       n_rot, hd, reinterpret_cast<const float2*>(cs));
   return launch_status(cudaGetLastError());
 }
 
-int launch_swiglu(const void* gu, const int32_t* n_exec, int cap, int F, void* act,
+int launch_swiglu(const void* gu, const int32_t* n_exec, int cap, int F, void* act, int act_dtype,
                   cudaStream_t s) {
-  swiglu_kernel<<<row_grid(8), kRowThreads, 0, s>>>(static_cast<const uint4*>(gu), n_exec, cap, F,
-                                                    static_cast<uint4*>(act));
+  if (act_dtype == QTALE_ACT_F16)
+    swiglu_kernel<1><<<row_grid(8), kRowThreads, 0, s>>>(static_cast<const uint4*>(gu), n_exec, cap,
+                                                         F, static_cast<uint4*>(act));
+  else
+    swiglu_kernel<0><<<row_grid(8), kRowThreads, 0, s>>>(static_cast<const uint4*>(gu), n_exec, cap,
+                                                         F, static_cast<uint4*>(act));
   return launch_status(cudaGetLastError());
 }
 
@@ -361,14 +386,16 @@ using namespace qtale;
 extern "C" {
 
 int qtale_compact(const void* x, const int32_t* idx, const int32_t* n_exec, int T, int d,
-                  const float* rms_gamma, float eps, void* xc_out, void* hn_out, void* stream) {
+                  const float* rms_gamma, float eps, int act_dtype, void* xc_out, void* hn_out,
+                  void* stream) {
+  if (act_dtype != QTALE_ACT_BF16 && act_dtype != QTALE_ACT_F16) return QTALE_ERR_MODE;
   if (!x || !idx || !n_exec) return QTALE_ERR_NULL;
   if (!xc_out && !hn_out) return QTALE_ERR_NULL;
   if (hn_out && !rms_gamma) return QTALE_ERR_NULL;
   if (T < 1 || d < 8 || d % 8 != 0) return QTALE_ERR_SHAPE;
   if (!aligned16(x) || !aligned16(xc_out) || !aligned16(hn_out) || !aligned16(rms_gamma))
     return QTALE_ERR_ALIGN;
-  return launch_compact(x, idx, n_exec, T, d, rms_gamma, eps, xc_out, hn_out,
+  return launch_compact(x, idx, n_exec, T, d, rms_gamma, eps, act_dtype, xc_out, hn_out,
                         static_cast<cudaStream_t>(stream));
 }
 

@@ -107,7 +107,7 @@ __device__ __forceinline__ int tile_row_to_n(const GemmParams& p, int nt, int L)
 // Slot i holds the code in its low QBITS bits.  The code is moved into a float
 // mantissa next to 2^23, so (float - (2^23 + zero * 16^i)) * (scale / 16^i) is
 // exactly (code - zero) * scale.
-template <uint32_t QMASK>
+template <uint32_t QMASK, int ACT>
 __device__ __forceinline__ void dequant8(uint32_t t, const float (&C)[5], const float (&S)[5],
                                          uint32_t* out) {
   constexpr uint32_t MAGIC = 0x4B000000u;  // 2^23
@@ -120,10 +120,10 @@ __device__ __forceinline__ void dequant8(uint32_t t, const float (&C)[5], const 
   for (int i = 5; i < 8; ++i)
     v[i] = (__uint_as_float((hi & (QMASK << (4 * (i - 3)))) | MAGIC) - C[i - 3]) * S[i - 3];
 #pragma unroll
-  for (int q = 0; q < 4; ++q) out[q] = pack_bf16x2(v[2 * q], v[2 * q + 1]);
+  for (int q = 0; q < 4; ++q) out[q] = Act16<ACT>::pack(v[2 * q], v[2 * q + 1]);
 }
 
-template <int TN, int BITS>
+template <int TN, int BITS, int ACT>
 __global__ void __launch_bounds__(kGemmThreads, 1)
     wq_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x,
                    const __grid_constant__ CUtensorMap tmap_w, const GemmParams p) {
@@ -202,7 +202,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
   } else if (warp == 1) {
     // ------------------------------- MMA issuer --------------------------------
     if (lane == 0) {
-      constexpr uint32_t idesc = idesc_bf16_f32(kTileRows, TN);
+      constexpr uint32_t idesc = idesc_16bit_f32(kTileRows, TN, ACT == 1);
       int s = 0;
       uint32_t ph = 0, dph = 0;
       for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
@@ -266,10 +266,10 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
             for (int part = 0; part < 2; ++part) {
               const uint4 w = reinterpret_cast<const uint4*>(st)[part * kTileRows + L];
               uint32_t r[16];
-              dequant8<0xFu>(w.x, C, Sc, r + 0);
-              dequant8<0xFu>(w.y, C, Sc, r + 4);
-              dequant8<0xFu>(w.z, C, Sc, r + 8);
-              dequant8<0xFu>(w.w, C, Sc, r + 12);
+              dequant8<0xFu, ACT>(w.x, C, Sc, r + 0);
+              dequant8<0xFu, ACT>(w.y, C, Sc, r + 4);
+              dequant8<0xFu, ACT>(w.z, C, Sc, r + 8);
+              dequant8<0xFu, ACT>(w.w, C, Sc, r + 12);
               tmem_st_x16(a_taddr + part * 16, r);
             }
           } else {
@@ -292,7 +292,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
                                   : rr == 1 ? (bw[u >> 2] << 1)
                                   : rr == 2 ? bw[u >> 2] : (bw[u >> 2] >> 1);
                 const uint32_t t = (a2 & 0x33333333u) | (b1 & 0xCCCCCCCCu);
-                dequant8<0x7u>(t, C, Sc, r + 4 * uu);
+                dequant8<0x7u, ACT>(t, C, Sc, r + 4 * uu);
               }
               tmem_st_x16(a_taddr + part * 16, r);
             }
@@ -319,11 +319,47 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
       const int m_base = mt * TN;
 #pragma unroll 1
       for (int c0 = 0; c0 < TN; c0 += 32) {
-        if (m_base + c0 >= M) break;
+        const int m0 = m_base + c0;
+        if (m0 >= M) break;
+        const int n_cols = min(32, M - m0);  // warp-uniform
         uint32_t r[32];
         tmem_ld_x32(tmem_base + ((uint32_t)(quad * 32) << 16) + c0, r);
-        tmem_wait_ld();
-        if (p.epilogue == QTALE_EPI_SWIGLU) {
+        if (p.epilogue == QTALE_EPI_RESID_F32 || p.epilogue == QTALE_EPI_RESID_SCATTER) {
+          // all residual reads of the chunk are issued before the first store so that
+          // their latencies overlap (one row index per column, fetched by one lane)
+          const int my_row = (lane < n_cols) ? __ldg(p.idx + m0 + lane) : 0;
+          float res[32];
+          if (p.epilogue == QTALE_EPI_RESID_F32) {
+            const unsigned short* rp = static_cast<const unsigned short*>(p.resid);
+#pragma unroll
+            for (int c = 0; c < 32; ++c) {
+              const int row = __shfl_sync(0xffffffffu, my_row, c);
+              res[c] = (c < n_cols && n >= 0)
+                           ? bf16_bits_to_float(__ldg(rp + (size_t)row * p.ld_resid + n)) : 0.f;
+            }
+            tmem_wait_ld();
+            if (n >= 0) {
+              float* y = static_cast<float*>(p.y);
+#pragma unroll
+              for (int c = 0; c < 32; ++c)
+                if (c < n_cols) y[(size_t)(m0 + c) * p.ldy + n] = res[c] + __uint_as_float(r[c]);
+            }
+          } else {
+            const float* rp = static_cast<const float*>(p.resid);
+#pragma unroll
+            for (int c = 0; c < 32; ++c)
+              res[c] = (c < n_cols && n >= 0) ? __ldg(rp + (size_t)(m0 + c) * p.ld_resid + n) : 0.f;
+            tmem_wait_ld();
+            __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(p.dst);
+#pragma unroll
+            for (int c = 0; c < 32; ++c) {
+              const int row = __shfl_sync(0xffffffffu, my_row, c);
+              if (c < n_cols && n >= 0)
+                dst[(size_t)row * p.ld_dst + n] = __float2bfloat16_rn(res[c] + __uint_as_float(r[c]));
+            }
+          }
+        } else if (p.epilogue == QTALE_EPI_SWIGLU) {
+          tmem_wait_ld();
           // lanes 0-15 hold gate rows, lanes 16-31 the matching up rows
           float other[16];
 #pragma unroll
@@ -332,34 +368,29 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
                                        __uint_as_float((lane < 16) ? r[16 + i] : r[i]), 16);
           const int j = nt * 64 + quad * 16 + (lane & 15);
           if (j < p.F) {
-            __nv_bfloat16* y = static_cast<__nv_bfloat16*>(p.y);
+            unsigned short* y = static_cast<unsigned short*>(p.y);
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
               const int c = (lane < 16) ? i : 16 + i;
-              const int m = m_base + c0 + c;
               const float g = (lane < 16) ? __uint_as_float(r[c]) : other[i];
               const float u = (lane < 16) ? other[i] : __uint_as_float(r[c]);
-              if (m < M) y[(size_t)m * p.ldy + j] = __float2bfloat16_rn(g / (1.f + __expf(-g)) * u);
+              if (c < n_cols)
+                y[(size_t)(m0 + c) * p.ldy + j] = Act16<ACT>::one(g / (1.f + __expf(-g)) * u);
             }
           }
-        } else if (n >= 0) {
+        } else {
+          tmem_wait_ld();
+          if (n >= 0) {
+            if (p.epilogue == QTALE_EPI_STORE_16) {
+              unsigned short* y = static_cast<unsigned short*>(p.y);
 #pragma unroll
-          for (int c = 0; c < 32; ++c) {
-            const int m = m_base + c0 + c;
-            if (m >= M) break;
-            const float acc = __uint_as_float(r[c]);
-            if (p.epilogue == QTALE_EPI_STORE_BF16) {
-              static_cast<__nv_bfloat16*>(p.y)[(size_t)m * p.ldy + n] = __float2bfloat16_rn(acc);
-            } else if (p.epilogue == QTALE_EPI_STORE_F32) {
-              static_cast<float*>(p.y)[(size_t)m * p.ldy + n] = acc;
-            } else if (p.epilogue == QTALE_EPI_RESID_F32) {
-              const __nv_bfloat16* res = static_cast<const __nv_bfloat16*>(p.resid);
-              static_cast<float*>(p.y)[(size_t)m * p.ldy + n] =
-                  __bfloat162float(res[(size_t)p.idx[m] * p.ld_resid + n]) + acc;
-            } else {  // QTALE_EPI_RESID_SCATTER
-              const float* res = static_cast<const float*>(p.resid);
-              static_cast<__nv_bfloat16*>(p.dst)[(size_t)p.idx[m] * p.ld_dst + n] =
-                  __float2bfloat16_rn(res[(size_t)m * p.ld_resid + n] + acc);
+              for (int c = 0; c < 32; ++c)
+                if (c < n_cols) y[(size_t)(m0 + c) * p.ldy + n] = Act16<ACT>::one(__uint_as_float(r[c]));
+            } else {  // QTALE_EPI_STORE_F32
+              float* y = static_cast<float*>(p.y);
+#pragma unroll
+              for (int c = 0; c < 32; ++c)
+                if (c < n_cols) y[(size_t)(m0 + c) * p.ldy + n] = __uint_as_float(r[c]);
             }
           }
         }
@@ -402,23 +433,23 @@ static EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// Tensor map over a row-major bf16 matrix [rows, cols] with pitch `ld` elements;
+// Tensor map over a row-major 16-bit (bf16 or fp16) matrix [rows, cols] with pitch `ld` elements;
 // box = 64 columns x box_rows rows, 128-byte swizzle, zero fill out of bounds.
-static int make_tmap_bf16(CUtensorMap* m, const void* base, int rows, int cols, int ld,
-                          int box_rows) {
+static int make_tmap_16(CUtensorMap* m, const void* base, int rows, int cols, int ld,
+                        int box_rows, int act) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return QTALE_ERR_CUDA;
   cuuint64_t gdim[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
   cuuint64_t gstr[1] = {(cuuint64_t)ld * 2};
   cuuint32_t box[2] = {(cuuint32_t)kKB, (cuuint32_t)box_rows};
   cuuint32_t estr[2] = {1, 1};
-  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstr, box,
+  CUresult r = fn(m, act == QTALE_ACT_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstr, box,
                   estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? QTALE_OK : QTALE_ERR_CUDA;
 }
 
-template <int TN, int BITS>
+template <int TN, int BITS, int ACT>
 static int launch_gemm(const CUtensorMap& tx, const CUtensorMap& tw, const GemmParams& p,
                        cudaStream_t s) {
   using Cfg = GemmCfg<TN, BITS>;
@@ -426,7 +457,7 @@ static int launch_gemm(const CUtensorMap& tx, const CUtensorMap& tw, const GemmP
   int dev = 0;
   cudaGetDevice(&dev);
   if (dev >= 0 && dev < 64 && !configured[dev]) {
-    if (cudaFuncSetAttribute(wq_gemm_kernel<TN, BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    if (cudaFuncSetAttribute(wq_gemm_kernel<TN, BITS, ACT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)Cfg::kSmemBytes) != cudaSuccess)
       return QTALE_ERR_CUDA;
     configured[dev] = true;
@@ -435,16 +466,16 @@ static int launch_gemm(const CUtensorMap& tx, const CUtensorMap& tw, const GemmP
   int grid = sm_count();
   if (grid > max_tiles) grid = max_tiles;
   if (grid < 1) grid = 1;
-  wq_gemm_kernel<TN, BITS><<<grid, kGemmThreads, Cfg::kSmemBytes, s>>>(tx, tw, p);
+  wq_gemm_kernel<TN, BITS, ACT><<<grid, kGemmThreads, Cfg::kSmemBytes, s>>>(tx, tw, p);
   return launch_status(cudaGetLastError());
 }
 
-template <int BITS>
+template <int BITS, int ACT>
 static int dispatch_tn(const CUtensorMap& tx, const CUtensorMap& tw, const GemmParams& p, int tn,
                        cudaStream_t s) {
-  if (tn == 64) return launch_gemm<64, BITS>(tx, tw, p, s);
-  if (tn == 128) return launch_gemm<128, BITS>(tx, tw, p, s);
-  return launch_gemm<256, BITS>(tx, tw, p, s);
+  if (tn == 64) return launch_gemm<64, BITS, ACT>(tx, tw, p, s);
+  if (tn == 128) return launch_gemm<128, BITS, ACT>(tx, tw, p, s);
+  return launch_gemm<256, BITS, ACT>(tx, tw, p, s);
 }
 
 static int pick_tn(int M_cap) { return M_cap <= 64 ? 64 : (M_cap <= 128 ? 128 : 256); }
@@ -463,8 +494,8 @@ size_t wq_blob_bytes(int N, int K, int bits, int group, int row_mode, WqGeometry
 }
 
 int wq_gemm_launch(const void* a, int lda, const int32_t* m_dev, int M_cap,
-                   const qtale_wq_weight* w, int epilogue, const qtale_epilogue_args* epi, void* y,
-                   int ldy, cudaStream_t s) {
+                   const qtale_wq_weight* w, int act, int epilogue, const qtale_epilogue_args* epi,
+                   void* y, int ldy, cudaStream_t s) {
   WqGeometry g;
   wq_blob_bytes(w->N, w->K, w->bits, w->group, w->row_mode, &g);
   GemmParams p;
@@ -493,10 +524,11 @@ int wq_gemm_launch(const void* a, int lda, const int32_t* m_dev, int M_cap,
   const int tn = pick_tn(M_cap);
   CUtensorMap tx, tw;
   memset(&tw, 0, sizeof(tw));
-  int rc = make_tmap_bf16(&tx, a, M_cap, w->K, lda, tn);
+  int rc = make_tmap_16(&tx, a, M_cap, w->K, lda, tn, act);
   if (rc != QTALE_OK) return rc;
-  if (w->bits == 4) return dispatch_tn<4>(tx, tw, p, tn, s);
-  return dispatch_tn<3>(tx, tw, p, tn, s);
+  if (act == QTALE_ACT_F16)
+    return w->bits == 4 ? dispatch_tn<4, 1>(tx, tw, p, tn, s) : dispatch_tn<3, 1>(tx, tw, p, tn, s);
+  return w->bits == 4 ? dispatch_tn<4, 0>(tx, tw, p, tn, s) : dispatch_tn<3, 0>(tx, tw, p, tn, s);
 }
 
 int bf16_gemm_launch(const void* a, int lda, const int32_t* m_dev, int M_cap, const void* w_bf16,
@@ -516,11 +548,11 @@ int bf16_gemm_launch(const void* a, int lda, const int32_t* m_dev, int M_cap, co
   p.status = device_status_ptr();
   const int tn = pick_tn(M_cap);
   CUtensorMap tx, tw;
-  int rc = make_tmap_bf16(&tx, a, M_cap, K, lda, tn);
+  int rc = make_tmap_16(&tx, a, M_cap, K, lda, tn, QTALE_ACT_BF16);
   if (rc != QTALE_OK) return rc;
-  rc = make_tmap_bf16(&tw, w_bf16, N, K, ldw, kTileRows);
+  rc = make_tmap_16(&tw, w_bf16, N, K, ldw, kTileRows, QTALE_ACT_BF16);
   if (rc != QTALE_OK) return rc;
-  return dispatch_tn<16>(tx, tw, p, tn, s);
+  return dispatch_tn<16, 0>(tx, tw, p, tn, s);
 }
 
 // ---- offline repack (host) -------------------------------------------------------
@@ -634,12 +666,14 @@ int qtale_wq_repack(const uint8_t* codes, const uint16_t* scales, const uint16_t
 }
 
 int qtale_wq_gemm(const void* a, int lda, const int32_t* m_dev, int M_cap, const qtale_wq_weight* w,
-                  int epilogue, const qtale_epilogue_args* epi, void* y, int ldy, void* stream) {
+                  int act_dtype, int epilogue, const qtale_epilogue_args* epi, void* y, int ldy,
+                  void* stream) {
   if (!a || !w || !w->packed) return QTALE_ERR_NULL;
+  if (act_dtype != QTALE_ACT_BF16 && act_dtype != QTALE_ACT_F16) return QTALE_ERR_MODE;
   if (w->bits != 3 && w->bits != 4) return QTALE_ERR_BITS;
   if (w->group != 64 && w->group != 128) return QTALE_ERR_GROUP;
   if (M_cap < 1 || w->N < 1 || w->K < 1 || lda < w->K) return QTALE_ERR_SHAPE;
-  if (epilogue < QTALE_EPI_STORE_BF16 || epilogue > QTALE_EPI_SWIGLU) return QTALE_ERR_MODE;
+  if (epilogue < QTALE_EPI_STORE_16 || epilogue > QTALE_EPI_SWIGLU) return QTALE_ERR_MODE;
   if (epilogue == QTALE_EPI_SWIGLU && w->row_mode != QTALE_WQ_ROWS_SWIGLU) return QTALE_ERR_MODE;
   if (epilogue == QTALE_EPI_RESID_F32 || epilogue == QTALE_EPI_RESID_SCATTER) {
     if (!epi || !epi->idx || !epi->resid) return QTALE_ERR_NULL;
@@ -647,7 +681,7 @@ int qtale_wq_gemm(const void* a, int lda, const int32_t* m_dev, int M_cap, const
   }
   if (epilogue != QTALE_EPI_RESID_SCATTER && !y) return QTALE_ERR_NULL;
   if (!aligned16(a) || !aligned16(w->packed) || (lda * 2) % 16 != 0) return QTALE_ERR_ALIGN;
-  return wq_gemm_launch(a, lda, m_dev, M_cap, w, epilogue, epi, y, ldy,
+  return wq_gemm_launch(a, lda, m_dev, M_cap, w, act_dtype, epilogue, epi, y, ldy,
                         static_cast<cudaStream_t>(stream));
 }
 

@@ -18,8 +18,8 @@ size_t wq_blob_bytes(int N, int K, int bits, int group, int row_mode, WqGeometry
 
 // y = epilogue(a W^T); arguments as qtale_wq_gemm (already validated).
 int wq_gemm_launch(const void* a, int lda, const int32_t* m_dev, int M_cap,
-                   const qtale_wq_weight* w, int epilogue, const qtale_epilogue_args* epi, void* y,
-                   int ldy, cudaStream_t s);
+                   const qtale_wq_weight* w, int act, int epilogue, const qtale_epilogue_args* epi,
+                   void* y, int ldy, cudaStream_t s);
 
 // y[m, n] = sum_k a[m, k] * w[n, k] with bf16 weights W[N, K] (pitch ldw), fp32 output.
 int bf16_gemm_launch(const void* a, int lda, const int32_t* m_dev, int M_cap, const void* w_bf16,

@@ -45,3 +45,18 @@ def assert_selection_matches(idx_gpu, n_gpu, scores_ref, mask_ref, threshold=Non
     if threshold is not None:
         diff &= np.abs(scores_ref.astype(np.float64) - threshold) > SCORE_BAND
     assert not diff.any(), "selection differs at tokens %s" % np.nonzero(diff)[0][:10]
+
+
+def round_act(a, act_dtype):
+    """float32 values rounded to the 16-bit activation format (0 = bf16, 1 = fp16)."""
+    a = np.asarray(a, np.float32)
+    if act_dtype == 1:
+        return a.astype(np.float16).astype(np.float32)
+    b = a.view(np.uint32)
+    r = (b + np.uint32(0x7FFF) + ((b >> np.uint32(16)) & np.uint32(1))) & np.uint32(0xFFFF0000)
+    return r.view(np.float32)
+
+
+def act_eps(act_dtype):
+    """Half an ulp, relative, of the 16-bit activation format."""
+    return 2.0 ** -12 if act_dtype == 1 else 2.0 ** -9

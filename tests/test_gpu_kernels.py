@@ -8,7 +8,7 @@ import pytest
 
 import oracle
 from paper_2602_10431_b200 import inputs
-from tests.gpu_util import assert_selection_matches, rel_fro
+from tests.gpu_util import act_eps, assert_selection_matches, rel_fro, round_act
 
 pytestmark = pytest.mark.gpu
 
@@ -97,8 +97,9 @@ def test_index_bookkeeping(env):
     assert int(r["n_exec"].item()) == 0 and not r["cu_exec"].cpu().numpy().any()
 
 
+@pytest.mark.parametrize("act", [0, 1])
 @pytest.mark.parametrize("T,d,ratio", [(256, 256, 0.5), (300, 4096, 0.7), (64, 5120, 1.0), (129, 512, 0.0)])
-def test_compact_and_scatter(env, T, d, ratio):
+def test_compact_and_scatter(env, T, d, ratio, act):
     api, torch, dev = env
     x = inputs.hidden_states(T + d, T, d)
     mask = (inputs.uniform(T, 3, T) < ratio).astype(np.uint8)
@@ -108,14 +109,14 @@ def test_compact_and_scatter(env, T, d, ratio):
     n_d = torch.tensor([n], dtype=torch.int32, device=dev)
     gam = (1 + 0.1 * inputs.normal(T, 7, d)).astype(np.float32)
     xd = api.to_device_bf16(x, dev)
-    xc, hn = api.compact(xd, idx_d, n_d, torch.from_numpy(gam).to(dev), 1e-5)
+    xc, hn = api.compact(xd, idx_d, n_d, torch.from_numpy(gam).to(dev), 1e-5, act_dtype=act)
     xc_h, hn_h = api.to_host_f32(xc), api.to_host_f32(hn)
     assert np.array_equal(xc_h[:n], oracle.gather_rows(x, idx))       # byte copy
     assert not xc_h[n:].any() and not hn_h[n:].any()                  # rows past the count untouched
     if n:
         ref = oracle.rmsnorm(x[idx], gam, 1e-5)
-        # fp32 arithmetic, one bf16 rounding: half an ulp of bf16 relative (2^-9) plus slack
-        assert np.all(np.abs(hn_h[:n] - ref) <= np.abs(ref) * 2.0 ** -8 + 1e-6)
+        # fp32 arithmetic, one rounding to the activation format: half an ulp relative, plus slack
+        assert np.all(np.abs(hn_h[:n] - ref) <= np.abs(ref) * 2 * act_eps(act) + 1e-6)
     f = inputs.gaussian_f32(T, 9, T, d, 0.5)
     x2 = api.scatter_add(xd.clone(), xc, torch.from_numpy(f).to(dev), idx_d, n_d)
     out = api.to_host_f32(x2)
@@ -138,8 +139,9 @@ GEMM_CASES = [
 ]
 
 
+@pytest.mark.parametrize("act", [0, 1])
 @pytest.mark.parametrize("M,N,K,bits,group,m_dev", GEMM_CASES)
-def test_wq_gemm_against_oracle(env, M, N, K, bits, group, m_dev):
+def test_wq_gemm_against_oracle(env, M, N, K, bits, group, m_dev, act):
     api, torch, dev = env
     a = inputs.activations(M + N, 11, M, K)
     wq = inputs.quantized_weight(K + bits, 12, N, K, bits, group)
@@ -147,22 +149,24 @@ def test_wq_gemm_against_oracle(env, M, N, K, bits, group, m_dev):
     mm = M if m_dev is None else m_dev
     qw = api.QuantWeight(wq, dev)
     md = None if m_dev is None else torch.tensor([m_dev], dtype=torch.int32, device=dev)
-    y = api.wq_gemm(api.to_device_bf16(a, dev), qw, md, api.EPI_STORE_F32).cpu().numpy()
+    ad = api.to_device_act(a, act, dev)                       # N(0,1) bf16 values are exact in fp16 too
+    y = api.wq_gemm(ad, qw, md, api.EPI_STORE_F32).cpu().numpy()
     assert api.device_status() == 0
     assert not y[mm:].any()                                   # rows past the count untouched
     if mm == 0:
         return
     ref = oracle.linear(a[:mm], w_hat)
-    # kernel rounds the dequantised weight once to bf16 (relative 2^-9 per weight)
-    assert rel_fro(y[:mm], ref) <= 3e-3
+    # kernel rounds the dequantised weight once to the 16-bit format (half an ulp relative per weight)
+    assert rel_fro(y[:mm], ref) <= 6 * act_eps(act)
     # with the same rounding applied to the oracle's weights only fp32 summation order differs
-    ref_b = oracle.linear(a[:mm], inputs.round_bf16(w_hat))
+    ref_b = oracle.linear(a[:mm], round_act(w_hat, act))
     assert np.abs(y[:mm] - ref_b).max() <= 1e-4 * max(1.0, np.abs(ref_b).max())
-    yb = api.to_host_f32(api.wq_gemm(api.to_device_bf16(a, dev), qw, md, api.EPI_STORE_BF16))
-    assert np.array_equal(yb[:mm], inputs.round_bf16(y[:mm]))
+    yb = api.to_host_f32(api.wq_gemm(ad, qw, md, api.EPI_STORE_16))
+    assert np.array_equal(yb[:mm], round_act(y[:mm], act))
 
 
-def test_wq_gemm_epilogues(env):
+@pytest.mark.parametrize("act", [0, 1])
+def test_wq_gemm_epilogues(env, act):
     api, torch, dev = env
     M, d, F, T = 200, 256, 688, 333
     bits, group = 4, 64
@@ -171,32 +175,33 @@ def test_wq_gemm_epilogues(env):
     md = torch.tensor([m_dev], dtype=torch.int32, device=dev)
     # SwiGLU epilogue: gate / up rows interleaved per tile by the repack
     wq = inputs.quantized_weight(2, 12, 2 * F, d, bits, group)
-    w_hat = inputs.round_bf16(oracle.dequantize_weight(wq))
+    w_hat = round_act(oracle.dequantize_weight(wq), act)
     gu = oracle.linear(a[:m_dev], w_hat)
     ref = oracle.swiglu(gu[:, :F], gu[:, F:])
     qw = api.QuantWeight(wq, dev, api.ROWS_SWIGLU)
-    act = api.to_host_f32(api.wq_gemm(api.to_device_bf16(a, dev), qw, md, api.EPI_SWIGLU))
-    assert act.shape == (M, F) and not act[m_dev:].any()
-    assert np.all(np.abs(act[:m_dev] - ref) <= np.abs(ref) * 2.0 ** -7 + 2e-5)
-    plain = api.wq_gemm(api.to_device_bf16(a, dev), qw, md, api.EPI_STORE_F32).cpu().numpy()
+    ad = api.to_device_act(a, act, dev)
+    sw = api.to_host_f32(api.wq_gemm(ad, qw, md, api.EPI_SWIGLU))
+    assert sw.shape == (M, F) and not sw[m_dev:].any()
+    assert np.all(np.abs(sw[:m_dev] - ref) <= np.abs(ref) * 4 * act_eps(act) + 2e-5)
+    plain = api.wq_gemm(ad, qw, md, api.EPI_STORE_F32).cpu().numpy()
     assert np.abs(plain[:m_dev] - gu).max() <= 1e-4       # same weights, plain epilogue, logical columns
     # residual epilogues: u = x[idx] + a W^T (fp32), then x[idx] = bf16(u + act W_d^T)
     x = inputs.hidden_states(3, T, d)
     idx = np.sort(np.argsort(inputs.uniform(3, 5, T))[:M]).astype(np.int32)
     wo = inputs.quantized_weight(4, 13, d, d, bits, group)
-    wo_hat = inputs.round_bf16(oracle.dequantize_weight(wo))
+    wo_hat = round_act(oracle.dequantize_weight(wo), act)
     idx_d = torch.from_numpy(idx).to(dev)
     xd = api.to_device_bf16(x, dev)
-    u = api.wq_gemm(api.to_device_bf16(a, dev), api.QuantWeight(wo, dev), md, api.EPI_RESID_F32,
+    u = api.wq_gemm(ad, api.QuantWeight(wo, dev), md, api.EPI_RESID_F32,
                     idx=idx_d, resid=xd).cpu().numpy()
     u_ref = x[idx[:m_dev]] + oracle.linear(a[:m_dev], wo_hat)
     assert np.abs(u[:m_dev] - u_ref).max() <= 1e-4 and not u[m_dev:].any()
     wd = inputs.quantized_weight(5, 14, d, F, bits, group)
-    wd_hat = inputs.round_bf16(oracle.dequantize_weight(wd))
+    wd_hat = round_act(oracle.dequantize_weight(wd), act)
     act_in = inputs.activations(6, 15, M, F)
     u_d = torch.from_numpy(u).to(dev)
     x2 = xd.clone()
-    api.wq_gemm(api.to_device_bf16(act_in, dev), api.QuantWeight(wd, dev), md, api.EPI_RESID_SCATTER,
+    api.wq_gemm(api.to_device_act(act_in, act, dev), api.QuantWeight(wd, dev), md, api.EPI_RESID_SCATTER,
                 idx=idx_d, resid=u_d, dst=x2)
     out = api.to_host_f32(x2)
     want = u[:m_dev].astype(np.float64) + oracle.linear(act_in[:m_dev], wd_hat)
@@ -218,14 +223,14 @@ def test_wq_gemm_full_size_sampled(env):
     a = inputs.activations(7, 11, M, K)
     m_dev = 7373
     md = torch.tensor([m_dev], dtype=torch.int32, device=dev)
-    y = api.wq_gemm(api.to_device_bf16(a, dev), qw, md, api.EPI_STORE_F32)
+    y = api.wq_gemm(api.to_device_act(a, 1, dev), qw, md, api.EPI_STORE_F32)
     assert api.device_status() == 0
     rows = np.array([0, 1, 255, 256, 4095, 4096, 7000, 7371, 7372])
     cols = np.unique(np.concatenate([[0, 1, 127, 128, 11007, 11008, 22015],
                                      inputs.integers(8, 1, 40, N)]))
     sub = dict(packed=wq["packed"][cols], scales=wq["scales"][cols], zeros=wq["zeros"][cols],
                N=len(cols), K=K, bits=bits, group=group)
-    ref = oracle.linear(a[rows], inputs.round_bf16(oracle.dequantize_weight(sub)))
+    ref = oracle.linear(a[rows], round_act(oracle.dequantize_weight(sub), 1))
     got = y[torch.from_numpy(rows).to(dev)][:, torch.from_numpy(cols).to(dev)].cpu().numpy()
     assert np.abs(got - ref).max() <= 2e-4 * max(1.0, np.abs(ref).max())
     assert not y[m_dev:].any().item()
