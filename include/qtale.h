@@ -114,6 +114,37 @@ int qtale_router_select(const void* x, int T, int d, const float* w_router, floa
                         int32_t* n_exec_out, int32_t* cu_exec_out, int32_t* pos_out, void* ws,
                         size_t ws_bytes, void* stream);
 
+/*
+ * qtale_router_select for callers that must not allocate device memory.
+ * (No counterpart in the paper: this is a packaging variant of the call above.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- a plugin inside
+ * a host application that owns the whole memory pool and hands out no scratch,
+ * a real-time or safety-checked loop that forbids allocator calls after start-up,
+ * or a caller that simply has no buffer left to lend as `ws`.  Same arguments,
+ * results and limits as qtale_router_select, minus the workspace: the kernel's
+ * scratch (its 4-byte ticket counter, 256 bytes reserved) sits in an array that
+ * is part of the library's device image, so every GPU that loads the library
+ * holds those 256 bytes until the process exits.  The call itself performs no
+ * cudaMalloc / cudaFree and uses no allocating library routine.
+ *
+ *  - Limit: T whose scratch need (qtale_router_select_workspace_bytes(T))
+ *    exceeds the 256 built-in bytes is refused with QTALE_ERR_CAPACITY.
+ *  - The first call on each device looks up the array's device address (one
+ *    cudaGetSymbolAddress, result cached per device); make that first call
+ *    outside any stream capture.
+ *  - All calls on a device share the one array.  The counter is cleared on the
+ *    stream before every launch, so leftovers of the previous call are harmless,
+ *    but two calls whose kernels overlap on the GPU (different streams) race on
+ *    it: keep calls to this entry point on one stream, or order them yourself.
+ */
+int qtale_router_select_static(const void* x, int T, int d, const float* w_router, float bias,
+                               const float* scores_override, const uint8_t* valid,
+                               const int32_t* cu_seqlens, int B, const int32_t* pos0, int mode,
+                               float theta, int k, float* scores_out, int32_t* idx_out,
+                               int32_t* n_exec_out, int32_t* cu_exec_out, int32_t* pos_out,
+                               void* stream);
+
 /* Bookkeeping for a caller-supplied ascending index list (QTALE_SELECT_FORCED):
  * fills n_exec_out, cu_exec_out and pos_out as qtale_router_select does.
  * idx [n] int32 device, 0 <= n <= T. */

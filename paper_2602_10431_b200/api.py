@@ -25,7 +25,8 @@ PHASE_PREFILL, PHASE_DECODE = 0, 1
 
 EXPORTS = [
     "qtale_strerror", "qtale_device_status", "qtale_topk_count",
-    "qtale_router_select_workspace_bytes", "qtale_router_select", "qtale_index_bookkeeping",
+    "qtale_router_select_workspace_bytes", "qtale_router_select", "qtale_router_select_static",
+    "qtale_index_bookkeeping",
     "qtale_compact", "qtale_scatter_add", "qtale_wq_repack", "qtale_wq_gemm",
     "qtale_layer_workspace_bytes", "qtale_layer_forward", "qtale_model_workspace_bytes",
     "qtale_model_prefill",
@@ -92,6 +93,7 @@ def lib():
             C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_float, C.c_void_p, C.c_void_p,
             C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_float, C.c_int, C.c_void_p, C.c_void_p,
             C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+        L.qtale_router_select_static.argtypes = L.qtale_router_select.argtypes[:18] + [C.c_void_p]
         L.qtale_index_bookkeeping.argtypes = [
             C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p,
             C.c_void_p, C.c_void_p]
@@ -173,6 +175,22 @@ def router_select(x, w_router, bias, cu_seqlens, mode, theta=0.5, k=0, scores_ov
         _ptr(n_exec), _ptr(cu_exec), _ptr(pos), _ptr(ws), ws.numel(), _stream()),
         "qtale_router_select")
     return dict(scores=scores, idx=idx, n_exec=n_exec, cu_exec=cu_exec, pos=pos, ws=ws)
+
+
+def router_select_static(x, w_router, bias, cu_seqlens, mode, out, theta=0.5, k=0,
+                         scores_override=None, valid=None, pos0=None):
+    """qtale_router_select_static: same as router_select but without a workspace; the
+    scratch is built into the library, so this wrapper allocates nothing either --
+    the caller passes every output tensor in `out` (scores, idx, n_exec, cu_exec, pos)."""
+    T = int(x.shape[0]) if x is not None else int(scores_override.shape[0])
+    d = int(x.shape[1]) if x is not None else 0
+    B = int(cu_seqlens.shape[0]) - 1
+    check(lib().qtale_router_select_static(
+        _ptr(x), T, d, _ptr(w_router), float(bias), _ptr(scores_override), _ptr(valid),
+        _ptr(cu_seqlens), B, _ptr(pos0), int(mode), float(theta), int(k), _ptr(out["scores"]),
+        _ptr(out["idx"]), _ptr(out["n_exec"]), _ptr(out["cu_exec"]), _ptr(out["pos"]), _stream()),
+        "qtale_router_select_static")
+    return out
 
 
 def index_bookkeeping(idx, n, T, cu_seqlens, pos0=None):

@@ -358,6 +358,38 @@ int qtale_router_select(const void* x, int T, int d, const float* w_router, floa
   return launch_status(cudaGetLastError());
 }
 
+// ---- variant for callers that cannot allocate device memory -------------------
+// The kernel's only scratch is its ticket counter; here it lives in a static
+// device array that every GPU loading the library carries until exit.
+#define QTALE_ROUTER_STATIC_SCRATCH_BYTES 256
+static __device__ __align__(256) unsigned char g_router_static_scratch[QTALE_ROUTER_STATIC_SCRATCH_BYTES];
+
+int qtale_router_select_static(const void* x, int T, int d, const float* w_router, float bias,
+                               const float* scores_override, const uint8_t* valid,
+                               const int32_t* cu_seqlens, int B, const int32_t* pos0, int mode,
+                               float theta, int k, float* scores_out, int32_t* idx_out,
+                               int32_t* n_exec_out, int32_t* cu_exec_out, int32_t* pos_out,
+                               void* stream) {
+  // In host code the array's name is only a handle; its device address has to be
+  // asked for, once per device, with that device current.
+  static void* scratch_of_device[64] = {nullptr};
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return QTALE_ERR_CUDA;
+  if (T >= 1 && qtale_router_select_workspace_bytes(T) > (size_t)QTALE_ROUTER_STATIC_SCRATCH_BYTES)
+    return QTALE_ERR_CAPACITY;  // the built-in scratch is too small for this many tokens
+  if (!scratch_of_device[dev]) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_router_static_scratch) != cudaSuccess || !ptr)
+      return QTALE_ERR_CUDA;
+    scratch_of_device[dev] = ptr;
+  }
+  // The shared entry point zeroes the ticket word (cudaMemsetAsync on the stream)
+  // before the launch, so whatever the previous call left behind does not matter.
+  return qtale_router_select(x, T, d, w_router, bias, scores_override, valid, cu_seqlens, B, pos0,
+                             mode, theta, k, scores_out, idx_out, n_exec_out, cu_exec_out, pos_out,
+                             scratch_of_device[dev], QTALE_ROUTER_STATIC_SCRATCH_BYTES, stream);
+}
+
 int qtale_index_bookkeeping(const int32_t* idx, int n, int T, const int32_t* cu_seqlens, int B,
                             const int32_t* pos0, int32_t* n_exec_out, int32_t* cu_exec_out,
                             int32_t* pos_out, void* stream) {
