@@ -3,18 +3,22 @@
 //
 // The product is computed transposed, D[n, m] = sum_k W[n, k] * A[m, k]:
 //   * the 128 weight rows of a tile are the MMA's M dimension; the packed codes
-//     are fetched by a bulk TMA copy, turned into bf16 in registers
-//     ((code - zero) * scale exactly in fp32, one rounding) and written with
-//     tcgen05.st into tensor memory, from where the MMA reads its A operand;
-//   * up to 256 tokens are the N dimension; their activations arrive by a tiled
-//     TMA load into 128-byte-swizzled shared memory (the B operand);
-//   * the fp32 accumulator D (128 lanes x TN columns) lives in tensor memory and
-//     is drained by four epilogue warps, one TMEM lane quadrant each.
-// The grid is persistent (one CTA per SM) and reads the number of executed
-// tokens from device memory, so no launch parameter depends on the routing.
+//     arrive by bulk TMA copies in a ring of their own, are turned into the 16-bit
+//     activation format in registers ((code - zero) * scale exactly in fp32, one
+//     rounding) and written with tcgen05.st into a ring of tensor-memory slots,
+//     from where the MMA reads its A operand;
+//   * up to 192 tokens are the N dimension; their activations arrive by tiled TMA
+//     loads into a ring of 128-byte-swizzled shared-memory stages (the B operand);
+//   * two fp32 accumulators (128 lanes x TN columns each) live in tensor memory, so
+//     the four epilogue warps drain tile i while the MMAs of tile i+1 run.
+// The three rings (weights, dequantised A slots, activations) are independent, so
+// the dequantisers run ahead of the activation loads instead of lengthening their
+// round trip.  The grid is persistent (one CTA per SM) and reads the number of
+// executed tokens from device memory: no launch parameter depends on the routing.
 //
-// Warp roles (320 threads): warp 0 TMA producer, warp 1 MMA issuer and TMEM
-// allocator, warps 2-5 dequantisers, warps 6-9 epilogue.
+// Warp roles (480 threads): warp 0 activation TMA producer, warp 1 MMA issuer and
+// TMEM allocator, warps 2-9 dequantisers (two sets of four that alternate K blocks),
+// warps 10-13 epilogue (one TMEM lane quadrant each), warp 14 weight TMA producer.
 #include <cuda.h>
 
 #include <string.h>
@@ -27,25 +31,36 @@ namespace qtale {
 
 using namespace ptx;
 
-constexpr int kGemmThreads = 320;
-constexpr int kTileRows = 128;          // weight rows per tile (MMA M)
-constexpr int kKB = 64;                 // K elements per pipeline stage (128 B of bf16)
+constexpr int kGemmThreads = 480;
+constexpr int kDequantGroups = 2;        // two sets of four dequantiser warps alternate K blocks
+constexpr int kTileRows = 128;           // weight rows per tile (MMA M)
+constexpr int kKB = 64;                  // K elements per pipeline step (128 B of 16-bit data)
 constexpr uint32_t kSpinLimit = 1u << 24;
 constexpr int kTmemCols = 512;
-constexpr int kTmemAColBase = 256;      // A-operand stages start here; D uses [0, TN)
-constexpr int kAColsPerStage = kKB / 2; // two bf16 per 32-bit column
+constexpr int kAColsPerSlot = kKB / 2;   // two 16-bit values per 32-bit TMEM column
+constexpr int kEpiRowWords = 36;         // padded row (32 fp32 + 4) of the epilogue staging tile
+constexpr int kEpiWarpBytes = 32 * kEpiRowWords * 4;
 
 template <int TN, int BITS>
 struct GemmCfg {
   static constexpr int kXBytes = TN * 128;
-  static constexpr int kWBytes = BITS == 16 ? kTileRows * 128 : kTileRows * kKB * BITS / 8;
+  // with 16-bit weights the weight tile travels with the activations (both from TMA)
+  static constexpr int kXStageBytes = kXBytes + (BITS == 16 ? kTileRows * 128 : 0);
+  static constexpr int kXStages = BITS == 16 ? 4 : (TN >= 192 ? 6 : 8);
+  static constexpr int kWCodeBytes = BITS == 16 ? 0 : kTileRows * kKB * BITS / 8;
   static constexpr int kSzBytes = BITS == 16 ? 0 : kTileRows * 4;
-  static constexpr int kStageBytes = (kXBytes + kWBytes + kSzBytes + 1023) / 1024 * 1024;
-  static constexpr int kMaxStages = (224 * 1024) / kStageBytes;
-  static constexpr int kStages = kMaxStages > 8 ? 8 : kMaxStages;
-  static constexpr size_t kSmemBytes = (size_t)kStages * kStageBytes + 1024;
-  static_assert(kStages >= 2, "pipeline needs at least two stages");
-  static_assert(kTmemAColBase + kStages * kAColsPerStage <= kTmemCols, "TMEM budget");
+  static constexpr int kWStageBytes = kWCodeBytes + kSzBytes;
+  static constexpr int kWStages = BITS == 16 ? 0 : 10;
+  static constexpr int kDCols = TN;                       // columns of one accumulator
+  static constexpr int kAColBase = 2 * kDCols;            // A slots follow the two accumulators
+  static constexpr int kASlotsMax = (kTmemCols - kAColBase) / kAColsPerSlot;
+  static constexpr int kASlots = kASlotsMax > 8 ? 8 : kASlotsMax;
+  static constexpr size_t kEpiOffset = (size_t)kXStages * kXStageBytes + (size_t)kWStages * kWStageBytes;
+  static constexpr size_t kSmemBytes = kEpiOffset + 4 * kEpiWarpBytes + 1024;
+  static_assert(kXStageBytes % 1024 == 0, "swizzled stages must stay 1024-byte aligned");
+  static_assert(kWStageBytes % 16 == 0, "bulk copies need 16-byte granularity");
+  static_assert(BITS == 16 || kASlots >= 4, "TMEM budget");
+  static_assert(kSmemBytes <= 232448 - 512, "shared memory budget");
 };
 
 struct GemmParams {
@@ -69,11 +84,10 @@ struct GemmParams {
 };
 
 struct __align__(8) GemmShared {
-  uint64_t full[8];
-  uint64_t empty[8];
-  uint64_t a_full[8];
-  uint64_t d_full;
-  uint64_t d_empty;
+  uint64_t full_x[8], empty_x[8];    // activation ring
+  uint64_t full_w[12], empty_w[12];  // packed-weight ring
+  uint64_t a_full[8], a_empty[8];    // dequantised A slots in tensor memory
+  uint64_t d_full[2], d_empty[2];    // the two accumulators
   uint32_t tmem_base;
   volatile int abort_flag;
 };
@@ -103,7 +117,7 @@ __device__ __forceinline__ int tile_row_to_n(const GemmParams& p, int nt, int L)
   return n < p.N ? n : -1;
 }
 
-// Eight codes sitting in the 4-bit slots of `t` -> four bf16x2 registers.
+// Eight codes sitting in the 4-bit slots of `t` -> four packed 16-bit pairs.
 // Slot i holds the code in its low QBITS bits.  The code is moved into a float
 // mantissa next to 2^23, so (float - (2^23 + zero * 16^i)) * (scale / 16^i) is
 // exactly (code - zero) * scale.
@@ -123,28 +137,141 @@ __device__ __forceinline__ void dequant8(uint32_t t, const float (&C)[5], const 
   for (int q = 0; q < 4; ++q) out[q] = Act16<ACT>::pack(v[2 * q], v[2 * q + 1]);
 }
 
+struct Ring {
+  int s = 0;
+  uint32_t ph = 0;
+  __device__ __forceinline__ void advance(int n) {
+    if (++s == n) { s = 0; ph ^= 1u; }
+  }
+};
+
+// ---- epilogue of one 32-column chunk, run by one warp on its 32 weight rows ----
+// `stage` holds the chunk transposed: stage[m * kEpiRowWords + lane_n] = D[lane_n, m].
+// Each lane then owns 8 consecutive output features of one token row, so global
+// accesses are 16 bytes per lane and 64 or 128 contiguous bytes per row.
+template <int ACT>
+__device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const float* stage, int lane,
+                                               int nt, int quad, int m0, int M) {
+  if (p.epilogue == QTALE_EPI_SWIGLU) {
+    // lanes n = 0..15 of the chunk are gate rows, n = 16..31 the matching up rows
+    const int jc = (lane & 1) * 8;
+    const int j0 = nt * 64 + quad * 16 + jc;
+    if (j0 >= p.F) return;
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      const int row = i * 16 + (lane >> 1);
+      const int m = m0 + row;
+      if (m >= M) continue;
+      const float4 g0 = *reinterpret_cast<const float4*>(stage + row * kEpiRowWords + jc);
+      const float4 g1 = *reinterpret_cast<const float4*>(stage + row * kEpiRowWords + jc + 4);
+      const float4 u0 = *reinterpret_cast<const float4*>(stage + row * kEpiRowWords + 16 + jc);
+      const float4 u1 = *reinterpret_cast<const float4*>(stage + row * kEpiRowWords + 16 + jc + 4);
+      const float g[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+      const float u[8] = {u0.x, u0.y, u0.z, u0.w, u1.x, u1.y, u1.z, u1.w};
+      uint32_t o[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e)
+        o[e] = Act16<ACT>::pack(g[2 * e] / (1.f + __expf(-g[2 * e])) * u[2 * e],
+                                g[2 * e + 1] / (1.f + __expf(-g[2 * e + 1])) * u[2 * e + 1]);
+      st_16(static_cast<unsigned short*>(p.y) + (size_t)m * p.ldy + j0,
+            make_uint4(o[0], o[1], o[2], o[3]));
+    }
+    return;
+  }
+  const int nc = (lane & 3) * 8;
+  const int n0 = tile_row_to_n(p, nt, quad * 32 + nc);  // 8 consecutive features, all valid or none
+  const bool n_ok = n0 >= 0;  // no early return: the shuffles below need the whole warp
+  const bool gathers = p.epilogue == QTALE_EPI_RESID_F32 || p.epilogue == QTALE_EPI_RESID_SCATTER;
+  int my_row = 0;
+  if (gathers && m0 + lane < M) my_row = __ldg(p.idx + m0 + lane);
+  // residual operands of all four row groups are requested before the first use
+  uint4 rb[4];
+  float4 rf[4][2];
+  int tok[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int row = i * 8 + (lane >> 2);
+    const int m = m0 + row;
+    tok[i] = __shfl_sync(0xffffffffu, my_row, row);
+    if (m < M && n_ok) {
+      if (p.epilogue == QTALE_EPI_RESID_F32) {
+        rb[i] = ld_nc_16(static_cast<const unsigned short*>(p.resid) + (size_t)tok[i] * p.ld_resid + n0);
+      } else if (p.epilogue == QTALE_EPI_RESID_SCATTER) {
+        const float* r = static_cast<const float*>(p.resid) + (size_t)m * p.ld_resid + n0;
+        rf[i][0] = __ldg(reinterpret_cast<const float4*>(r));
+        rf[i][1] = __ldg(reinterpret_cast<const float4*>(r) + 1);
+      }
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int row = i * 8 + (lane >> 2);
+    const int m = m0 + row;
+    if (m >= M || !n_ok) continue;
+    const float4 a0 = *reinterpret_cast<const float4*>(stage + row * kEpiRowWords + nc);
+    const float4 a1 = *reinterpret_cast<const float4*>(stage + row * kEpiRowWords + nc + 4);
+    float v[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+    if (p.epilogue == QTALE_EPI_STORE_16) {
+      st_16(static_cast<unsigned short*>(p.y) + (size_t)m * p.ldy + n0,
+            make_uint4(Act16<ACT>::pack(v[0], v[1]), Act16<ACT>::pack(v[2], v[3]),
+                       Act16<ACT>::pack(v[4], v[5]), Act16<ACT>::pack(v[6], v[7])));
+    } else if (p.epilogue == QTALE_EPI_STORE_F32 || p.epilogue == QTALE_EPI_RESID_F32) {
+      if (p.epilogue == QTALE_EPI_RESID_F32) {
+        const uint32_t w[4] = {rb[i].x, rb[i].y, rb[i].z, rb[i].w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          v[2 * e] += bf16_lo(w[e]);
+          v[2 * e + 1] += bf16_hi(w[e]);
+        }
+      }
+      float* y = static_cast<float*>(p.y) + (size_t)m * p.ldy + n0;
+      st_16(y, make_uint4(__float_as_uint(v[0]), __float_as_uint(v[1]), __float_as_uint(v[2]),
+                          __float_as_uint(v[3])));
+      st_16(y + 4, make_uint4(__float_as_uint(v[4]), __float_as_uint(v[5]), __float_as_uint(v[6]),
+                              __float_as_uint(v[7])));
+    } else {  // QTALE_EPI_RESID_SCATTER: x[idx[m]] = bf16(u + acc)   (Eq. 3)
+      const float r[8] = {rf[i][0].x, rf[i][0].y, rf[i][0].z, rf[i][0].w,
+                          rf[i][1].x, rf[i][1].y, rf[i][1].z, rf[i][1].w};
+      st_16(static_cast<unsigned short*>(p.dst) + (size_t)tok[i] * p.ld_dst + n0,
+            make_uint4(pack_bf16x2(v[0] + r[0], v[1] + r[1]), pack_bf16x2(v[2] + r[2], v[3] + r[3]),
+                       pack_bf16x2(v[4] + r[4], v[5] + r[5]), pack_bf16x2(v[6] + r[6], v[7] + r[7])));
+    }
+  }
+}
+
 template <int TN, int BITS, int ACT>
 __global__ void __launch_bounds__(kGemmThreads, 1)
     wq_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x,
                    const __grid_constant__ CUtensorMap tmap_w, const GemmParams p) {
   using Cfg = GemmCfg<TN, BITS>;
-  constexpr int S = Cfg::kStages;
+  constexpr int SX = Cfg::kXStages;
+  constexpr int SW = Cfg::kWStages;
+  constexpr int SA = Cfg::kASlots;
   extern __shared__ unsigned char smem_dyn[];
   __shared__ GemmShared sh;
-  unsigned char* stage_base = reinterpret_cast<unsigned char*>(
+  unsigned char* x_base = reinterpret_cast<unsigned char*>(
       (reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~static_cast<uintptr_t>(1023));
+  unsigned char* w_base = x_base + (size_t)SX * Cfg::kXStageBytes;
+  float* epi_base = reinterpret_cast<float*>(x_base + Cfg::kEpiOffset);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < S; ++s) {
-      mbar_init(&sh.full[s], 1);
-      mbar_init(&sh.empty[s], 1);
+    for (int s = 0; s < 8; ++s) {
+      mbar_init(&sh.full_x[s], 1);
+      mbar_init(&sh.empty_x[s], 1);
       mbar_init(&sh.a_full[s], 4);
+      mbar_init(&sh.a_empty[s], 1);
     }
-    mbar_init(&sh.d_full, 1);
-    mbar_init(&sh.d_empty, 4);
+    for (int s = 0; s < 12; ++s) {
+      mbar_init(&sh.full_w[s], 1);
+      mbar_init(&sh.empty_w[s], 4);
+    }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&sh.d_full[s], 1);
+      mbar_init(&sh.d_empty[s], 4);
+    }
     sh.abort_flag = 0;
     fence_barrier_init();
   }
@@ -169,88 +296,123 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
   const int nkb = p.nkb;
 
   if (warp == 0) {
-    // ------------------------------ TMA producer ------------------------------
+    // -------------------------- activation TMA producer --------------------------
     if (lane == 0) {
-      int s = 0;
-      uint32_t ph = 0;
+      Ring rx;
       for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
         const int nt = tile / n_mt, mt = tile % n_mt;
         for (int kb = 0; kb < nkb; ++kb) {
-          if (!wait_or_abort(&sh.empty[s], ph ^ 1u, &sh, p.status)) goto producer_done;
-          unsigned char* st = stage_base + (size_t)s * Cfg::kStageBytes;
-          const bool with_sz = BITS != 16 && (kb % p.kb_per_group) == 0;
-          mbar_arrive_expect_tx(&sh.full[s],
-                                Cfg::kXBytes + Cfg::kWBytes + (with_sz ? Cfg::kSzBytes : 0));
-          tma_load_2d(st, &tmap_x, &sh.full[s], kb * kKB, mt * TN);
-          if (BITS == 16) {
-            tma_load_2d(st + Cfg::kXBytes, &tmap_w, &sh.full[s], kb * kKB, nt * kTileRows);
-          } else {
-            bulk_load(st + Cfg::kXBytes, p.packed + ((size_t)nt * nkb + kb) * Cfg::kWBytes,
-                      Cfg::kWBytes, &sh.full[s]);
-            if (with_sz)
-              bulk_load(st + Cfg::kXBytes + Cfg::kWBytes,
-                        p.packed + p.sz_offset +
-                            ((size_t)nt * (nkb / p.kb_per_group) + kb / p.kb_per_group) *
-                                Cfg::kSzBytes,
-                        Cfg::kSzBytes, &sh.full[s]);
-          }
-          if (++s == S) { s = 0; ph ^= 1u; }
+          if (!wait_or_abort(&sh.empty_x[rx.s], rx.ph ^ 1u, &sh, p.status)) goto x_done;
+          unsigned char* st = x_base + (size_t)rx.s * Cfg::kXStageBytes;
+          mbar_arrive_expect_tx(&sh.full_x[rx.s], Cfg::kXStageBytes);
+          tma_load_2d(st, &tmap_x, &sh.full_x[rx.s], kb * kKB, mt * TN);
+          if (BITS == 16)
+            tma_load_2d(st + Cfg::kXBytes, &tmap_w, &sh.full_x[rx.s], kb * kKB, nt * kTileRows);
+          rx.advance(SX);
         }
       }
-    producer_done:;
+    x_done:;
+    }
+  } else if (warp == 14) {
+    // ---------------------------- weight TMA producer ----------------------------
+    if (BITS != 16 && lane == 0) {
+      Ring rw;
+      const int ng = nkb / p.kb_per_group;
+      for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+        const int nt = tile / n_mt;
+        for (int kb = 0; kb < nkb; ++kb) {
+          if (!wait_or_abort(&sh.empty_w[rw.s], rw.ph ^ 1u, &sh, p.status)) goto w_done;
+          unsigned char* st = w_base + (size_t)rw.s * Cfg::kWStageBytes;
+          // every stage carries the scale / zero words of its group
+          mbar_arrive_expect_tx(&sh.full_w[rw.s], Cfg::kWStageBytes);
+          bulk_load(st, p.packed + ((size_t)nt * nkb + kb) * Cfg::kWCodeBytes, Cfg::kWCodeBytes,
+                    &sh.full_w[rw.s]);
+          bulk_load(st + Cfg::kWCodeBytes,
+                    p.packed + p.sz_offset +
+                        ((size_t)nt * ng + kb / p.kb_per_group) * Cfg::kSzBytes,
+                    Cfg::kSzBytes, &sh.full_w[rw.s]);
+          rw.advance(SW);
+        }
+      }
+    w_done:;
     }
   } else if (warp == 1) {
     // ------------------------------- MMA issuer --------------------------------
     if (lane == 0) {
       constexpr uint32_t idesc = idesc_16bit_f32(kTileRows, TN, ACT == 1);
-      int s = 0;
-      uint32_t ph = 0, dph = 0;
-      for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
-        if (!wait_or_abort(&sh.d_empty, dph ^ 1u, &sh, p.status)) goto mma_done;
+      Ring rx, ra;
+      int it = 0;
+      for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++it) {
+        const int buf = it & 1;
+        const uint32_t dph = (uint32_t)(it >> 1) & 1u;
+        if (!wait_or_abort(&sh.d_empty[buf], dph ^ 1u, &sh, p.status)) goto mma_done;
         tc_fence_after();
+        const uint32_t d_tmem = tmem_base + buf * Cfg::kDCols;
         for (int kb = 0; kb < nkb; ++kb) {
-          if (!wait_or_abort(&sh.full[s], ph, &sh, p.status)) goto mma_done;
+          if (!wait_or_abort(&sh.full_x[rx.s], rx.ph, &sh, p.status)) goto mma_done;
           if (BITS != 16) {
-            if (!wait_or_abort(&sh.a_full[s], ph, &sh, p.status)) goto mma_done;
+            if (!wait_or_abort(&sh.a_full[ra.s], ra.ph, &sh, p.status)) goto mma_done;
           }
           tc_fence_after();
-          unsigned char* st = stage_base + (size_t)s * Cfg::kStageBytes;
+          unsigned char* st = x_base + (size_t)rx.s * Cfg::kXStageBytes;
           const uint64_t b_desc = smem_desc_sw128(smem_u32(st));
 #pragma unroll
           for (int j = 0; j < kKB / 16; ++j) {
             const uint32_t acc = (kb | j) != 0 ? 1u : 0u;
             if (BITS == 16) {
               const uint64_t a_desc = smem_desc_sw128(smem_u32(st + Cfg::kXBytes));
-              mma_ss(tmem_base, a_desc + 2u * j, b_desc + 2u * j, idesc, acc);
+              mma_ss(d_tmem, a_desc + 2u * j, b_desc + 2u * j, idesc, acc);
             } else {
-              mma_ts(tmem_base, tmem_base + kTmemAColBase + s * kAColsPerStage + j * 8,
+              mma_ts(d_tmem, tmem_base + Cfg::kAColBase + ra.s * kAColsPerSlot + j * 8,
                      b_desc + 2u * j, idesc, acc);
             }
           }
-          mma_commit(&sh.empty[s]);  // frees the smem stage and the TMEM A slot
-          if (++s == S) { s = 0; ph ^= 1u; }
+          mma_commit(&sh.empty_x[rx.s]);             // frees the activation stage
+          if (BITS != 16) mma_commit(&sh.a_empty[ra.s]);  // frees the A slot
+          rx.advance(SX);
+          ra.advance(SA);
         }
-        mma_commit(&sh.d_full);
-        dph ^= 1u;
+        mma_commit(&sh.d_full[buf]);
       }
     mma_done:;
     }
-  } else if (warp < 6) {
+  } else if (warp < 2 + 4 * kDequantGroups) {
     // ------------------------------- dequantisers --------------------------------
     if (BITS != 16) {
       const int quad = warp & 3;
       const int L = quad * 32 + lane;
-      int s = 0;
-      uint32_t ph = 0;
-      float C[5], Sc[5];
-#pragma unroll
-      for (int i = 0; i < 5; ++i) { C[i] = 0.f; Sc[i] = 0.f; }
+      const int my_group = (warp - 2) >> 2;
+      int turn = 0;  // which set owns the current K block
+      Ring rw, ra;
       for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
         for (int kb = 0; kb < nkb; ++kb) {
-          if (!wait_or_abort(&sh.full[s], ph, &sh, p.status)) goto dequant_done;
-          const unsigned char* st = stage_base + (size_t)s * Cfg::kStageBytes + Cfg::kXBytes;
-          if ((kb % p.kb_per_group) == 0) {
-            const uint32_t sz = reinterpret_cast<const uint32_t*>(st + Cfg::kWBytes)[L];
+          const bool mine = (turn == my_group);
+          if (++turn == kDequantGroups) turn = 0;
+          if (!mine) {
+            rw.advance(SW);
+            ra.advance(SA);
+            continue;
+          }
+          if (!wait_or_abort(&sh.full_w[rw.s], rw.ph, &sh, p.status)) goto dequant_done;
+          const unsigned char* st = w_base + (size_t)rw.s * Cfg::kWStageBytes;
+          // packed codes and the group's scale / zero into registers, then release the stage
+          const uint32_t sz = reinterpret_cast<const uint32_t*>(st + Cfg::kWCodeBytes)[L];
+          uint32_t cw[8];
+          if (BITS == 4) {
+            const uint4 w0 = reinterpret_cast<const uint4*>(st)[L];
+            const uint4 w1 = reinterpret_cast<const uint4*>(st)[kTileRows + L];
+            cw[0] = w0.x; cw[1] = w0.y; cw[2] = w0.z; cw[3] = w0.w;
+            cw[4] = w1.x; cw[5] = w1.y; cw[6] = w1.z; cw[7] = w1.w;
+          } else {
+            const uint4 a = reinterpret_cast<const uint4*>(st)[L];
+            const uint2 b = reinterpret_cast<const uint2*>(st + kTileRows * 16)[L];
+            cw[0] = a.x; cw[1] = a.y; cw[2] = a.z; cw[3] = a.w;
+            cw[4] = b.x; cw[5] = b.y; cw[6] = 0; cw[7] = 0;
+          }
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&sh.empty_w[rw.s]);
+          float C[5], Sc[5];
+          {
             const float scale = __half2float(__ushort_as_half((unsigned short)(sz & 0xFFFFu)));
             const float zero = __half2float(__ushort_as_half((unsigned short)(sz >> 16)));
 #pragma unroll
@@ -259,146 +421,71 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
               Sc[i] = scale * (1.f / (float)(1 << (4 * i)));
             }
           }
+          if (!wait_or_abort(&sh.a_empty[ra.s], ra.ph ^ 1u, &sh, p.status)) goto dequant_done;
+          tc_fence_after();
           const uint32_t a_taddr =
-              tmem_base + ((uint32_t)(quad * 32) << 16) + kTmemAColBase + s * kAColsPerStage;
-          if (BITS == 4) {
+              tmem_base + ((uint32_t)(quad * 32) << 16) + Cfg::kAColBase + ra.s * kAColsPerSlot;
 #pragma unroll
-            for (int part = 0; part < 2; ++part) {
-              const uint4 w = reinterpret_cast<const uint4*>(st)[part * kTileRows + L];
-              uint32_t r[16];
-              dequant8<0xFu, ACT>(w.x, C, Sc, r + 0);
-              dequant8<0xFu, ACT>(w.y, C, Sc, r + 4);
-              dequant8<0xFu, ACT>(w.z, C, Sc, r + 8);
-              dequant8<0xFu, ACT>(w.w, C, Sc, r + 12);
-              tmem_st_x16(a_taddr + part * 16, r);
-            }
-          } else {
-            // 3-bit: low two bits of 16 codes per word (plane A), high bit of 32 codes
-            // per word (plane B).  A nibble-style word with the code in the low 3 bits
-            // of each 4-bit slot is assembled with one bitwise select.
-            const uint4 a = reinterpret_cast<const uint4*>(st)[L];
-            const uint2 b = reinterpret_cast<const uint2*>(st + kTileRows * 16)[L];
-            const uint32_t aw[4] = {a.x, a.y, a.z, a.w};
-            const uint32_t bw[2] = {b.x, b.y};
+          for (int part = 0; part < 2; ++part) {
+            uint32_t r[16];
+            if (BITS == 4) {
 #pragma unroll
-            for (int part = 0; part < 2; ++part) {
-              uint32_t r[16];
+              for (int j = 0; j < 4; ++j) dequant8<0xFu, ACT>(cw[part * 4 + j], C, Sc, r + 4 * j);
+            } else {
+              // 3-bit: low two bits of 16 codes per word (plane A: cw[0..3]), high bit of 32
+              // codes per word (plane B: cw[4..5]).  A nibble-style word with the code in
+              // the low 3 bits of each 4-bit slot is assembled with one bitwise select.
 #pragma unroll
               for (int uu = 0; uu < 4; ++uu) {
                 const int u = part * 4 + uu;
-                const uint32_t a2 = (u & 1) ? (aw[u >> 1] >> 2) : aw[u >> 1];
+                const uint32_t a2 = (u & 1) ? (cw[u >> 1] >> 2) : cw[u >> 1];
                 const int rr = u & 3;
-                const uint32_t b1 = rr == 0 ? (bw[u >> 2] << 2)
-                                  : rr == 1 ? (bw[u >> 2] << 1)
-                                  : rr == 2 ? bw[u >> 2] : (bw[u >> 2] >> 1);
+                const uint32_t bw = cw[4 + (u >> 2)];
+                const uint32_t b1 = rr == 0 ? (bw << 2) : rr == 1 ? (bw << 1) : rr == 2 ? bw : (bw >> 1);
                 const uint32_t t = (a2 & 0x33333333u) | (b1 & 0xCCCCCCCCu);
                 dequant8<0x7u, ACT>(t, C, Sc, r + 4 * uu);
               }
-              tmem_st_x16(a_taddr + part * 16, r);
             }
+            tmem_st_x16(a_taddr + part * 16, r);
           }
           tmem_wait_st();
           tc_fence_before();
           __syncwarp();
-          if (lane == 0) mbar_arrive(&sh.a_full[s]);
-          if (++s == S) { s = 0; ph ^= 1u; }
+          if (lane == 0) mbar_arrive(&sh.a_full[ra.s]);
+          rw.advance(SW);
+          ra.advance(SA);
         }
       }
     dequant_done:;
     }
-  } else {
+  } else if (warp < 14) {
     // --------------------------------- epilogue -----------------------------------
     const int quad = warp & 3;
-    const int L = quad * 32 + lane;
-    uint32_t dph = 0;
-    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+    float* stage = epi_base + (size_t)(warp - 10) * (kEpiWarpBytes / 4);
+    int it = 0;
+    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++it) {
       const int nt = tile / n_mt, mt = tile % n_mt;
-      if (!wait_or_abort(&sh.d_full, dph, &sh, p.status)) break;
+      const int buf = it & 1;
+      const uint32_t dph = (uint32_t)(it >> 1) & 1u;
+      if (!wait_or_abort(&sh.d_full[buf], dph, &sh, p.status)) break;
       tc_fence_after();
-      const int n = tile_row_to_n(p, nt, L);
       const int m_base = mt * TN;
 #pragma unroll 1
       for (int c0 = 0; c0 < TN; c0 += 32) {
         const int m0 = m_base + c0;
         if (m0 >= M) break;
-        const int n_cols = min(32, M - m0);  // warp-uniform
         uint32_t r[32];
-        tmem_ld_x32(tmem_base + ((uint32_t)(quad * 32) << 16) + c0, r);
-        if (p.epilogue == QTALE_EPI_RESID_F32 || p.epilogue == QTALE_EPI_RESID_SCATTER) {
-          // all residual reads of the chunk are issued before the first store so that
-          // their latencies overlap (one row index per column, fetched by one lane)
-          const int my_row = (lane < n_cols) ? __ldg(p.idx + m0 + lane) : 0;
-          float res[32];
-          if (p.epilogue == QTALE_EPI_RESID_F32) {
-            const unsigned short* rp = static_cast<const unsigned short*>(p.resid);
+        tmem_ld_x32(tmem_base + ((uint32_t)(quad * 32) << 16) + buf * Cfg::kDCols + c0, r);
+        tmem_wait_ld();
 #pragma unroll
-            for (int c = 0; c < 32; ++c) {
-              const int row = __shfl_sync(0xffffffffu, my_row, c);
-              res[c] = (c < n_cols && n >= 0)
-                           ? bf16_bits_to_float(__ldg(rp + (size_t)row * p.ld_resid + n)) : 0.f;
-            }
-            tmem_wait_ld();
-            if (n >= 0) {
-              float* y = static_cast<float*>(p.y);
-#pragma unroll
-              for (int c = 0; c < 32; ++c)
-                if (c < n_cols) y[(size_t)(m0 + c) * p.ldy + n] = res[c] + __uint_as_float(r[c]);
-            }
-          } else {
-            const float* rp = static_cast<const float*>(p.resid);
-#pragma unroll
-            for (int c = 0; c < 32; ++c)
-              res[c] = (c < n_cols && n >= 0) ? __ldg(rp + (size_t)(m0 + c) * p.ld_resid + n) : 0.f;
-            tmem_wait_ld();
-            __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(p.dst);
-#pragma unroll
-            for (int c = 0; c < 32; ++c) {
-              const int row = __shfl_sync(0xffffffffu, my_row, c);
-              if (c < n_cols && n >= 0)
-                dst[(size_t)row * p.ld_dst + n] = __float2bfloat16_rn(res[c] + __uint_as_float(r[c]));
-            }
-          }
-        } else if (p.epilogue == QTALE_EPI_SWIGLU) {
-          tmem_wait_ld();
-          // lanes 0-15 hold gate rows, lanes 16-31 the matching up rows
-          float other[16];
-#pragma unroll
-          for (int i = 0; i < 16; ++i)
-            other[i] = __shfl_xor_sync(0xffffffffu,
-                                       __uint_as_float((lane < 16) ? r[16 + i] : r[i]), 16);
-          const int j = nt * 64 + quad * 16 + (lane & 15);
-          if (j < p.F) {
-            unsigned short* y = static_cast<unsigned short*>(p.y);
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-              const int c = (lane < 16) ? i : 16 + i;
-              const float g = (lane < 16) ? __uint_as_float(r[c]) : other[i];
-              const float u = (lane < 16) ? other[i] : __uint_as_float(r[c]);
-              if (c < n_cols)
-                y[(size_t)(m0 + c) * p.ldy + j] = Act16<ACT>::one(g / (1.f + __expf(-g)) * u);
-            }
-          }
-        } else {
-          tmem_wait_ld();
-          if (n >= 0) {
-            if (p.epilogue == QTALE_EPI_STORE_16) {
-              unsigned short* y = static_cast<unsigned short*>(p.y);
-#pragma unroll
-              for (int c = 0; c < 32; ++c)
-                if (c < n_cols) y[(size_t)(m0 + c) * p.ldy + n] = Act16<ACT>::one(__uint_as_float(r[c]));
-            } else {  // QTALE_EPI_STORE_F32
-              float* y = static_cast<float*>(p.y);
-#pragma unroll
-              for (int c = 0; c < 32; ++c)
-                if (c < n_cols) y[(size_t)(m0 + c) * p.ldy + n] = __uint_as_float(r[c]);
-            }
-          }
-        }
+        for (int c = 0; c < 32; ++c) stage[c * kEpiRowWords + lane] = __uint_as_float(r[c]);
+        __syncwarp();
+        epilogue_chunk<ACT>(p, stage, lane, nt, quad, m0, M);
+        __syncwarp();
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&sh.d_empty);
-      dph ^= 1u;
+      if (lane == 0) mbar_arrive(&sh.d_empty[buf]);
     }
   }
 
@@ -475,10 +562,10 @@ static int dispatch_tn(const CUtensorMap& tx, const CUtensorMap& tw, const GemmP
                        cudaStream_t s) {
   if (tn == 64) return launch_gemm<64, BITS, ACT>(tx, tw, p, s);
   if (tn == 128) return launch_gemm<128, BITS, ACT>(tx, tw, p, s);
-  return launch_gemm<256, BITS, ACT>(tx, tw, p, s);
+  return launch_gemm<192, BITS, ACT>(tx, tw, p, s);
 }
 
-static int pick_tn(int M_cap) { return M_cap <= 64 ? 64 : (M_cap <= 128 ? 128 : 256); }
+static int pick_tn(int M_cap) { return M_cap <= 64 ? 64 : (M_cap <= 128 ? 128 : 192); }
 
 size_t wq_blob_bytes(int N, int K, int bits, int group, int row_mode, WqGeometry* g) {
   WqGeometry q;
@@ -681,6 +768,12 @@ int qtale_wq_gemm(const void* a, int lda, const int32_t* m_dev, int M_cap, const
   }
   if (epilogue != QTALE_EPI_RESID_SCATTER && !y) return QTALE_ERR_NULL;
   if (!aligned16(a) || !aligned16(w->packed) || (lda * 2) % 16 != 0) return QTALE_ERR_ALIGN;
+  // the epilogue moves 8 consecutive output features (16 bytes of 16-bit data) per lane
+  if (w->N % 8 != 0 || (w->row_mode == QTALE_WQ_ROWS_SWIGLU && (w->N / 2) % 8 != 0))
+    return QTALE_ERR_SHAPE;
+  if (y && (!aligned16(y) || ldy % 8 != 0)) return QTALE_ERR_ALIGN;
+  if (epi && epi->resid && (!aligned16(epi->resid) || epi->ld_resid % 8 != 0)) return QTALE_ERR_ALIGN;
+  if (epi && epi->dst && (!aligned16(epi->dst) || epi->ld_dst % 8 != 0)) return QTALE_ERR_ALIGN;
   return wq_gemm_launch(a, lda, m_dev, M_cap, w, act_dtype, epilogue, epi, y, ldy,
                         static_cast<cudaStream_t>(stream));
 }
