@@ -229,7 +229,7 @@ typedef struct {
  * y = epilogue(a W^T) on the tensor cores; rows m >= *m_dev (or >= M_cap when
  * m_dev == NULL) are neither computed nor written.
  *   a  act_dtype [M_cap, lda]  (lda >= K elements, lda * 2 bytes % 16 == 0)
- *   y  [M_cap, ldy]; element type set by the epilogue
+ *   y  [M_cap, ldy]; element type set by the epilogue; N % 8 == 0, ldy % 8 == 0
  * The packed weights are dequantised inside the kernel to the 16-bit format of
  * `a` (exact (code - zero) * scale in fp32, one rounding) and accumulated in
  * fp32.

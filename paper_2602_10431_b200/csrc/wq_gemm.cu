@@ -1,24 +1,30 @@
 // Weight-only quantised GEMM on the tcgen05 tensor cores (Sec. 4.1: 4-bit /
 // 3-bit integer weights with per-group parameters; the layer's four linears).
 //
-// The product is computed transposed, D[n, m] = sum_k W[n, k] * A[m, k]:
-//   * the 128 weight rows of a tile are the MMA's M dimension; the packed codes
-//     arrive by bulk TMA copies in a ring of their own, are turned into the 16-bit
-//     activation format in registers ((code - zero) * scale exactly in fp32, one
-//     rounding) and written with tcgen05.st into a ring of tensor-memory slots,
-//     from where the MMA reads its A operand;
-//   * up to 192 tokens are the N dimension; their activations arrive by tiled TMA
-//     loads into a ring of 128-byte-swizzled shared-memory stages (the B operand);
-//   * two fp32 accumulators (128 lanes x TN columns each) live in tensor memory, so
-//     the four epilogue warps drain tile i while the MMAs of tile i+1 run.
-// The three rings (weights, dequantised A slots, activations) are independent, so
-// the dequantisers run ahead of the activation loads instead of lengthening their
+// The product is computed transposed, D[n, m] = sum_k W[n, k] * A[m, k].  One CTA
+// tile is 256 weight rows (two MMA row tiles of 128) x up to 192 tokens:
+//   * the packed codes of both row tiles arrive by bulk TMA copies in a ring of
+//     their own, are turned into the 16-bit activation format in registers
+//     ((code - zero) * scale exactly in fp32, one rounding) and written with
+//     tcgen05.st into a ring of tensor-memory slots, from where the MMAs read
+//     their A operand;
+//   * the tokens' activations arrive by tiled TMA loads into a ring of
+//     128-byte-swizzled shared-memory stages (the B operand).  Both row tiles use
+//     the same stage, which halves the L2 -> SM traffic per flop; with one row
+//     tile per stage the loop is bound by L2 bandwidth (about 72 B/clk/SM), not
+//     by the tensor cores;
+//   * two fp32 accumulators (128 lanes x TN columns, one per row tile) live in
+//     tensor memory and are drained through a transposing shared-memory tile so
+//     that every global access of the epilogue is 16 bytes per lane.
+// The rings (weights, dequantised A slots, activations) are independent, so the
+// dequantisers run ahead of the activation loads instead of lengthening their
 // round trip.  The grid is persistent (one CTA per SM) and reads the number of
 // executed tokens from device memory: no launch parameter depends on the routing.
 //
-// Warp roles (480 threads): warp 0 activation TMA producer, warp 1 MMA issuer and
-// TMEM allocator, warps 2-9 dequantisers (two sets of four that alternate K blocks),
-// warps 10-13 epilogue (one TMEM lane quadrant each), warp 14 weight TMA producer.
+// Warp roles (384 threads): warps 0 and 2 activation TMA producers (even / odd K
+// blocks), warp 1 MMA issuer and TMEM allocator, warp 3 weight TMA producer,
+// warps 4-11 dequantisers and, at the end of a tile, epilogue: set g = 0, 1 (four
+// warps, one TMEM lane quadrant each) owns row tile g.
 #include <cuda.h>
 
 #include <string.h>
@@ -31,8 +37,7 @@ namespace qtale {
 
 using namespace ptx;
 
-constexpr int kGemmThreads = 480;
-constexpr int kDequantGroups = 2;        // two sets of four dequantiser warps alternate K blocks
+constexpr int kGemmThreads = 384;
 constexpr int kTileRows = 128;           // weight rows per tile (MMA M)
 constexpr int kKB = 64;                  // K elements per pipeline step (128 B of 16-bit data)
 constexpr uint32_t kSpinLimit = 1u << 24;
@@ -43,23 +48,25 @@ constexpr int kEpiWarpBytes = 32 * kEpiRowWords * 4;
 
 template <int TN, int BITS>
 struct GemmCfg {
+  static constexpr int kRowTiles = BITS == 16 ? 1 : 2;    // 128-row weight tiles per CTA tile
   static constexpr int kXBytes = TN * 128;
   // with 16-bit weights the weight tile travels with the activations (both from TMA)
   static constexpr int kXStageBytes = kXBytes + (BITS == 16 ? kTileRows * 128 : 0);
   static constexpr int kXStages = BITS == 16 ? 4 : (TN >= 192 ? 6 : 8);
   static constexpr int kWCodeBytes = BITS == 16 ? 0 : kTileRows * kKB * BITS / 8;
   static constexpr int kSzBytes = BITS == 16 ? 0 : kTileRows * 4;
-  static constexpr int kWStageBytes = kWCodeBytes + kSzBytes;
-  static constexpr int kWStages = BITS == 16 ? 0 : 10;
-  static constexpr int kDCols = TN;                       // columns of one accumulator
-  static constexpr int kAColBase = 2 * kDCols;            // A slots follow the two accumulators
-  static constexpr int kASlotsMax = (kTmemCols - kAColBase) / kAColsPerSlot;
-  static constexpr int kASlots = kASlotsMax > 8 ? 8 : kASlotsMax;
+  static constexpr int kWTileBytes = kWCodeBytes + kSzBytes;       // one row tile, one K block
+  static constexpr int kWStageBytes = kRowTiles * kWTileBytes;
+  static constexpr int kWStages = BITS == 16 ? 0 : 4;
+  static constexpr int kDCols = TN;                                // columns of one accumulator
+  static constexpr int kAColBase = kRowTiles * kDCols;             // A slots follow the accumulators
+  static constexpr int kAEntriesMax = (kTmemCols - kAColBase) / (kRowTiles * kAColsPerSlot);
+  static constexpr int kAEntries = kAEntriesMax > 4 ? 4 : kAEntriesMax;  // K blocks of A in flight
   static constexpr size_t kEpiOffset = (size_t)kXStages * kXStageBytes + (size_t)kWStages * kWStageBytes;
-  static constexpr size_t kSmemBytes = kEpiOffset + 4 * kEpiWarpBytes + 1024;
+  static constexpr size_t kSmemBytes = kEpiOffset + 8 * kEpiWarpBytes + 1024;
   static_assert(kXStageBytes % 1024 == 0, "swizzled stages must stay 1024-byte aligned");
-  static_assert(kWStageBytes % 16 == 0, "bulk copies need 16-byte granularity");
-  static_assert(BITS == 16 || kASlots >= 4, "TMEM budget");
+  static_assert(BITS == 16 || kWTileBytes % 16 == 0, "bulk copies need 16-byte granularity");
+  static_assert(BITS == 16 || kAEntries >= 2, "TMEM budget");
   static_assert(kSmemBytes <= 232448 - 512, "shared memory budget");
 };
 
@@ -84,10 +91,10 @@ struct GemmParams {
 };
 
 struct __align__(8) GemmShared {
-  uint64_t full_x[8], empty_x[8];    // activation ring
-  uint64_t full_w[12], empty_w[12];  // packed-weight ring
-  uint64_t a_full[8], a_empty[8];    // dequantised A slots in tensor memory
-  uint64_t d_full[2], d_empty[2];    // the two accumulators
+  uint64_t full_x[8], empty_x[8];  // activation ring
+  uint64_t full_w[8], empty_w[8];  // packed-weight ring
+  uint64_t a_full[8], a_empty[8];  // dequantised A slots in tensor memory, one entry per K block
+  uint64_t d_full, d_empty;        // the accumulators of the CTA tile
   uint32_t tmem_base;
   volatile int abort_flag;
 };
@@ -118,9 +125,13 @@ __device__ __forceinline__ int tile_row_to_n(const GemmParams& p, int nt, int L)
 }
 
 // Eight codes sitting in the 4-bit slots of `t` -> four packed 16-bit pairs.
-// Slot i holds the code in its low QBITS bits.  The code is moved into a float
-// mantissa next to 2^23, so (float - (2^23 + zero * 16^i)) * (scale / 16^i) is
-// exactly (code - zero) * scale.
+// Slot i holds, in its low QBITS bits, the code of input feature 2i (i < 4) or
+// 2(i-4)+1 (i >= 4) of the word's eight features, so slots i and i+4 form the
+// pair that shares a 32-bit TMEM column.
+//
+// Generic path (bf16 output): the code is moved into a float mantissa next to
+// 2^23, so (float - (2^23 + zero * 16^i)) * (scale / 16^i) is exactly
+// (code - zero) * scale in fp32, rounded once.
 template <uint32_t QMASK, int ACT>
 __device__ __forceinline__ void dequant8(uint32_t t, const float (&C)[5], const float (&S)[5],
                                          uint32_t* out) {
@@ -134,7 +145,41 @@ __device__ __forceinline__ void dequant8(uint32_t t, const float (&C)[5], const 
   for (int i = 5; i < 8; ++i)
     v[i] = (__uint_as_float((hi & (QMASK << (4 * (i - 3)))) | MAGIC) - C[i - 3]) * S[i - 3];
 #pragma unroll
-  for (int q = 0; q < 4; ++q) out[q] = Act16<ACT>::pack(v[2 * q], v[2 * q + 1]);
+  for (int q = 0; q < 4; ++q) out[q] = Act16<ACT>::pack(v[q], v[q + 4]);
+}
+
+// fp16 path: two codes at a time in packed half arithmetic.  0x6400 | code is the
+// half 1024 + code (1024 + 16 code for a code in bits 4-7); subtracting 1024 + zero
+// (or one fused multiply-add by 1/16 and -(64 + zero)) leaves the exact integer
+// code - zero, and the product with the fp16 scale is rounded once: the same value
+// as rounding the exact fp32 product.
+__device__ __forceinline__ uint32_t h2_sub(uint32_t a, uint32_t b) {
+  uint32_t r;
+  asm("sub.rn.f16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+  return r;
+}
+__device__ __forceinline__ uint32_t h2_mul(uint32_t a, uint32_t b) {
+  uint32_t r;
+  asm("mul.rn.f16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+  return r;
+}
+__device__ __forceinline__ uint32_t h2_fma(uint32_t a, uint32_t b, uint32_t c) {
+  uint32_t r;
+  asm("fma.rn.f16x2 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(c));
+  return r;
+}
+template <uint32_t QMASK>
+__device__ __forceinline__ void dequant8_f16(uint32_t t, uint32_t z_lo, uint32_t z_hi,
+                                             uint32_t scale2, uint32_t* out) {
+  constexpr uint32_t MAGIC = 0x64006400u;        // (1024, 1024)
+  constexpr uint32_t M0 = QMASK * 0x00010001u;   // codes in bits 0-3 of each half
+  constexpr uint32_t M1 = M0 << 4;               // codes in bits 4-7 of each half
+  constexpr uint32_t SIXTEENTH = 0x2C002C00u;    // (1/16, 1/16)
+  const uint32_t t8 = t >> 8;
+  out[0] = h2_mul(h2_sub((t & M0) | MAGIC, z_lo), scale2);               // slots 0, 4
+  out[1] = h2_mul(h2_fma((t & M1) | MAGIC, SIXTEENTH, z_hi), scale2);    // slots 1, 5
+  out[2] = h2_mul(h2_sub((t8 & M0) | MAGIC, z_lo), scale2);              // slots 2, 6
+  out[3] = h2_mul(h2_fma((t8 & M1) | MAGIC, SIXTEENTH, z_hi), scale2);   // slots 3, 7
 }
 
 struct Ring {
@@ -246,7 +291,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
   using Cfg = GemmCfg<TN, BITS>;
   constexpr int SX = Cfg::kXStages;
   constexpr int SW = Cfg::kWStages;
-  constexpr int SA = Cfg::kASlots;
+  constexpr int SA = Cfg::kAEntries;
+  constexpr int RT = Cfg::kRowTiles;  // weight row tiles (of 128) sharing one activation tile
   extern __shared__ unsigned char smem_dyn[];
   __shared__ GemmShared sh;
   unsigned char* x_base = reinterpret_cast<unsigned char*>(
@@ -261,17 +307,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
     for (int s = 0; s < 8; ++s) {
       mbar_init(&sh.full_x[s], 1);
       mbar_init(&sh.empty_x[s], 1);
-      mbar_init(&sh.a_full[s], 4);
+      mbar_init(&sh.full_w[s], 1);
+      mbar_init(&sh.empty_w[s], 8);
+      mbar_init(&sh.a_full[s], 8);
       mbar_init(&sh.a_empty[s], 1);
     }
-    for (int s = 0; s < 12; ++s) {
-      mbar_init(&sh.full_w[s], 1);
-      mbar_init(&sh.empty_w[s], 4);
-    }
-    for (int s = 0; s < 2; ++s) {
-      mbar_init(&sh.d_full[s], 1);
-      mbar_init(&sh.d_empty[s], 4);
-    }
+    mbar_init(&sh.d_full, 1);
+    mbar_init(&sh.d_empty, 8);
     sh.abort_flag = 0;
     fence_barrier_init();
   }
@@ -292,45 +334,59 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
   if (p.m_dev) M = min(M, *p.m_dev);
   M = max(M, 0);
   const int n_mt = (M + TN - 1) / TN;
-  const int total_tiles = n_mt * p.n_tiles;
+  const int n_rp = (p.n_tiles + RT - 1) / RT;  // groups of RT row tiles
+  const int total_tiles = n_mt * n_rp;
   const int nkb = p.nkb;
 
-  if (warp == 0) {
-    // -------------------------- activation TMA producer --------------------------
+  if (warp == 0 || warp == 2) {
+    // ---------------- activation TMA producers: warp 0 even, warp 2 odd K blocks ----------------
     if (lane == 0) {
+      const int parity = warp >> 1;
       Ring rx;
+      int count = 0;
       for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
-        const int nt = tile / n_mt, mt = tile % n_mt;
-        for (int kb = 0; kb < nkb; ++kb) {
-          if (!wait_or_abort(&sh.empty_x[rx.s], rx.ph ^ 1u, &sh, p.status)) goto x_done;
-          unsigned char* st = x_base + (size_t)rx.s * Cfg::kXStageBytes;
-          mbar_arrive_expect_tx(&sh.full_x[rx.s], Cfg::kXStageBytes);
-          tma_load_2d(st, &tmap_x, &sh.full_x[rx.s], kb * kKB, mt * TN);
-          if (BITS == 16)
-            tma_load_2d(st + Cfg::kXBytes, &tmap_w, &sh.full_x[rx.s], kb * kKB, nt * kTileRows);
+        const int rp = tile / n_mt, mt = tile % n_mt;
+        for (int kb = 0; kb < nkb; ++kb, ++count) {
+          if ((count & 1) == parity) {
+            if (!wait_or_abort(&sh.empty_x[rx.s], rx.ph ^ 1u, &sh, p.status)) goto x_done;
+            unsigned char* st = x_base + (size_t)rx.s * Cfg::kXStageBytes;
+            mbar_arrive_expect_tx(&sh.full_x[rx.s], Cfg::kXStageBytes);
+            tma_load_2d(st, &tmap_x, &sh.full_x[rx.s], kb * kKB, mt * TN);
+            if (BITS == 16)
+              tma_load_2d(st + Cfg::kXBytes, &tmap_w, &sh.full_x[rx.s], kb * kKB, rp * kTileRows);
+          }
           rx.advance(SX);
         }
       }
     x_done:;
     }
-  } else if (warp == 14) {
+  } else if (warp == 3) {
     // ---------------------------- weight TMA producer ----------------------------
     if (BITS != 16 && lane == 0) {
       Ring rw;
       const int ng = nkb / p.kb_per_group;
       for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
-        const int nt = tile / n_mt;
+        const int rp = tile / n_mt;
         for (int kb = 0; kb < nkb; ++kb) {
           if (!wait_or_abort(&sh.empty_w[rw.s], rw.ph ^ 1u, &sh, p.status)) goto w_done;
           unsigned char* st = w_base + (size_t)rw.s * Cfg::kWStageBytes;
-          // every stage carries the scale / zero words of its group
-          mbar_arrive_expect_tx(&sh.full_w[rw.s], Cfg::kWStageBytes);
-          bulk_load(st, p.packed + ((size_t)nt * nkb + kb) * Cfg::kWCodeBytes, Cfg::kWCodeBytes,
-                    &sh.full_w[rw.s]);
-          bulk_load(st + Cfg::kWCodeBytes,
-                    p.packed + p.sz_offset +
-                        ((size_t)nt * ng + kb / p.kb_per_group) * Cfg::kSzBytes,
-                    Cfg::kSzBytes, &sh.full_w[rw.s]);
+          int n_valid = 0;
+#pragma unroll
+          for (int r = 0; r < RT; ++r) n_valid += (rp * RT + r < p.n_tiles);
+          // every stage carries, per row tile, the codes and the scale / zero words of its group
+          mbar_arrive_expect_tx(&sh.full_w[rw.s], n_valid * Cfg::kWTileBytes);
+#pragma unroll
+          for (int r = 0; r < RT; ++r) {
+            const int nt = rp * RT + r;
+            if (nt >= p.n_tiles) continue;
+            unsigned char* d = st + r * Cfg::kWTileBytes;
+            bulk_load(d, p.packed + ((size_t)nt * nkb + kb) * Cfg::kWCodeBytes, Cfg::kWCodeBytes,
+                      &sh.full_w[rw.s]);
+            bulk_load(d + Cfg::kWCodeBytes,
+                      p.packed + p.sz_offset +
+                          ((size_t)nt * ng + kb / p.kb_per_group) * Cfg::kSzBytes,
+                      Cfg::kSzBytes, &sh.full_w[rw.s]);
+          }
           rw.advance(SW);
         }
       }
@@ -341,13 +397,12 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
     if (lane == 0) {
       constexpr uint32_t idesc = idesc_16bit_f32(kTileRows, TN, ACT == 1);
       Ring rx, ra;
-      int it = 0;
-      for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++it) {
-        const int buf = it & 1;
-        const uint32_t dph = (uint32_t)(it >> 1) & 1u;
-        if (!wait_or_abort(&sh.d_empty[buf], dph ^ 1u, &sh, p.status)) goto mma_done;
+      uint32_t dph = 0;
+      for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+        const int rp = tile / n_mt;
+        // the accumulators are free once the previous tile has been drained
+        if (!wait_or_abort(&sh.d_empty, dph ^ 1u, &sh, p.status)) goto mma_done;
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + buf * Cfg::kDCols;
         for (int kb = 0; kb < nkb; ++kb) {
           if (!wait_or_abort(&sh.full_x[rx.s], rx.ph, &sh, p.status)) goto mma_done;
           if (BITS != 16) {
@@ -357,136 +412,153 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
           unsigned char* st = x_base + (size_t)rx.s * Cfg::kXStageBytes;
           const uint64_t b_desc = smem_desc_sw128(smem_u32(st));
 #pragma unroll
-          for (int j = 0; j < kKB / 16; ++j) {
-            const uint32_t acc = (kb | j) != 0 ? 1u : 0u;
-            if (BITS == 16) {
-              const uint64_t a_desc = smem_desc_sw128(smem_u32(st + Cfg::kXBytes));
-              mma_ss(d_tmem, a_desc + 2u * j, b_desc + 2u * j, idesc, acc);
-            } else {
-              mma_ts(d_tmem, tmem_base + Cfg::kAColBase + ra.s * kAColsPerSlot + j * 8,
-                     b_desc + 2u * j, idesc, acc);
+          for (int r = 0; r < RT; ++r) {
+            if (rp * RT + r >= p.n_tiles) continue;
+            const uint32_t d_tmem = tmem_base + r * Cfg::kDCols;
+#pragma unroll
+            for (int j = 0; j < kKB / 16; ++j) {
+              const uint32_t acc = (kb | j) != 0 ? 1u : 0u;
+              if (BITS == 16) {
+                const uint64_t a_desc = smem_desc_sw128(smem_u32(st + Cfg::kXBytes));
+                mma_ss(d_tmem, a_desc + 2u * j, b_desc + 2u * j, idesc, acc);
+              } else {
+                mma_ts(d_tmem,
+                       tmem_base + Cfg::kAColBase + (ra.s * RT + r) * kAColsPerSlot + j * 8,
+                       b_desc + 2u * j, idesc, acc);
+              }
             }
           }
-          mma_commit(&sh.empty_x[rx.s]);             // frees the activation stage
-          if (BITS != 16) mma_commit(&sh.a_empty[ra.s]);  // frees the A slot
+          mma_commit(&sh.empty_x[rx.s]);                   // frees the activation stage
+          if (BITS != 16) mma_commit(&sh.a_empty[ra.s]);   // frees the A slots of this K block
           rx.advance(SX);
           ra.advance(SA);
         }
-        mma_commit(&sh.d_full[buf]);
+        mma_commit(&sh.d_full);
+        dph ^= 1u;
       }
     mma_done:;
     }
-  } else if (warp < 2 + 4 * kDequantGroups) {
-    // ------------------------------- dequantisers --------------------------------
-    if (BITS != 16) {
-      const int quad = warp & 3;
-      const int L = quad * 32 + lane;
-      const int my_group = (warp - 2) >> 2;
-      int turn = 0;  // which set owns the current K block
-      Ring rw, ra;
-      for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+  } else {
+    // ----------- dequantisers, then epilogue: set g (4 warps) owns row tile g of the CTA -----------
+    const int quad = warp & 3;
+    const int L = quad * 32 + lane;
+    const int g = (warp - 4) >> 2;
+    float* stage = epi_base + (size_t)(warp - 4) * (kEpiWarpBytes / 4);
+    Ring rw, ra;
+    uint32_t dph = 0;
+    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+      const int rp = tile / n_mt, mt = tile % n_mt;
+      const int nt = rp * RT + g;
+      const bool has_tile = g < RT && nt < p.n_tiles;
+      if (BITS != 16) {
         for (int kb = 0; kb < nkb; ++kb) {
-          const bool mine = (turn == my_group);
-          if (++turn == kDequantGroups) turn = 0;
-          if (!mine) {
-            rw.advance(SW);
-            ra.advance(SA);
-            continue;
-          }
-          if (!wait_or_abort(&sh.full_w[rw.s], rw.ph, &sh, p.status)) goto dequant_done;
-          const unsigned char* st = w_base + (size_t)rw.s * Cfg::kWStageBytes;
-          // packed codes and the group's scale / zero into registers, then release the stage
-          const uint32_t sz = reinterpret_cast<const uint32_t*>(st + Cfg::kWCodeBytes)[L];
           uint32_t cw[8];
-          if (BITS == 4) {
-            const uint4 w0 = reinterpret_cast<const uint4*>(st)[L];
-            const uint4 w1 = reinterpret_cast<const uint4*>(st)[kTileRows + L];
-            cw[0] = w0.x; cw[1] = w0.y; cw[2] = w0.z; cw[3] = w0.w;
-            cw[4] = w1.x; cw[5] = w1.y; cw[6] = w1.z; cw[7] = w1.w;
-          } else {
-            const uint4 a = reinterpret_cast<const uint4*>(st)[L];
-            const uint2 b = reinterpret_cast<const uint2*>(st + kTileRows * 16)[L];
-            cw[0] = a.x; cw[1] = a.y; cw[2] = a.z; cw[3] = a.w;
-            cw[4] = b.x; cw[5] = b.y; cw[6] = 0; cw[7] = 0;
+          uint32_t sz = 0;
+          // every warp, with or without a tile, takes part in each handshake exactly once
+          if (!wait_or_abort(&sh.full_w[rw.s], rw.ph, &sh, p.status)) goto role_done;
+          if (has_tile) {
+            const unsigned char* st = w_base + (size_t)rw.s * Cfg::kWStageBytes + g * Cfg::kWTileBytes;
+            sz = reinterpret_cast<const uint32_t*>(st + Cfg::kWCodeBytes)[L];
+            if (BITS == 4) {
+              const uint4 w0 = reinterpret_cast<const uint4*>(st)[L];
+              const uint4 w1 = reinterpret_cast<const uint4*>(st)[kTileRows + L];
+              cw[0] = w0.x; cw[1] = w0.y; cw[2] = w0.z; cw[3] = w0.w;
+              cw[4] = w1.x; cw[5] = w1.y; cw[6] = w1.z; cw[7] = w1.w;
+            } else {
+              const uint4 a = reinterpret_cast<const uint4*>(st)[L];
+              const uint2 b = reinterpret_cast<const uint2*>(st + kTileRows * 16)[L];
+              cw[0] = a.x; cw[1] = a.y; cw[2] = a.z; cw[3] = a.w;
+              cw[4] = b.x; cw[5] = b.y; cw[6] = 0; cw[7] = 0;
+            }
           }
           __syncwarp();
           if (lane == 0) mbar_arrive(&sh.empty_w[rw.s]);
-          float C[5], Sc[5];
-          {
-            const float scale = __half2float(__ushort_as_half((unsigned short)(sz & 0xFFFFu)));
-            const float zero = __half2float(__ushort_as_half((unsigned short)(sz >> 16)));
-#pragma unroll
-            for (int i = 0; i < 5; ++i) {
-              C[i] = 8388608.f + zero * (float)(1 << (4 * i));
-              Sc[i] = scale * (1.f / (float)(1 << (4 * i)));
-            }
-          }
-          if (!wait_or_abort(&sh.a_empty[ra.s], ra.ph ^ 1u, &sh, p.status)) goto dequant_done;
-          tc_fence_after();
-          const uint32_t a_taddr =
-              tmem_base + ((uint32_t)(quad * 32) << 16) + Cfg::kAColBase + ra.s * kAColsPerSlot;
-#pragma unroll
-          for (int part = 0; part < 2; ++part) {
-            uint32_t r[16];
-            if (BITS == 4) {
-#pragma unroll
-              for (int j = 0; j < 4; ++j) dequant8<0xFu, ACT>(cw[part * 4 + j], C, Sc, r + 4 * j);
+          if (!wait_or_abort(&sh.a_empty[ra.s], ra.ph ^ 1u, &sh, p.status)) goto role_done;
+          if (has_tile) {
+            float C[5], Sc[5];
+            uint32_t z_lo = 0, z_hi = 0, scale2 = 0;
+            if (ACT == 1) {
+              const uint32_t zero2 = (sz >> 16) * 0x00010001u;          // (zero, zero) as halves
+              scale2 = (sz & 0xFFFFu) * 0x00010001u;
+              z_lo = h2_sub(zero2, 0xE400E400u);                        // zero - (-1024) = 1024 + zero
+              z_hi = h2_sub(0xD400D400u, zero2);                        // -64 - zero
             } else {
-              // 3-bit: low two bits of 16 codes per word (plane A: cw[0..3]), high bit of 32
-              // codes per word (plane B: cw[4..5]).  A nibble-style word with the code in
-              // the low 3 bits of each 4-bit slot is assembled with one bitwise select.
+              const float scale = __half2float(__ushort_as_half((unsigned short)(sz & 0xFFFFu)));
+              const float zero = __half2float(__ushort_as_half((unsigned short)(sz >> 16)));
 #pragma unroll
-              for (int uu = 0; uu < 4; ++uu) {
-                const int u = part * 4 + uu;
-                const uint32_t a2 = (u & 1) ? (cw[u >> 1] >> 2) : cw[u >> 1];
-                const int rr = u & 3;
-                const uint32_t bw = cw[4 + (u >> 2)];
-                const uint32_t b1 = rr == 0 ? (bw << 2) : rr == 1 ? (bw << 1) : rr == 2 ? bw : (bw >> 1);
-                const uint32_t t = (a2 & 0x33333333u) | (b1 & 0xCCCCCCCCu);
-                dequant8<0x7u, ACT>(t, C, Sc, r + 4 * uu);
+              for (int i = 0; i < 5; ++i) {
+                C[i] = 8388608.f + zero * (float)(1 << (4 * i));
+                Sc[i] = scale * (1.f / (float)(1 << (4 * i)));
               }
             }
-            tmem_st_x16(a_taddr + part * 16, r);
+            tc_fence_after();
+            const uint32_t a_taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + Cfg::kAColBase +
+                                     (ra.s * RT + g) * kAColsPerSlot;
+#pragma unroll
+            for (int part = 0; part < 2; ++part) {
+              uint32_t r[16];
+              if (BITS == 4) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                  if (ACT == 1) dequant8_f16<0xFu>(cw[part * 4 + j], z_lo, z_hi, scale2, r + 4 * j);
+                  else dequant8<0xFu, ACT>(cw[part * 4 + j], C, Sc, r + 4 * j);
+                }
+              } else {
+                // 3-bit: low two bits of 16 codes per word (plane A: cw[0..3]), high bit of 32
+                // codes per word (plane B: cw[4..5]).  A nibble-style word with the code in
+                // the low 3 bits of each 4-bit slot is assembled with one bitwise select.
+#pragma unroll
+                for (int uu = 0; uu < 4; ++uu) {
+                  const int u = part * 4 + uu;
+                  const uint32_t a2 = (u & 1) ? (cw[u >> 1] >> 2) : cw[u >> 1];
+                  const int rr = u & 3;
+                  const uint32_t bw = cw[4 + (u >> 2)];
+                  const uint32_t b1 = rr == 0 ? (bw << 2) : rr == 1 ? (bw << 1) : rr == 2 ? bw : (bw >> 1);
+                  const uint32_t t = (a2 & 0x33333333u) | (b1 & 0xCCCCCCCCu);
+                  if (ACT == 1) dequant8_f16<0x7u>(t, z_lo, z_hi, scale2, r + 4 * uu);
+                  else dequant8<0x7u, ACT>(t, C, Sc, r + 4 * uu);
+                }
+              }
+              tmem_st_x16(a_taddr + part * 16, r);
+            }
+            tmem_wait_st();
+            tc_fence_before();
           }
-          tmem_wait_st();
-          tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(&sh.a_full[ra.s]);
           rw.advance(SW);
           ra.advance(SA);
         }
       }
-    dequant_done:;
-    }
-  } else if (warp < 14) {
-    // --------------------------------- epilogue -----------------------------------
-    const int quad = warp & 3;
-    float* stage = epi_base + (size_t)(warp - 10) * (kEpiWarpBytes / 4);
-    int it = 0;
-    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++it) {
-      const int nt = tile / n_mt, mt = tile % n_mt;
-      const int buf = it & 1;
-      const uint32_t dph = (uint32_t)(it >> 1) & 1u;
-      if (!wait_or_abort(&sh.d_full[buf], dph, &sh, p.status)) break;
+      // ---- epilogue of this tile: set g drains accumulator g, one lane quadrant per warp ----
+      if (!wait_or_abort(&sh.d_full, dph, &sh, p.status)) goto role_done;
       tc_fence_after();
-      const int m_base = mt * TN;
-#pragma unroll 1
-      for (int c0 = 0; c0 < TN; c0 += 32) {
-        const int m0 = m_base + c0;
-        if (m0 >= M) break;
+      if (has_tile) {
+        const int m_base = mt * TN;
+        const uint32_t d_taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + g * Cfg::kDCols;
         uint32_t r[32];
-        tmem_ld_x32(tmem_base + ((uint32_t)(quad * 32) << 16) + buf * Cfg::kDCols + c0, r);
-        tmem_wait_ld();
+        tmem_ld_x32(d_taddr, r);
+#pragma unroll 1
+        for (int c0 = 0; c0 < TN; c0 += 32) {
+          const int m0 = m_base + c0;
+          if (m0 >= M) break;
+          tmem_wait_ld();
 #pragma unroll
-        for (int c = 0; c < 32; ++c) stage[c * kEpiRowWords + lane] = __uint_as_float(r[c]);
-        __syncwarp();
-        epilogue_chunk<ACT>(p, stage, lane, nt, quad, m0, M);
-        __syncwarp();
+          for (int c = 0; c < 32; ++c) stage[c * kEpiRowWords + lane] = __uint_as_float(r[c]);
+          __syncwarp();
+          // the next chunk's accumulator read overlaps this chunk's global traffic
+          if (c0 + 32 < TN && m0 + 32 < M) tmem_ld_x32(d_taddr + c0 + 32, r);
+          epilogue_chunk<ACT>(p, stage, lane, nt, quad, m0, M);
+          __syncwarp();
+        }
+        tmem_wait_ld();
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&sh.d_empty[buf]);
+      if (lane == 0) mbar_arrive(&sh.d_empty);
+      dph ^= 1u;
     }
+  role_done:;
   }
 
   // teardown: every thread arrives here, also after an abort
@@ -549,7 +621,7 @@ static int launch_gemm(const CUtensorMap& tx, const CUtensorMap& tw, const GemmP
       return QTALE_ERR_CUDA;
     configured[dev] = true;
   }
-  const int max_tiles = ((p.M_cap + TN - 1) / TN) * p.n_tiles;
+  const int max_tiles = ((p.M_cap + TN - 1) / TN) * ((p.n_tiles + Cfg::kRowTiles - 1) / Cfg::kRowTiles);
   int grid = sm_count();
   if (grid > max_tiles) grid = max_tiles;
   if (grid < 1) grid = 1;
@@ -717,30 +789,34 @@ int qtale_wq_repack(const uint8_t* codes, const uint16_t* scales, const uint16_t
             q[i] = (unsigned)z;
           }
         }
+        // slot i of an 8-code word holds feature 2i (i < 4) or 2(i-4)+1 (i >= 4) of the word
+        auto slot_k = [](int i) { return i < 4 ? 2 * i : 2 * (i - 4) + 1; };
         if (bits == 4) {
-          // [part][lane][4 words]; word j of part p: k = 32p + 8j + i in nibble i
+          // [part][lane][4 words]; word j of part p covers k = 32p + 8j .. +7, slot i in nibble i
           for (int part = 0; part < 2; ++part) {
             uint32_t* wdst = reinterpret_cast<uint32_t*>(blk) + ((size_t)part * kTileRows + L) * 4;
             for (int j = 0; j < 4; ++j) {
               uint32_t wv = 0;
-              for (int i = 0; i < 8; ++i) wv |= (q[32 * part + 8 * j + i] & 0xFu) << (4 * i);
+              for (int i = 0; i < 8; ++i) wv |= (q[32 * part + 8 * j + slot_k(i)] & 0xFu) << (4 * i);
               wdst[j] = wv;
             }
           }
         } else {
-          // plane A: [lane][4 words], 2-bit field f of word w2 <- code k = 8(2 w2 + f%2) + f/2
-          // plane B: [lane][2 words], bit 4i + u%4 of word u/4 <- high bit of code 8u + i
+          // plane A: [lane][4 words], 2-bit field f of word w2 <- low bits of slot f/2 of word
+          //          u = 2 w2 + f%2;  plane B: [lane][2 words], bit 4i + u%4 of word u/4 <- high
+          //          bit of slot i of word u
           uint32_t* a = reinterpret_cast<uint32_t*>(blk) + (size_t)L * 4;
           uint32_t* b = reinterpret_cast<uint32_t*>(blk + kTileRows * 16) + (size_t)L * 2;
           for (int w2 = 0; w2 < 4; ++w2) {
             uint32_t wv = 0;
-            for (int f = 0; f < 16; ++f) wv |= (q[8 * (2 * w2 + (f & 1)) + (f >> 1)] & 3u) << (2 * f);
+            for (int f = 0; f < 16; ++f)
+              wv |= (q[8 * (2 * w2 + (f & 1)) + slot_k(f >> 1)] & 3u) << (2 * f);
             a[w2] = wv;
           }
           uint32_t b0 = 0, b1 = 0;
           for (int u = 0; u < 8; ++u)
             for (int i = 0; i < 8; ++i) {
-              const uint32_t hb = (q[8 * u + i] >> 2) & 1u;
+              const uint32_t hb = (q[8 * u + slot_k(i)] >> 2) & 1u;
               if (u < 4) b0 |= hb << (4 * i + (u & 3)); else b1 |= hb << (4 * i + (u & 3));
             }
           b[0] = b0;
