@@ -70,6 +70,11 @@ struct GemmCfg {
   static_assert(kSmemBytes <= 232448 - 512, "shared memory budget");
 };
 
+// Activation tensor maps for token tiles of 32, 64, ... , 192 rows (index w / 32 - 1).
+struct TmapSet {
+  CUtensorMap m[6];
+};
+
 struct GemmParams {
   const uint8_t* packed;   // repacked blob (codes, then scale/zero words)
   size_t sz_offset;        // byte offset of the scale/zero region
@@ -286,7 +291,7 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const float*
 
 template <int TN, int BITS, int ACT>
 __global__ void __launch_bounds__(kGemmThreads, 1)
-    wq_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x,
+    wq_gemm_kernel(const __grid_constant__ TmapSet tmaps_x,
                    const __grid_constant__ CUtensorMap tmap_w, const GemmParams p) {
   using Cfg = GemmCfg<TN, BITS>;
   constexpr int SX = Cfg::kXStages;
@@ -322,7 +327,6 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
     tmem_relinquish();
   }
   if (warp == 0 && lane == 0) {
-    prefetch_tmap(&tmap_x);
     if (BITS == 16) prefetch_tmap(&tmap_w);
   }
   tc_fence_before();
@@ -333,10 +337,29 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
   int M = p.M_cap;
   if (p.m_dev) M = min(M, *p.m_dev);
   M = max(M, 0);
-  const int n_mt = (M + TN - 1) / TN;
   const int n_rp = (p.n_tiles + RT - 1) / RT;  // groups of RT row tiles
-  const int total_tiles = n_mt * n_rp;
   const int nkb = p.nkb;
+  // Token-tile width: the multiple of 32 (at most TN) that minimises
+  // (waves of the persistent grid) x (columns per tile + fixed per-tile cost), so
+  // that a tile count just above a multiple of the grid does not cost a whole wave.
+  int TW = TN;
+  {
+    // per-tile time in columns of MMA work: the K loop costs max(w, 128) per block (below
+    // about 128 tokens the dequantisers, not the MMAs, set the pace) plus epilogue / restart
+    const int fixed = 1408 / max(nkb, 1);
+    long best = -1;
+    for (int w = TN; w >= 32; w -= 32) {
+      const long tiles = (long)((M + w - 1) / w) * n_rp;
+      const long cost = ((tiles + gridDim.x - 1) / gridDim.x) * (max(w, 128) + fixed);
+      if (best < 0 || cost < best) { best = cost; TW = w; }
+    }
+  }
+  const CUtensorMap* tmap_x = &tmaps_x.m[TW / 32 - 1];
+  // tile index = mt * n_rp + rp: CTAs running at the same time share a few token tiles and
+  // sweep the (small, L2-resident) packed weights, so activations stream from HBM once
+  const int n_mt = (M + TW - 1) / TW;
+  const int total_tiles = n_mt * n_rp;
+  const uint32_t x_stage_tx = (uint32_t)TW * 128u + (BITS == 16 ? kTileRows * 128 : 0);
 
   if (warp == 0 || warp == 2) {
     // ---------------- activation TMA producers: warp 0 even, warp 2 odd K blocks ----------------
@@ -345,13 +368,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
       Ring rx;
       int count = 0;
       for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
-        const int rp = tile / n_mt, mt = tile % n_mt;
+        const int rp = tile % n_rp, mt = tile / n_rp;
         for (int kb = 0; kb < nkb; ++kb, ++count) {
           if ((count & 1) == parity) {
             if (!wait_or_abort(&sh.empty_x[rx.s], rx.ph ^ 1u, &sh, p.status)) goto x_done;
             unsigned char* st = x_base + (size_t)rx.s * Cfg::kXStageBytes;
-            mbar_arrive_expect_tx(&sh.full_x[rx.s], Cfg::kXStageBytes);
-            tma_load_2d(st, &tmap_x, &sh.full_x[rx.s], kb * kKB, mt * TN);
+            mbar_arrive_expect_tx(&sh.full_x[rx.s], x_stage_tx);
+            tma_load_2d(st, tmap_x, &sh.full_x[rx.s], kb * kKB, mt * TW);
             if (BITS == 16)
               tma_load_2d(st + Cfg::kXBytes, &tmap_w, &sh.full_x[rx.s], kb * kKB, rp * kTileRows);
           }
@@ -364,29 +387,16 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
     // ---------------------------- weight TMA producer ----------------------------
     if (BITS != 16 && lane == 0) {
       Ring rw;
-      const int ng = nkb / p.kb_per_group;
       for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
-        const int rp = tile / n_mt;
+        const int rp = tile % n_rp;
         for (int kb = 0; kb < nkb; ++kb) {
           if (!wait_or_abort(&sh.empty_w[rw.s], rw.ph ^ 1u, &sh, p.status)) goto w_done;
           unsigned char* st = w_base + (size_t)rw.s * Cfg::kWStageBytes;
-          int n_valid = 0;
-#pragma unroll
-          for (int r = 0; r < RT; ++r) n_valid += (rp * RT + r < p.n_tiles);
-          // every stage carries, per row tile, the codes and the scale / zero words of its group
-          mbar_arrive_expect_tx(&sh.full_w[rw.s], n_valid * Cfg::kWTileBytes);
-#pragma unroll
-          for (int r = 0; r < RT; ++r) {
-            const int nt = rp * RT + r;
-            if (nt >= p.n_tiles) continue;
-            unsigned char* d = st + r * Cfg::kWTileBytes;
-            bulk_load(d, p.packed + ((size_t)nt * nkb + kb) * Cfg::kWCodeBytes, Cfg::kWCodeBytes,
-                      &sh.full_w[rw.s]);
-            bulk_load(d + Cfg::kWCodeBytes,
-                      p.packed + p.sz_offset +
-                          ((size_t)nt * ng + kb / p.kb_per_group) * Cfg::kSzBytes,
-                      Cfg::kSzBytes, &sh.full_w[rw.s]);
-          }
+          // one contiguous chunk per (row-tile pair, K block): both tiles' codes, each
+          // followed by the scale / zero words of its group
+          mbar_arrive_expect_tx(&sh.full_w[rw.s], Cfg::kWStageBytes);
+          bulk_load(st, p.packed + ((size_t)rp * nkb + kb) * Cfg::kWStageBytes, Cfg::kWStageBytes,
+                    &sh.full_w[rw.s]);
           rw.advance(SW);
         }
       }
@@ -395,11 +405,11 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
   } else if (warp == 1) {
     // ------------------------------- MMA issuer --------------------------------
     if (lane == 0) {
-      constexpr uint32_t idesc = idesc_16bit_f32(kTileRows, TN, ACT == 1);
+      const uint32_t idesc = idesc_16bit_f32(kTileRows, TW, ACT == 1);
       Ring rx, ra;
       uint32_t dph = 0;
       for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
-        const int rp = tile / n_mt;
+        const int rp = tile % n_rp;
         // the accumulators are free once the previous tile has been drained
         if (!wait_or_abort(&sh.d_empty, dph ^ 1u, &sh, p.status)) goto mma_done;
         tc_fence_after();
@@ -447,7 +457,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
     Ring rw, ra;
     uint32_t dph = 0;
     for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
-      const int rp = tile / n_mt, mt = tile % n_mt;
+      const int rp = tile % n_rp, mt = tile / n_rp;
       const int nt = rp * RT + g;
       const bool has_tile = g < RT && nt < p.n_tiles;
       if (BITS != 16) {
@@ -473,7 +483,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
           }
           __syncwarp();
           if (lane == 0) mbar_arrive(&sh.empty_w[rw.s]);
-          if (!wait_or_abort(&sh.a_empty[ra.s], ra.ph ^ 1u, &sh, p.status)) goto role_done;
+          // dequantise into registers first; only the TMEM stores wait for the free A slot
+          uint32_t r[32];
           if (has_tile) {
             float C[5], Sc[5];
             uint32_t z_lo = 0, z_hi = 0, scale2 = 0;
@@ -491,36 +502,32 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
                 Sc[i] = scale * (1.f / (float)(1 << (4 * i)));
               }
             }
-            tc_fence_after();
-            const uint32_t a_taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + Cfg::kAColBase +
-                                     (ra.s * RT + g) * kAColsPerSlot;
 #pragma unroll
-            for (int part = 0; part < 2; ++part) {
-              uint32_t r[16];
+            for (int u = 0; u < 8; ++u) {
+              uint32_t t;
               if (BITS == 4) {
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                  if (ACT == 1) dequant8_f16<0xFu>(cw[part * 4 + j], z_lo, z_hi, scale2, r + 4 * j);
-                  else dequant8<0xFu, ACT>(cw[part * 4 + j], C, Sc, r + 4 * j);
-                }
+                t = cw[u];
               } else {
                 // 3-bit: low two bits of 16 codes per word (plane A: cw[0..3]), high bit of 32
                 // codes per word (plane B: cw[4..5]).  A nibble-style word with the code in
                 // the low 3 bits of each 4-bit slot is assembled with one bitwise select.
-#pragma unroll
-                for (int uu = 0; uu < 4; ++uu) {
-                  const int u = part * 4 + uu;
-                  const uint32_t a2 = (u & 1) ? (cw[u >> 1] >> 2) : cw[u >> 1];
-                  const int rr = u & 3;
-                  const uint32_t bw = cw[4 + (u >> 2)];
-                  const uint32_t b1 = rr == 0 ? (bw << 2) : rr == 1 ? (bw << 1) : rr == 2 ? bw : (bw >> 1);
-                  const uint32_t t = (a2 & 0x33333333u) | (b1 & 0xCCCCCCCCu);
-                  if (ACT == 1) dequant8_f16<0x7u>(t, z_lo, z_hi, scale2, r + 4 * uu);
-                  else dequant8<0x7u, ACT>(t, C, Sc, r + 4 * uu);
-                }
+                const uint32_t a2 = (u & 1) ? (cw[u >> 1] >> 2) : cw[u >> 1];
+                const int rr = u & 3;
+                const uint32_t bw = cw[4 + (u >> 2)];
+                const uint32_t b1 = rr == 0 ? (bw << 2) : rr == 1 ? (bw << 1) : rr == 2 ? bw : (bw >> 1);
+                t = (a2 & 0x33333333u) | (b1 & 0xCCCCCCCCu);
               }
-              tmem_st_x16(a_taddr + part * 16, r);
+              constexpr uint32_t QM = BITS == 4 ? 0xFu : 0x7u;
+              if (ACT == 1) dequant8_f16<QM>(t, z_lo, z_hi, scale2, r + 4 * u);
+              else dequant8<QM, ACT>(t, C, Sc, r + 4 * u);
             }
+          }
+          if (!wait_or_abort(&sh.a_empty[ra.s], ra.ph ^ 1u, &sh, p.status)) goto role_done;
+          if (has_tile) {
+            tc_fence_after();
+            const uint32_t a_taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + Cfg::kAColBase +
+                                     (ra.s * RT + g) * kAColsPerSlot;
+            tmem_st_x32(a_taddr, r);
             tmem_wait_st();
             tc_fence_before();
           }
@@ -534,12 +541,12 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
       if (!wait_or_abort(&sh.d_full, dph, &sh, p.status)) goto role_done;
       tc_fence_after();
       if (has_tile) {
-        const int m_base = mt * TN;
+        const int m_base = mt * TW;
         const uint32_t d_taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + g * Cfg::kDCols;
         uint32_t r[32];
         tmem_ld_x32(d_taddr, r);
 #pragma unroll 1
-        for (int c0 = 0; c0 < TN; c0 += 32) {
+        for (int c0 = 0; c0 < TW; c0 += 32) {
           const int m0 = m_base + c0;
           if (m0 >= M) break;
           tmem_wait_ld();
@@ -547,7 +554,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
           for (int c = 0; c < 32; ++c) stage[c * kEpiRowWords + lane] = __uint_as_float(r[c]);
           __syncwarp();
           // the next chunk's accumulator read overlaps this chunk's global traffic
-          if (c0 + 32 < TN && m0 + 32 < M) tmem_ld_x32(d_taddr + c0 + 32, r);
+          if (c0 + 32 < TW && m0 + 32 < M) tmem_ld_x32(d_taddr + c0 + 32, r);
           epilogue_chunk<ACT>(p, stage, lane, nt, quad, m0, M);
           __syncwarp();
         }
@@ -608,8 +615,18 @@ static int make_tmap_16(CUtensorMap* m, const void* base, int rows, int cols, in
   return r == CUDA_SUCCESS ? QTALE_OK : QTALE_ERR_CUDA;
 }
 
+// tensor maps for every token-tile width (multiples of 32) up to tn
+static int make_tmap_set(TmapSet* set, const void* base, int rows, int cols, int ld, int tn,
+                         int act) {
+  for (int w = 32; w <= tn; w += 32) {
+    const int rc = make_tmap_16(&set->m[w / 32 - 1], base, rows, cols, ld, w, act);
+    if (rc != QTALE_OK) return rc;
+  }
+  return QTALE_OK;
+}
+
 template <int TN, int BITS, int ACT>
-static int launch_gemm(const CUtensorMap& tx, const CUtensorMap& tw, const GemmParams& p,
+static int launch_gemm(const TmapSet& tx, const CUtensorMap& tw, const GemmParams& p,
                        cudaStream_t s) {
   using Cfg = GemmCfg<TN, BITS>;
   static bool configured[64] = {false};
@@ -621,7 +638,7 @@ static int launch_gemm(const CUtensorMap& tx, const CUtensorMap& tw, const GemmP
       return QTALE_ERR_CUDA;
     configured[dev] = true;
   }
-  const int max_tiles = ((p.M_cap + TN - 1) / TN) * ((p.n_tiles + Cfg::kRowTiles - 1) / Cfg::kRowTiles);
+  const int max_tiles = ((p.M_cap + 31) / 32) * ((p.n_tiles + Cfg::kRowTiles - 1) / Cfg::kRowTiles);
   int grid = sm_count();
   if (grid > max_tiles) grid = max_tiles;
   if (grid < 1) grid = 1;
@@ -630,7 +647,7 @@ static int launch_gemm(const CUtensorMap& tx, const CUtensorMap& tw, const GemmP
 }
 
 template <int BITS, int ACT>
-static int dispatch_tn(const CUtensorMap& tx, const CUtensorMap& tw, const GemmParams& p, int tn,
+static int dispatch_tn(const TmapSet& tx, const CUtensorMap& tw, const GemmParams& p, int tn,
                        cudaStream_t s) {
   if (tn == 64) return launch_gemm<64, BITS, ACT>(tx, tw, p, s);
   if (tn == 128) return launch_gemm<128, BITS, ACT>(tx, tw, p, s);
@@ -646,8 +663,10 @@ size_t wq_blob_bytes(int N, int K, int bits, int group, int row_mode, WqGeometry
   q.ng = q.K_pad / group;
   q.n_tiles = row_mode == QTALE_WQ_ROWS_SWIGLU ? ((N / 2) + 63) / 64 : (N + kTileRows - 1) / kTileRows;
   q.block_bytes = kTileRows * kKB * bits / 8;
-  q.sz_offset = (size_t)q.n_tiles * q.nkb * q.block_bytes;
-  q.total = q.sz_offset + (size_t)q.n_tiles * q.ng * kTileRows * 4;
+  q.tile_bytes = q.block_bytes + kTileRows * 4;  // codes + (scale, zero) words of one row tile, one K block
+  q.n_rp = (q.n_tiles + 1) / 2;                  // row tiles are stored in pairs
+  q.sz_offset = 0;
+  q.total = (size_t)q.n_rp * q.nkb * 2 * q.tile_bytes;
   if (g) *g = q;
   return q.total;
 }
@@ -681,9 +700,11 @@ int wq_gemm_launch(const void* a, int lda, const int32_t* m_dev, int M_cap,
   }
   p.status = device_status_ptr();
   const int tn = pick_tn(M_cap);
-  CUtensorMap tx, tw;
+  TmapSet tx;
+  CUtensorMap tw;
+  memset(&tx, 0, sizeof(tx));
   memset(&tw, 0, sizeof(tw));
-  int rc = make_tmap_16(&tx, a, M_cap, w->K, lda, tn, act);
+  int rc = make_tmap_set(&tx, a, M_cap, w->K, lda, tn, act);
   if (rc != QTALE_OK) return rc;
   if (act == QTALE_ACT_F16)
     return w->bits == 4 ? dispatch_tn<4, 1>(tx, tw, p, tn, s) : dispatch_tn<3, 1>(tx, tw, p, tn, s);
@@ -706,8 +727,10 @@ int bf16_gemm_launch(const void* a, int lda, const int32_t* m_dev, int M_cap, co
   p.ldy = ldy;
   p.status = device_status_ptr();
   const int tn = pick_tn(M_cap);
-  CUtensorMap tx, tw;
-  int rc = make_tmap_16(&tx, a, M_cap, K, lda, tn, QTALE_ACT_BF16);
+  TmapSet tx;
+  CUtensorMap tw;
+  memset(&tx, 0, sizeof(tx));
+  int rc = make_tmap_set(&tx, a, M_cap, K, lda, tn, QTALE_ACT_BF16);
   if (rc != QTALE_OK) return rc;
   rc = make_tmap_16(&tw, w_bf16, N, K, ldw, kTileRows, QTALE_ACT_BF16);
   if (rc != QTALE_OK) return rc;
@@ -767,17 +790,21 @@ int qtale_wq_repack(const uint8_t* codes, const uint16_t* scales, const uint16_t
         n = nt * kTileRows + L;
         if (n >= N) n = -1;
       }
-      uint32_t* sz = reinterpret_cast<uint32_t*>(out + g.sz_offset) + (size_t)nt * g.ng * kTileRows;
-      for (int gi = 0; gi < g.ng; ++gi) {
-        uint32_t v = 0;  // padding rows: scale 0, zero 0
-        if (n >= 0 && gi < ng_in)
+      // chunk of (pair nt/2, K block kb): [tile nt%2]{codes, 128 (scale | zero << 16) words}
+      auto chunk = [&](int kb) {
+        return out + (((size_t)(nt >> 1) * g.nkb + kb) * 2 + (nt & 1)) * g.tile_bytes;
+      };
+      if (n < 0) continue;  // padding rows keep scale 0, zero 0, codes 0
+      for (int kb = 0; kb < g.nkb; ++kb) {
+        const int gi = kb * kKB / group;
+        uint32_t v = 0;
+        if (gi < ng_in)
           v = (uint32_t)scales[(size_t)n * ng_in + gi] | ((uint32_t)zeros[(size_t)n * ng_in + gi] << 16);
-        sz[(size_t)gi * kTileRows + L] = v;
+        reinterpret_cast<uint32_t*>(chunk(kb) + g.block_bytes)[L] = v;
       }
-      if (n < 0) continue;
       const uint8_t* row = codes + (size_t)n * row_bytes;
       for (int kb = 0; kb < g.nkb; ++kb) {
-        uint8_t* blk = out + ((size_t)nt * g.nkb + kb) * g.block_bytes;
+        uint8_t* blk = chunk(kb);
         unsigned q[64];
         for (int i = 0; i < 64; ++i) {
           const int k = kb * 64 + i;

@@ -10,7 +10,9 @@ struct WqGeometry {
   int ng;             // groups per row
   int n_tiles;        // 128-row tiles
   int block_bytes;    // code bytes of one (tile, K block)
-  size_t sz_offset;   // start of the scale / zero-point words
+  int tile_bytes;     // codes + scale / zero words of one (tile, K block)
+  int n_rp;           // pairs of row tiles
+  size_t sz_offset;   // unused (scale / zero words travel with the codes)
   size_t total;       // blob size in bytes
 };
 
