@@ -87,8 +87,9 @@ size_t qtale_router_select_workspace_bytes(int T);
  * Score (Eq. 9 specialised to a linear two-class router): the router emits
  * two class logits (g0 execute, g1 bypass); with a linear router their
  * difference is z_t = w_router . x_t + bias and softmax([g0,g1])[0] =
- * 1 / (1 + exp(-z_t)).  The dot product accumulates in fp64; the score is
- * stored as fp32.  If scores_override != NULL the router is skipped and those
+ * 1 / (1 + exp(-z_t)).  The dot product is formed from fp32 partial sums of 8
+ * products accumulated in fp64 (within about 1e-8 of an all-fp64 sum); the
+ * logistic is evaluated in fp64 and the score is stored as fp32.  If scores_override != NULL the router is skipped and those
  * scores are used (and copied to scores_out).
  *
  * Decision: THRESHOLD: execute iff score >= theta (fp32 compare, ties

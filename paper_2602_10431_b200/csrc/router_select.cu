@@ -41,66 +41,129 @@ __device__ void select_and_compact(const RouterParams& p, uint32_t* sh_hist, int
   const int nthr = blockDim.x;
   const int T = p.T;
   __shared__ uint32_t s_prefix, s_mask;
-  __shared__ int s_remaining, s_need_eq, s_total;
+  __shared__ int s_remaining, s_total, s_bucket, s_new_remaining;
 
   uint32_t tau = 0;  // key of the k-th largest score (top-k)
   int need_eq = 0;   // how many tokens with key == tau execute (lowest indices first)
 
   if (p.mode == QTALE_SELECT_TOPK) {
-    // MSB-first radix select of the k-th largest key among valid tokens.
+    // MSB-first radix select of the k-th largest key among valid tokens.  Keys are read
+    // in batches of kBatch independent loads per thread (token t = (batch*kBatch + j) * nthr
+    // + tid); when a thread's share fits one batch it is read once and kept in registers.
+    constexpr int kBatch = 16;
+    constexpr uint32_t kInvalid = 0u;  // key 0 is below every real key (those have a set bit)
     if (tid == 0) {
       s_prefix = 0;
       s_mask = 0;
       s_remaining = p.k;
     }
+    const int per = (T + nthr - 1) / nthr;
+    const int n_batches = (per + kBatch - 1) / kBatch;
+    uint32_t keys[kBatch];
+    auto load_batch = [&](int bi) {
+#pragma unroll
+      for (int j = 0; j < kBatch; ++j) {
+        const int t = (bi * kBatch + j) * nthr + tid;
+        float sc = 0.f;
+        bool ok = t < T;
+        if (ok) sc = __ldcg(p.scores + t);
+        if (ok && p.valid) ok = p.valid[t] != 0;
+        keys[j] = ok ? score_key(sc) : kInvalid;
+      }
+    };
+    if (n_batches == 1) load_batch(0);
     __syncthreads();
     for (int pass = 0; pass < 4 && p.k > 0; ++pass) {
       const int shift = 24 - 8 * pass;
       for (int i = tid; i < 256; i += nthr) sh_hist[i] = 0;
+      if (tid == 0) {  // defaults if k exceeds the number of valid tokens: lowest bucket
+        s_bucket = 0;
+        s_new_remaining = s_remaining;
+      }
       __syncthreads();
       const uint32_t prefix = s_prefix, mask = s_mask;
-      for (int t = tid; t < T; t += nthr) {
-        if (p.valid && !p.valid[t]) continue;
-        uint32_t key = score_key(__ldcg(p.scores + t));
-        if ((key & mask) == prefix) {
+      for (int bi = 0; bi < n_batches; ++bi) {
+        if (n_batches > 1) load_batch(bi);
+#pragma unroll
+        for (int j = 0; j < kBatch; ++j) {
+          const uint32_t key = keys[j];
+          const bool in = key != kInvalid && (key & mask) == prefix;
           // scores cluster in a few buckets: one atomic per distinct bucket per warp
-          const uint32_t bucket = (key >> shift) & 0xFF;
-          const uint32_t peers = __match_any_sync(__activemask(), bucket);
-          if ((int)(__ffs(peers) - 1) == (threadIdx.x & 31)) atomicAdd(&sh_hist[bucket], __popc(peers));
+          const uint32_t bucket = in ? ((key >> shift) & 0xFF) : 256u;
+          const uint32_t peers = __match_any_sync(0xffffffffu, bucket);
+          if (in && (int)(__ffs(peers) - 1) == (tid & 31)) atomicAdd(&sh_hist[bucket], __popc(peers));
         }
       }
       __syncthreads();
-      if (tid == 0) {
-        int rem = s_remaining;
-        int b = 255;
-        for (; b > 0; --b) {
-          int c = (int)sh_hist[b];
-          if (c >= rem) break;
-          rem -= c;
+      // bucket holding the target: suffix sums over the 256 buckets, one bucket per thread
+      {
+        const int lane = tid & 31, wid = tid >> 5;
+        int h = 0, inc = 0;
+        if (tid < 256) {
+          h = (int)sh_hist[255 - tid];  // descending bucket order
+          inc = h;
+#pragma unroll
+          for (int o = 1; o < 32; o <<= 1) {
+            const int n = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o) inc += n;
+          }
+          if (lane == 31) sh_scan[wid] = inc;
         }
-        s_remaining = rem;  // rank of the target inside bucket b (1-based)
-        s_prefix = prefix | ((uint32_t)b << shift);
-        s_mask = mask | (0xFFu << shift);
+        __syncthreads();
+        if (tid < 256) {
+          int before = 0;
+          for (int w = 0; w < wid; ++w) before += sh_scan[w];
+          inc += before;
+          const int rem = s_remaining;
+          if (inc >= rem && inc - h < rem) {  // exactly one thread (bucket counts are >= 0)
+            s_bucket = 255 - tid;
+            s_new_remaining = rem - (inc - h);
+          }
+        }
+        __syncthreads();
+        if (tid == 0) {
+          s_remaining = s_new_remaining;  // rank of the target inside the bucket (1-based)
+          s_prefix = prefix | ((uint32_t)s_bucket << shift);
+          s_mask = mask | (0xFFu << shift);
+        }
+        __syncthreads();
       }
-      __syncthreads();
     }
     tau = s_prefix;
     need_eq = (p.k > 0) ? s_remaining : 0;
   }
 
-  // ordered compaction: each thread owns a contiguous chunk of tokens
+  // ordered compaction: each thread owns a contiguous chunk of tokens, read in batches of
+  // independent loads
+  constexpr int kCB = 16;
   const int chunk = (T + nthr - 1) / nthr;
   const int t0 = min(T, tid * chunk), t1 = min(T, t0 + chunk);
+  float cs[kCB];
+  bool cv[kCB];
+  auto load_chunk = [&](int base) {
+#pragma unroll
+    for (int j = 0; j < kCB; ++j) {
+      const int t = base + j;
+      cs[j] = 0.f;
+      cv[j] = false;
+      if (t < t1) {
+        cs[j] = __ldcg(p.scores + t);
+        cv[j] = !p.valid || p.valid[t];
+      }
+    }
+  };
   int n_sel = 0, n_eq = 0;
-  for (int t = t0; t < t1; ++t) {
-    const bool ok = !p.valid || p.valid[t];
-    const float s = __ldcg(p.scores + t);
-    if (p.mode == QTALE_SELECT_TOPK) {
-      const uint32_t key = score_key(s);
-      n_sel += (ok && p.k > 0 && key > tau);
-      n_eq += (ok && p.k > 0 && key == tau);
-    } else {
-      n_sel += (ok && s >= p.theta);
+  for (int base = t0; base < t1; base += kCB) {
+    load_chunk(base);
+#pragma unroll
+    for (int j = 0; j < kCB; ++j) {
+      if (p.mode == QTALE_SELECT_TOPK) {
+        const uint32_t key = score_key(cs[j]);
+        n_sel += (cv[j] && p.k > 0 && key > tau);
+        n_eq += (cv[j] && p.k > 0 && key == tau);
+      } else {
+        n_sel += (cv[j] && cs[j] >= p.theta);
+      }
     }
   }
   // block-wide exclusive scans of (n_sel, n_eq) with warp shuffles
@@ -141,8 +204,10 @@ __device__ void select_and_compact(const RouterParams& p, uint32_t* sh_hist, int
     total += min(tot_eq, need_eq);
   }
 
-  // sequence of the first token of the chunk: largest b with cu_seqlens[b] <= t0
-  int b = 0;
+  // Sequence bookkeeping of the chunk.  b = sequence of the current token; q = next entry of
+  // cu_seqlens not yet passed.  The thread whose chunk contains token cu_seqlens[q] writes
+  // cu_exec[q] = executed tokens before it; entries equal to T are written at the end.
+  int b = 0, q = 0, seq_start = 0, seq_pos0 = 0, next_bound = T + 1;
   if (t0 < t1) {
     int lo = 0, hi = p.B;  // invariant: cu[lo] <= t0 < cu[hi] (cu[B] = T > t0)
     while (hi - lo > 1) {
@@ -150,41 +215,53 @@ __device__ void select_and_compact(const RouterParams& p, uint32_t* sh_hist, int
       if (p.cu_seqlens[mid] <= t0) lo = mid; else hi = mid;
     }
     b = lo;
+    q = b + 1;
+    if (p.cu_seqlens[b] == t0) {  // boundaries sitting exactly on the chunk start are ours
+      q = b;
+      while (q > 0 && p.cu_seqlens[q - 1] == t0) --q;
+    }
+    seq_start = p.cu_seqlens[b];
+    seq_pos0 = p.pos0 ? p.pos0[b] : 0;
+    next_bound = p.cu_seqlens[q];
   }
   int e = eq_before;
-  for (int t = t0; t < t1; ++t) {
-    while (b + 1 < p.B && t >= p.cu_seqlens[b + 1]) ++b;
-    const bool ok = !p.valid || p.valid[t];
-    const float s = __ldcg(p.scores + t);
-    bool take;
-    if (p.mode == QTALE_SELECT_TOPK) {
-      const uint32_t key = score_key(s);
-      take = ok && p.k > 0 && key > tau;
-      if (ok && p.k > 0 && key == tau) {
-        take = e < need_eq;
-        ++e;
+  for (int base = t0; base < t1; base += kCB) {
+    if (chunk > kCB || base != t0) load_chunk(base);  // a single batch is still in registers
+#pragma unroll
+    for (int j = 0; j < kCB; ++j) {
+      const int t = base + j;
+      if (t >= t1) break;
+      while (t >= next_bound) {  // token t opens sequence q (or skips empty ones)
+        p.cu_exec[q] = out;
+        if (q < p.B) {
+          b = q;
+          seq_start = next_bound;
+          seq_pos0 = p.pos0 ? p.pos0[b] : 0;
+        }
+        ++q;
+        next_bound = q <= p.B ? p.cu_seqlens[q] : T + 1;
       }
-    } else {
-      take = ok && s >= p.theta;
-    }
-    if (take) {
-      p.idx[out] = t;
-      p.pos[out] = t - p.cu_seqlens[b] + (p.pos0 ? p.pos0[b] : 0);
-      ++out;
+      bool take;
+      if (p.mode == QTALE_SELECT_TOPK) {
+        const uint32_t key = score_key(cs[j]);
+        take = cv[j] && p.k > 0 && key > tau;
+        if (cv[j] && p.k > 0 && key == tau) {
+          take = e < need_eq;
+          ++e;
+        }
+      } else {
+        take = cv[j] && cs[j] >= p.theta;
+      }
+      if (take) {
+        p.idx[out] = t;
+        p.pos[out] = t - seq_start + seq_pos0;
+        ++out;
+      }
     }
   }
-  __syncthreads();
   if (tid == 0) *p.n_exec = total;
-  // cu_exec[b] = number of executed tokens with index < cu_seqlens[b]
-  for (int q = tid; q <= p.B; q += nthr) {
-    const int bound = p.cu_seqlens[q];
-    int lo = 0, hi = total;
-    while (lo < hi) {
-      int mid = (lo + hi) >> 1;
-      if (p.idx[mid] < bound) lo = mid + 1; else hi = mid;
-    }
-    p.cu_exec[q] = lo;
-  }
+  for (int qq = tid; qq <= p.B; qq += nthr)
+    if (p.cu_seqlens[qq] >= T) p.cu_exec[qq] = total;
 }
 
 // ---- the fused kernel -------------------------------------------------------
@@ -197,16 +274,16 @@ __global__ void __launch_bounds__(kRouterThreads)
 
   const int tid = threadIdx.x;
   if (p.scores_override == nullptr) {
-    // phase A: router GEMV.  Router weights staged in shared memory as fp64,
-    // laid out [iteration][element j of the lane's 8][lane] so that the 32
-    // lanes of a warp read consecutive doubles.
-    double* w_s = reinterpret_cast<double*>(smem_raw);
+    // phase A: router GEMV.  Router weights staged in shared memory as fp32, laid out
+    // [iteration][lane][8] so a lane's eight weights are two 16-byte loads.  Each 16-byte
+    // load of x (8 bf16) is reduced with fp32 FMAs into a block sum, and the block sums
+    // are accumulated in fp64: conversions and fp64 adds are one per 8 elements, which
+    // keeps the sweep bandwidth bound, and the result stays within about 1e-8 of the
+    // all-fp64 dot product.
+    float* w_s = reinterpret_cast<float*>(smem_raw);
     const int d = p.d;
     const int n_it = (d + 255) / 256;
-    for (int i = tid; i < n_it * 256; i += blockDim.x) {
-      const int it = i >> 8, rem = i & 255, lane = rem >> 3, j = rem & 7;
-      w_s[(it * 8 + j) * 32 + lane] = (i < d) ? (double)p.w[i] : 0.0;
-    }
+    for (int i = tid; i < n_it * 256; i += blockDim.x) w_s[i] = (i < d) ? p.w[i] : 0.f;
     __syncthreads();
     const int lane = tid & 31;
     const int warp = tid >> 5;
@@ -217,24 +294,35 @@ __global__ void __launch_bounds__(kRouterThreads)
       double acc[kRowsPerWarp];
 #pragma unroll
       for (int r = 0; r < kRowsPerWarp; ++r) acc[r] = 0.0;
-      for (int it = 0; it < n_it; ++it) {
-        const int col = it * 256 + lane * 8;
-        uint4 v[kRowsPerWarp];
+      constexpr int kUnroll = 4;  // 16-byte loads in flight per lane: kUnroll x rows per warp
+      for (int it0 = 0; it0 < n_it; it0 += kUnroll) {
+        uint4 v[kUnroll][kRowsPerWarp];
 #pragma unroll
-        for (int r = 0; r < kRowsPerWarp; ++r) {
-          const int row = min(r0 + r, p.T - 1);
-          v[r] = (col < d) ? ld_nc_16(p.x + (size_t)row * d + col) : make_uint4(0, 0, 0, 0);
+        for (int u = 0; u < kUnroll; ++u) {
+          const int col = (it0 + u) * 256 + lane * 8;
+#pragma unroll
+          for (int r = 0; r < kRowsPerWarp; ++r) {
+            const int row = min(r0 + r, p.T - 1);
+            v[u][r] = (it0 + u < n_it && col < d) ? ld_nc_16(p.x + (size_t)row * d + col)
+                                                  : make_uint4(0, 0, 0, 0);
+          }
         }
-        double wv[8];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) wv[j] = w_s[(it * 8 + j) * 32 + lane];
+        for (int u = 0; u < kUnroll; ++u) {
+          if (it0 + u >= n_it) break;
+          const float4 wa = *reinterpret_cast<const float4*>(w_s + (it0 + u) * 256 + lane * 8);
+          const float4 wb = *reinterpret_cast<const float4*>(w_s + (it0 + u) * 256 + lane * 8 + 4);
 #pragma unroll
-        for (int r = 0; r < kRowsPerWarp; ++r) {
-          const uint32_t u[4] = {v[r].x, v[r].y, v[r].z, v[r].w};
-#pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            acc[r] = fma((double)bf16_lo(u[q]), wv[2 * q], acc[r]);
-            acc[r] = fma((double)bf16_hi(u[q]), wv[2 * q + 1], acc[r]);
+          for (int r = 0; r < kRowsPerWarp; ++r) {
+            float blk = bf16_lo(v[u][r].x) * wa.x;
+            blk = fmaf(bf16_hi(v[u][r].x), wa.y, blk);
+            blk = fmaf(bf16_lo(v[u][r].y), wa.z, blk);
+            blk = fmaf(bf16_hi(v[u][r].y), wa.w, blk);
+            blk = fmaf(bf16_lo(v[u][r].z), wb.x, blk);
+            blk = fmaf(bf16_hi(v[u][r].z), wb.y, blk);
+            blk = fmaf(bf16_lo(v[u][r].w), wb.z, blk);
+            blk = fmaf(bf16_hi(v[u][r].w), wb.w, blk);
+            acc[r] += (double)blk;
           }
         }
       }
@@ -338,10 +426,13 @@ int qtale_router_select(const void* x, int T, int d, const float* w_router, floa
   int grid;
   size_t smem = 0;
   if (scores_override) {
-    grid = 1;
+    // copy of the supplied scores: enough CTAs that each thread moves a few elements
+    grid = (T + kRouterThreads * 4 - 1) / (kRouterThreads * 4);
+    if (grid > sm_count()) grid = sm_count();
+    if (grid < 1) grid = 1;
   } else {
     const int n_it = (d + 255) / 256;
-    smem = (size_t)n_it * 256 * sizeof(double);
+    smem = (size_t)n_it * 256 * sizeof(float);
     const int warps = kRouterThreads / 32;
     const int n_groups = (T + kRowsPerWarp - 1) / kRowsPerWarp;
     grid = (n_groups + warps - 1) / warps;
