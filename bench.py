@@ -103,6 +103,23 @@ class ClockSampler:
                     samples=len(sm), power_w_max=max(power) if power else None)
 
 
+def max_over_ranks(ms: float, device=None) -> float:
+    """Slowest rank's time: every rank runs its own replica of the batch, the job's
+    throughput is set by the last one to finish.  No-op without a process group."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(ms)
+    t = torch.tensor([ms], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_tokens_per_s(tokens_per_rank: int, world: int, ms_per_step: float) -> float:
+    """Whole-job throughput of `world` replicas that each process tokens_per_rank per step."""
+    return world * tokens_per_rank / (ms_per_step * 1e-3)
+
+
 def build_layer_inputs(seed, cfg_name):
     c = inputs.CONFIG_SHAPES[cfg_name]
     sh, B, S = c["shape"], c["B"], c["S"]
@@ -212,12 +229,7 @@ def run_ours(args):
             fn(i)
         e1.record()
         barrier()
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return max_over_ranks(e0.elapsed_time(e1), dev if world > 1 else None)
 
     # ---- headline: device-resident inputs ----
     sampler = ClockSampler(local)
@@ -225,7 +237,7 @@ def run_ours(args):
     ms = timed(step, args.steps, args.warmup)
     clocks = sampler.stop()
     ms_per_step = ms / args.steps
-    value = world * T / (ms_per_step * 1e-3)
+    value = aggregate_tokens_per_s(T, world, ms_per_step)
     rc = api.device_status()
     if rc != 0:
         raise RuntimeError("device status: " + api.strerror(rc))

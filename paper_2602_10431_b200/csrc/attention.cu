@@ -60,9 +60,9 @@ __device__ __forceinline__ void mma_16816(float (&c)[4], const uint32_t (&a)[4],
 // ---------------------------------------------------------------------------
 // prefill
 // ---------------------------------------------------------------------------
-constexpr int kBQ = 64;   // query rows per CTA (16 per warp)
+constexpr int kBQ = 128;  // query rows per CTA (16 per warp, 8 warps)
 constexpr int kBK = 64;   // keys per tile
-constexpr int kAttnThreads = 128;
+constexpr int kAttnThreads = 256;
 
 // byte offset of 16-byte chunk c of row r in a tile with HD bf16 per row
 template <int HD>
@@ -70,11 +70,11 @@ __device__ __forceinline__ int sw_off(int r, int c) {
   return r * (HD * 2) + (((c & ~7) | ((c ^ r) & 7)) << 4);
 }
 
-template <int HD>
+template <int HD, int ROWS>
 __device__ __forceinline__ void load_tile(unsigned char* smem, const __nv_bfloat16* base, int ld,
                                           int row0, int n_rows_valid) {
   constexpr int CPR = HD / 8;  // chunks per row
-  for (int e = threadIdx.x; e < kBK * CPR; e += kAttnThreads) {
+  for (int e = threadIdx.x; e < ROWS * CPR; e += kAttnThreads) {
     const int r = e / CPR, c = e % CPR;
     const bool ok = r < n_rows_valid;
     const __nv_bfloat16* src = base + (size_t)(row0 + (ok ? r : 0)) * ld + c * 8;
@@ -89,9 +89,10 @@ __global__ void __launch_bounds__(kAttnThreads)
                         __nv_bfloat16* __restrict__ out, int ldo, float scale_log2) {
   extern __shared__ __align__(128) unsigned char smem[];
   constexpr int TILE_BYTES = kBK * HD * 2;
+  constexpr int Q_BYTES = kBQ * HD * 2;
   unsigned char* sQ = smem;
-  unsigned char* sK = smem + TILE_BYTES;       // two buffers
-  unsigned char* sV = smem + 3 * TILE_BYTES;   // two buffers
+  unsigned char* sK = smem + Q_BYTES;                    // two buffers
+  unsigned char* sV = smem + Q_BYTES + 2 * TILE_BYTES;   // two buffers
 
   // locate (sequence, query tile) of this CTA; heavy (late) tiles are scheduled first
   int b = -1, qt = 0;
@@ -117,11 +118,12 @@ __global__ void __launch_bounds__(kAttnThreads)
   const __nv_bfloat16* kbase = qkv + k_off + (size_t)hk * HD;
   const __nv_bfloat16* vbase = qkv + v_off + (size_t)hk * HD;
 
-  load_tile<HD>(sQ, qbase, ld, seq0 + q0, min(kBQ, len - q0));
+  load_tile<HD, kBQ>(sQ, qbase, ld, seq0 + q0, min(kBQ, len - q0));
   cp_async_commit();
-  const int n_kt = qt + 1;  // causal: key tiles 0 .. qt
-  load_tile<HD>(sK, kbase, ld, seq0, min(kBK, len));
-  load_tile<HD>(sV, vbase, ld, seq0, min(kBK, len));
+  // causal: key tiles that hold a key <= the last query row of this CTA
+  const int n_kt = min((len + kBK - 1) / kBK, (q0 + kBQ) / kBK);
+  load_tile<HD, kBK>(sK, kbase, ld, seq0, min(kBK, len));
+  load_tile<HD, kBK>(sV, vbase, ld, seq0, min(kBK, len));
   cp_async_commit();
 
   cp_async_wait<1>();
@@ -146,8 +148,8 @@ __global__ void __launch_bounds__(kAttnThreads)
     const int buf = kt & 1;
     if (kt + 1 < n_kt) {
       const int k0n = (kt + 1) * kBK;
-      load_tile<HD>(sK + (buf ^ 1) * TILE_BYTES, kbase, ld, seq0 + k0n, min(kBK, len - k0n));
-      load_tile<HD>(sV + (buf ^ 1) * TILE_BYTES, vbase, ld, seq0 + k0n, min(kBK, len - k0n));
+      load_tile<HD, kBK>(sK + (buf ^ 1) * TILE_BYTES, kbase, ld, seq0 + k0n, min(kBK, len - k0n));
+      load_tile<HD, kBK>(sV + (buf ^ 1) * TILE_BYTES, vbase, ld, seq0 + k0n, min(kBK, len - k0n));
       cp_async_commit();
       cp_async_wait<1>();
     } else {
@@ -156,6 +158,10 @@ __global__ void __launch_bounds__(kAttnThreads)
     __syncthreads();
     const unsigned char* k_s = sK + buf * TILE_BYTES;
     const unsigned char* v_s = sV + buf * TILE_BYTES;
+    const int k0 = kt * kBK;
+    const int warp_row0 = q0 + warp * 16;
+    // a key tile entirely above this warp's rows contributes nothing (warp-uniform skip)
+    if (k0 <= warp_row0 + 15) {
 
     // S = Q K^T for this warp's 16 rows x 64 keys
     float s[kBK / 8][4];
@@ -174,10 +180,10 @@ __global__ void __launch_bounds__(kAttnThreads)
         mma_16816<ACT>(s[2 * np + 1], qf[ks], kf[2], kf[3]);
       }
     }
-    // scale, causal / length mask (only the diagonal tile needs it)
-    const int k0 = kt * kBK;
-    const bool diag = (kt == qt);
-    const int row_a = q0 + warp * 16 + g, row_b = row_a + 8;
+    // scale, causal / length mask (only tiles that reach past this warp's first row or the
+    // end of the sequence need it)
+    const bool diag = (k0 + kBK - 1 > warp_row0) || (k0 + kBK > len);
+    const int row_a = warp_row0 + g, row_b = row_a + 8;
 #pragma unroll
     for (int i = 0; i < kBK / 8; ++i) {
 #pragma unroll
@@ -237,6 +243,7 @@ __global__ void __launch_bounds__(kAttnThreads)
         mma_16816<ACT>(o[2 * np], pf[kk], vf[0], vf[1]);
         mma_16816<ACT>(o[2 * np + 1], pf[kk], vf[2], vf[3]);
       }
+    }
     }
     __syncthreads();  // all warps done with this buffer before it is refilled
   }
@@ -381,7 +388,7 @@ __global__ void __launch_bounds__(kDecThreads)
 template <int HD, int ACT>
 static int launch_prefill_hd(const void* qkv, int ld, int k_off, int v_off, const int32_t* cu_exec,
                              int B, int H, int Hkv, int T_cap, void* out, int ldo, cudaStream_t s) {
-  const size_t smem = (size_t)5 * kBK * HD * 2;
+  const size_t smem = (size_t)(kBQ + 4 * kBK) * HD * 2;
   static bool configured[64] = {false};
   int dev = 0;
   cudaGetDevice(&dev);
