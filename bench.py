@@ -33,7 +33,7 @@ UNIT = "tokens/s"
 SWEEP = [1.0, 0.9, 0.75, 0.5]
 WORKLOAD = ("c2: 7B-shaped layer (hidden 4096, 32 heads, FFN 11008), int4 g128, "
             "batch 4 x seq 2048 prefill")
-KERNELS_PER_STEP = 10  # router, gather+norm, 4 GEMMs, rotary table, rotary, attention, RMSNorm
+KERNELS_PER_STEP = 11  # router, gather+norm, 4 GEMMs, rotary table, rotary, tail zeroing, attention, RMSNorm
 
 
 def measured_peaks():

@@ -1,0 +1,378 @@
+// Causal attention among the executed tokens of each sequence (prefill) on the
+// tcgen05 tensor cores (Eq. 3: bypassed tokens have no query, key or value here).
+//
+// One CTA handles 128 consecutive executed tokens (query rows) of one sequence and
+// one head, streaming that sequence's executed keys / values in tiles of 128:
+//   S = Q K^T     SS MMA, Q and K tiles from 128-byte-swizzled shared memory (TMA),
+//                 fp32 scores in tensor memory, double buffered;
+//   softmax       four warps, one query row per thread: running max / sum in the
+//                 log2 domain, probabilities written back to tensor memory in the
+//                 16-bit activation format (the A operand of the next MMA);
+//   O += P V      TS MMA with V read straight from its row-major tile (MN-major B
+//                 operand), fp32 output accumulator in tensor memory, rescaled by the
+//                 softmax warps only when a row's running maximum moves.
+// Warp roles (192 threads): warp 0 TMA producer, warp 1 MMA issuer and TMEM
+// allocator, warps 2-5 softmax / correction / output.  Every wait is bounded.
+#include <cuda.h>
+
+#include <string.h>
+
+#include "attention.cuh"
+#include "ptx.cuh"
+
+namespace qtale {
+
+using namespace ptx;
+
+constexpr int kTcThreads = 192;
+constexpr int kTcTile = 128;  // query rows per CTA and keys per tile
+constexpr uint32_t kTcSpin = 1u << 24;
+
+struct TcShared {
+  uint64_t q_full;
+  uint64_t k_full[2], v_full[2], kv_empty[2];
+  uint64_t s_full[2], p_full[2];
+  uint64_t pv_done;
+  uint32_t tmem_base;
+  volatile int abort_flag;
+};
+
+struct TcParams {
+  const int32_t* cu_exec;
+  int B, rep, H;
+  int k_off, v_off;      // column offsets of the K and V heads inside a qkv row
+  void* out;
+  int ldo;
+  float scale_log2;
+  int* status;
+};
+
+__device__ __forceinline__ bool tc_wait(uint64_t* bar, uint32_t parity, TcShared* sh, int* status) {
+  for (uint32_t it = 0; it < kTcSpin; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 255u) == 255u && sh->abort_flag) return false;
+  }
+  sh->abort_flag = 1;
+  report_device_error(status, QTALE_ERR_TIMEOUT);
+  return false;
+}
+
+// K-major tile of 128 rows x 64 elements per 16 KB chunk (128-byte swizzle): descriptor
+// of the 16-element K step `kk` (chunks follow each other every 16 KB)
+__device__ __forceinline__ uint64_t kmajor_desc(uint32_t smem_addr, int kk) {
+  return smem_desc_sw128(smem_addr + (kk >> 2) * 16384) + 2u * (kk & 3);
+}
+// V tile used as the MN-major B operand: rows are keys (the MMA's K), a row holds 64
+// head-dim elements per chunk.  Eight key rows form one 1024-byte group (stride offset),
+// the next 64 head-dim elements are 16 KB further (leading offset).
+__device__ __forceinline__ uint64_t v_desc(uint32_t smem_addr, int key16) {
+  uint64_t d = 0;
+  d |= (uint64_t)(((smem_addr + key16 * 2048) & 0x3FFFFu) >> 4);
+  d |= (uint64_t)(16384 >> 4) << 16;
+  d |= (uint64_t)(1024 >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+
+template <int HD, int ACT>
+__global__ void __launch_bounds__(kTcThreads, 1)
+    attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap, const TcParams p) {
+  constexpr int CH = HD / 64;                       // 16 KB chunks per tile
+  constexpr int TILE_BYTES = kTcTile * HD * 2;
+  constexpr int S_COL = 0;                          // two score buffers of 128 columns
+  constexpr int P_COL = 256;                        // two probability buffers of 64 columns
+  constexpr int O_COL = 384;                        // output accumulator, HD columns
+  extern __shared__ unsigned char smem_dyn[];
+  __shared__ TcShared sh;
+  unsigned char* base = reinterpret_cast<unsigned char*>(
+      (reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~static_cast<uintptr_t>(1023));
+  unsigned char* sQ = base;
+  unsigned char* sK = base + TILE_BYTES;            // two stages
+  unsigned char* sV = base + 3 * TILE_BYTES;        // two stages
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  // locate (sequence, query tile); late (long) tiles first
+  int b = -1, qt = 0;
+  {
+    int tile = blockIdx.x;
+    for (int s = p.B - 1; s >= 0; --s) {
+      const int len = p.cu_exec[s + 1] - p.cu_exec[s];
+      const int nt = (len + kTcTile - 1) / kTcTile;
+      if (tile < nt) { b = s; qt = nt - 1 - tile; break; }
+      tile -= nt;
+    }
+  }
+  if (b < 0) return;  // uniform for the CTA: nothing allocated yet
+  const int h = blockIdx.y, hk = h / p.rep;
+  const int seq0 = p.cu_exec[b];
+  const int len = p.cu_exec[b + 1] - seq0;
+  const int q0 = qt * kTcTile;
+  const int n_kt = qt + 1;
+
+  if (threadIdx.x == 0) {
+    mbar_init(&sh.q_full, 1);
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&sh.k_full[s], 1);
+      mbar_init(&sh.v_full[s], 1);
+      mbar_init(&sh.kv_empty[s], 1);
+      mbar_init(&sh.s_full[s], 1);
+      mbar_init(&sh.p_full[s], 4);
+    }
+    mbar_init(&sh.pv_done, 1);
+    sh.abort_flag = 0;
+    fence_barrier_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(&sh.tmem_base, 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = sh.tmem_base;
+
+  if (warp == 0) {
+    // ------------------------------ TMA producer ------------------------------
+    if (lane == 0) {
+      mbar_arrive_expect_tx(&sh.q_full, TILE_BYTES);
+      for (int c = 0; c < CH; ++c)
+        tma_load_2d(sQ + c * 16384, &tmap, &sh.q_full, h * HD + c * 64, seq0 + q0);
+      for (int j = 0; j < n_kt; ++j) {
+        const int s = j & 1;
+        const uint32_t ph = (uint32_t)(j >> 1) & 1u;
+        if (!tc_wait(&sh.kv_empty[s], ph ^ 1u, &sh, p.status)) break;
+        mbar_arrive_expect_tx(&sh.k_full[s], TILE_BYTES);
+        for (int c = 0; c < CH; ++c)
+          tma_load_2d(sK + s * TILE_BYTES + c * 16384, &tmap, &sh.k_full[s],
+                      p.k_off + hk * HD + c * 64, seq0 + j * kTcTile);
+        mbar_arrive_expect_tx(&sh.v_full[s], TILE_BYTES);
+        for (int c = 0; c < CH; ++c)
+          tma_load_2d(sV + s * TILE_BYTES + c * 16384, &tmap, &sh.v_full[s],
+                      p.v_off + hk * HD + c * 64, seq0 + j * kTcTile);
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------- MMA issuer -------------------------------
+    if (lane == 0) {
+      constexpr uint32_t idesc_qk = idesc_16bit_f32(128, kTcTile, ACT == 1);
+      constexpr uint32_t idesc_pv = idesc_16bit_f32(128, HD, ACT == 1) | (1u << 16);  // B is MN-major
+      bool ok = tc_wait(&sh.q_full, 0, &sh, p.status);
+      auto issue_qk = [&](int j) {
+        const int s = j & 1;
+        if (!tc_wait(&sh.k_full[s], (uint32_t)(j >> 1) & 1u, &sh, p.status)) return false;
+        tc_fence_after();
+        const uint32_t qa = smem_u32(sQ), ka = smem_u32(sK + s * TILE_BYTES);
+#pragma unroll
+        for (int kk = 0; kk < HD / 16; ++kk)
+          mma_ss(tmem + S_COL + s * 128, kmajor_desc(qa, kk), kmajor_desc(ka, kk), idesc_qk,
+                 kk != 0 ? 1u : 0u);
+        mma_commit(&sh.s_full[s]);
+        return true;
+      };
+      if (ok) ok = issue_qk(0);
+      for (int j = 0; ok && j < n_kt; ++j) {
+        const int s = j & 1;
+        const uint32_t ph = (uint32_t)(j >> 1) & 1u;
+        // scores of the next tile are computed while the softmax of this one runs
+        if (j + 1 < n_kt) ok = issue_qk(j + 1);
+        if (!ok) break;
+        if (!tc_wait(&sh.p_full[s], ph, &sh, p.status)) break;
+        if (!tc_wait(&sh.v_full[s], ph, &sh, p.status)) break;
+        tc_fence_after();
+        const uint32_t va = smem_u32(sV + s * TILE_BYTES);
+#pragma unroll
+        for (int kk = 0; kk < kTcTile / 16; ++kk)
+          mma_ts(tmem + O_COL, tmem + P_COL + s * 64 + kk * 8, v_desc(va, kk), idesc_pv,
+                 (j | kk) != 0 ? 1u : 0u);
+        mma_commit(&sh.kv_empty[s]);
+        mma_commit(&sh.pv_done);
+      }
+    }
+  } else {
+    // ------------------ softmax, correction and output: one query row per thread ------------------
+    const int quad = warp & 3;
+    const int row = quad * 32 + lane;          // TMEM lane = query row of the tile
+    const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+    float m_run = -INFINITY, l_run = 0.f;
+    bool alive = true;
+    for (int j = 0; j < n_kt && alive; ++j) {
+      const int s = j & 1;
+      const uint32_t ph = (uint32_t)(j >> 1) & 1u;
+      if (!tc_wait(&sh.s_full[s], ph, &sh, p.status)) { alive = false; break; }
+      tc_fence_after();
+      const uint32_t s_addr = tmem + lane_addr + S_COL + s * 128;
+      const int k0 = j * kTcTile;
+      const bool masked = (j == qt) || (k0 + kTcTile > len);
+      const int q_row = q0 + row;
+      // the whole score row (128 keys) in registers: scaled and masked once
+      float sc[128];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t r[32];
+        tmem_ld_x32(s_addr + c * 32, r);
+        tmem_wait_ld();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) sc[c * 32 + i] = __uint_as_float(r[i]) * p.scale_log2;
+      }
+      if (masked) {
+#pragma unroll
+        for (int i = 0; i < 128; ++i) {
+          const int key = k0 + i;
+          if (key > q_row || key >= len) sc[i] = -INFINITY;
+        }
+      }
+      float mx = m_run;
+#pragma unroll
+      for (int i = 0; i < 128; ++i) mx = fmaxf(mx, sc[i]);
+      const float m_safe = (mx == -INFINITY) ? 0.f : mx;
+      const float corr = exp2f(m_run - m_safe);
+      const bool moved = mx > m_run;
+      m_run = mx;
+      l_run *= corr;
+      // probabilities in the 16-bit format, two keys per 32-bit column
+      float sum = 0.f;
+      uint32_t pr[64];
+#pragma unroll
+      for (int i = 0; i < 64; ++i) {
+        const float p0 = exp2f(sc[2 * i] - m_safe), p1 = exp2f(sc[2 * i + 1] - m_safe);
+        sum += p0 + p1;
+        pr[i] = Act16<ACT>::pack(p0, p1);
+      }
+      // the previous P V must be complete before O is rescaled or P is overwritten
+      if (j > 0) {
+        if (!tc_wait(&sh.pv_done, (uint32_t)(j - 1) & 1u, &sh, p.status)) { alive = false; break; }
+        tc_fence_after();
+        if (__any_sync(0xffffffffu, moved)) {
+#pragma unroll 1
+          for (int c = 0; c < HD / 32; ++c) {
+            uint32_t r[32];
+            tmem_ld_x32(tmem + lane_addr + O_COL + c * 32, r);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * corr);
+            tmem_st_x32(tmem + lane_addr + O_COL + c * 32, r);
+          }
+        }
+      }
+      {
+        uint32_t lo[32], hi[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) { lo[i] = pr[i]; hi[i] = pr[32 + i]; }
+        tmem_st_x32(tmem + lane_addr + P_COL + s * 64, lo);
+        tmem_st_x32(tmem + lane_addr + P_COL + s * 64 + 32, hi);
+      }
+      l_run += sum;
+      tmem_wait_st();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh.p_full[s]);
+    }
+    // output: O / l for the rows that exist
+    if (alive && tc_wait(&sh.pv_done, (uint32_t)(n_kt - 1) & 1u, &sh, p.status)) {
+      tc_fence_after();
+      const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+      const int q_row = q0 + row;
+      unsigned short* out = static_cast<unsigned short*>(p.out) + (size_t)(seq0 + q_row) * p.ldo + (size_t)h * HD;
+#pragma unroll 1
+      for (int c = 0; c < HD / 32; ++c) {
+        uint32_t r[32];
+        tmem_ld_x32(tmem + lane_addr + O_COL + c * 32, r);
+        tmem_wait_ld();
+        if (q_row < len) {
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            uint4 o;
+            o.x = Act16<ACT>::pack(__uint_as_float(r[8 * i + 0]) * inv, __uint_as_float(r[8 * i + 1]) * inv);
+            o.y = Act16<ACT>::pack(__uint_as_float(r[8 * i + 2]) * inv, __uint_as_float(r[8 * i + 3]) * inv);
+            o.z = Act16<ACT>::pack(__uint_as_float(r[8 * i + 4]) * inv, __uint_as_float(r[8 * i + 5]) * inv);
+            o.w = Act16<ACT>::pack(__uint_as_float(r[8 * i + 6]) * inv, __uint_as_float(r[8 * i + 7]) * inv);
+            st_16(out + c * 32 + i * 8, o);
+          }
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 512);
+  }
+}
+
+// ---------------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFnA)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                   const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                   const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFnA encode_fn_a() {
+  static EncodeTiledFnA fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) ==
+            cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFnA>(p);
+  }
+  return fn;
+}
+
+template <int HD, int ACT>
+static int launch_tc(const CUtensorMap& tm, const TcParams& p, int max_tiles, int H, cudaStream_t s) {
+  const size_t smem = (size_t)5 * kTcTile * HD * 2 + 1024;
+  static bool configured[64] = {false};
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (dev >= 0 && dev < 64 && !configured[dev]) {
+    if (cudaFuncSetAttribute(attn_prefill_tc_kernel<HD, ACT>,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return QTALE_ERR_CUDA;
+    configured[dev] = true;
+  }
+  dim3 grid(max_tiles, H);
+  attn_prefill_tc_kernel<HD, ACT><<<grid, kTcThreads, smem, s>>>(tm, p);
+  return launch_status(cudaGetLastError());
+}
+
+int launch_attn_prefill(const void* qkv, int ld, int H, int Hkv, int hd, int act,
+                        const int32_t* cu_exec, int B, int T_cap, void* out, int ldo,
+                        cudaStream_t s) {
+  EncodeTiledFnA fn = encode_fn_a();
+  if (!fn) return QTALE_ERR_CUDA;
+  CUtensorMap tm;
+  cuuint64_t gdim[2] = {(cuuint64_t)ld, (cuuint64_t)T_cap};
+  cuuint64_t gstr[1] = {(cuuint64_t)ld * 2};
+  cuuint32_t box[2] = {64, (cuuint32_t)kTcTile};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(&tm, act == QTALE_ACT_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
+                  2, const_cast<void*>(qkv), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return QTALE_ERR_CUDA;
+  TcParams p;
+  p.cu_exec = cu_exec;
+  p.B = B;
+  p.rep = H / Hkv;
+  p.H = H;
+  p.k_off = H * hd;
+  p.v_off = (H + Hkv) * hd;
+  p.out = out;
+  p.ldo = ldo;
+  p.scale_log2 = 1.4426950408889634f / sqrtf((float)hd);
+  p.status = device_status_ptr();
+  const int max_tiles = (T_cap + kTcTile - 1) / kTcTile + B;
+  if (hd == 128)
+    return act == QTALE_ACT_F16 ? launch_tc<128, 1>(tm, p, max_tiles, H, s) : launch_tc<128, 0>(tm, p, max_tiles, H, s);
+  if (hd == 64)
+    return act == QTALE_ACT_F16 ? launch_tc<64, 1>(tm, p, max_tiles, H, s) : launch_tc<64, 0>(tm, p, max_tiles, H, s);
+  return QTALE_ERR_SHAPE;
+}
+
+}  // namespace qtale

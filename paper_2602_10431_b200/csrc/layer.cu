@@ -121,6 +121,7 @@ static int layer_forward_impl(const qtale_layer_config* c, const qtale_layer_wei
     QTALE_TRY(launch_attn_decode(ws.qkv, nqkv, H, Hkv, hd, act, idx, ws.n_exec, T, kv->k, kv->v,
                                  kv->kv_len, kv->cap, ws.ao, qd, s));
   } else {
+    QTALE_TRY(launch_zero_tail_rows(ws.qkv, ws.n_exec, T, nqkv, 128, s));
     QTALE_TRY(launch_attn_prefill(ws.qkv, nqkv, H, Hkv, hd, act, ws.cu_exec, B, T, ws.ao, qd, s));
   }
   // 6. output projection + residual: u = x[idx] + attention branch (fp32)

@@ -255,6 +255,19 @@ __global__ void kv_len_update_kernel(int32_t* kv_len, const int32_t* cu_exec, in
     kv_len[b] = min(cap, kv_len[b] + cu_exec[b + 1] - cu_exec[b]);
 }
 
+// ---- zero the rows between the executed count and the next multiple of `tile` ----
+// (tiled loads of the attention kernel read whole tiles; rows past the count must be finite)
+__global__ void zero_tail_rows_kernel(uint4* __restrict__ buf, const int32_t* __restrict__ n_exec,
+                                      int cap, int ld, int tile) {
+  const int n = min(*n_exec, cap);
+  const int end = min(cap, (n + tile - 1) / tile * tile);
+  const int ldc = ld >> 3;
+  const size_t total = (size_t)(end - n) * ldc;
+  for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < total;
+       e += (size_t)gridDim.x * blockDim.x)
+    buf[(size_t)n * ldc + e] = make_uint4(0, 0, 0, 0);
+}
+
 // ---- embedding gather ------------------------------------------------------------
 __global__ void __launch_bounds__(kRowThreads)
     embed_kernel(const uint4* __restrict__ embed, const int32_t* __restrict__ ids, int T, int d,
@@ -369,6 +382,12 @@ int launch_kv_append(const void* qkv, const int32_t* n_exec, int cap_rows, int l
       static_cast<uint4*>(cache_k), static_cast<uint4*>(cache_v), kv_len, cap);
   if (cudaGetLastError() != cudaSuccess) return QTALE_ERR_CUDA;
   kv_len_update_kernel<<<(B + 255) / 256, 256, 0, s>>>(kv_len, cu_exec, B, cap);
+  return launch_status(cudaGetLastError());
+}
+
+int launch_zero_tail_rows(void* buf, const int32_t* n_exec, int cap, int ld, int tile,
+                          cudaStream_t s) {
+  zero_tail_rows_kernel<<<64, 256, 0, s>>>(static_cast<uint4*>(buf), n_exec, cap, ld, tile);
   return launch_status(cudaGetLastError());
 }
 
