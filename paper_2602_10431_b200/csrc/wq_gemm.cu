@@ -21,8 +21,9 @@
 // round trip.  The grid is persistent (one CTA per SM) and reads the number of
 // executed tokens from device memory: no launch parameter depends on the routing.
 //
-// Warp roles (384 threads): warps 0 and 2 activation TMA producers (even / odd K
-// blocks), warp 1 MMA issuer and TMEM allocator, warp 3 weight TMA producer,
+// Warp roles (384 threads): warps 0 and 2 TMA producers (even / odd K blocks,
+// activations and weights), warps 1 and 3 MMA issuers (one per row tile; warp 1
+// also allocates tensor memory),
 // warps 4-11 dequantisers and, at the end of a tile, epilogue: set g = 0, 1 (four
 // warps, one TMEM lane quadrant each) owns row tile g.
 #include <cuda.h>
@@ -98,8 +99,8 @@ struct GemmParams {
 struct __align__(8) GemmShared {
   uint64_t full_x[8], empty_x[8];  // activation ring
   uint64_t full_w[8], empty_w[8];  // packed-weight ring
-  uint64_t a_full[8], a_empty[8];  // dequantised A slots in tensor memory, one entry per K block
-  uint64_t d_full, d_empty;        // the accumulators of the CTA tile
+  uint64_t a_full[2][4], a_empty[2][4];  // dequantised A slots in tensor memory, per row tile
+  uint64_t d_full[2], d_empty[2];        // the accumulators, per row tile
   uint32_t tmem_base;
   volatile int abort_flag;
 };
@@ -311,14 +312,18 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
   if (threadIdx.x == 0) {
     for (int s = 0; s < 8; ++s) {
       mbar_init(&sh.full_x[s], 1);
-      mbar_init(&sh.empty_x[s], 1);
+      mbar_init(&sh.empty_x[s], 2);  // released by both MMA issuers
       mbar_init(&sh.full_w[s], 1);
       mbar_init(&sh.empty_w[s], 8);
-      mbar_init(&sh.a_full[s], 8);
-      mbar_init(&sh.a_empty[s], 1);
     }
-    mbar_init(&sh.d_full, 1);
-    mbar_init(&sh.d_empty, 8);
+    for (int r = 0; r < 2; ++r) {
+      for (int s = 0; s < 4; ++s) {
+        mbar_init(&sh.a_full[r][s], 4);
+        mbar_init(&sh.a_empty[r][s], 1);
+      }
+      mbar_init(&sh.d_full[r], 1);
+      mbar_init(&sh.d_empty[r], 4);
+    }
     sh.abort_flag = 0;
     fence_barrier_init();
   }
@@ -362,15 +367,24 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
   const uint32_t x_stage_tx = (uint32_t)TW * 128u + (BITS == 16 ? kTileRows * 128 : 0);
 
   if (warp == 0 || warp == 2) {
-    // ---------------- activation TMA producers: warp 0 even, warp 2 odd K blocks ----------------
+    // ------- TMA producers: warp 0 serves even, warp 2 odd K blocks (activations + weights) -------
     if (lane == 0) {
       const int parity = warp >> 1;
-      Ring rx;
+      Ring rx, rw;
       int count = 0;
       for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
         const int rp = tile % n_rp, mt = tile / n_rp;
         for (int kb = 0; kb < nkb; ++kb, ++count) {
           if ((count & 1) == parity) {
+            if (BITS != 16) {
+              // one contiguous chunk per (row-tile pair, K block): both tiles' codes, each
+              // followed by the scale / zero words of its group
+              if (!wait_or_abort(&sh.empty_w[rw.s], rw.ph ^ 1u, &sh, p.status)) goto x_done;
+              mbar_arrive_expect_tx(&sh.full_w[rw.s], Cfg::kWStageBytes);
+              bulk_load(w_base + (size_t)rw.s * Cfg::kWStageBytes,
+                        p.packed + ((size_t)rp * nkb + kb) * Cfg::kWStageBytes, Cfg::kWStageBytes,
+                        &sh.full_w[rw.s]);
+            }
             if (!wait_or_abort(&sh.empty_x[rx.s], rx.ph ^ 1u, &sh, p.status)) goto x_done;
             unsigned char* st = x_base + (size_t)rx.s * Cfg::kXStageBytes;
             mbar_arrive_expect_tx(&sh.full_x[rx.s], x_stage_tx);
@@ -379,52 +393,37 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
               tma_load_2d(st + Cfg::kXBytes, &tmap_w, &sh.full_x[rx.s], kb * kKB, rp * kTileRows);
           }
           rx.advance(SX);
+          rw.advance(SW);
         }
       }
     x_done:;
     }
-  } else if (warp == 3) {
-    // ---------------------------- weight TMA producer ----------------------------
-    if (BITS != 16 && lane == 0) {
-      Ring rw;
-      for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
-        const int rp = tile % n_rp;
-        for (int kb = 0; kb < nkb; ++kb) {
-          if (!wait_or_abort(&sh.empty_w[rw.s], rw.ph ^ 1u, &sh, p.status)) goto w_done;
-          unsigned char* st = w_base + (size_t)rw.s * Cfg::kWStageBytes;
-          // one contiguous chunk per (row-tile pair, K block): both tiles' codes, each
-          // followed by the scale / zero words of its group
-          mbar_arrive_expect_tx(&sh.full_w[rw.s], Cfg::kWStageBytes);
-          bulk_load(st, p.packed + ((size_t)rp * nkb + kb) * Cfg::kWStageBytes, Cfg::kWStageBytes,
-                    &sh.full_w[rw.s]);
-          rw.advance(SW);
-        }
-      }
-    w_done:;
-    }
-  } else if (warp == 1) {
-    // ------------------------------- MMA issuer --------------------------------
+  } else if (warp == 1 || warp == 3) {
+    // ---- MMA issuers: warp 1 drives row tile 0, warp 3 row tile 1; they share the activation
+    // ---- stages and are otherwise independent (own A slots, own accumulator).  The tensor
+    // ---- core's queue is only a few MMAs deep, so the waits, fence and commits of one issuer
+    // ---- are covered by the MMAs of the other.
     if (lane == 0) {
+      const int r = warp >> 1;
       const uint32_t idesc = idesc_16bit_f32(kTileRows, TW, ACT == 1);
+      const uint32_t d_tmem = tmem_base + r * Cfg::kDCols;
       Ring rx, ra;
       uint32_t dph = 0;
       for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
         const int rp = tile % n_rp;
-        // the accumulators are free once the previous tile has been drained
-        if (!wait_or_abort(&sh.d_empty, dph ^ 1u, &sh, p.status)) goto mma_done;
+        const bool has_tile = r < RT && rp * RT + r < p.n_tiles;
+        // the accumulator is free once the previous tile has been drained
+        if (!wait_or_abort(&sh.d_empty[r], dph ^ 1u, &sh, p.status)) goto mma_done;
         tc_fence_after();
         for (int kb = 0; kb < nkb; ++kb) {
           if (!wait_or_abort(&sh.full_x[rx.s], rx.ph, &sh, p.status)) goto mma_done;
           if (BITS != 16) {
-            if (!wait_or_abort(&sh.a_full[ra.s], ra.ph, &sh, p.status)) goto mma_done;
+            if (!wait_or_abort(&sh.a_full[r][ra.s], ra.ph, &sh, p.status)) goto mma_done;
           }
-          tc_fence_after();
-          unsigned char* st = x_base + (size_t)rx.s * Cfg::kXStageBytes;
-          const uint64_t b_desc = smem_desc_sw128(smem_u32(st));
-#pragma unroll
-          for (int r = 0; r < RT; ++r) {
-            if (rp * RT + r >= p.n_tiles) continue;
-            const uint32_t d_tmem = tmem_base + r * Cfg::kDCols;
+          if (has_tile) {
+            tc_fence_after();
+            unsigned char* st = x_base + (size_t)rx.s * Cfg::kXStageBytes;
+            const uint64_t b_desc = smem_desc_sw128(smem_u32(st));
 #pragma unroll
             for (int j = 0; j < kKB / 16; ++j) {
               const uint32_t acc = (kb | j) != 0 ? 1u : 0u;
@@ -437,13 +436,17 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
                        b_desc + 2u * j, idesc, acc);
               }
             }
+            mma_commit(&sh.empty_x[rx.s]);                      // one of the two releases of the stage
+            if (BITS != 16) mma_commit(&sh.a_empty[r][ra.s]);   // frees this row tile's A slot
+          } else {
+            // nothing to multiply for this row tile: keep the handshakes in step
+            mbar_arrive(&sh.empty_x[rx.s]);
+            if (BITS != 16) mbar_arrive(&sh.a_empty[r][ra.s]);
           }
-          mma_commit(&sh.empty_x[rx.s]);                   // frees the activation stage
-          if (BITS != 16) mma_commit(&sh.a_empty[ra.s]);   // frees the A slots of this K block
           rx.advance(SX);
           ra.advance(SA);
         }
-        mma_commit(&sh.d_full);
+        if (has_tile) mma_commit(&sh.d_full[r]); else mbar_arrive(&sh.d_full[r]);
         dph ^= 1u;
       }
     mma_done:;
@@ -522,7 +525,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
               else dequant8<QM, ACT>(t, C, Sc, r + 4 * u);
             }
           }
-          if (!wait_or_abort(&sh.a_empty[ra.s], ra.ph ^ 1u, &sh, p.status)) goto role_done;
+          if (!wait_or_abort(&sh.a_empty[g][ra.s], ra.ph ^ 1u, &sh, p.status)) goto role_done;
           if (has_tile) {
             tc_fence_after();
             const uint32_t a_taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + Cfg::kAColBase +
@@ -532,13 +535,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
             tc_fence_before();
           }
           __syncwarp();
-          if (lane == 0) mbar_arrive(&sh.a_full[ra.s]);
+          if (lane == 0) mbar_arrive(&sh.a_full[g][ra.s]);
           rw.advance(SW);
           ra.advance(SA);
         }
       }
       // ---- epilogue of this tile: set g drains accumulator g, one lane quadrant per warp ----
-      if (!wait_or_abort(&sh.d_full, dph, &sh, p.status)) goto role_done;
+      if (!wait_or_abort(&sh.d_full[g], dph, &sh, p.status)) goto role_done;
       tc_fence_after();
       if (has_tile) {
         const int m_base = mt * TW;
@@ -562,7 +565,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&sh.d_empty);
+      if (lane == 0) mbar_arrive(&sh.d_empty[g]);
       dph ^= 1u;
     }
   role_done:;
