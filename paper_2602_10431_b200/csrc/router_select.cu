@@ -11,7 +11,6 @@ namespace qtale {
 
 constexpr int kRouterThreads = 512;  // 16 warps
 constexpr int kRowsPerWarp = 2;
-constexpr int kSelectThreads = 1024;  // upper bound of the CTA size the selection code supports
 
 struct RouterParams {
   const __nv_bfloat16* x;
@@ -35,228 +34,244 @@ __device__ __forceinline__ uint32_t score_key(float s) {
   return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
 }
 
-// ---- phase B: decision + compaction, executed by one CTA of kSelectThreads ----
+// ---- phase B: decision + compaction, executed by one CTA ----------------------
+// Every sweep over the scores is warp-cooperative and coalesced: warp w owns the
+// contiguous token segment [w * seg, (w + 1) * seg) and walks it 32 tokens at a
+// time (token = segment start + 32 i + lane), so ballots give each selected
+// token its rank in token order.  When a lane's share is at most kKeep scores
+// they are read once and kept in registers for all sweeps.
+constexpr int kKeep = 16;
+
 __device__ void select_and_compact(const RouterParams& p, uint32_t* sh_hist, int* sh_scan) {
   const int tid = threadIdx.x;
   const int nthr = blockDim.x;
+  const int lane = tid & 31, wid = tid >> 5, nwarps = nthr >> 5;
   const int T = p.T;
   __shared__ uint32_t s_prefix, s_mask;
-  __shared__ int s_remaining, s_total, s_bucket, s_new_remaining;
+  __shared__ int s_remaining;
+
+  const int seg = ((T + nwarps - 1) / nwarps + 31) & ~31;  // tokens per warp, multiple of 32
+  const int w0 = min(T, wid * seg), w1 = min(T, w0 + seg);
+  const int n_it = (w1 - w0 + 31) >> 5;                    // 32-token steps of this warp
+  const bool keep = seg <= 32 * kKeep;                     // uniform over the CTA
+
+  // score and validity of the token of step i (0 and false past the end)
+  auto load_one = [&](int i, float& sc, bool& ok) {
+    const int t = w0 + 32 * i + lane;
+    ok = t < w1;
+    sc = 0.f;
+    if (ok) {
+      sc = __ldcg(p.scores + t);
+      if (p.valid) ok = p.valid[t] != 0;
+    }
+  };
+  float ksc[kKeep];
+  uint32_t kok = 0;  // bit i: token of step i is valid
+  if (keep) {
+#pragma unroll
+    for (int i = 0; i < kKeep; ++i) {
+      bool ok;
+      load_one(i, ksc[i], ok);
+      kok |= (ok ? 1u : 0u) << i;
+    }
+  }
 
   uint32_t tau = 0;  // key of the k-th largest score (top-k)
   int need_eq = 0;   // how many tokens with key == tau execute (lowest indices first)
 
-  if (p.mode == QTALE_SELECT_TOPK) {
-    // MSB-first radix select of the k-th largest key among valid tokens.  Keys are read
-    // in batches of kBatch independent loads per thread (token t = (batch*kBatch + j) * nthr
-    // + tid); when a thread's share fits one batch it is read once and kept in registers.
-    constexpr int kBatch = 16;
-    constexpr uint32_t kInvalid = 0u;  // key 0 is below every real key (those have a set bit)
+  if (p.mode == QTALE_SELECT_TOPK && p.k > 0) {
+    // MSB-first radix select (four 8-bit digits) of the k-th largest key among valid tokens
     if (tid == 0) {
       s_prefix = 0;
       s_mask = 0;
       s_remaining = p.k;
     }
-    const int per = (T + nthr - 1) / nthr;
-    const int n_batches = (per + kBatch - 1) / kBatch;
-    uint32_t keys[kBatch];
-    auto load_batch = [&](int bi) {
-#pragma unroll
-      for (int j = 0; j < kBatch; ++j) {
-        const int t = (bi * kBatch + j) * nthr + tid;
-        float sc = 0.f;
-        bool ok = t < T;
-        if (ok) sc = __ldcg(p.scores + t);
-        if (ok && p.valid) ok = p.valid[t] != 0;
-        keys[j] = ok ? score_key(sc) : kInvalid;
-      }
-    };
-    if (n_batches == 1) load_batch(0);
-    __syncthreads();
-    for (int pass = 0; pass < 4 && p.k > 0; ++pass) {
+    for (int pass = 0; pass < 4; ++pass) {
       const int shift = 24 - 8 * pass;
       for (int i = tid; i < 256; i += nthr) sh_hist[i] = 0;
-      if (tid == 0) {  // defaults if k exceeds the number of valid tokens: lowest bucket
-        s_bucket = 0;
-        s_new_remaining = s_remaining;
-      }
       __syncthreads();
       const uint32_t prefix = s_prefix, mask = s_mask;
-      for (int bi = 0; bi < n_batches; ++bi) {
-        if (n_batches > 1) load_batch(bi);
+      auto count_key = [&](float sc, bool ok) {
+        const uint32_t key = score_key(sc);
+        const bool in = ok && (key & mask) == prefix;
+        const uint32_t bucket = (key >> shift) & 0xFFu;
+        // scores cluster in few buckets of the leading digits: one atomic when the warp agrees
+        const uint32_t members = __ballot_sync(0xffffffffu, in);
+        if (members == 0) return;
+        const int first = __ffs(members) - 1;
+        const uint32_t b0 = __shfl_sync(0xffffffffu, bucket, first);
+        if (__all_sync(0xffffffffu, !in || bucket == b0)) {
+          if (lane == first) atomicAdd(&sh_hist[b0], (uint32_t)__popc(members));
+        } else if (in) {
+          atomicAdd(&sh_hist[bucket], 1u);
+        }
+      };
+      if (keep) {
 #pragma unroll
-        for (int j = 0; j < kBatch; ++j) {
-          const uint32_t key = keys[j];
-          const bool in = key != kInvalid && (key & mask) == prefix;
-          // scores cluster in a few buckets: one atomic per distinct bucket per warp
-          const uint32_t bucket = in ? ((key >> shift) & 0xFF) : 256u;
-          const uint32_t peers = __match_any_sync(0xffffffffu, bucket);
-          if (in && (int)(__ffs(peers) - 1) == (tid & 31)) atomicAdd(&sh_hist[bucket], __popc(peers));
+        for (int i = 0; i < kKeep; ++i) count_key(ksc[i], (kok >> i) & 1u);
+      } else {
+        for (int i0 = 0; i0 < n_it; i0 += 8) {
+          float sc[8];
+          bool ok[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) load_one(i0 + j, sc[j], ok[j]);
+#pragma unroll
+          for (int j = 0; j < 8; ++j) count_key(sc[j], ok[j]);
         }
       }
       __syncthreads();
-      // bucket holding the target: suffix sums over the 256 buckets, one bucket per thread
-      {
-        const int lane = tid & 31, wid = tid >> 5;
-        int h = 0, inc = 0;
-        if (tid < 256) {
-          h = (int)sh_hist[255 - tid];  // descending bucket order
-          inc = h;
+      // bucket holding the target rank: warp 0 scans the 256 counts from the top, 8 per lane
+      if (wid == 0) {
+        int c[8], sum = 0;
 #pragma unroll
-          for (int o = 1; o < 32; o <<= 1) {
-            const int n = __shfl_up_sync(0xffffffffu, inc, o);
-            if (lane >= o) inc += n;
-          }
-          if (lane == 31) sh_scan[wid] = inc;
+        for (int j = 0; j < 8; ++j) {
+          c[j] = (int)sh_hist[255 - (lane * 8 + j)];
+          sum += c[j];
         }
-        __syncthreads();
-        if (tid < 256) {
-          int before = 0;
-          for (int w = 0; w < wid; ++w) before += sh_scan[w];
-          inc += before;
-          const int rem = s_remaining;
-          if (inc >= rem && inc - h < rem) {  // exactly one thread (bucket counts are >= 0)
-            s_bucket = 255 - tid;
-            s_new_remaining = rem - (inc - h);
-          }
+        int inc = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int n = __shfl_up_sync(0xffffffffu, inc, o);
+          if (lane >= o) inc += n;
         }
-        __syncthreads();
-        if (tid == 0) {
-          s_remaining = s_new_remaining;  // rank of the target inside the bucket (1-based)
-          s_prefix = prefix | ((uint32_t)s_bucket << shift);
+        const int rem = s_remaining;
+        int before = inc - sum;  // keys in buckets above this lane's eight
+        int found = -1, new_rem = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          if (found < 0 && before + c[j] >= rem && before < rem) {
+            found = 255 - (lane * 8 + j);
+            new_rem = rem - before;
+          }
+          before += c[j];
+        }
+        const uint32_t owner = __ballot_sync(0xffffffffu, found >= 0);
+        if (owner == 0) {
+          // k exceeds the number of valid tokens: everything valid executes (lowest bucket)
+          if (lane == 0) {
+            s_prefix = prefix;
+            s_mask = mask | (0xFFu << shift);
+          }
+        } else if (lane == __ffs(owner) - 1) {
+          s_remaining = new_rem;  // rank of the target inside the bucket (1-based)
+          s_prefix = prefix | ((uint32_t)found << shift);
           s_mask = mask | (0xFFu << shift);
         }
-        __syncthreads();
       }
+      __syncthreads();
     }
     tau = s_prefix;
-    need_eq = (p.k > 0) ? s_remaining : 0;
+    need_eq = s_remaining;
   }
 
-  // ordered compaction: each thread owns a contiguous chunk of tokens, read in batches of
-  // independent loads
-  constexpr int kCB = 16;
-  const int chunk = (T + nthr - 1) / nthr;
-  const int t0 = min(T, tid * chunk), t1 = min(T, t0 + chunk);
-  float cs[kCB];
-  bool cv[kCB];
-  auto load_chunk = [&](int base) {
-#pragma unroll
-    for (int j = 0; j < kCB; ++j) {
-      const int t = base + j;
-      cs[j] = 0.f;
-      cv[j] = false;
-      if (t < t1) {
-        cs[j] = __ldcg(p.scores + t);
-        cv[j] = !p.valid || p.valid[t];
-      }
+  const bool topk = p.mode == QTALE_SELECT_TOPK;
+  const bool none = topk && p.k <= 0;
+  // (executes for sure, executes if among the first need_eq equal keys)
+  auto classify = [&](float sc, bool ok, bool& sure, bool& eq) {
+    if (topk) {
+      const uint32_t key = score_key(sc);
+      sure = ok && !none && key > tau;
+      eq = ok && !none && key == tau;
+    } else {
+      sure = ok && sc >= p.theta;
+      eq = false;
     }
   };
-  int n_sel = 0, n_eq = 0;
-  for (int base = t0; base < t1; base += kCB) {
-    load_chunk(base);
-#pragma unroll
-    for (int j = 0; j < kCB; ++j) {
-      if (p.mode == QTALE_SELECT_TOPK) {
-        const uint32_t key = score_key(cs[j]);
-        n_sel += (cv[j] && p.k > 0 && key > tau);
-        n_eq += (cv[j] && p.k > 0 && key == tau);
-      } else {
-        n_sel += (cv[j] && cs[j] >= p.theta);
-      }
-    }
-  }
-  // block-wide exclusive scans of (n_sel, n_eq) with warp shuffles
-  auto block_exclusive = [&](int v, int& total) -> int {
-    const int lane = tid & 31, wid = tid >> 5;
-    int inc = v;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      int n = __shfl_up_sync(0xffffffffu, inc, o);
-      if (lane >= o) inc += n;
-    }
-    __syncthreads();
-    if (lane == 31) sh_scan[wid] = inc;
-    __syncthreads();
-    if (wid == 0) {
-      int w = (lane < (nthr >> 5)) ? sh_scan[lane] : 0;
-      int winc = w;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        int n = __shfl_up_sync(0xffffffffu, winc, o);
-        if (lane >= o) winc += n;
-      }
-      sh_scan[32 + lane] = winc - w;  // exclusive warp offsets
-      if (lane == 31) s_total = winc;
-    }
-    __syncthreads();
-    total = s_total;
-    return inc - v + sh_scan[32 + wid];
-  };
-  int tot_eq = 0, tot_sel = 0;
-  int eq_before = 0;
-  if (p.mode == QTALE_SELECT_TOPK) eq_before = block_exclusive(n_eq, tot_eq);
-  int sel_before = block_exclusive(n_sel, tot_sel);
-  int out = sel_before;
-  int total = tot_sel;
-  if (p.mode == QTALE_SELECT_TOPK) {
-    out += min(eq_before, need_eq);
-    total += min(tot_eq, need_eq);
-  }
 
-  // Sequence bookkeeping of the chunk.  b = sequence of the current token; q = next entry of
-  // cu_seqlens not yet passed.  The thread whose chunk contains token cu_seqlens[q] writes
-  // cu_exec[q] = executed tokens before it; entries equal to T are written at the end.
-  int b = 0, q = 0, seq_start = 0, seq_pos0 = 0, next_bound = T + 1;
-  if (t0 < t1) {
-    int lo = 0, hi = p.B;  // invariant: cu[lo] <= t0 < cu[hi] (cu[B] = T > t0)
+  // sweep 1: executed tokens and tied tokens of each warp's segment
+  int n_sure = 0, n_eq = 0;
+  if (keep) {
+#pragma unroll
+    for (int i = 0; i < kKeep; ++i) {
+      bool sure, eq;
+      classify(ksc[i], (kok >> i) & 1u, sure, eq);
+      n_sure += __popc(__ballot_sync(0xffffffffu, sure));
+      n_eq += __popc(__ballot_sync(0xffffffffu, eq));
+    }
+  } else {
+    for (int i0 = 0; i0 < n_it; i0 += 8) {
+      float sc[8];
+      bool ok[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) load_one(i0 + j, sc[j], ok[j]);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        bool sure, eq;
+        classify(sc[j], ok[j], sure, eq);
+        n_sure += __popc(__ballot_sync(0xffffffffu, sure));
+        n_eq += __popc(__ballot_sync(0xffffffffu, eq));
+      }
+    }
+  }
+  // exclusive scans over the warps (at most 32 of them): sh_scan[0..31] sure, [32..63] tied
+  if (lane == 0) {
+    sh_scan[wid] = n_sure;
+    sh_scan[32 + wid] = n_eq;
+  }
+  __syncthreads();
+  int eq_before = 0, sure_before = 0, tot_eq = 0, tot_sure = 0;
+  for (int w = 0; w < nwarps; ++w) {
+    const int a = sh_scan[w], b = sh_scan[32 + w];
+    if (w < wid) {
+      sure_before += a;
+      eq_before += b;
+    }
+    tot_sure += a;
+    tot_eq += b;
+  }
+  const int total = tot_sure + min(tot_eq, need_eq);
+  int out = sure_before + min(eq_before, need_eq);
+
+  // sweep 2: ordered write of idx / pos, and cu_exec at every sequence start.
+  // b = sequence holding the lane's current token (largest b with cu_seqlens[b] <= t).
+  int b = 0;
+  {
+    const int t = min(w0 + lane, T - 1);
+    int lo = 0, hi = p.B;  // cu[lo] <= t < cu[hi]
     while (hi - lo > 1) {
-      int mid = (lo + hi) >> 1;
-      if (p.cu_seqlens[mid] <= t0) lo = mid; else hi = mid;
+      const int mid = (lo + hi) >> 1;
+      if (__ldg(p.cu_seqlens + mid) <= t) lo = mid; else hi = mid;
     }
     b = lo;
-    q = b + 1;
-    if (p.cu_seqlens[b] == t0) {  // boundaries sitting exactly on the chunk start are ours
-      q = b;
-      while (q > 0 && p.cu_seqlens[q - 1] == t0) --q;
-    }
-    seq_start = p.cu_seqlens[b];
-    seq_pos0 = p.pos0 ? p.pos0[b] : 0;
-    next_bound = p.cu_seqlens[q];
   }
-  int e = eq_before;
-  for (int base = t0; base < t1; base += kCB) {
-    if (chunk > kCB || base != t0) load_chunk(base);  // a single batch is still in registers
-#pragma unroll
-    for (int j = 0; j < kCB; ++j) {
-      const int t = base + j;
-      if (t >= t1) break;
-      while (t >= next_bound) {  // token t opens sequence q (or skips empty ones)
-        p.cu_exec[q] = out;
-        if (q < p.B) {
-          b = q;
-          seq_start = next_bound;
-          seq_pos0 = p.pos0 ? p.pos0[b] : 0;
-        }
-        ++q;
-        next_bound = q <= p.B ? p.cu_seqlens[q] : T + 1;
+  int seq_start = __ldg(p.cu_seqlens + b), seq_end = __ldg(p.cu_seqlens + b + 1);
+  const uint32_t lt = (1u << lane) - 1u;
+  auto emit = [&](int i, float sc, bool ok) {
+    const int t = w0 + 32 * i + lane;
+    bool sure, eq;
+    classify(sc, ok, sure, eq);
+    const uint32_t m_eq = __ballot_sync(0xffffffffu, eq);
+    const bool take = sure || (eq && eq_before + __popc(m_eq & lt) < need_eq);
+    const uint32_t m_take = __ballot_sync(0xffffffffu, take);
+    const int my_out = out + __popc(m_take & lt);
+    if (t < w1) {
+      while (t >= seq_end) {  // move to the sequence holding t (skips empty ones)
+        ++b;
+        seq_start = seq_end;
+        seq_end = __ldg(p.cu_seqlens + b + 1);
       }
-      bool take;
-      if (p.mode == QTALE_SELECT_TOPK) {
-        const uint32_t key = score_key(cs[j]);
-        take = cv[j] && p.k > 0 && key > tau;
-        if (cv[j] && p.k > 0 && key == tau) {
-          take = e < need_eq;
-          ++e;
-        }
-      } else {
-        take = cv[j] && cs[j] >= p.theta;
+      if (t == seq_start) {  // first token of sequence b and of the empty sequences before it
+        for (int q = b; q >= 0 && __ldg(p.cu_seqlens + q) == t; --q) p.cu_exec[q] = my_out;
       }
       if (take) {
-        p.idx[out] = t;
-        p.pos[out] = t - seq_start + seq_pos0;
-        ++out;
+        p.idx[my_out] = t;
+        p.pos[my_out] = t - seq_start + (p.pos0 ? __ldg(p.pos0 + b) : 0);
       }
+    }
+    out += __popc(m_take);
+    eq_before += __popc(m_eq);
+  };
+  if (keep) {
+#pragma unroll
+    for (int i = 0; i < kKeep; ++i) emit(i, ksc[i], (kok >> i) & 1u);
+  } else {
+    for (int i0 = 0; i0 < n_it; i0 += 8) {
+      float sc[8];
+      bool ok[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) load_one(i0 + j, sc[j], ok[j]);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) emit(i0 + j, sc[j], ok[j]);
     }
   }
   if (tid == 0) *p.n_exec = total;

@@ -21,11 +21,16 @@
 // round trip.  The grid is persistent (one CTA per SM) and reads the number of
 // executed tokens from device memory: no launch parameter depends on the routing.
 //
-// Warp roles (384 threads): warps 0 and 2 TMA producers (even / odd K blocks,
+// Warp roles (640 threads): warps 0 and 2 TMA producers (even / odd K blocks,
 // activations and weights), warps 1 and 3 MMA issuers (one per row tile; warp 1
-// also allocates tensor memory),
-// warps 4-11 dequantisers and, at the end of a tile, epilogue: set g = 0, 1 (four
-// warps, one TMEM lane quadrant each) owns row tile g.
+// also allocates tensor memory), warps 4-19 dequantisers and, at the end of a
+// tile, epilogue.  The sixteen form four sets of four warps (one TMEM lane
+// quadrant each): set (g, h) owns row tile g and the K blocks whose running
+// number has parity h, so that one set's "wait for the free slot, store to
+// tensor memory, wait for the store" never delays the arithmetic of the next
+// block: a single set per row tile needs about 1300 cycles per K block, the
+// MMAs of a block 768.  In the epilogue set (g, h) drains every other 16-column
+// chunk of accumulator g.
 #include <cuda.h>
 
 #include <string.h>
@@ -38,14 +43,17 @@ namespace qtale {
 
 using namespace ptx;
 
-constexpr int kGemmThreads = 384;
+constexpr int kGemmThreads = 640;
+constexpr int kDequantWarps = 16;
 constexpr int kTileRows = 128;           // weight rows per tile (MMA M)
 constexpr int kKB = 64;                  // K elements per pipeline step (128 B of 16-bit data)
-constexpr uint32_t kSpinLimit = 1u << 24;
+constexpr uint32_t kWaitSliceNs = 20000;  // longest hardware suspension of one barrier test
+constexpr uint32_t kWaitSlices = 1u << 16;  // tests before a wait gives up (about a second)
 constexpr int kTmemCols = 512;
 constexpr int kAColsPerSlot = kKB / 2;   // two 16-bit values per 32-bit TMEM column
+constexpr int kEpiCols = 16;             // tokens per epilogue chunk
 constexpr int kEpiRowWords = 36;         // padded row (32 fp32 + 4) of the epilogue staging tile
-constexpr int kEpiWarpBytes = 32 * kEpiRowWords * 4;
+constexpr int kEpiWarpBytes = kEpiCols * kEpiRowWords * 4;
 
 template <int TN, int BITS>
 struct GemmCfg {
@@ -64,10 +72,12 @@ struct GemmCfg {
   static constexpr int kAEntriesMax = (kTmemCols - kAColBase) / (kRowTiles * kAColsPerSlot);
   static constexpr int kAEntries = kAEntriesMax > 4 ? 4 : kAEntriesMax;  // K blocks of A in flight
   static constexpr size_t kEpiOffset = (size_t)kXStages * kXStageBytes + (size_t)kWStages * kWStageBytes;
-  static constexpr size_t kSmemBytes = kEpiOffset + 8 * kEpiWarpBytes + 1024;
+  static constexpr size_t kSmemBytes = kEpiOffset + kDequantWarps * kEpiWarpBytes + 1024;
   static_assert(kXStageBytes % 1024 == 0, "swizzled stages must stay 1024-byte aligned");
   static_assert(BITS == 16 || kWTileBytes % 16 == 0, "bulk copies need 16-byte granularity");
   static_assert(BITS == 16 || kAEntries >= 2, "TMEM budget");
+  static_assert(BITS == 16 || (kAEntries % 2 == 0 && kWStages % 2 == 0),
+                "a ring slot must always meet the same parity of the running K block number");
   static_assert(kSmemBytes <= 232448 - 512, "shared memory budget");
 };
 
@@ -105,13 +115,14 @@ struct __align__(8) GemmShared {
   volatile int abort_flag;
 };
 
-// Bounded wait: gives up after kSpinLimit polls, records a timeout and raises
+// Bounded wait: gives up after kWaitSlices suspended tests, records a timeout and raises
 // the CTA-wide abort flag so that every role leaves its loop.
 __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, GemmShared* sh,
                                               int* status) {
-  for (uint32_t it = 0; it < kSpinLimit; ++it) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 255u) == 255u && sh->abort_flag) return false;
+  if (mbar_try_wait(bar, parity)) return true;
+  for (uint32_t it = 0; it < kWaitSlices; ++it) {
+    if (mbar_try_wait_suspend(bar, parity, kWaitSliceNs)) return true;
+    if (sh->abort_flag) return false;
   }
   sh->abort_flag = 1;
   report_device_error(status, QTALE_ERR_TIMEOUT);
@@ -196,7 +207,7 @@ struct Ring {
   }
 };
 
-// ---- epilogue of one 32-column chunk, run by one warp on its 32 weight rows ----
+// ---- epilogue of one 16-column chunk, run by one warp on its 32 weight rows ----
 // `stage` holds the chunk transposed: stage[m * kEpiRowWords + lane_n] = D[lane_n, m].
 // Each lane then owns 8 consecutive output features of one token row, so global
 // accesses are 16 bytes per lane and 64 or 128 contiguous bytes per row.
@@ -208,11 +219,10 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const float*
     const int jc = (lane & 1) * 8;
     const int j0 = nt * 64 + quad * 16 + jc;
     if (j0 >= p.F) return;
-#pragma unroll
-    for (int i = 0; i < 2; ++i) {
-      const int row = i * 16 + (lane >> 1);
+    {
+      const int row = lane >> 1;
       const int m = m0 + row;
-      if (m >= M) continue;
+      if (m >= M) return;
       const float4 g0 = *reinterpret_cast<const float4*>(stage + row * kEpiRowWords + jc);
       const float4 g1 = *reinterpret_cast<const float4*>(stage + row * kEpiRowWords + jc + 4);
       const float4 u0 = *reinterpret_cast<const float4*>(stage + row * kEpiRowWords + 16 + jc);
@@ -234,13 +244,14 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const float*
   const bool n_ok = n0 >= 0;  // no early return: the shuffles below need the whole warp
   const bool gathers = p.epilogue == QTALE_EPI_RESID_F32 || p.epilogue == QTALE_EPI_RESID_SCATTER;
   int my_row = 0;
-  if (gathers && m0 + lane < M) my_row = __ldg(p.idx + m0 + lane);
-  // residual operands of all four row groups are requested before the first use
-  uint4 rb[4];
-  float4 rf[4][2];
-  int tok[4];
+  if (gathers && lane < kEpiCols && m0 + lane < M) my_row = __ldg(p.idx + m0 + lane);
+  // residual operands of both row groups are requested before the first use
+  constexpr int kRowGroups = kEpiCols / 8;
+  uint4 rb[kRowGroups];
+  float4 rf[kRowGroups][2];
+  int tok[kRowGroups];
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
+  for (int i = 0; i < kRowGroups; ++i) {
     const int row = i * 8 + (lane >> 2);
     const int m = m0 + row;
     tok[i] = __shfl_sync(0xffffffffu, my_row, row);
@@ -255,7 +266,7 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const float*
     }
   }
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
+  for (int i = 0; i < kRowGroups; ++i) {
     const int row = i * 8 + (lane >> 2);
     const int m = m0 + row;
     if (m >= M || !n_ok) continue;
@@ -322,7 +333,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
         mbar_init(&sh.a_empty[r][s], 1);
       }
       mbar_init(&sh.d_full[r], 1);
-      mbar_init(&sh.d_empty[r], 4);
+      mbar_init(&sh.d_empty[r], 8);
     }
     sh.abort_flag = 0;
     fence_barrier_init();
@@ -452,22 +463,29 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
     mma_done:;
     }
   } else {
-    // ----------- dequantisers, then epilogue: set g (4 warps) owns row tile g of the CTA -----------
+    // ---- dequantisers, then epilogue: set (g, h) owns row tile g and the K blocks of parity h ----
     const int quad = warp & 3;
     const int L = quad * 32 + lane;
-    const int g = (warp - 4) >> 2;
+    const int g = ((warp - 4) >> 2) & 1;
+    const int h = (warp - 4) >> 3;
     float* stage = epi_base + (size_t)(warp - 4) * (kEpiWarpBytes / 4);
     Ring rw, ra;
     uint32_t dph = 0;
+    int count = 0;  // running K block number, as in the producers
     for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
       const int rp = tile % n_rp, mt = tile / n_rp;
       const int nt = rp * RT + g;
       const bool has_tile = g < RT && nt < p.n_tiles;
       if (BITS != 16) {
-        for (int kb = 0; kb < nkb; ++kb) {
+        for (int kb = 0; kb < nkb; ++kb, ++count) {
+          if ((count & 1) != h) {  // the other set's block (ring slots alternate with the parity)
+            rw.advance(SW);
+            ra.advance(SA);
+            continue;
+          }
           uint32_t cw[8];
           uint32_t sz = 0;
-          // every warp, with or without a tile, takes part in each handshake exactly once
+          // every warp of the set, with or without a tile, takes part in each handshake once
           if (!wait_or_abort(&sh.full_w[rw.s], rw.ph, &sh, p.status)) goto role_done;
           if (has_tile) {
             const unsigned char* st = w_base + (size_t)rw.s * Cfg::kWStageBytes + g * Cfg::kWTileBytes;
@@ -486,27 +504,29 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
           }
           __syncwarp();
           if (lane == 0) mbar_arrive(&sh.empty_w[rw.s]);
-          // dequantise into registers first; only the TMEM stores wait for the free A slot
-          uint32_t r[32];
-          if (has_tile) {
-            float C[5], Sc[5];
-            uint32_t z_lo = 0, z_hi = 0, scale2 = 0;
-            if (ACT == 1) {
-              const uint32_t zero2 = (sz >> 16) * 0x00010001u;          // (zero, zero) as halves
-              scale2 = (sz & 0xFFFFu) * 0x00010001u;
-              z_lo = h2_sub(zero2, 0xE400E400u);                        // zero - (-1024) = 1024 + zero
-              z_hi = h2_sub(0xD400D400u, zero2);                        // -64 - zero
-            } else {
-              const float scale = __half2float(__ushort_as_half((unsigned short)(sz & 0xFFFFu)));
-              const float zero = __half2float(__ushort_as_half((unsigned short)(sz >> 16)));
+          // The first half of the block (32 input features) is dequantised before the wait for
+          // the free A slot, the second half while the first half's store is in flight.
+          uint32_t r[16];
+          float C[5], Sc[5];
+          uint32_t z_lo = 0, z_hi = 0, scale2 = 0;
+          if (ACT == 1) {
+            const uint32_t zero2 = (sz >> 16) * 0x00010001u;          // (zero, zero) as halves
+            scale2 = (sz & 0xFFFFu) * 0x00010001u;
+            z_lo = h2_sub(zero2, 0xE400E400u);                        // zero - (-1024) = 1024 + zero
+            z_hi = h2_sub(0xD400D400u, zero2);                        // -64 - zero
+          } else {
+            const float scale = __half2float(__ushort_as_half((unsigned short)(sz & 0xFFFFu)));
+            const float zero = __half2float(__ushort_as_half((unsigned short)(sz >> 16)));
 #pragma unroll
-              for (int i = 0; i < 5; ++i) {
-                C[i] = 8388608.f + zero * (float)(1 << (4 * i));
-                Sc[i] = scale * (1.f / (float)(1 << (4 * i)));
-              }
+            for (int i = 0; i < 5; ++i) {
+              C[i] = 8388608.f + zero * (float)(1 << (4 * i));
+              Sc[i] = scale * (1.f / (float)(1 << (4 * i)));
             }
+          }
+          auto dequant_half = [&](int half) {
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
+            for (int v = 0; v < 4; ++v) {
+              const int u = half * 4 + v;
               uint32_t t;
               if (BITS == 4) {
                 t = cw[u];
@@ -521,16 +541,19 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
                 t = (a2 & 0x33333333u) | (b1 & 0xCCCCCCCCu);
               }
               constexpr uint32_t QM = BITS == 4 ? 0xFu : 0x7u;
-              if (ACT == 1) dequant8_f16<QM>(t, z_lo, z_hi, scale2, r + 4 * u);
-              else dequant8<QM, ACT>(t, C, Sc, r + 4 * u);
+              if (ACT == 1) dequant8_f16<QM>(t, z_lo, z_hi, scale2, r + 4 * v);
+              else dequant8<QM, ACT>(t, C, Sc, r + 4 * v);
             }
-          }
+          };
+          if (has_tile) dequant_half(0);
           if (!wait_or_abort(&sh.a_empty[g][ra.s], ra.ph ^ 1u, &sh, p.status)) goto role_done;
           if (has_tile) {
             tc_fence_after();
             const uint32_t a_taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + Cfg::kAColBase +
                                      (ra.s * RT + g) * kAColsPerSlot;
-            tmem_st_x32(a_taddr, r);
+            tmem_st_x16(a_taddr, r);
+            dequant_half(1);  // the store has taken its operands: the registers are free again
+            tmem_st_x16(a_taddr + kAColsPerSlot / 2, r);
             tmem_wait_st();
             tc_fence_before();
           }
@@ -540,24 +563,25 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
           ra.advance(SA);
         }
       }
-      // ---- epilogue of this tile: set g drains accumulator g, one lane quadrant per warp ----
+      // ---- epilogue of this tile: sets (g, 0) and (g, 1) drain alternate 16-column chunks of
+      // ---- accumulator g, one lane quadrant per warp ----
       if (!wait_or_abort(&sh.d_full[g], dph, &sh, p.status)) goto role_done;
       tc_fence_after();
       if (has_tile) {
         const int m_base = mt * TW;
         const uint32_t d_taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + g * Cfg::kDCols;
-        uint32_t r[32];
-        tmem_ld_x32(d_taddr, r);
+        uint32_t r[kEpiCols];
+        if (m_base + h * kEpiCols < M) tmem_ld_x16(d_taddr + h * kEpiCols, r);
 #pragma unroll 1
-        for (int c0 = 0; c0 < TW; c0 += 32) {
+        for (int c0 = h * kEpiCols; c0 < TW; c0 += 2 * kEpiCols) {
           const int m0 = m_base + c0;
           if (m0 >= M) break;
           tmem_wait_ld();
 #pragma unroll
-          for (int c = 0; c < 32; ++c) stage[c * kEpiRowWords + lane] = __uint_as_float(r[c]);
+          for (int c = 0; c < kEpiCols; ++c) stage[c * kEpiRowWords + lane] = __uint_as_float(r[c]);
           __syncwarp();
           // the next chunk's accumulator read overlaps this chunk's global traffic
-          if (c0 + 32 < TW && m0 + 32 < M) tmem_ld_x32(d_taddr + c0 + 32, r);
+          if (c0 + 2 * kEpiCols < TW && m0 + 2 * kEpiCols < M) tmem_ld_x16(d_taddr + c0 + 2 * kEpiCols, r);
           epilogue_chunk<ACT>(p, stage, lane, nt, quad, m0, M);
           __syncwarp();
         }
@@ -577,6 +601,331 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// ------------------------------------------------------------------------------
+// CTA-pair kernel (prefill shapes): one tile = 256 weight rows x up to 256 tokens,
+// computed by two CTAs of a cluster with tcgen05.mma.cta_group::2.
+//
+// Each CTA dequantises its own 128 weight rows into its own tensor memory (A
+// operand, ring of 8 slots of 64 input features) and loads its own half of the
+// tile's tokens into its own shared memory (B operand, ring of 8 stages of 16 KB);
+// the pair leader (cluster rank 0) issues the MMAs for both CTAs.  Against the
+// single-CTA kernel this halves the B-operand shared-memory reads and the
+// activation bytes loaded per flop, makes every dequantised weight serve 256
+// tokens instead of 192, and leaves room for eight A slots instead of two, so the
+// chain "MMA done -> slot free -> store to tensor memory -> MMA" is no longer exposed.
+//
+// Warp roles per CTA (640 threads): warp 0 activation producer, warp 2 weight
+// producer, warp 1 MMA issuer (leader only; in both CTAs it allocates tensor memory),
+// warp 3 idle, warps 4-19 dequantisers / epilogue in four sets of four warps: set j
+// owns the K blocks whose running number is j modulo 4.
+//
+// Barriers.  slot_free[s] (both CTAs, multicast commit of the leader): activation stage
+// s and A slot s have been consumed.  ready[s] (leader): both CTAs' activation loads of
+// stage s have landed and both CTAs have stored A slot s, so the issuer tests one barrier
+// per K block.  full_w / empty_w (local): packed weights.  d_full (both, multicast commit):
+// the accumulator is complete.  d_empty (leader): both CTAs have drained it.
+// ------------------------------------------------------------------------------
+constexpr int kPairStages = 8;           // activation stages = A slots = weight stages
+constexpr int kPairTokens = 256;         // tokens per pair tile (128 per CTA)
+constexpr int kPairDCols = kPairTokens;  // accumulator columns
+
+template <int BITS>
+struct PairCfg {
+  static constexpr int kXStageBytes = (kPairTokens / 2) * 128;
+  static constexpr int kWCodeBytes = kTileRows * kKB * BITS / 8;
+  static constexpr int kWTileBytes = kWCodeBytes + kTileRows * 4;
+  static constexpr size_t kWOffset = (size_t)kPairStages * kXStageBytes;
+  static constexpr size_t kEpiOffset = kWOffset + (size_t)kPairStages * kWTileBytes;
+  static constexpr size_t kSmemBytes = kEpiOffset + kDequantWarps * kEpiWarpBytes + 1024;
+  static_assert(kWTileBytes % 16 == 0, "bulk copies need 16-byte granularity");
+  static_assert(kPairDCols + kPairStages * kAColsPerSlot <= kTmemCols, "TMEM budget");
+  static_assert(kPairStages == 8, "ring index and phase are taken from the low bits of the block count");
+  static_assert(kSmemBytes <= 232448 - 512, "shared memory budget");
+};
+
+// Activation tensor maps for per-CTA token boxes of 16, 32, ..., 128 rows (index rows / 16 - 1).
+struct PairTmapSet {
+  CUtensorMap m[8];
+};
+
+struct __align__(8) PairShared {
+  uint64_t ready[kPairStages];
+  uint64_t slot_free[kPairStages];
+  uint64_t full_w[kPairStages], empty_w[kPairStages];
+  uint64_t d_full, d_empty;
+  uint32_t tmem_base;
+  volatile int abort_flag;
+};
+
+__device__ __forceinline__ bool pair_wait(uint64_t* bar, uint32_t parity, PairShared* sh, int* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  for (uint32_t it = 0; it < kWaitSlices; ++it) {
+    if (mbar_try_wait_suspend(bar, parity, kWaitSliceNs)) return true;
+    if (sh->abort_flag) return false;
+  }
+  sh->abort_flag = 1;
+  report_device_error(status, QTALE_ERR_TIMEOUT);
+  return false;
+}
+
+template <int BITS, int ACT>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
+    wq_gemm_pair_kernel(const __grid_constant__ PairTmapSet tmaps_x, const GemmParams p) {
+  using Cfg = PairCfg<BITS>;
+  constexpr int S = kPairStages;
+  extern __shared__ unsigned char smem_dyn[];
+  __shared__ PairShared sh;
+  unsigned char* x_base = reinterpret_cast<unsigned char*>(
+      (reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~static_cast<uintptr_t>(1023));
+  unsigned char* w_base = x_base + Cfg::kWOffset;
+  float* epi_base = reinterpret_cast<float*>(x_base + Cfg::kEpiOffset);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();  // 0: pair leader
+  const bool leader = rank == 0;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < S; ++s) {
+      mbar_init(&sh.ready[s], 9);      // the leader's producer (expecting both halves' bytes) and
+                                       // four dequantiser warps of each CTA
+      mbar_init(&sh.slot_free[s], 1);  // one multicast commit
+      mbar_init(&sh.full_w[s], 1);
+      mbar_init(&sh.empty_w[s], 4);    // the four warps of the set that read the stage
+    }
+    mbar_init(&sh.d_full, 1);
+    mbar_init(&sh.d_empty, 2 * kDequantWarps);
+    sh.abort_flag = 0;
+    fence_barrier_init();
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(&sh.tmem_base, kTmemCols);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync();  // both CTAs' barriers exist before anything is signalled across the pair
+  tc_fence_after();
+  const uint32_t tmem_base = sh.tmem_base;
+
+  int M = p.M_cap;
+  if (p.m_dev) M = min(M, *p.m_dev);
+  M = max(M, 0);
+  const int n_rp = (p.n_tiles + 1) / 2;  // pairs of row tiles: one per tile of the CTA pair
+  const int nkb = p.nkb;
+  const int n_clusters = gridDim.x >> 1;
+  const int cluster_id = blockIdx.x >> 1;
+  // Token-tile width: the multiple of 32 (at most 256) that minimises (waves of the persistent
+  // grid) x (columns per tile + fixed per-tile cost).
+  int TW = kPairTokens;
+  {
+    const int fixed = 1408 / max(nkb, 1);
+    long best = -1;
+    for (int w = kPairTokens; w >= 32; w -= 32) {
+      const long tiles = (long)((M + w - 1) / w) * n_rp;
+      const long cost = ((tiles + n_clusters - 1) / n_clusters) * (max(w, 128) + fixed);
+      if (best < 0 || cost < best) { best = cost; TW = w; }
+    }
+  }
+  const int HW = TW >> 1;  // tokens of this CTA's half
+  const CUtensorMap* tmap_x = &tmaps_x.m[HW / 16 - 1];
+  const int n_mt = (M + TW - 1) / TW;
+  const int total_tiles = n_mt * n_rp;
+
+  if (warp == 0) {
+    // ---------------- activation producer: this CTA's half of the tile's tokens ----------------
+    if (lane == 0) {
+      const uint32_t ready_leader = map_to_cta(smem_u32(&sh.ready[0]), 0);
+      int count = 0;
+      for (int tile = cluster_id; tile < total_tiles; tile += n_clusters) {
+        const int mt = tile / n_rp;
+        for (int kb = 0; kb < nkb; ++kb, ++count) {
+          const int s = count % S;
+          const uint32_t ph = (uint32_t)(count / S) & 1u;
+          if (!pair_wait(&sh.slot_free[s], ph ^ 1u, &sh, p.status)) goto x_done;
+          if (leader) mbar_arrive_expect_tx(&sh.ready[s], (uint32_t)TW * 128u);  // both halves
+          tma_load_2d_pair(x_base + (size_t)s * Cfg::kXStageBytes, tmap_x, ready_leader + 8u * s,
+                           kb * kKB, mt * TW + (int)rank * HW);
+        }
+      }
+    x_done:;
+    }
+  } else if (warp == 2) {
+    // ---------------- weight producer: this CTA's row tile ----------------
+    if (lane == 0) {
+      int count = 0;
+      for (int tile = cluster_id; tile < total_tiles; tile += n_clusters) {
+        const int rp = tile % n_rp;
+        for (int kb = 0; kb < nkb; ++kb, ++count) {
+          const int s = count % S;
+          const uint32_t ph = (uint32_t)(count / S) & 1u;
+          if (!pair_wait(&sh.empty_w[s], ph ^ 1u, &sh, p.status)) goto w_done;
+          mbar_arrive_expect_tx(&sh.full_w[s], Cfg::kWTileBytes);
+          bulk_load(w_base + (size_t)s * Cfg::kWTileBytes,
+                    p.packed + (((size_t)rp * nkb + kb) * 2 + rank) * Cfg::kWTileBytes,
+                    Cfg::kWTileBytes, &sh.full_w[s]);
+        }
+      }
+    w_done:;
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer (pair leader) ----------------
+    // One thread, so every instruction's latency is exposed: the loop tests one barrier per K
+    // block, and tests the next block's barrier before it issues this block's MMAs so that the
+    // answer arrives while they are being issued.
+    if (leader && lane == 0) {
+      const uint32_t idesc = idesc_16bit_f32(256, TW, ACT == 1);
+      const uint64_t b_desc0 = smem_desc_sw128(smem_u32(x_base));
+      const uint32_t a_tmem0 = tmem_base + kPairDCols;
+      const long total_kb = (long)((total_tiles - cluster_id + n_clusters - 1) / n_clusters) * nkb;
+      uint32_t count = 0;
+      uint32_t dph = 0;
+      bool ready_now = false;  // the barrier of block `count` is already known to be complete
+      for (int tile = cluster_id; tile < total_tiles; tile += n_clusters) {
+        if (!pair_wait(&sh.d_empty, dph ^ 1u, &sh, p.status)) goto mma_done;
+        for (int kb = 0; kb < nkb; ++kb, ++count) {
+          const uint32_t s = count & (S - 1);
+          if (!ready_now && !pair_wait(&sh.ready[s], (count >> 3) & 1u, &sh, p.status)) goto mma_done;
+          tc_fence_after();
+          const uint32_t nxt = count + 1;
+          const bool more = (long)nxt < total_kb;
+          const bool next_ok = more && mbar_try_wait(&sh.ready[nxt & (S - 1)], (nxt >> 3) & 1u);
+          const uint64_t b_desc = b_desc0 + (uint64_t)(s * (Cfg::kXStageBytes >> 4));
+          const uint32_t a_tmem = a_tmem0 + s * kAColsPerSlot;
+#pragma unroll
+          for (int j = 0; j < kKB / 16; ++j)
+            mma_ts_pair(tmem_base, a_tmem + j * 8, b_desc + 2u * j, idesc, (kb | j) != 0 ? 1u : 0u);
+          mma_commit_pair(&sh.slot_free[s], 3);
+          ready_now = next_ok;
+        }
+        mma_commit_pair(&sh.d_full, 3);
+        dph ^= 1u;
+      }
+    mma_done:;
+    }
+  } else if (warp >= 4) {
+    // ---------------- dequantisers, then epilogue ----------------
+    const int quad = warp & 3;
+    const int L = quad * 32 + lane;
+    const int set = (warp - 4) >> 2;
+    float* stage = epi_base + (size_t)(warp - 4) * (kEpiWarpBytes / 4);
+    const uint32_t ready_leader = map_to_cta(smem_u32(&sh.ready[0]), 0);
+    const uint32_t d_empty_leader = map_to_cta(smem_u32(&sh.d_empty), 0);
+    uint32_t dph = 0;
+    int count = 0;
+    for (int tile = cluster_id; tile < total_tiles; tile += n_clusters) {
+      const int rp = tile % n_rp, mt = tile / n_rp;
+      const int nt = rp * 2 + (int)rank;
+      for (int kb = 0; kb < nkb; ++kb, ++count) {
+        if ((count & 3) != set) continue;
+        const int s = count % S;
+        const uint32_t ph = (uint32_t)(count / S) & 1u;
+        uint32_t cw[8];
+        if (!pair_wait(&sh.full_w[s], ph, &sh, p.status)) goto role_done;
+        const unsigned char* st = w_base + (size_t)s * Cfg::kWTileBytes;
+        const uint32_t sz = reinterpret_cast<const uint32_t*>(st + Cfg::kWCodeBytes)[L];
+        if (BITS == 4) {
+          const uint4 w0 = reinterpret_cast<const uint4*>(st)[L];
+          const uint4 w1 = reinterpret_cast<const uint4*>(st)[kTileRows + L];
+          cw[0] = w0.x; cw[1] = w0.y; cw[2] = w0.z; cw[3] = w0.w;
+          cw[4] = w1.x; cw[5] = w1.y; cw[6] = w1.z; cw[7] = w1.w;
+        } else {
+          const uint4 a = reinterpret_cast<const uint4*>(st)[L];
+          const uint2 b = reinterpret_cast<const uint2*>(st + kTileRows * 16)[L];
+          cw[0] = a.x; cw[1] = a.y; cw[2] = a.z; cw[3] = a.w;
+          cw[4] = b.x; cw[5] = b.y; cw[6] = 0; cw[7] = 0;
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh.empty_w[s]);
+        uint32_t r[16];
+        float C[5], Sc[5];
+        uint32_t z_lo = 0, z_hi = 0, scale2 = 0;
+        if (ACT == 1) {
+          const uint32_t zero2 = (sz >> 16) * 0x00010001u;
+          scale2 = (sz & 0xFFFFu) * 0x00010001u;
+          z_lo = h2_sub(zero2, 0xE400E400u);
+          z_hi = h2_sub(0xD400D400u, zero2);
+        } else {
+          const float scale = __half2float(__ushort_as_half((unsigned short)(sz & 0xFFFFu)));
+          const float zero = __half2float(__ushort_as_half((unsigned short)(sz >> 16)));
+#pragma unroll
+          for (int i = 0; i < 5; ++i) {
+            C[i] = 8388608.f + zero * (float)(1 << (4 * i));
+            Sc[i] = scale * (1.f / (float)(1 << (4 * i)));
+          }
+        }
+        auto dequant_half = [&](int half) {
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            const int u = half * 4 + v;
+            uint32_t t;
+            if (BITS == 4) {
+              t = cw[u];
+            } else {
+              const uint32_t a2 = (u & 1) ? (cw[u >> 1] >> 2) : cw[u >> 1];
+              const int rr = u & 3;
+              const uint32_t bw = cw[4 + (u >> 2)];
+              const uint32_t b1 = rr == 0 ? (bw << 2) : rr == 1 ? (bw << 1) : rr == 2 ? bw : (bw >> 1);
+              t = (a2 & 0x33333333u) | (b1 & 0xCCCCCCCCu);
+            }
+            constexpr uint32_t QM = BITS == 4 ? 0xFu : 0x7u;
+            if (ACT == 1) dequant8_f16<QM>(t, z_lo, z_hi, scale2, r + 4 * v);
+            else dequant8<QM, ACT>(t, C, Sc, r + 4 * v);
+          }
+        };
+        dequant_half(0);
+        if (!pair_wait(&sh.slot_free[s], ph ^ 1u, &sh, p.status)) goto role_done;
+        tc_fence_after();
+        const uint32_t a_taddr =
+            tmem_base + ((uint32_t)(quad * 32) << 16) + kPairDCols + s * kAColsPerSlot;
+        tmem_st_x16(a_taddr, r);
+        dequant_half(1);
+        tmem_st_x16(a_taddr + kAColsPerSlot / 2, r);
+        tmem_wait_st();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(ready_leader + 8u * s);
+      }
+      // ---- epilogue: set j drains the 16-column chunks j, j + 4, ... of this CTA's accumulator ----
+      if (!pair_wait(&sh.d_full, dph, &sh, p.status)) goto role_done;
+      tc_fence_after();
+      {
+        const int m_base = mt * TW;
+        const uint32_t d_taddr = tmem_base + ((uint32_t)(quad * 32) << 16);
+        uint32_t r[kEpiCols];
+        if (set * kEpiCols < TW && m_base + set * kEpiCols < M) tmem_ld_x16(d_taddr + set * kEpiCols, r);
+#pragma unroll 1
+        for (int c0 = set * kEpiCols; c0 < TW; c0 += 4 * kEpiCols) {
+          const int m0 = m_base + c0;
+          if (m0 >= M) break;
+          tmem_wait_ld();
+#pragma unroll
+          for (int c = 0; c < kEpiCols; ++c) stage[c * kEpiRowWords + lane] = __uint_as_float(r[c]);
+          __syncwarp();
+          if (c0 + 4 * kEpiCols < TW && m0 + 4 * kEpiCols < M) tmem_ld_x16(d_taddr + c0 + 4 * kEpiCols, r);
+          epilogue_chunk<ACT>(p, stage, lane, nt, quad, m0, M);
+          __syncwarp();
+        }
+        tmem_wait_ld();
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(d_empty_leader);
+      dph ^= 1u;
+    }
+  role_done:;
+  }
+
+  // teardown: both CTAs are done with tensor memory and with each other's barriers
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc_pair(tmem_base, kTmemCols);
   }
 }
 
@@ -657,6 +1006,57 @@ static int dispatch_tn(const TmapSet& tx, const CUtensorMap& tw, const GemmParam
   return launch_gemm<192, BITS, ACT>(tx, tw, p, s);
 }
 
+// ---- CTA-pair kernel ----
+template <int BITS, int ACT>
+static int launch_pair(const PairTmapSet& tx, const GemmParams& p, cudaStream_t s) {
+  using Cfg = PairCfg<BITS>;
+  static int clusters_of_device[64] = {0};
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (dev < 0 || dev >= 64) return QTALE_ERR_CUDA;
+  if (clusters_of_device[dev] == 0) {
+    if (cudaFuncSetAttribute(wq_gemm_pair_kernel<BITS, ACT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)Cfg::kSmemBytes) != cudaSuccess)
+      return QTALE_ERR_CUDA;
+    // how many CTA pairs the device can hold at once: the persistent grid is sized to it
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3((unsigned)sm_count() & ~1u);
+    cfg.blockDim = dim3(kGemmThreads);
+    cfg.dynamicSmemBytes = Cfg::kSmemBytes;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2;
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, wq_gemm_pair_kernel<BITS, ACT>, &cfg) != cudaSuccess || n < 1) {
+      cudaGetLastError();
+      n = sm_count() / 2;
+    }
+    clusters_of_device[dev] = n;
+  }
+  const int max_tiles = ((p.M_cap + 31) / 32) * ((p.n_tiles + 1) / 2);
+  int clusters = clusters_of_device[dev];
+  if (clusters > max_tiles) clusters = max_tiles;
+  if (clusters < 1) clusters = 1;
+  wq_gemm_pair_kernel<BITS, ACT><<<2 * clusters, kGemmThreads, Cfg::kSmemBytes, s>>>(tx, p);
+  return launch_status(cudaGetLastError());
+}
+
+static int make_pair_tmaps(PairTmapSet* set, const void* base, int rows, int cols, int ld, int act) {
+  for (int h = 16; h <= kPairTokens / 2; h += 16) {
+    const int rc = make_tmap_16(&set->m[h / 16 - 1], base, rows, cols, ld, h, act);
+    if (rc != QTALE_OK) return rc;
+  }
+  return QTALE_OK;
+}
+
+// Token counts from which the CTA-pair kernel is used (below, a tile of 256 tokens is mostly padding).
+constexpr int kPairMinTokens = 129;
+
 static int pick_tn(int M_cap) { return M_cap <= 64 ? 64 : (M_cap <= 128 ? 128 : 192); }
 
 size_t wq_blob_bytes(int N, int K, int bits, int group, int row_mode, WqGeometry* g) {
@@ -702,6 +1102,15 @@ int wq_gemm_launch(const void* a, int lda, const int32_t* m_dev, int M_cap,
     p.ld_dst = epi->ld_dst;
   }
   p.status = device_status_ptr();
+  if (M_cap >= kPairMinTokens) {
+    PairTmapSet px;
+    memset(&px, 0, sizeof(px));
+    const int rc = make_pair_tmaps(&px, a, M_cap, w->K, lda, act);
+    if (rc != QTALE_OK) return rc;
+    if (act == QTALE_ACT_F16)
+      return w->bits == 4 ? launch_pair<4, 1>(px, p, s) : launch_pair<3, 1>(px, p, s);
+    return w->bits == 4 ? launch_pair<4, 0>(px, p, s) : launch_pair<3, 0>(px, p, s);
+  }
   const int tn = pick_tn(M_cap);
   TmapSet tx;
   CUtensorMap tw;
