@@ -609,40 +609,48 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
 // computed by two CTAs of a cluster with tcgen05.mma.cta_group::2.
 //
 // Each CTA dequantises its own 128 weight rows into its own tensor memory (A
-// operand, ring of 8 slots of 64 input features) and loads its own half of the
-// tile's tokens into its own shared memory (B operand, ring of 8 stages of 16 KB);
+// operand, ring of 4 slots of 128 input features) and loads its own half of the
+// tile's tokens into its own shared memory (B operand, ring of 4 stages of 32 KB);
+// a pipeline step is two 64-wide K blocks, so that the single issuing thread and
+// the dequantisers pay their barrier traffic once per eight MMAs;
 // the pair leader (cluster rank 0) issues the MMAs for both CTAs.  Against the
 // single-CTA kernel this halves the B-operand shared-memory reads and the
 // activation bytes loaded per flop, makes every dequantised weight serve 256
-// tokens instead of 192, and leaves room for eight A slots instead of two, so the
-// chain "MMA done -> slot free -> store to tensor memory -> MMA" is no longer exposed.
+// tokens instead of 192, and leaves room for 512 input features of dequantised weights
+// in flight instead of 128, so the chain "MMA done -> slot free -> store to tensor
+// memory -> MMA" is no longer exposed.
 //
 // Warp roles per CTA (640 threads): warp 0 activation producer, warp 2 weight
 // producer, warp 1 MMA issuer (leader only; in both CTAs it allocates tensor memory),
 // warp 3 idle, warps 4-19 dequantisers / epilogue in four sets of four warps: set j
-// owns the K blocks whose running number is j modulo 4.
+// owns the pipeline steps whose running number is j modulo 4, i.e. ring slot j.
 //
 // Barriers.  slot_free[s] (both CTAs, multicast commit of the leader): activation stage
 // s and A slot s have been consumed.  ready[s] (leader): both CTAs' activation loads of
 // stage s have landed and both CTAs have stored A slot s, so the issuer tests one barrier
-// per K block.  full_w / empty_w (local): packed weights.  d_full (both, multicast commit):
+// per step.  full_w / empty_w (local): packed weights.  d_full (both, multicast commit):
 // the accumulator is complete.  d_empty (leader): both CTAs have drained it.
 // ------------------------------------------------------------------------------
-constexpr int kPairStages = 8;           // activation stages = A slots = weight stages
+constexpr int kPairStages = 4;           // activation stages = A slots = weight stages
+constexpr int kPairBlocks = 2;           // 64-wide K blocks per pipeline step
 constexpr int kPairTokens = 256;         // tokens per pair tile (128 per CTA)
 constexpr int kPairDCols = kPairTokens;  // accumulator columns
 
 template <int BITS>
 struct PairCfg {
-  static constexpr int kXStageBytes = (kPairTokens / 2) * 128;
+  static constexpr int kXBlockBytes = (kPairTokens / 2) * 128;   // one K block of this CTA's tokens
+  static constexpr int kXStageBytes = kPairBlocks * kXBlockBytes;
   static constexpr int kWCodeBytes = kTileRows * kKB * BITS / 8;
-  static constexpr int kWTileBytes = kWCodeBytes + kTileRows * 4;
+  static constexpr int kWTileBytes = kWCodeBytes + kTileRows * 4;  // one row tile, one K block
+  static constexpr int kWStageBytes = kPairBlocks * kWTileBytes;
+  static constexpr int kAColsPerStage = kPairBlocks * kAColsPerSlot;
   static constexpr size_t kWOffset = (size_t)kPairStages * kXStageBytes;
-  static constexpr size_t kEpiOffset = kWOffset + (size_t)kPairStages * kWTileBytes;
+  static constexpr size_t kEpiOffset = kWOffset + (size_t)kPairStages * kWStageBytes;
   static constexpr size_t kSmemBytes = kEpiOffset + kDequantWarps * kEpiWarpBytes + 1024;
   static_assert(kWTileBytes % 16 == 0, "bulk copies need 16-byte granularity");
-  static_assert(kPairDCols + kPairStages * kAColsPerSlot <= kTmemCols, "TMEM budget");
-  static_assert(kPairStages == 8, "ring index and phase are taken from the low bits of the block count");
+  static_assert(kPairDCols + kPairStages * kAColsPerStage <= kTmemCols, "TMEM budget");
+  static_assert(kPairStages == 4, "ring slot = low two bits of the step count = dequantiser set");
+  static_assert(kXBlockBytes % 1024 == 0, "swizzled blocks must stay 1024-byte aligned");
   static_assert(kSmemBytes <= 232448 - 512, "shared memory budget");
 };
 
@@ -719,14 +727,15 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
   const int n_clusters = gridDim.x >> 1;
   const int cluster_id = blockIdx.x >> 1;
   // Token-tile width: the multiple of 32 (at most 256) that minimises (waves of the persistent
-  // grid) x (columns per tile + fixed per-tile cost).
+  // grid) x (time of a tile).  Below about 224 tokens a pipeline step is paced by the
+  // dequantisers and the issuing thread, not by the MMAs, so narrower tiles are not faster.
   int TW = kPairTokens;
   {
     const int fixed = 1408 / max(nkb, 1);
     long best = -1;
     for (int w = kPairTokens; w >= 32; w -= 32) {
       const long tiles = (long)((M + w - 1) / w) * n_rp;
-      const long cost = ((tiles + n_clusters - 1) / n_clusters) * (max(w, 128) + fixed);
+      const long cost = ((tiles + n_clusters - 1) / n_clusters) * (max(w, 224) + fixed);
       if (best < 0 || cost < best) { best = cost; TW = w; }
     }
   }
@@ -735,20 +744,23 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
   const int n_mt = (M + TW - 1) / TW;
   const int total_tiles = n_mt * n_rp;
 
+  const int n_st = (nkb + kPairBlocks - 1) / kPairBlocks;  // pipeline steps per tile
+
   if (warp == 0) {
     // ---------------- activation producer: this CTA's half of the tile's tokens ----------------
     if (lane == 0) {
       const uint32_t ready_leader = map_to_cta(smem_u32(&sh.ready[0]), 0);
-      int count = 0;
+      uint32_t count = 0;
       for (int tile = cluster_id; tile < total_tiles; tile += n_clusters) {
         const int mt = tile / n_rp;
-        for (int kb = 0; kb < nkb; ++kb, ++count) {
-          const int s = count % S;
-          const uint32_t ph = (uint32_t)(count / S) & 1u;
+        for (int st = 0; st < n_st; ++st, ++count) {
+          const uint32_t s = count & (S - 1), ph = (count >> 2) & 1u;
+          const int nb = min(kPairBlocks, nkb - st * kPairBlocks);
           if (!pair_wait(&sh.slot_free[s], ph ^ 1u, &sh, p.status)) goto x_done;
-          if (leader) mbar_arrive_expect_tx(&sh.ready[s], (uint32_t)TW * 128u);  // both halves
-          tma_load_2d_pair(x_base + (size_t)s * Cfg::kXStageBytes, tmap_x, ready_leader + 8u * s,
-                           kb * kKB, mt * TW + (int)rank * HW);
+          if (leader) mbar_arrive_expect_tx(&sh.ready[s], (uint32_t)(TW * 128 * nb));  // both halves
+          for (int b = 0; b < nb; ++b)
+            tma_load_2d_pair(x_base + (size_t)s * Cfg::kXStageBytes + (size_t)b * Cfg::kXBlockBytes, tmap_x,
+                             ready_leader + 8u * s, (st * kPairBlocks + b) * kKB, mt * TW + (int)rank * HW);
         }
       }
     x_done:;
@@ -756,48 +768,56 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
   } else if (warp == 2) {
     // ---------------- weight producer: this CTA's row tile ----------------
     if (lane == 0) {
-      int count = 0;
+      uint32_t count = 0;
       for (int tile = cluster_id; tile < total_tiles; tile += n_clusters) {
         const int rp = tile % n_rp;
-        for (int kb = 0; kb < nkb; ++kb, ++count) {
-          const int s = count % S;
-          const uint32_t ph = (uint32_t)(count / S) & 1u;
+        for (int st = 0; st < n_st; ++st, ++count) {
+          const uint32_t s = count & (S - 1), ph = (count >> 2) & 1u;
+          const int nb = min(kPairBlocks, nkb - st * kPairBlocks);
           if (!pair_wait(&sh.empty_w[s], ph ^ 1u, &sh, p.status)) goto w_done;
-          mbar_arrive_expect_tx(&sh.full_w[s], Cfg::kWTileBytes);
-          bulk_load(w_base + (size_t)s * Cfg::kWTileBytes,
-                    p.packed + (((size_t)rp * nkb + kb) * 2 + rank) * Cfg::kWTileBytes,
-                    Cfg::kWTileBytes, &sh.full_w[s]);
+          mbar_arrive_expect_tx(&sh.full_w[s], (uint32_t)(Cfg::kWTileBytes * nb));
+          for (int b = 0; b < nb; ++b)
+            bulk_load(w_base + (size_t)s * Cfg::kWStageBytes + (size_t)b * Cfg::kWTileBytes,
+                      p.packed + (((size_t)rp * nkb + st * kPairBlocks + b) * 2 + rank) * Cfg::kWTileBytes,
+                      Cfg::kWTileBytes, &sh.full_w[s]);
         }
       }
     w_done:;
     }
   } else if (warp == 1) {
     // ---------------- MMA issuer (pair leader) ----------------
-    // One thread, so every instruction's latency is exposed: the loop tests one barrier per K
-    // block, and tests the next block's barrier before it issues this block's MMAs so that the
+    // One thread, so every instruction's latency is exposed: the loop tests one barrier per
+    // step, and tests the next step's barrier before it issues this step's MMAs so that the
     // answer arrives while they are being issued.
     if (leader && lane == 0) {
       const uint32_t idesc = idesc_16bit_f32(256, TW, ACT == 1);
       const uint64_t b_desc0 = smem_desc_sw128(smem_u32(x_base));
       const uint32_t a_tmem0 = tmem_base + kPairDCols;
-      const long total_kb = (long)((total_tiles - cluster_id + n_clusters - 1) / n_clusters) * nkb;
+      const long total_st = (long)((total_tiles - cluster_id + n_clusters - 1) / n_clusters) * n_st;
       uint32_t count = 0;
       uint32_t dph = 0;
-      bool ready_now = false;  // the barrier of block `count` is already known to be complete
+      bool ready_now = false;  // the barrier of step `count` is already known to be complete
       for (int tile = cluster_id; tile < total_tiles; tile += n_clusters) {
         if (!pair_wait(&sh.d_empty, dph ^ 1u, &sh, p.status)) goto mma_done;
-        for (int kb = 0; kb < nkb; ++kb, ++count) {
+        for (int st = 0; st < n_st; ++st, ++count) {
           const uint32_t s = count & (S - 1);
-          if (!ready_now && !pair_wait(&sh.ready[s], (count >> 3) & 1u, &sh, p.status)) goto mma_done;
+          if (!ready_now && !pair_wait(&sh.ready[s], (count >> 2) & 1u, &sh, p.status)) goto mma_done;
           tc_fence_after();
           const uint32_t nxt = count + 1;
-          const bool more = (long)nxt < total_kb;
-          const bool next_ok = more && mbar_try_wait(&sh.ready[nxt & (S - 1)], (nxt >> 3) & 1u);
+          const bool more = (long)nxt < total_st;
+          const bool next_ok = more && mbar_try_wait(&sh.ready[nxt & (S - 1)], (nxt >> 2) & 1u);
           const uint64_t b_desc = b_desc0 + (uint64_t)(s * (Cfg::kXStageBytes >> 4));
-          const uint32_t a_tmem = a_tmem0 + s * kAColsPerSlot;
+          const uint32_t a_tmem = a_tmem0 + s * Cfg::kAColsPerStage;
+          const bool two = st * kPairBlocks + 1 < nkb;
 #pragma unroll
           for (int j = 0; j < kKB / 16; ++j)
-            mma_ts_pair(tmem_base, a_tmem + j * 8, b_desc + 2u * j, idesc, (kb | j) != 0 ? 1u : 0u);
+            mma_ts_pair(tmem_base, a_tmem + j * 8, b_desc + 2u * j, idesc, (st | j) != 0 ? 1u : 0u);
+          if (two) {
+#pragma unroll
+            for (int j = 0; j < kKB / 16; ++j)
+              mma_ts_pair(tmem_base, a_tmem + kAColsPerSlot + j * 8,
+                          b_desc + (uint64_t)(Cfg::kXBlockBytes >> 4) + 2u * j, idesc, 1u);
+          }
           mma_commit_pair(&sh.slot_free[s], 3);
           ready_now = next_ok;
         }
@@ -814,60 +834,74 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
     float* stage = epi_base + (size_t)(warp - 4) * (kEpiWarpBytes / 4);
     const uint32_t ready_leader = map_to_cta(smem_u32(&sh.ready[0]), 0);
     const uint32_t d_empty_leader = map_to_cta(smem_u32(&sh.d_empty), 0);
+    const uint32_t a_taddr0 =
+        tmem_base + ((uint32_t)(quad * 32) << 16) + kPairDCols + set * Cfg::kAColsPerStage;
+    const unsigned char* w_stage = w_base + (size_t)set * Cfg::kWStageBytes;
     uint32_t dph = 0;
-    int count = 0;
+    uint32_t count = 0;
     for (int tile = cluster_id; tile < total_tiles; tile += n_clusters) {
       const int rp = tile % n_rp, mt = tile / n_rp;
       const int nt = rp * 2 + (int)rank;
-      for (int kb = 0; kb < nkb; ++kb, ++count) {
-        if ((count & 3) != set) continue;
-        const int s = count % S;
-        const uint32_t ph = (uint32_t)(count / S) & 1u;
-        uint32_t cw[8];
-        if (!pair_wait(&sh.full_w[s], ph, &sh, p.status)) goto role_done;
-        const unsigned char* st = w_base + (size_t)s * Cfg::kWTileBytes;
-        const uint32_t sz = reinterpret_cast<const uint32_t*>(st + Cfg::kWCodeBytes)[L];
-        if (BITS == 4) {
-          const uint4 w0 = reinterpret_cast<const uint4*>(st)[L];
-          const uint4 w1 = reinterpret_cast<const uint4*>(st)[kTileRows + L];
-          cw[0] = w0.x; cw[1] = w0.y; cw[2] = w0.z; cw[3] = w0.w;
-          cw[4] = w1.x; cw[5] = w1.y; cw[6] = w1.z; cw[7] = w1.w;
-        } else {
-          const uint4 a = reinterpret_cast<const uint4*>(st)[L];
-          const uint2 b = reinterpret_cast<const uint2*>(st + kTileRows * 16)[L];
-          cw[0] = a.x; cw[1] = a.y; cw[2] = a.z; cw[3] = a.w;
-          cw[4] = b.x; cw[5] = b.y; cw[6] = 0; cw[7] = 0;
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&sh.empty_w[s]);
-        uint32_t r[16];
-        float C[5], Sc[5];
-        uint32_t z_lo = 0, z_hi = 0, scale2 = 0;
-        if (ACT == 1) {
-          const uint32_t zero2 = (sz >> 16) * 0x00010001u;
-          scale2 = (sz & 0xFFFFu) * 0x00010001u;
-          z_lo = h2_sub(zero2, 0xE400E400u);
-          z_hi = h2_sub(0xD400D400u, zero2);
-        } else {
-          const float scale = __half2float(__ushort_as_half((unsigned short)(sz & 0xFFFFu)));
-          const float zero = __half2float(__ushort_as_half((unsigned short)(sz >> 16)));
+      for (int st = 0; st < n_st; ++st, ++count) {
+        if ((int)(count & 3u) != set) continue;  // ring slot = set
+        const uint32_t ph = (count >> 2) & 1u;
+        const bool two = st * kPairBlocks + 1 < nkb;
+        uint32_t cw[kPairBlocks][8];
+        uint32_t sz[kPairBlocks];
+        if (!pair_wait(&sh.full_w[set], ph, &sh, p.status)) goto role_done;
 #pragma unroll
-          for (int i = 0; i < 5; ++i) {
-            C[i] = 8388608.f + zero * (float)(1 << (4 * i));
-            Sc[i] = scale * (1.f / (float)(1 << (4 * i)));
+        for (int b = 0; b < kPairBlocks; ++b) {
+          const unsigned char* wt = w_stage + (size_t)b * Cfg::kWTileBytes;
+          if (b == 0 || two) {
+            sz[b] = reinterpret_cast<const uint32_t*>(wt + Cfg::kWCodeBytes)[L];
+            if (BITS == 4) {
+              const uint4 w0 = reinterpret_cast<const uint4*>(wt)[L];
+              const uint4 w1 = reinterpret_cast<const uint4*>(wt)[kTileRows + L];
+              cw[b][0] = w0.x; cw[b][1] = w0.y; cw[b][2] = w0.z; cw[b][3] = w0.w;
+              cw[b][4] = w1.x; cw[b][5] = w1.y; cw[b][6] = w1.z; cw[b][7] = w1.w;
+            } else {
+              const uint4 a = reinterpret_cast<const uint4*>(wt)[L];
+              const uint2 bb = reinterpret_cast<const uint2*>(wt + kTileRows * 16)[L];
+              cw[b][0] = a.x; cw[b][1] = a.y; cw[b][2] = a.z; cw[b][3] = a.w;
+              cw[b][4] = bb.x; cw[b][5] = bb.y; cw[b][6] = 0; cw[b][7] = 0;
+            }
+          } else {
+            sz[b] = 0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) cw[b][i] = 0;
           }
         }
-        auto dequant_half = [&](int half) {
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh.empty_w[set]);
+        uint32_t r[16];
+        // one K block (64 input features of this thread's weight row) in two halves of 16 registers
+        auto dequant_half = [&](const uint32_t (&c8)[8], uint32_t szw, int half) {
+          float C[5], Sc[5];
+          uint32_t z_lo = 0, z_hi = 0, scale2 = 0;
+          if (ACT == 1) {
+            const uint32_t zero2 = (szw >> 16) * 0x00010001u;          // (zero, zero) as halves
+            scale2 = (szw & 0xFFFFu) * 0x00010001u;
+            z_lo = h2_sub(zero2, 0xE400E400u);                         // zero - (-1024) = 1024 + zero
+            z_hi = h2_sub(0xD400D400u, zero2);                         // -64 - zero
+          } else {
+            const float scale = __half2float(__ushort_as_half((unsigned short)(szw & 0xFFFFu)));
+            const float zero = __half2float(__ushort_as_half((unsigned short)(szw >> 16)));
+#pragma unroll
+            for (int i = 0; i < 5; ++i) {
+              C[i] = 8388608.f + zero * (float)(1 << (4 * i));
+              Sc[i] = scale * (1.f / (float)(1 << (4 * i)));
+            }
+          }
 #pragma unroll
           for (int v = 0; v < 4; ++v) {
             const int u = half * 4 + v;
             uint32_t t;
             if (BITS == 4) {
-              t = cw[u];
+              t = c8[u];
             } else {
-              const uint32_t a2 = (u & 1) ? (cw[u >> 1] >> 2) : cw[u >> 1];
+              const uint32_t a2 = (u & 1) ? (c8[u >> 1] >> 2) : c8[u >> 1];
               const int rr = u & 3;
-              const uint32_t bw = cw[4 + (u >> 2)];
+              const uint32_t bw = c8[4 + (u >> 2)];
               const uint32_t b1 = rr == 0 ? (bw << 2) : rr == 1 ? (bw << 1) : rr == 2 ? bw : (bw >> 1);
               t = (a2 & 0x33333333u) | (b1 & 0xCCCCCCCCu);
             }
@@ -876,18 +910,24 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
             else dequant8<QM, ACT>(t, C, Sc, r + 4 * v);
           }
         };
-        dequant_half(0);
-        if (!pair_wait(&sh.slot_free[s], ph ^ 1u, &sh, p.status)) goto role_done;
+        // the first quarter is dequantised before the wait for the free A slot; every store has
+        // taken its operands when it returns, so the registers are reused at once
+        dequant_half(cw[0], sz[0], 0);
+        if (!pair_wait(&sh.slot_free[set], ph ^ 1u, &sh, p.status)) goto role_done;
         tc_fence_after();
-        const uint32_t a_taddr =
-            tmem_base + ((uint32_t)(quad * 32) << 16) + kPairDCols + s * kAColsPerSlot;
-        tmem_st_x16(a_taddr, r);
-        dequant_half(1);
-        tmem_st_x16(a_taddr + kAColsPerSlot / 2, r);
+        tmem_st_x16(a_taddr0, r);
+        dequant_half(cw[0], sz[0], 1);
+        tmem_st_x16(a_taddr0 + 16, r);
+        if (two) {
+          dequant_half(cw[1], sz[1], 0);
+          tmem_st_x16(a_taddr0 + 32, r);
+          dequant_half(cw[1], sz[1], 1);
+          tmem_st_x16(a_taddr0 + 48, r);
+        }
         tmem_wait_st();
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive_cluster(ready_leader + 8u * s);
+        if (lane == 0) mbar_arrive_cluster(ready_leader + 8u * set);
       }
       // ---- epilogue: set j drains the 16-column chunks j, j + 4, ... of this CTA's accumulator ----
       if (!pair_wait(&sh.d_full, dph, &sh, p.status)) goto role_done;
