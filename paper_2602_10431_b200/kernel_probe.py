@@ -21,10 +21,30 @@ import torch
 from . import api, inputs
 
 
+GRAPH = False  # --graph: replay the calls from a CUDA graph, so that short kernels are not timed
+               # at the rate the host can launch them
+
+
 def _time(fn, iters, warmup=3):
     for _ in range(warmup):
         fn()
     torch.cuda.synchronize()
+    if GRAPH:
+        side = torch.cuda.Stream()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(g, stream=side):
+                for _ in range(iters):
+                    fn()
+            g.replay()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(side)
+            for _ in range(5):
+                g.replay()
+            e1.record(side)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / (5 * iters) * 1e-3
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(iters):
@@ -162,7 +182,10 @@ def main():
     ap.add_argument("--select-only", dest="select_only", action="store_true")
     ap.add_argument("--config", default="c2")
     ap.add_argument("--iters", type=int, default=20)
+    ap.add_argument("--graph", action="store_true")
     a = ap.parse_args()
+    global GRAPH
+    GRAPH = a.graph
     api.lib()
     dev = torch.device("cuda", 0)
     {"gemm": probe_gemm, "router": probe_router, "compact": probe_compact, "scatter": probe_scatter,
