@@ -57,7 +57,10 @@ __global__ void __launch_bounds__(kDecThreads)
   const __nv_bfloat16* kb = cache_k + ((size_t)b * cap) * row_stride + (size_t)hk * HD + sub * 8;
   const __nv_bfloat16* vb = cache_v + ((size_t)b * cap) * row_stride + (size_t)hk * HD + sub * 8;
   constexpr int UNROLL = 4;
-  for (int k0 = grp; k0 < n_keys; k0 += GROUPS * UNROLL) {
+  // the trip count is the same for every lane (the shuffles below name the whole warp); keys
+  // past the end are masked by `ok`
+  for (int kbase = 0; kbase < n_keys; kbase += GROUPS * UNROLL) {
+    const int k0 = kbase + grp;
     uint4 kv[UNROLL], vv[UNROLL];
 #pragma unroll
     for (int u = 0; u < UNROLL; ++u) {
@@ -65,6 +68,9 @@ __global__ void __launch_bounds__(kDecThreads)
       if (key < n_keys) {
         kv[u] = ld_nc_16(kb + (size_t)key * row_stride);
         vv[u] = ld_nc_16(vb + (size_t)key * row_stride);
+      } else {
+        kv[u] = make_uint4(0, 0, 0, 0);
+        vv[u] = make_uint4(0, 0, 0, 0);
       }
     }
 #pragma unroll

@@ -5,6 +5,7 @@
     python -m paper_2602_10431_b200.kernel_probe compact --T 8192 --d 4096 --ratio 0.5
     python -m paper_2602_10431_b200.kernel_probe scatter --T 8192 --d 4096 --ratio 0.5
     python -m paper_2602_10431_b200.kernel_probe layer --config c2 --ratio 0.5
+    python -m paper_2602_10431_b200.kernel_probe decode --config c3_int3 --ratio 0.9 --graph
 
 Prints one line with the mean duration (CUDA events on the launching stream, after
 warm-up) and the achieved algorithmic rate: bytes the method must move (or FLOPs it must
@@ -163,9 +164,49 @@ def probe_layer(a, dev):
         a.config, a.ratio, sec * 1e6, T / sec, int(nex.item()), T, api.device_status()))
 
 
+def probe_decode(a, dev):
+    """One decode step of the layer: B sequences with one new token each, a per-layer cache of
+    `--kv-len` executed tokens per sequence, router scores supplied so that round(ratio * B)
+    sequences execute.  Bytes counted: packed weights once, cached K and V of the executed
+    sequences once."""
+    c = inputs.CONFIG_SHAPES[a.config]
+    sh, B = c["shape"], c["B"]
+    w = inputs.layer_weights(0, 0, sh)
+    lw = api.LayerWeights(w, dev)
+    k = api.topk_count(a.ratio, B)
+    logits = inputs.normal(3, 77, B)
+    scores = (1.0 / (1.0 + np.exp(-logits))).astype(np.float32)
+    order = np.sort(scores)[::-1]
+    theta = float((order[k - 1] + order[k]) / 2) if 0 < k < B else (0.0 if k == B else 2.0)
+    cfg = api.layer_config(sh, api.SELECT_THRESHOLD, theta=theta)
+    cap = a.kv_len + 8
+    kv = api.KvCache(B, cap, sh.kv_dim, dev, act_dtype=cfg.act_dtype)
+    kv.k.normal_()
+    kv.v.normal_()
+    ws = torch.zeros(api.layer_workspace_bytes(cfg, B, B), dtype=torch.uint8, device=dev)
+    x = torch.randn(B, sh.d, device=dev).to(torch.bfloat16)
+    cu = torch.arange(B + 1, dtype=torch.int32, device=dev)
+    pos0 = torch.full((B,), a.kv_len, dtype=torch.int32, device=dev)
+    sc = torch.from_numpy(scores).to(dev)
+    nex = torch.zeros(1, dtype=torch.int32, device=dev)
+
+    def step():
+        kv.kv_len.fill_(a.kv_len)  # every step appends at the same place
+        api.layer_forward(cfg, lw, x, cu, ws, nex, pos0=pos0, scores_override=sc, kv=kv,
+                          phase=api.PHASE_DECODE)
+
+    sec = _time(step, a.iters)
+    wbytes = sum(q.blob.numel() for q in (lw.qkv, lw.o, lw.gate_up, lw.down))
+    kvbytes = k * a.kv_len * sh.kv_dim * 2 * 2
+    print("decode %s ratio=%.2f (%d of %d sequences, kv_len %d): %.1f us, %.0f GB/s of %d algorithmic "
+          "bytes (weights %d + cache %d) (status %d)" % (
+              a.config, a.ratio, int(nex.item()), B, a.kv_len, sec * 1e6, (wbytes + kvbytes) / sec / 1e9,
+              wbytes + kvbytes, wbytes, kvbytes, api.device_status()))
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("kernel", choices=["gemm", "router", "compact", "scatter", "layer"])
+    ap.add_argument("kernel", choices=["gemm", "router", "compact", "scatter", "layer", "decode"])
     ap.add_argument("--M", type=int, default=4096)
     ap.add_argument("--M_cap", type=int, default=0)
     ap.add_argument("--N", type=int, default=4096)
@@ -181,6 +222,7 @@ def main():
     ap.add_argument("--norm", action="store_true")
     ap.add_argument("--select-only", dest="select_only", action="store_true")
     ap.add_argument("--config", default="c2")
+    ap.add_argument("--kv-len", dest="kv_len", type=int, default=2048)
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--graph", action="store_true")
     a = ap.parse_args()
@@ -189,7 +231,7 @@ def main():
     api.lib()
     dev = torch.device("cuda", 0)
     {"gemm": probe_gemm, "router": probe_router, "compact": probe_compact, "scatter": probe_scatter,
-     "layer": probe_layer}[a.kernel](a, dev)
+     "layer": probe_layer, "decode": probe_decode}[a.kernel](a, dev)
 
 
 if __name__ == "__main__":

@@ -188,6 +188,49 @@ def test_decode_step_with_executed_only_cache(env, bits, group, Hkv, act):
     assert_layer_close(out_new, ref_new, strict=True)
 
 
+@pytest.mark.timeout(120)
+def test_decode_step_ragged_cache_lengths(env):
+    """Decode against caches whose lengths differ per sequence and leave every remainder
+    modulo the key-loop stride of the decode attention (1 key, a stride plus one, ...):
+    the whole warp must leave that loop together."""
+    api, torch, dev = env
+    sh = inputs.LayerShape(256, 2, 2, 128, 512, 4, 64)
+    lens = [0, 1, 31, 32, 33, 40, 63, 64, 65, 97, 127, 130]
+    B, cap = len(lens), 136
+    case = Case(api, torch, dev, sh, inputs.cu_seqlens_uniform(B, 1), seed=6, router_std=0.05)
+    kvd = sh.kv_dim
+    kl = np.array(lens, np.int32)
+    ck = inputs.round_bf16(inputs.normal(6, 300, B * cap * kvd).reshape(B, cap, kvd).astype(np.float32))
+    cv = inputs.round_bf16(inputs.normal(6, 301, B * cap * kvd).reshape(B, cap, kvd).astype(np.float32))
+    for b in range(B):
+        ck[b, kl[b]:] = 0
+        cv[b, kl[b]:] = 0
+    kv = api.KvCache(B, cap, kvd, dev, act_dtype=1)
+    kv.k.copy_(torch.from_numpy(ck).to(dev).to(kv.k.dtype))   # bf16-valued normals are exact in fp16
+    kv.v.copy_(torch.from_numpy(cv).to(dev).to(kv.v.dtype))
+    kv.kv_len.copy_(torch.from_numpy(kl).to(dev))
+    scores = np.full(B, 0.9, np.float32)
+    scores[3] = 0.1                                            # one sequence bypasses the layer
+    m_new = oracle.select_threshold(scores, 0.5)
+    pos0 = kl.copy()
+    ck_ref, cv_ref, kl_ref = ck.copy(), cv.copy(), kl.copy()
+    ref, n_ref = oracle.layer_forward(case.layer, case.x, case.cu, m_new, pos0=pos0,
+                                      cache_k=ck_ref, cache_v=cv_ref, kv_len=kl_ref)
+    cfg = case.cfg(api.SELECT_THRESHOLD, 1, theta=0.5)
+    ws = torch.zeros(api.layer_workspace_bytes(cfg, B, B), dtype=torch.uint8, device=dev)
+    xd = api.to_device_bf16(case.x, dev)
+    nex = torch.zeros(1, dtype=torch.int32, device=dev)
+    api.layer_forward(cfg, case.lw, xd, case.cud, ws, nex, pos0=torch.from_numpy(pos0).to(dev),
+                      scores_override=torch.from_numpy(scores).to(dev), kv=kv, phase=api.PHASE_DECODE)
+    torch.cuda.synchronize()
+    assert api.device_status() == 0
+    assert int(nex.item()) == n_ref == B - 1
+    assert np.array_equal(kv.kv_len.cpu().numpy(), kl_ref)
+    out = api.to_host_f32(xd)
+    assert np.array_equal(out[3], case.x[3])
+    assert_layer_close(out, ref, strict=True)
+
+
 def test_model_prefill_teacher_forced(env):
     """Stack of layers with one global theta: each layer's selection is checked
     against the oracle's router on the SAME input (the GPU's x_l), the layer output
