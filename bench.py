@@ -33,6 +33,9 @@ UNIT = "tokens/s"
 SWEEP = [1.0, 0.9, 0.75, 0.5]
 WORKLOAD = ("c2: 7B-shaped layer (hidden 4096, 32 heads, FFN 11008), int4 g128, "
             "batch 4 x seq 2048 prefill")
+# DRAM traffic of the four GEMM launches of one step at ratio 0.5 (4096 executed tokens), from
+# one ncu capture of the kernel as it stands; None at other ratios.
+GEMM_DRAM_BYTES = 716259840
 KERNELS_PER_STEP = 11  # router, gather+norm, 4 GEMMs, rotary table, rotary, tail zeroing, attention, RMSNorm
 
 
@@ -289,7 +292,10 @@ def run_ours(args):
     peak = peaks["bf16_tflops_sustained"]
     roofline = dict(bound="tensor", kernel="wq_gemm_pair_kernel<4,1> (4 launches per step)",
                     achieved=achieved, peak=peak, unit="TFLOP/s", frac=achieved / peak,
-                    peak_source="%s (sustained bf16)" % peaks["source"], traffic=None,
+                    peak_source="%s (sustained bf16)" % peaks["source"],
+                    traffic=GEMM_DRAM_BYTES if abs(ratio - 0.5) < 1e-9 else None,
+                    traffic_unit="bytes per 4 launches (dram__bytes_read.sum + dram__bytes_write.sum, "
+                                 "ncu, ratio 0.5; profiles/wq_gemm_pair_layer_step_traffic.md)",
                     ms_per_4_launches=g_ms, share_of_step=g_ms / ms_per_step)
 
     # ---- end to end: host buffers, H2D of the inputs and D2H of the result every step ----
