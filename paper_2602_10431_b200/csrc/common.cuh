@@ -90,6 +90,11 @@ __device__ __forceinline__ double warp_sum(double v) {
   return v;
 }
 
+// barrier among `threads` threads (a multiple of 32) of the CTA; id 1..15 (0 is __syncthreads)
+__device__ __forceinline__ void named_barrier(int id, int threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
 // 16-byte global accesses
 __device__ __forceinline__ uint4 ld_nc_16(const void* p) {
   uint4 v;

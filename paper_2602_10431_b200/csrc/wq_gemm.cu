@@ -970,6 +970,248 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
 }
 
 // ------------------------------------------------------------------------------
+// Small-M kernel (up to 64 tokens: the decode step).  Here the product is bound by the
+// stream of packed weights, and the tcgen05 kernels above, whose dequantised operand makes a
+// round trip through tensor memory and three barriers per K block, cannot pull it fast
+// enough: a CTA needs about 0.6 us per 64-wide block whatever the token count.  This kernel
+// keeps everything in registers: one CTA owns 64 weight rows (half a blob tile) over the
+// whole K, eight warps = four 16-row blocks x two K halves (even / odd K blocks), a ninth
+// warp feeds an 8-stage ring with bulk copies of the codes and a tiled load of the
+// activations; each warp rebuilds its m16n8k16 A fragments from the packed codes (one shift,
+// one logic op, one exact subtract, one multiply per pair of weights) and issues warp MMAs
+// against ldmatrix-loaded activation fragments.  With 64 to 344 CTAs per linear and two CTAs
+// per SM the weight stream is spread over the whole device.
+// ------------------------------------------------------------------------------
+constexpr int kSmallStages = 8;
+constexpr int kSmallMmaWarps = 8;
+constexpr int kSmallThreads = (kSmallMmaWarps + 1) * 32;
+constexpr int kSmallTokens = 64;  // token capacity
+
+// ROWS = weight rows per CTA (32, 64 or 128: a quarter, a half or a whole blob tile), chosen on
+// the host so that a linear gives between one and two CTAs per SM; the eight MMA warps are
+// ROWS / 16 row blocks x 8 / (ROWS / 16) K groups (K block kb belongs to group kb modulo that).
+template <int BITS, int ROWS>
+struct SmallCfg {
+  static constexpr int kRowBlocks = ROWS / 16;
+  static constexpr int kGroups = kSmallMmaWarps / kRowBlocks;
+  static constexpr int kQuads = ROWS / 32;
+  static constexpr int kXBytes = kSmallTokens * 128;                   // 64 tokens x 64 k
+  static constexpr int kCodeA = ROWS * 16;                             // 16 bytes per row
+  static constexpr int kCodeB = BITS == 4 ? ROWS * 16 : ROWS * 8;
+  static constexpr int kSzBytes = ROWS * 4;
+  static constexpr int kWBytes = kCodeA + kCodeB + kSzBytes;
+  static constexpr int kTileCodeBytes = kTileRows * kKB * BITS / 8;    // code bytes of a full tile block
+  static constexpr int kTileBytes = kTileCodeBytes + kTileRows * 4;
+  static constexpr size_t kWOffset = (size_t)kSmallStages * kXBytes;
+  static constexpr size_t kSmemBytes = kWOffset + (size_t)kSmallStages * kWBytes + 1024;
+  // after the K loop the activation ring is reused: partial sums of the K groups but the first,
+  // then the output tile for the epilogue
+  static constexpr int kRedBytes = (kGroups - 1) * kRowBlocks * 32 * 32 * 4;
+  static constexpr int kOutBytes = kQuads * kSmallTokens * kEpiRowWords * 4;
+  static_assert(ROWS == 32 || ROWS == 64 || ROWS == 128, "rows per CTA");
+  static_assert(kSmallStages % kGroups == 0, "a ring stage always meets the same K group");
+  static_assert(kRedBytes + kOutBytes <= kSmallStages * kXBytes, "epilogue buffers fit the ring");
+};
+
+struct __align__(8) SmallShared {
+  uint64_t full[kSmallStages], empty[kSmallStages];
+  volatile int abort_flag;
+};
+
+__device__ __forceinline__ bool small_wait(uint64_t* bar, uint32_t parity, SmallShared* sh, int* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  for (uint32_t it = 0; it < kWaitSlices; ++it) {
+    if (mbar_try_wait_suspend(bar, parity, kWaitSliceNs)) return true;
+    if (sh->abort_flag) return false;
+  }
+  sh->abort_flag = 1;
+  report_device_error(status, QTALE_ERR_TIMEOUT);
+  return false;
+}
+
+// two weights of one row (the codes in bits 4 t .. 4 t + 3 of both halves of `word`) as a pair of
+// 16-bit values: (code - zero) * scale, exact difference, one rounding
+template <int BITS, int ACT>
+__device__ __forceinline__ uint32_t small_dequant_pair(uint32_t word, int shift, uint32_t z_lo,
+                                                       uint32_t scale2, float zero, float scale) {
+  constexpr uint32_t QM = BITS == 4 ? 0x000F000Fu : 0x00070007u;
+  const uint32_t q = (word >> shift) & QM;
+  if (ACT == 1) return h2_mul(h2_sub(q | 0x64006400u, z_lo), scale2);
+  return pack_bf16x2(((float)(q & 0xFFFFu) - zero) * scale, ((float)(q >> 16) - zero) * scale);
+}
+
+template <int BITS, int ACT, int ROWS>
+__global__ void __launch_bounds__(kSmallThreads, 2)
+    wq_gemm_small_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmParams p) {
+  using Cfg = SmallCfg<BITS, ROWS>;
+  constexpr int S = kSmallStages;
+  constexpr int RB = Cfg::kRowBlocks, KG = Cfg::kGroups;
+  constexpr int SLICES = kTileRows / ROWS;  // CTAs per blob tile
+  extern __shared__ unsigned char smem_dyn[];
+  __shared__ SmallShared sh;
+  unsigned char* x_base = reinterpret_cast<unsigned char*>(
+      (reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~static_cast<uintptr_t>(1023));
+  unsigned char* w_base = x_base + Cfg::kWOffset;
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  int M = p.M_cap;
+  if (p.m_dev) M = min(M, *p.m_dev);
+  if (M <= 0) return;  // every thread: nothing to do
+  M = min(M, kSmallTokens);
+  const int nt = blockIdx.x / SLICES;     // blob tile
+  const int slice = blockIdx.x % SLICES;  // rows ROWS * slice .. of the tile
+  const int nkb = p.nkb;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < S; ++s) {
+      mbar_init(&sh.full[s], 1);
+      mbar_init(&sh.empty[s], RB);  // the warps of the K group that reads the stage
+    }
+    sh.abort_flag = 0;
+    fence_barrier_init();
+  }
+  __syncthreads();
+
+  if (warp == kSmallMmaWarps) {
+    // ---------------- producer ----------------
+    if (lane == 0) {
+      const uint8_t* tile0 = p.packed + (((size_t)(nt >> 1) * nkb) * 2 + (nt & 1)) * Cfg::kTileBytes;
+      for (int kb = 0; kb < nkb; ++kb) {
+        const int s = kb & (S - 1);
+        const uint32_t ph = (uint32_t)(kb >> 3) & 1u;
+        if (!small_wait(&sh.empty[s], ph ^ 1u, &sh, p.status)) break;
+        mbar_arrive_expect_tx(&sh.full[s], Cfg::kXBytes + Cfg::kWBytes);
+        tma_load_2d(x_base + (size_t)s * Cfg::kXBytes, &tmap_x, &sh.full[s], kb * kKB, 0);
+        const uint8_t* blk = tile0 + (size_t)kb * 2 * Cfg::kTileBytes;  // (pair, kb) chunks are two tiles apart
+        unsigned char* w = w_base + (size_t)s * Cfg::kWBytes;
+        // int4: two 32-feature parts of 16 bytes per row; int3: a 2-bit plane of 16 and a 1-bit
+        // plane of 8 bytes per row; either way the second piece starts 2 KB into the block
+        bulk_load(w, blk + slice * Cfg::kCodeA, Cfg::kCodeA, &sh.full[s]);
+        bulk_load(w + Cfg::kCodeA, blk + kTileRows * 16 + slice * Cfg::kCodeB, Cfg::kCodeB, &sh.full[s]);
+        bulk_load(w + Cfg::kCodeA + Cfg::kCodeB, blk + Cfg::kTileCodeBytes + slice * Cfg::kSzBytes,
+                  Cfg::kSzBytes, &sh.full[s]);
+      }
+    }
+    return;  // the producer takes no part in the epilogue barriers
+  }
+
+  // ---------------- MMA warps ----------------
+  const int kgroup = warp / RB;  // K blocks kb with kb % KG == kgroup
+  const int rb = warp % RB;      // 16-row block of the CTA's rows
+  const int g = lane >> 2, t = lane & 3;
+  const int r0 = rb * 16 + g, r1 = r0 + 8;
+  float acc[8][4];
+#pragma unroll
+  for (int i = 0; i < 8; ++i)
+#pragma unroll
+    for (int e = 0; e < 4; ++e) acc[i][e] = 0.f;
+  for (int kb = kgroup; kb < nkb; kb += KG) {
+    const int s = kb & (S - 1);
+    const uint32_t ph = (uint32_t)(kb >> 3) & 1u;
+    if (!small_wait(&sh.full[s], ph, &sh, p.status)) break;
+    const unsigned char* w = w_base + (size_t)s * Cfg::kWBytes;
+    uint32_t c[2][8];  // eight nibble-style words (8 codes each) of rows r0 and r1
+    uint32_t szw[2];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const int r = h ? r1 : r0;
+      szw[h] = reinterpret_cast<const uint32_t*>(w + Cfg::kCodeA + Cfg::kCodeB)[r];
+      if (BITS == 4) {
+        const uint4 a = reinterpret_cast<const uint4*>(w)[r];
+        const uint4 b = reinterpret_cast<const uint4*>(w + Cfg::kCodeA)[r];
+        c[h][0] = a.x; c[h][1] = a.y; c[h][2] = a.z; c[h][3] = a.w;
+        c[h][4] = b.x; c[h][5] = b.y; c[h][6] = b.z; c[h][7] = b.w;
+      } else {
+        const uint4 a = reinterpret_cast<const uint4*>(w)[r];
+        const uint2 b = reinterpret_cast<const uint2*>(w + Cfg::kCodeA)[r];
+        const uint32_t pa[4] = {a.x, a.y, a.z, a.w};
+        const uint32_t pb[2] = {b.x, b.y};
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const uint32_t a2 = (u & 1) ? (pa[u >> 1] >> 2) : pa[u >> 1];
+          const int rr = u & 3;
+          const uint32_t bw = pb[u >> 2];
+          const uint32_t b1 = rr == 0 ? (bw << 2) : rr == 1 ? (bw << 1) : rr == 2 ? bw : (bw >> 1);
+          c[h][u] = (a2 & 0x33333333u) | (b1 & 0xCCCCCCCCu);
+        }
+      }
+    }
+    uint32_t z_lo[2], scale2[2];
+    float zf[2], sf[2];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const uint32_t zero2 = (szw[h] >> 16) * 0x00010001u;
+      scale2[h] = (szw[h] & 0xFFFFu) * 0x00010001u;
+      z_lo[h] = h2_sub(zero2, 0xE400E400u);  // 1024 + zero
+      zf[h] = __half2float(__ushort_as_half((unsigned short)(szw[h] >> 16)));
+      sf[h] = __half2float(__ushort_as_half((unsigned short)(szw[h] & 0xFFFFu)));
+    }
+    const uint32_t x_stage = smem_u32(x_base + (size_t)s * Cfg::kXBytes);
+#pragma unroll
+    for (int s16 = 0; s16 < 4; ++s16) {
+      // word 2 s16 holds k = 16 s16 .. + 7, word 2 s16 + 1 the next eight; in a word, bits 4 t of
+      // the low half are feature 2 t and of the high half feature 2 t + 1
+      uint32_t a[4];
+      a[0] = small_dequant_pair<BITS, ACT>(c[0][2 * s16], 4 * t, z_lo[0], scale2[0], zf[0], sf[0]);
+      a[1] = small_dequant_pair<BITS, ACT>(c[1][2 * s16], 4 * t, z_lo[1], scale2[1], zf[1], sf[1]);
+      a[2] = small_dequant_pair<BITS, ACT>(c[0][2 * s16 + 1], 4 * t, z_lo[0], scale2[0], zf[0], sf[0]);
+      a[3] = small_dequant_pair<BITS, ACT>(c[1][2 * s16 + 1], 4 * t, z_lo[1], scale2[1], zf[1], sf[1]);
+#pragma unroll
+      for (int tg2 = 0; tg2 < 4; ++tg2) {
+        // matrices: (tokens 16 tg2 .. + 7, k chunk 2 s16), (same tokens, chunk 2 s16 + 1),
+        //           (tokens 16 tg2 + 8 .., chunk 2 s16), (.., chunk 2 s16 + 1); 128-byte swizzle
+        const int mi = lane >> 3;
+        const int token = tg2 * 16 + (mi >> 1) * 8 + (lane & 7);
+        const int chunk = 2 * s16 + (mi & 1);
+        uint32_t b[4];
+        ldmatrix_x4(x_stage + token * 128 + ((chunk ^ (token & 7)) << 4), b);
+        mma_m16n8k16<ACT == 1>(acc[2 * tg2], a, b[0], b[1]);
+        mma_m16n8k16<ACT == 1>(acc[2 * tg2 + 1], a, b[2], b[3]);
+      }
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&sh.empty[s]);
+  }
+  // ---- the other K groups hand their sums to the first; then the tile goes through the common epilogue ----
+  named_barrier(1, kSmallMmaWarps * 32);  // every stage has been read: the ring is free
+  float* red = reinterpret_cast<float*>(x_base);
+  float* out = reinterpret_cast<float*>(x_base + Cfg::kRedBytes);
+  if (kgroup > 0) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+#pragma unroll
+      for (int e = 0; e < 4; ++e)
+        red[((((kgroup - 1) * RB + rb) * 32) + i * 4 + e) * 32 + lane] = acc[i][e];
+  }
+  named_barrier(1, kSmallMmaWarps * 32);
+  if (kgroup == 0) {
+    const int ql = rb >> 1;              // quadrant (32 rows) of the CTA's rows
+    const int nl = (rb & 1) * 16 + g;    // row inside the quadrant
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        float v = acc[i][e];
+#pragma unroll
+        for (int kg = 1; kg < KG; ++kg) v += red[((((kg - 1) * RB + rb) * 32) + i * 4 + e) * 32 + lane];
+        const int token = i * 8 + 2 * t + (e & 1);
+        out[(ql * kSmallTokens + token) * kEpiRowWords + nl + (e >> 1) * 8] = v;
+      }
+    }
+  }
+  named_barrier(1, kSmallMmaWarps * 32);
+  // units of (quadrant, 16-token chunk) over the eight warps
+  for (int unit = warp; unit < Cfg::kQuads * (kSmallTokens / kEpiCols); unit += kSmallMmaWarps) {
+    const int ql = unit % Cfg::kQuads, chunk = unit / Cfg::kQuads;
+    const int m0 = chunk * kEpiCols;
+    if (m0 < M)
+      epilogue_chunk<ACT>(p, out + (ql * kSmallTokens + m0) * kEpiRowWords, lane, nt,
+                          slice * Cfg::kQuads + ql, m0, M);
+  }
+}
+
+// ------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------
 
@@ -1094,6 +1336,36 @@ static int make_pair_tmaps(PairTmapSet* set, const void* base, int rows, int col
   return QTALE_OK;
 }
 
+// ---- small-M kernel ----
+template <int BITS, int ACT, int ROWS>
+static int launch_small_rows(const CUtensorMap& tx, const GemmParams& p, cudaStream_t s) {
+  using Cfg = SmallCfg<BITS, ROWS>;
+  static bool configured[64] = {false};
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (dev < 0 || dev >= 64) return QTALE_ERR_CUDA;
+  if (!configured[dev]) {
+    if (cudaFuncSetAttribute(wq_gemm_small_kernel<BITS, ACT, ROWS>,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)Cfg::kSmemBytes) != cudaSuccess)
+      return QTALE_ERR_CUDA;
+    configured[dev] = true;
+  }
+  wq_gemm_small_kernel<BITS, ACT, ROWS>
+      <<<p.n_tiles * (kTileRows / ROWS), kSmallThreads, Cfg::kSmemBytes, s>>>(tx, p);
+  return launch_status(cudaGetLastError());
+}
+
+// Rows per CTA: the most that still fills the device (each CTA streams all the activations, so
+// fewer, taller CTAs read less); a quarter tile at the least.
+template <int BITS, int ACT>
+static int launch_small(const CUtensorMap& tx, const GemmParams& p, cudaStream_t s) {
+  const int sms = sm_count();  // two CTAs fit an SM
+  if (p.n_tiles >= 2 * sms) return launch_small_rows<BITS, ACT, 128>(tx, p, s);
+  if (2 * p.n_tiles >= sms) return launch_small_rows<BITS, ACT, 64>(tx, p, s);
+  return launch_small_rows<BITS, ACT, 32>(tx, p, s);
+}
+
 // Token counts from which the CTA-pair kernel is used (below, a tile of 256 tokens is mostly padding).
 constexpr int kPairMinTokens = 129;
 
@@ -1150,6 +1422,15 @@ int wq_gemm_launch(const void* a, int lda, const int32_t* m_dev, int M_cap,
     if (act == QTALE_ACT_F16)
       return w->bits == 4 ? launch_pair<4, 1>(px, p, s) : launch_pair<3, 1>(px, p, s);
     return w->bits == 4 ? launch_pair<4, 0>(px, p, s) : launch_pair<3, 0>(px, p, s);
+  }
+  if (M_cap <= kSmallTokens) {
+    CUtensorMap tx1;
+    memset(&tx1, 0, sizeof(tx1));
+    const int rc = make_tmap_16(&tx1, a, M_cap, w->K, lda, kSmallTokens, act);
+    if (rc != QTALE_OK) return rc;
+    if (act == QTALE_ACT_F16)
+      return w->bits == 4 ? launch_small<4, 1>(tx1, p, s) : launch_small<3, 1>(tx1, p, s);
+    return w->bits == 4 ? launch_small<4, 0>(tx1, p, s) : launch_small<3, 0>(tx1, p, s);
   }
   const int tn = pick_tn(M_cap);
   TmapSet tx;
