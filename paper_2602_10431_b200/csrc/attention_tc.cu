@@ -26,7 +26,7 @@ using namespace ptx;
 
 constexpr int kTcThreads = 192;
 constexpr int kTcTile = 128;  // query rows per CTA and keys per tile
-constexpr uint32_t kTcSpin = 1u << 24;
+constexpr uint32_t kTcSlices = 1u << 16;  // suspended barrier tests before a wait gives up
 
 struct TcShared {
   uint64_t q_full;
@@ -48,9 +48,12 @@ struct TcParams {
 };
 
 __device__ __forceinline__ bool tc_wait(uint64_t* bar, uint32_t parity, TcShared* sh, int* status) {
-  for (uint32_t it = 0; it < kTcSpin; ++it) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 255u) == 255u && sh->abort_flag) return false;
+  // the first test is plain; after that the thread lets the hardware suspend it (up to 20 us a
+  // test), so waiting roles leave the issue slots to the softmax warps
+  if (mbar_try_wait(bar, parity)) return true;
+  for (uint32_t it = 0; it < kTcSlices; ++it) {
+    if (mbar_try_wait_suspend(bar, parity, 20000u)) return true;
+    if (sh->abort_flag) return false;
   }
   sh->abort_flag = 1;
   report_device_error(status, QTALE_ERR_TIMEOUT);

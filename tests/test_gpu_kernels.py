@@ -136,6 +136,8 @@ GEMM_CASES = [
     (64, 384, 256, 3, 64, 1),              # 3-bit, a single token
     (520, 256, 1024, 3, 128, 513),         # 3-bit, several token tiles and a tail of one
     (256, 512, 128, 4, 128, 0),            # nothing to do
+    (129, 384, 192, 4, 64, None),          # smallest CTA-pair case: three row tiles (one padded), one and a half K steps
+    (700, 640, 384, 3, 128, 651),          # CTA-pair, 3-bit, five row tiles, ragged tokens over three tiles
     (64, 9600, 128, 4, 128, 37),           # decode kernel, half a row tile per CTA
     (48, 38016, 64, 3, 64, None),          # decode kernel, a whole row tile per CTA, 3-bit
     (33, 256, 704, 4, 64, 33),             # decode kernel, a quarter tile per CTA, four K groups, odd K blocks
