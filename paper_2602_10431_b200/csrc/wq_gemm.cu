@@ -1161,6 +1161,7 @@ __global__ void __launch_bounds__(kSmallThreads, 2)
       for (int tg2 = 0; tg2 < 4; ++tg2) {
         // matrices: (tokens 16 tg2 .. + 7, k chunk 2 s16), (same tokens, chunk 2 s16 + 1),
         //           (tokens 16 tg2 + 8 .., chunk 2 s16), (.., chunk 2 s16 + 1); 128-byte swizzle
+        if (tg2 * 16 >= M) break;  // no executed token in these sixteen (same for the whole CTA)
         const int mi = lane >> 3;
         const int token = tg2 * 16 + (mi >> 1) * 8 + (lane & 7);
         const int chunk = 2 * s16 + (mi & 1);
