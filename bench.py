@@ -227,15 +227,19 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    def timed(fn, steps, warmup, sampler=None):
+    def timed(fn, steps, warmup, sampler=None, drain=None):
         for i in range(warmup):
             fn(i)
+        if drain is not None:
+            drain()
         barrier()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         t_start = time.time()
         e0.record()
         for i in range(steps):
             fn(i)
+        if drain is not None:
+            drain()  # the timed stream waits for the copies still in flight on the others
         e1.record()
         barrier()
         if sampler is not None:
@@ -299,17 +303,42 @@ def run_ours(args):
                     ms_per_4_launches=g_ms, share_of_step=g_ms / ms_per_step)
 
     # ---- end to end: host buffers, H2D of the inputs and D2H of the result every step ----
-    def e2e_step(i):
-        buf = bufs[i % n_buf]
-        buf.copy_(x_host, non_blocking=True)
-        api.layer_forward(cfg, lw, buf, cud, ws, nex)
-        out_host.copy_(buf, non_blocking=True)
+    # Every step copies its input from pinned host memory, runs the layer through the public
+    # call and copies its result back; the copies run on two streams of their own, so step
+    # i + 1's input and step i - 1's result travel while step i computes (n_buf device buffers).
+    main = torch.cuda.current_stream()
+    copy_in, copy_out = torch.cuda.Stream(), torch.cuda.Stream()
+    ev_in = [torch.cuda.Event() for _ in range(n_buf)]
+    ev_done = [torch.cuda.Event() for _ in range(n_buf)]
+    ev_out = [torch.cuda.Event() for _ in range(n_buf)]
+    out_hosts = [out_host] + [torch.empty_like(x_host).pin_memory() for _ in range(n_buf - 1)]
 
+    def e2e_step(i):
+        j = i % n_buf
+        buf = bufs[j]
+        with torch.cuda.stream(copy_in):
+            copy_in.wait_event(ev_out[j])  # the buffer's previous result has left the device
+            buf.copy_(x_host, non_blocking=True)
+            ev_in[j].record(copy_in)
+        main.wait_event(ev_in[j])
+        api.layer_forward(cfg, lw, buf, cud, ws, nex)
+        ev_done[j].record(main)
+        with torch.cuda.stream(copy_out):
+            copy_out.wait_event(ev_done[j])
+            out_hosts[j].copy_(buf, non_blocking=True)
+            ev_out[j].record(copy_out)
+
+    def e2e_drain():
+        main.wait_stream(copy_in)
+        main.wait_stream(copy_out)
+
+    main.wait_stream(copy_in)
     e_steps = max(3, min(50, args.steps // 2))
-    e_ms = timed(e2e_step, e_steps, 3) / e_steps
+    e_ms = timed(e2e_step, e_steps, 3, drain=e2e_drain) / e_steps
     nbytes = x_host.numel() * 2
     e2e = dict(value=world * T / (e_ms * 1e-3), unit=UNIT, h2d_bytes_per_step=nbytes,
-               d2h_bytes_per_step=nbytes, ms_per_step=e_ms)
+               d2h_bytes_per_step=nbytes, ms_per_step=e_ms,
+               note="copies on their own streams, overlapped with the neighbouring steps' compute")
 
     line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps,
                 warmup=args.warmup, ms_per_step=ms_per_step, higher_is_better=True, scaling="weak",
