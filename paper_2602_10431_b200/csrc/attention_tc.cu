@@ -47,6 +47,14 @@ struct TcParams {
   int* status;
 };
 
+// 2^x by the special-function unit alone (about 2 ulp; -inf gives 0): the softmax is bound by
+// this unit, so nothing is spent on the range fix-ups of exp2f
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
 __device__ __forceinline__ bool tc_wait(uint64_t* bar, uint32_t parity, TcShared* sh, int* status) {
   // the first test is plain; after that the thread lets the hardware suspend it (up to 20 us a
   // test), so waiting roles leave the issue slots to the softmax warps
@@ -209,7 +217,8 @@ __global__ void __launch_bounds__(kTcThreads, 1)
       const int k0 = j * kTcTile;
       const bool masked = (j == qt) || (k0 + kTcTile > len);
       const int q_row = q0 + row;
-      // the whole score row (128 keys) in registers: scaled and masked once
+      // the whole score row (128 keys) in registers, unscaled; the scale (positive) is folded
+      // into the exponent's multiply-add, so an element costs one max, one fma, one ex2, one add
       float sc[128];
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
@@ -217,7 +226,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
         tmem_ld_x32(s_addr + c * 32, r);
         tmem_wait_ld();
 #pragma unroll
-        for (int i = 0; i < 32; ++i) sc[c * 32 + i] = __uint_as_float(r[i]) * p.scale_log2;
+        for (int i = 0; i < 32; ++i) sc[c * 32 + i] = __uint_as_float(r[i]);
       }
       if (masked) {
 #pragma unroll
@@ -226,23 +235,33 @@ __global__ void __launch_bounds__(kTcThreads, 1)
           if (key > q_row || key >= len) sc[i] = -INFINITY;
         }
       }
-      float mx = m_run;
+      // four independent chains for the maximum
+      float mq[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-      for (int i = 0; i < 128; ++i) mx = fmaxf(mx, sc[i]);
+      for (int i = 0; i < 128; i += 4) {
+        mq[0] = fmaxf(mq[0], sc[i]);
+        mq[1] = fmaxf(mq[1], sc[i + 1]);
+        mq[2] = fmaxf(mq[2], sc[i + 2]);
+        mq[3] = fmaxf(mq[3], sc[i + 3]);
+      }
+      const float mx = fmaxf(m_run, fmaxf(fmaxf(mq[0], mq[1]), fmaxf(mq[2], mq[3])) * p.scale_log2);
       const float m_safe = (mx == -INFINITY) ? 0.f : mx;
-      const float corr = exp2f(m_run - m_safe);
+      const float corr = ex2_approx(m_run - m_safe);
       const bool moved = mx > m_run;
       m_run = mx;
       l_run *= corr;
       // probabilities in the 16-bit format, two keys per 32-bit column
-      float sum = 0.f;
+      const float neg_m = -m_safe;
+      float sq[4] = {0.f, 0.f, 0.f, 0.f};
       uint32_t pr[64];
 #pragma unroll
       for (int i = 0; i < 64; ++i) {
-        const float p0 = exp2f(sc[2 * i] - m_safe), p1 = exp2f(sc[2 * i + 1] - m_safe);
-        sum += p0 + p1;
+        const float p0 = ex2_approx(fmaf(sc[2 * i], p.scale_log2, neg_m));
+        const float p1 = ex2_approx(fmaf(sc[2 * i + 1], p.scale_log2, neg_m));
+        sq[i & 3] += p0 + p1;
         pr[i] = Act16<ACT>::pack(p0, p1);
       }
+      const float sum = (sq[0] + sq[1]) + (sq[2] + sq[3]);
       // the previous P V must be complete before O is rescaled or P is overwritten
       if (j > 0) {
         if (!tc_wait(&sh.pv_done, (uint32_t)(j - 1) & 1u, &sh, p.status)) { alive = false; break; }
