@@ -220,13 +220,21 @@ __global__ void __launch_bounds__(kTcThreads, 1)
       // the whole score row (128 keys) in registers, unscaled; the scale (positive) is folded
       // into the exponent's multiply-add, so an element costs one max, one fma, one ex2, one add
       float sc[128];
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint32_t r[32];
-        tmem_ld_x32(s_addr + c * 32, r);
+      {
+        // the four reads are issued back to back and waited for once
+        uint32_t r0[32], r1[32], r2[32], r3[32];
+        tmem_ld_x32(s_addr, r0);
+        tmem_ld_x32(s_addr + 32, r1);
+        tmem_ld_x32(s_addr + 64, r2);
+        tmem_ld_x32(s_addr + 96, r3);
         tmem_wait_ld();
 #pragma unroll
-        for (int i = 0; i < 32; ++i) sc[c * 32 + i] = __uint_as_float(r[i]);
+        for (int i = 0; i < 32; ++i) {
+          sc[i] = __uint_as_float(r0[i]);
+          sc[32 + i] = __uint_as_float(r1[i]);
+          sc[64 + i] = __uint_as_float(r2[i]);
+          sc[96 + i] = __uint_as_float(r3[i]);
+        }
       }
       if (masked) {
 #pragma unroll
