@@ -1,16 +1,20 @@
 // Causal attention among the executed tokens of each sequence (prefill) on the
 // tcgen05 tensor cores (Eq. 3: bypassed tokens have no query, key or value here).
 //
-// One CTA handles 128 consecutive executed tokens (query rows) of one sequence and
-// one head, streaming that sequence's executed keys / values in tiles of 128:
+// A work item is 128 consecutive executed tokens (query rows) of one sequence and one
+// head; the grid is persistent (one CTA per SM walks the items, longest first) and an item
+// streams that sequence's executed keys / values in tiles of 128:
 //   S = Q K^T     SS MMA, Q and K tiles from 128-byte-swizzled shared memory (TMA),
 //                 fp32 scores in tensor memory, double buffered;
 //   softmax       four warps, one query row per thread: running max / sum in the
-//                 log2 domain, probabilities written back to tensor memory in the
-//                 16-bit activation format (the A operand of the next MMA);
+//                 log2 domain (one fma and one ex2.approx per score), probabilities written
+//                 back to tensor memory in the 16-bit activation format (the A operand of
+//                 the next MMA);
 //   O += P V      TS MMA with V read straight from its row-major tile (MN-major B
 //                 operand), fp32 output accumulator in tensor memory, rescaled by the
 //                 softmax warps only when a row's running maximum moves.
+// Barrier phases run on across items (key tiles are counted per CTA), so the loads and
+// the first Q K^T of the next item overlap the output stage of the current one.
 // Warp roles (192 threads): warp 0 TMA producer, warp 1 MMA issuer and TMEM
 // allocator, warps 2-5 softmax / correction / output.  Every wait is bounded.
 #include <cuda.h>
@@ -29,7 +33,7 @@ constexpr int kTcTile = 128;  // query rows per CTA and keys per tile
 constexpr uint32_t kTcSlices = 1u << 16;  // suspended barrier tests before a wait gives up
 
 struct TcShared {
-  uint64_t q_full;
+  uint64_t q_full, q_empty, o_empty;
   uint64_t k_full[2], v_full[2], kv_empty[2];
   uint64_t s_full[2], p_full[2];
   uint64_t pv_done;
@@ -86,6 +90,43 @@ __device__ __forceinline__ uint64_t v_desc(uint32_t smem_addr, int key16) {
   return d;
 }
 
+// Work items of the persistent grid: (sequence, query tile) pairs sorted by query tile, longest
+// first, each for every head; item i -> pair i / H, head i % H.  CTA c takes items c, c + grid,
+// ... in that order, so its pair rank only grows and the cursor below is advanced, never rewound.
+struct ItemCursor {
+  int lvl;    // query tile index of the pairs being enumerated
+  int base;   // rank of the first pair with this query tile
+  int cnt;    // sequences that have this query tile
+};
+
+__device__ __forceinline__ int seq_tiles(const TcParams& p, int s) {
+  return (p.cu_exec[s + 1] - p.cu_exec[s] + kTcTile - 1) / kTcTile;
+}
+
+// pair of rank r (r must not decrease between calls): returns false past the last pair
+__device__ __forceinline__ bool pair_of_rank(const TcParams& p, ItemCursor& c, int r, int& b, int& qt) {
+  while (c.lvl >= 0) {
+    if (c.cnt < 0) {  // count the sequences of this level once
+      c.cnt = 0;
+      for (int s = 0; s < p.B; ++s) c.cnt += seq_tiles(p, s) > c.lvl ? 1 : 0;
+    }
+    if (r < c.base + c.cnt) {
+      int k = r - c.base;
+      for (int s = 0; s < p.B; ++s) {
+        if (seq_tiles(p, s) > c.lvl) {
+          if (k == 0) { b = s; qt = c.lvl; return true; }
+          --k;
+        }
+      }
+      return false;
+    }
+    c.base += c.cnt;
+    c.cnt = -1;
+    --c.lvl;
+  }
+  return false;
+}
+
 template <int HD, int ACT>
 __global__ void __launch_bounds__(kTcThreads, 1)
     attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap, const TcParams p) {
@@ -104,26 +145,18 @@ __global__ void __launch_bounds__(kTcThreads, 1)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-  // locate (sequence, query tile); late (long) tiles first
-  int b = -1, qt = 0;
-  {
-    int tile = blockIdx.x;
-    for (int s = p.B - 1; s >= 0; --s) {
-      const int len = p.cu_exec[s + 1] - p.cu_exec[s];
-      const int nt = (len + kTcTile - 1) / kTcTile;
-      if (tile < nt) { b = s; qt = nt - 1 - tile; break; }
-      tile -= nt;
-    }
+  int max_nt = 0, n_pairs = 0;
+  for (int s = 0; s < p.B; ++s) {
+    const int nt = seq_tiles(p, s);
+    max_nt = max(max_nt, nt);
+    n_pairs += nt;
   }
-  if (b < 0) return;  // uniform for the CTA: nothing allocated yet
-  const int h = blockIdx.y, hk = h / p.rep;
-  const int seq0 = p.cu_exec[b];
-  const int len = p.cu_exec[b + 1] - seq0;
-  const int q0 = qt * kTcTile;
-  const int n_kt = qt + 1;
+  const int n_items = n_pairs * p.H;
+  if ((int)blockIdx.x >= n_items) return;  // uniform for the CTA: nothing allocated yet
 
   if (threadIdx.x == 0) {
     mbar_init(&sh.q_full, 1);
+    mbar_init(&sh.q_empty, 1);
     for (int s = 0; s < 2; ++s) {
       mbar_init(&sh.k_full[s], 1);
       mbar_init(&sh.v_full[s], 1);
@@ -132,6 +165,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
       mbar_init(&sh.p_full[s], 4);
     }
     mbar_init(&sh.pv_done, 1);
+    mbar_init(&sh.o_empty, 4);
     sh.abort_flag = 0;
     fence_barrier_init();
   }
@@ -144,24 +178,41 @@ __global__ void __launch_bounds__(kTcThreads, 1)
   tc_fence_after();
   const uint32_t tmem = sh.tmem_base;
 
+  // every role walks the same item sequence with its own cursor and its own running counters:
+  // t = key tiles so far (ring stage t & 1, phase (t >> 1) & 1), it = items so far
+  ItemCursor cur;
+  cur.lvl = max_nt - 1;
+  cur.base = 0;
+  cur.cnt = -1;
+
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
     if (lane == 0) {
-      mbar_arrive_expect_tx(&sh.q_full, TILE_BYTES);
-      for (int c = 0; c < CH; ++c)
-        tma_load_2d(sQ + c * 16384, &tmap, &sh.q_full, h * HD + c * 64, seq0 + q0);
-      for (int j = 0; j < n_kt; ++j) {
-        const int s = j & 1;
-        const uint32_t ph = (uint32_t)(j >> 1) & 1u;
-        if (!tc_wait(&sh.kv_empty[s], ph ^ 1u, &sh, p.status)) break;
-        mbar_arrive_expect_tx(&sh.k_full[s], TILE_BYTES);
+      uint32_t t = 0, it = 0;
+      for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++it) {
+        int b, qt;
+        if (!pair_of_rank(p, cur, item / p.H, b, qt)) break;
+        const int h = item % p.H, hk = h / p.rep;
+        const int seq0 = p.cu_exec[b];
+        if (!tc_wait(&sh.q_empty, (it & 1u) ^ 1u, &sh, p.status)) break;
+        mbar_arrive_expect_tx(&sh.q_full, TILE_BYTES);
         for (int c = 0; c < CH; ++c)
-          tma_load_2d(sK + s * TILE_BYTES + c * 16384, &tmap, &sh.k_full[s],
-                      p.k_off + hk * HD + c * 64, seq0 + j * kTcTile);
-        mbar_arrive_expect_tx(&sh.v_full[s], TILE_BYTES);
-        for (int c = 0; c < CH; ++c)
-          tma_load_2d(sV + s * TILE_BYTES + c * 16384, &tmap, &sh.v_full[s],
-                      p.v_off + hk * HD + c * 64, seq0 + j * kTcTile);
+          tma_load_2d(sQ + c * 16384, &tmap, &sh.q_full, h * HD + c * 64, seq0 + qt * kTcTile);
+        bool ok = true;
+        for (int j = 0; j <= qt; ++j, ++t) {
+          const int s = t & 1;
+          const uint32_t ph = (t >> 1) & 1u;
+          if (!tc_wait(&sh.kv_empty[s], ph ^ 1u, &sh, p.status)) { ok = false; break; }
+          mbar_arrive_expect_tx(&sh.k_full[s], TILE_BYTES);
+          for (int c = 0; c < CH; ++c)
+            tma_load_2d(sK + s * TILE_BYTES + c * 16384, &tmap, &sh.k_full[s],
+                        p.k_off + hk * HD + c * 64, seq0 + j * kTcTile);
+          mbar_arrive_expect_tx(&sh.v_full[s], TILE_BYTES);
+          for (int c = 0; c < CH; ++c)
+            tma_load_2d(sV + s * TILE_BYTES + c * 16384, &tmap, &sh.v_full[s],
+                        p.v_off + hk * HD + c * 64, seq0 + j * kTcTile);
+        }
+        if (!ok) break;
       }
     }
   } else if (warp == 1) {
@@ -169,12 +220,12 @@ __global__ void __launch_bounds__(kTcThreads, 1)
     if (lane == 0) {
       constexpr uint32_t idesc_qk = idesc_16bit_f32(128, kTcTile, ACT == 1);
       constexpr uint32_t idesc_pv = idesc_16bit_f32(128, HD, ACT == 1) | (1u << 16);  // B is MN-major
-      bool ok = tc_wait(&sh.q_full, 0, &sh, p.status);
-      auto issue_qk = [&](int j) {
-        const int s = j & 1;
-        if (!tc_wait(&sh.k_full[s], (uint32_t)(j >> 1) & 1u, &sh, p.status)) return false;
+      const uint32_t qa = smem_u32(sQ);
+      auto issue_qk = [&](uint32_t tt) {
+        const int s = tt & 1;
+        if (!tc_wait(&sh.k_full[s], (tt >> 1) & 1u, &sh, p.status)) return false;
         tc_fence_after();
-        const uint32_t qa = smem_u32(sQ), ka = smem_u32(sK + s * TILE_BYTES);
+        const uint32_t ka = smem_u32(sK + s * TILE_BYTES);
 #pragma unroll
         for (int kk = 0; kk < HD / 16; ++kk)
           mma_ss(tmem + S_COL + s * 128, kmajor_desc(qa, kk), kmajor_desc(ka, kk), idesc_qk,
@@ -182,23 +233,40 @@ __global__ void __launch_bounds__(kTcThreads, 1)
         mma_commit(&sh.s_full[s]);
         return true;
       };
-      if (ok) ok = issue_qk(0);
-      for (int j = 0; ok && j < n_kt; ++j) {
-        const int s = j & 1;
-        const uint32_t ph = (uint32_t)(j >> 1) & 1u;
-        // scores of the next tile are computed while the softmax of this one runs
-        if (j + 1 < n_kt) ok = issue_qk(j + 1);
-        if (!ok) break;
-        if (!tc_wait(&sh.p_full[s], ph, &sh, p.status)) break;
-        if (!tc_wait(&sh.v_full[s], ph, &sh, p.status)) break;
-        tc_fence_after();
-        const uint32_t va = smem_u32(sV + s * TILE_BYTES);
+      uint32_t t = 0, it = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x, ++it) {
+        int b, qt;
+        if (!pair_of_rank(p, cur, item / p.H, b, qt)) break;
+        const int n_kt = qt + 1;
+        if (!tc_wait(&sh.q_full, it & 1u, &sh, p.status)) break;
+        ok = issue_qk(t);
+        if (ok && n_kt == 1) mma_commit(&sh.q_empty);  // the query tile has been read for the last time
+        for (int j = 0; ok && j < n_kt; ++j) {
+          const uint32_t tt = t + j;
+          const int s = tt & 1;
+          const uint32_t ph = (tt >> 1) & 1u;
+          // scores of the next tile are computed while the softmax of this one runs
+          if (j + 1 < n_kt) {
+            ok = issue_qk(tt + 1);
+            if (ok && j + 2 == n_kt) mma_commit(&sh.q_empty);
+          }
+          if (!ok) break;
+          if (!tc_wait(&sh.p_full[s], ph, &sh, p.status)) { ok = false; break; }
+          if (!tc_wait(&sh.v_full[s], ph, &sh, p.status)) { ok = false; break; }
+          // the first P V of an item overwrites the accumulator: the previous item's output
+          // must have been read
+          if (j == 0 && !tc_wait(&sh.o_empty, (it & 1u) ^ 1u, &sh, p.status)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t va = smem_u32(sV + s * TILE_BYTES);
 #pragma unroll
-        for (int kk = 0; kk < kTcTile / 16; ++kk)
-          mma_ts(tmem + O_COL, tmem + P_COL + s * 64 + kk * 8, v_desc(va, kk), idesc_pv,
-                 (j | kk) != 0 ? 1u : 0u);
-        mma_commit(&sh.kv_empty[s]);
-        mma_commit(&sh.pv_done);
+          for (int kk = 0; kk < kTcTile / 16; ++kk)
+            mma_ts(tmem + O_COL, tmem + P_COL + s * 64 + kk * 8, v_desc(va, kk), idesc_pv,
+                   (j | kk) != 0 ? 1u : 0u);
+          mma_commit(&sh.kv_empty[s]);
+          mma_commit(&sh.pv_done);
+        }
+        t += n_kt;
       }
     }
   } else {
@@ -206,110 +274,126 @@ __global__ void __launch_bounds__(kTcThreads, 1)
     const int quad = warp & 3;
     const int row = quad * 32 + lane;          // TMEM lane = query row of the tile
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
-    float m_run = -INFINITY, l_run = 0.f;
+    uint32_t t = 0, it = 0;
     bool alive = true;
-    for (int j = 0; j < n_kt && alive; ++j) {
-      const int s = j & 1;
-      const uint32_t ph = (uint32_t)(j >> 1) & 1u;
-      if (!tc_wait(&sh.s_full[s], ph, &sh, p.status)) { alive = false; break; }
-      tc_fence_after();
-      const uint32_t s_addr = tmem + lane_addr + S_COL + s * 128;
-      const int k0 = j * kTcTile;
-      const bool masked = (j == qt) || (k0 + kTcTile > len);
+    for (int item = blockIdx.x; alive && item < n_items; item += gridDim.x, ++it) {
+      int b, qt;
+      if (!pair_of_rank(p, cur, item / p.H, b, qt)) break;
+      const int h = item % p.H;
+      const int seq0 = p.cu_exec[b];
+      const int len = p.cu_exec[b + 1] - seq0;
+      const int q0 = qt * kTcTile;
+      const int n_kt = qt + 1;
       const int q_row = q0 + row;
-      // the whole score row (128 keys) in registers, unscaled; the scale (positive) is folded
-      // into the exponent's multiply-add, so an element costs one max, one fma, one ex2, one add
-      float sc[128];
-      {
-        // the four reads are issued back to back and waited for once
-        uint32_t r0[32], r1[32], r2[32], r3[32];
-        tmem_ld_x32(s_addr, r0);
-        tmem_ld_x32(s_addr + 32, r1);
-        tmem_ld_x32(s_addr + 64, r2);
-        tmem_ld_x32(s_addr + 96, r3);
-        tmem_wait_ld();
-#pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          sc[i] = __uint_as_float(r0[i]);
-          sc[32 + i] = __uint_as_float(r1[i]);
-          sc[64 + i] = __uint_as_float(r2[i]);
-          sc[96 + i] = __uint_as_float(r3[i]);
-        }
-      }
-      if (masked) {
-#pragma unroll
-        for (int i = 0; i < 128; ++i) {
-          const int key = k0 + i;
-          if (key > q_row || key >= len) sc[i] = -INFINITY;
-        }
-      }
-      // four independent chains for the maximum
-      float mq[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-      for (int i = 0; i < 128; i += 4) {
-        mq[0] = fmaxf(mq[0], sc[i]);
-        mq[1] = fmaxf(mq[1], sc[i + 1]);
-        mq[2] = fmaxf(mq[2], sc[i + 2]);
-        mq[3] = fmaxf(mq[3], sc[i + 3]);
-      }
-      const float mx = fmaxf(m_run, fmaxf(fmaxf(mq[0], mq[1]), fmaxf(mq[2], mq[3])) * p.scale_log2);
-      const float m_safe = (mx == -INFINITY) ? 0.f : mx;
-      const float corr = ex2_approx(m_run - m_safe);
-      const bool moved = mx > m_run;
-      m_run = mx;
-      l_run *= corr;
-      // probabilities in the 16-bit format, two keys per 32-bit column
-      const float neg_m = -m_safe;
-      float sq[4] = {0.f, 0.f, 0.f, 0.f};
-      uint32_t pr[64];
-#pragma unroll
-      for (int i = 0; i < 64; ++i) {
-        const float p0 = ex2_approx(fmaf(sc[2 * i], p.scale_log2, neg_m));
-        const float p1 = ex2_approx(fmaf(sc[2 * i + 1], p.scale_log2, neg_m));
-        sq[i & 3] += p0 + p1;
-        pr[i] = Act16<ACT>::pack(p0, p1);
-      }
-      const float sum = (sq[0] + sq[1]) + (sq[2] + sq[3]);
-      // the previous P V must be complete before O is rescaled or P is overwritten
-      if (j > 0) {
-        if (!tc_wait(&sh.pv_done, (uint32_t)(j - 1) & 1u, &sh, p.status)) { alive = false; break; }
+      float m_run = -INFINITY, l_run = 0.f;
+      for (int j = 0; j < n_kt && alive; ++j) {
+        const uint32_t tt = t + j;
+        const int s = tt & 1;
+        const uint32_t ph = (tt >> 1) & 1u;
+        if (!tc_wait(&sh.s_full[s], ph, &sh, p.status)) { alive = false; break; }
         tc_fence_after();
-        if (__any_sync(0xffffffffu, moved)) {
-#pragma unroll 1
-          for (int c = 0; c < HD / 32; ++c) {
-            uint32_t r[32];
-            tmem_ld_x32(tmem + lane_addr + O_COL + c * 32, r);
-            tmem_wait_ld();
+        const uint32_t s_addr = tmem + lane_addr + S_COL + s * 128;
+        const int k0 = j * kTcTile;
+        const bool masked = (j == qt) || (k0 + kTcTile > len);
+        // the whole score row (128 keys) in registers, unscaled; the scale (positive) is folded
+        // into the exponent's multiply-add, so an element costs one max, one fma, one ex2, one add
+        float sc[128];
+        {
+          // the four reads are issued back to back and waited for once
+          uint32_t r0[32], r1[32], r2[32], r3[32];
+          tmem_ld_x32(s_addr, r0);
+          tmem_ld_x32(s_addr + 32, r1);
+          tmem_ld_x32(s_addr + 64, r2);
+          tmem_ld_x32(s_addr + 96, r3);
+          tmem_wait_ld();
 #pragma unroll
-            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * corr);
-            tmem_st_x32(tmem + lane_addr + O_COL + c * 32, r);
+          for (int i = 0; i < 32; ++i) {
+            sc[i] = __uint_as_float(r0[i]);
+            sc[32 + i] = __uint_as_float(r1[i]);
+            sc[64 + i] = __uint_as_float(r2[i]);
+            sc[96 + i] = __uint_as_float(r3[i]);
           }
         }
-      }
-      {
-        uint32_t lo[32], hi[32];
+        if (masked) {
 #pragma unroll
-        for (int i = 0; i < 32; ++i) { lo[i] = pr[i]; hi[i] = pr[32 + i]; }
-        tmem_st_x32(tmem + lane_addr + P_COL + s * 64, lo);
-        tmem_st_x32(tmem + lane_addr + P_COL + s * 64 + 32, hi);
+          for (int i = 0; i < 128; ++i) {
+            const int key = k0 + i;
+            if (key > q_row || key >= len) sc[i] = -INFINITY;
+          }
+        }
+        // four independent chains for the maximum
+        float mq[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+        for (int i = 0; i < 128; i += 4) {
+          mq[0] = fmaxf(mq[0], sc[i]);
+          mq[1] = fmaxf(mq[1], sc[i + 1]);
+          mq[2] = fmaxf(mq[2], sc[i + 2]);
+          mq[3] = fmaxf(mq[3], sc[i + 3]);
+        }
+        const float mx = fmaxf(m_run, fmaxf(fmaxf(mq[0], mq[1]), fmaxf(mq[2], mq[3])) * p.scale_log2);
+        const float m_safe = (mx == -INFINITY) ? 0.f : mx;
+        const float corr = ex2_approx(m_run - m_safe);
+        const bool moved = mx > m_run;
+        m_run = mx;
+        l_run *= corr;
+        // probabilities in the 16-bit format, two keys per 32-bit column
+        const float neg_m = -m_safe;
+        float sq[4] = {0.f, 0.f, 0.f, 0.f};
+        uint32_t pr[64];
+#pragma unroll
+        for (int i = 0; i < 64; ++i) {
+          const float p0 = ex2_approx(fmaf(sc[2 * i], p.scale_log2, neg_m));
+          const float p1 = ex2_approx(fmaf(sc[2 * i + 1], p.scale_log2, neg_m));
+          sq[i & 3] += p0 + p1;
+          pr[i] = Act16<ACT>::pack(p0, p1);
+        }
+        const float sum = (sq[0] + sq[1]) + (sq[2] + sq[3]);
+        // the previous P V must be complete before O is rescaled or P is overwritten (for the
+        // first tile of an item the output stage of the item before has waited for it)
+        if (j > 0) {
+          if (!tc_wait(&sh.pv_done, (tt - 1) & 1u, &sh, p.status)) { alive = false; break; }
+          tc_fence_after();
+          if (__any_sync(0xffffffffu, moved)) {
+#pragma unroll 1
+            for (int c = 0; c < HD / 32; ++c) {
+              uint32_t r[32];
+              tmem_ld_x32(tmem + lane_addr + O_COL + c * 32, r);
+              tmem_wait_ld();
+#pragma unroll
+              for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * corr);
+              tmem_st_x32(tmem + lane_addr + O_COL + c * 32, r);
+            }
+          }
+        }
+        {
+          uint32_t lo[32], hi[32];
+#pragma unroll
+          for (int i = 0; i < 32; ++i) { lo[i] = pr[i]; hi[i] = pr[32 + i]; }
+          tmem_st_x32(tmem + lane_addr + P_COL + s * 64, lo);
+          tmem_st_x32(tmem + lane_addr + P_COL + s * 64 + 32, hi);
+        }
+        l_run += sum;
+        tmem_wait_st();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh.p_full[s]);
       }
-      l_run += sum;
-      tmem_wait_st();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&sh.p_full[s]);
-    }
-    // output: O / l for the rows that exist
-    if (alive && tc_wait(&sh.pv_done, (uint32_t)(n_kt - 1) & 1u, &sh, p.status)) {
+      if (!alive) break;
+      // output: O / l for the rows that exist; then the accumulator is handed back
+      if (!tc_wait(&sh.pv_done, (t + n_kt - 1) & 1u, &sh, p.status)) { alive = false; break; }
       tc_fence_after();
       const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-      const int q_row = q0 + row;
       unsigned short* out = static_cast<unsigned short*>(p.out) + (size_t)(seq0 + q_row) * p.ldo + (size_t)h * HD;
 #pragma unroll 1
       for (int c = 0; c < HD / 32; ++c) {
         uint32_t r[32];
         tmem_ld_x32(tmem + lane_addr + O_COL + c * 32, r);
         tmem_wait_ld();
+        if (c == HD / 32 - 1) {  // every column of this warp's rows is in registers
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&sh.o_empty);
+        }
         if (q_row < len) {
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
@@ -322,6 +406,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
           }
         }
       }
+      t += n_kt;
     }
   }
 
@@ -366,8 +451,10 @@ static int launch_tc(const CUtensorMap& tm, const TcParams& p, int max_tiles, in
       return QTALE_ERR_CUDA;
     configured[dev] = true;
   }
-  dim3 grid(max_tiles, H);
-  attn_prefill_tc_kernel<HD, ACT><<<grid, kTcThreads, smem, s>>>(tm, p);
+  // persistent grid: one CTA per SM walks the (sequence, query tile, head) items, longest first
+  (void)max_tiles;
+  (void)H;
+  attn_prefill_tc_kernel<HD, ACT><<<sm_count(), kTcThreads, smem, s>>>(tm, p);
   return launch_status(cudaGetLastError());
 }
 
