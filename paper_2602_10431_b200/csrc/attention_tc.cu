@@ -6,17 +6,21 @@
 // streams that sequence's executed keys / values in tiles of 128:
 //   S = Q K^T     SS MMA, Q and K tiles from 128-byte-swizzled shared memory (TMA),
 //                 fp32 scores in tensor memory, double buffered;
-//   softmax       four warps, one query row per thread: running max / sum in the
-//                 log2 domain (one fma and one ex2.approx per score), probabilities written
-//                 back to tensor memory in the 16-bit activation format (the A operand of
-//                 the next MMA);
+//   softmax       eight warps, two threads per query row (64 keys each; the half-row maxima
+//                 meet through shared memory): running max / sum in the log2 domain (one fma
+//                 and one ex2.approx per score), probabilities written back to tensor memory
+//                 in the 16-bit activation format (the A operand of the next MMA);
 //   O += P V      TS MMA with V read straight from its row-major tile (MN-major B
 //                 operand), fp32 output accumulator in tensor memory, rescaled by the
 //                 softmax warps only when a row's running maximum moves.
-// Barrier phases run on across items (key tiles are counted per CTA), so the loads and
-// the first Q K^T of the next item overlap the output stage of the current one.
-// Warp roles (192 threads): warp 0 TMA producer, warp 1 MMA issuer and TMEM
-// allocator, warps 2-5 softmax / correction / output.  Every wait is bounded.
+// Keys and values have rings of their own (three and two tiles) and a producer thread each:
+// a key tile is free as soon as its scores exist, so its successor is loaded three tiles
+// ahead; with one two-stage ring released after P V the load latency (about 1800 cycles) sat
+// in the loop of every tile.  Barrier phases run on across items (tiles are counted per
+// CTA), so the loads and the first Q K^T of the next item overlap the output stage of the
+// current one.
+// Warp roles (352 threads): warp 0 Q / K producer, warp 1 MMA issuer and TMEM allocator,
+// warps 2-9 softmax / correction / output, warp 10 V producer.  Every wait is bounded.
 #include <cuda.h>
 
 #include <string.h>
@@ -28,13 +32,19 @@ namespace qtale {
 
 using namespace ptx;
 
-constexpr int kTcThreads = 192;
+constexpr int kTcThreads = 352;  // K producer, issuer, eight softmax warps, V producer
+constexpr int kTcKStages = 3;    // key tiles in flight (the first thing a tile needs)
+constexpr int kTcVStages = 2;    // value tiles in flight
 constexpr int kTcTile = 128;  // query rows per CTA and keys per tile
 constexpr uint32_t kTcSlices = 1u << 16;  // suspended barrier tests before a wait gives up
 
 struct TcShared {
   uint64_t q_full, q_empty, o_empty;
-  uint64_t k_full[2], v_full[2], kv_empty[2];
+  uint64_t k_full[kTcKStages], k_empty[kTcKStages];
+  uint64_t v_full[kTcVStages], v_empty[kTcVStages];
+  uint64_t max_bar, sum_bar;  // the two threads of a query row exchange their half-row maximum / sum
+  float row_max[2][2][kTcTile];  // [tile parity][half][row]
+  float row_sum[2][kTcTile];     // [half][row]
   uint64_t s_full[2], p_full[2];
   uint64_t pv_done;
   uint32_t tmem_base;
@@ -140,8 +150,8 @@ __global__ void __launch_bounds__(kTcThreads, 1)
   unsigned char* base = reinterpret_cast<unsigned char*>(
       (reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~static_cast<uintptr_t>(1023));
   unsigned char* sQ = base;
-  unsigned char* sK = base + TILE_BYTES;            // two stages
-  unsigned char* sV = base + 3 * TILE_BYTES;        // two stages
+  unsigned char* sK = base + TILE_BYTES;                     // kTcKStages stages
+  unsigned char* sV = base + (1 + kTcKStages) * TILE_BYTES;  // kTcVStages stages
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -158,14 +168,21 @@ __global__ void __launch_bounds__(kTcThreads, 1)
     mbar_init(&sh.q_full, 1);
     mbar_init(&sh.q_empty, 1);
     for (int s = 0; s < 2; ++s) {
-      mbar_init(&sh.k_full[s], 1);
-      mbar_init(&sh.v_full[s], 1);
-      mbar_init(&sh.kv_empty[s], 1);
       mbar_init(&sh.s_full[s], 1);
-      mbar_init(&sh.p_full[s], 4);
+      mbar_init(&sh.p_full[s], 8);
     }
+    for (int s = 0; s < kTcKStages; ++s) {
+      mbar_init(&sh.k_full[s], 1);
+      mbar_init(&sh.k_empty[s], 1);
+    }
+    for (int s = 0; s < kTcVStages; ++s) {
+      mbar_init(&sh.v_full[s], 1);
+      mbar_init(&sh.v_empty[s], 1);
+    }
+    mbar_init(&sh.max_bar, 8);
+    mbar_init(&sh.sum_bar, 8);
     mbar_init(&sh.pv_done, 1);
-    mbar_init(&sh.o_empty, 4);
+    mbar_init(&sh.o_empty, 8);
     sh.abort_flag = 0;
     fence_barrier_init();
   }
@@ -200,19 +217,37 @@ __global__ void __launch_bounds__(kTcThreads, 1)
           tma_load_2d(sQ + c * 16384, &tmap, &sh.q_full, h * HD + c * 64, seq0 + qt * kTcTile);
         bool ok = true;
         for (int j = 0; j <= qt; ++j, ++t) {
-          const int s = t & 1;
-          const uint32_t ph = (t >> 1) & 1u;
-          if (!tc_wait(&sh.kv_empty[s], ph ^ 1u, &sh, p.status)) { ok = false; break; }
+          const int s = t % kTcKStages;
+          const uint32_t ph = (t / kTcKStages) & 1u;
+          if (!tc_wait(&sh.k_empty[s], ph ^ 1u, &sh, p.status)) { ok = false; break; }
           mbar_arrive_expect_tx(&sh.k_full[s], TILE_BYTES);
           for (int c = 0; c < CH; ++c)
             tma_load_2d(sK + s * TILE_BYTES + c * 16384, &tmap, &sh.k_full[s],
                         p.k_off + hk * HD + c * 64, seq0 + j * kTcTile);
+        }
+        if (!ok) break;
+      }
+    }
+  } else if (warp == 10) {
+    // ------------------------------ TMA producer of the value tiles ------------------------------
+    // (a thread of its own: a full value ring must not hold back the key loads)
+    if (lane == 0) {
+      uint32_t t = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
+        int b, qt;
+        if (!pair_of_rank(p, cur, item / p.H, b, qt)) break;
+        const int hk = (item % p.H) / p.rep;
+        const int seq0 = p.cu_exec[b];
+        for (int j = 0; j <= qt; ++j, ++t) {
+          const int s = t % kTcVStages;
+          const uint32_t ph = (t / kTcVStages) & 1u;
+          if (!tc_wait(&sh.v_empty[s], ph ^ 1u, &sh, p.status)) { ok = false; break; }
           mbar_arrive_expect_tx(&sh.v_full[s], TILE_BYTES);
           for (int c = 0; c < CH; ++c)
             tma_load_2d(sV + s * TILE_BYTES + c * 16384, &tmap, &sh.v_full[s],
                         p.v_off + hk * HD + c * 64, seq0 + j * kTcTile);
         }
-        if (!ok) break;
       }
     }
   } else if (warp == 1) {
@@ -223,14 +258,16 @@ __global__ void __launch_bounds__(kTcThreads, 1)
       const uint32_t qa = smem_u32(sQ);
       auto issue_qk = [&](uint32_t tt) {
         const int s = tt & 1;
-        if (!tc_wait(&sh.k_full[s], (tt >> 1) & 1u, &sh, p.status)) return false;
+        const int ks = tt % kTcKStages;
+        if (!tc_wait(&sh.k_full[ks], (tt / kTcKStages) & 1u, &sh, p.status)) return false;
         tc_fence_after();
-        const uint32_t ka = smem_u32(sK + s * TILE_BYTES);
+        const uint32_t ka = smem_u32(sK + ks * TILE_BYTES);
 #pragma unroll
         for (int kk = 0; kk < HD / 16; ++kk)
           mma_ss(tmem + S_COL + s * 128, kmajor_desc(qa, kk), kmajor_desc(ka, kk), idesc_qk,
                  kk != 0 ? 1u : 0u);
         mma_commit(&sh.s_full[s]);
+        mma_commit(&sh.k_empty[ks]);  // the key tile is free as soon as its scores exist
         return true;
       };
       uint32_t t = 0, it = 0;
@@ -253,27 +290,34 @@ __global__ void __launch_bounds__(kTcThreads, 1)
           }
           if (!ok) break;
           if (!tc_wait(&sh.p_full[s], ph, &sh, p.status)) { ok = false; break; }
-          if (!tc_wait(&sh.v_full[s], ph, &sh, p.status)) { ok = false; break; }
+          const int vs = tt % kTcVStages;
+          if (!tc_wait(&sh.v_full[vs], (tt / kTcVStages) & 1u, &sh, p.status)) { ok = false; break; }
           // the first P V of an item overwrites the accumulator: the previous item's output
           // must have been read
           if (j == 0 && !tc_wait(&sh.o_empty, (it & 1u) ^ 1u, &sh, p.status)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t va = smem_u32(sV + s * TILE_BYTES);
+          const uint32_t va = smem_u32(sV + vs * TILE_BYTES);
 #pragma unroll
           for (int kk = 0; kk < kTcTile / 16; ++kk)
             mma_ts(tmem + O_COL, tmem + P_COL + s * 64 + kk * 8, v_desc(va, kk), idesc_pv,
                    (j | kk) != 0 ? 1u : 0u);
-          mma_commit(&sh.kv_empty[s]);
+          mma_commit(&sh.v_empty[vs]);
           mma_commit(&sh.pv_done);
         }
         t += n_kt;
       }
     }
   } else {
-    // ------------------ softmax, correction and output: one query row per thread ------------------
+    // ---------- softmax, correction and output: two threads per query row ----------
+    // Warps 2-5 take keys 0..63 of a tile, warps 6-9 keys 64..127 (the same split of the output
+    // columns at the end); a warp reaches the TMEM lanes 32 (warp % 4) .. + 31.  The two threads
+    // of a row exchange their half-row maximum through shared memory and an mbarrier (bounded
+    // wait, like every other wait here), and their partial sums once per item.
     const int quad = warp & 3;
+    const int half = (warp - 2) >> 2;
     const int row = quad * 32 + lane;          // TMEM lane = query row of the tile
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+    constexpr int OC = HD / 2;                 // output columns of this thread
     uint32_t t = 0, it = 0;
     bool alive = true;
     for (int item = blockIdx.x; alive && item < n_items; item += gridDim.x, ++it) {
@@ -285,52 +329,52 @@ __global__ void __launch_bounds__(kTcThreads, 1)
       const int q0 = qt * kTcTile;
       const int n_kt = qt + 1;
       const int q_row = q0 + row;
-      float m_run = -INFINITY, l_run = 0.f;
+      float m_run = -INFINITY, l_run = 0.f;  // l_run: this thread's half of the row sum
       for (int j = 0; j < n_kt && alive; ++j) {
         const uint32_t tt = t + j;
         const int s = tt & 1;
         const uint32_t ph = (tt >> 1) & 1u;
         if (!tc_wait(&sh.s_full[s], ph, &sh, p.status)) { alive = false; break; }
         tc_fence_after();
-        const uint32_t s_addr = tmem + lane_addr + S_COL + s * 128;
-        const int k0 = j * kTcTile;
-        const bool masked = (j == qt) || (k0 + kTcTile > len);
-        // the whole score row (128 keys) in registers, unscaled; the scale (positive) is folded
-        // into the exponent's multiply-add, so an element costs one max, one fma, one ex2, one add
-        float sc[128];
+        const uint32_t s_addr = tmem + lane_addr + S_COL + s * 128 + half * 64;
+        const int k0 = j * kTcTile + half * 64;
+        const bool masked = (j == qt) || (j * kTcTile + kTcTile > len);
+        // half a score row (64 keys) in registers, unscaled; the scale (positive) is folded into
+        // the exponent's multiply-add, so an element costs one max, one fma, one ex2, one add
+        float sc[64];
         {
-          // the four reads are issued back to back and waited for once
-          uint32_t r0[32], r1[32], r2[32], r3[32];
+          uint32_t r0[32], r1[32];
           tmem_ld_x32(s_addr, r0);
           tmem_ld_x32(s_addr + 32, r1);
-          tmem_ld_x32(s_addr + 64, r2);
-          tmem_ld_x32(s_addr + 96, r3);
           tmem_wait_ld();
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
             sc[i] = __uint_as_float(r0[i]);
             sc[32 + i] = __uint_as_float(r1[i]);
-            sc[64 + i] = __uint_as_float(r2[i]);
-            sc[96 + i] = __uint_as_float(r3[i]);
           }
         }
         if (masked) {
 #pragma unroll
-          for (int i = 0; i < 128; ++i) {
+          for (int i = 0; i < 64; ++i) {
             const int key = k0 + i;
             if (key > q_row || key >= len) sc[i] = -INFINITY;
           }
         }
-        // four independent chains for the maximum
         float mq[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-        for (int i = 0; i < 128; i += 4) {
+        for (int i = 0; i < 64; i += 4) {
           mq[0] = fmaxf(mq[0], sc[i]);
           mq[1] = fmaxf(mq[1], sc[i + 1]);
           mq[2] = fmaxf(mq[2], sc[i + 2]);
           mq[3] = fmaxf(mq[3], sc[i + 3]);
         }
-        const float mx = fmaxf(m_run, fmaxf(fmaxf(mq[0], mq[1]), fmaxf(mq[2], mq[3])) * p.scale_log2);
+        const float my_max = fmaxf(fmaxf(mq[0], mq[1]), fmaxf(mq[2], mq[3]));
+        sh.row_max[tt & 1][half][row] = my_max;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh.max_bar);
+        if (!tc_wait(&sh.max_bar, tt & 1u, &sh, p.status)) { alive = false; break; }
+        const float row_raw = fmaxf(my_max, sh.row_max[tt & 1][half ^ 1][row]);
+        const float mx = fmaxf(m_run, row_raw * p.scale_log2);
         const float m_safe = (mx == -INFINITY) ? 0.f : mx;
         const float corr = ex2_approx(m_run - m_safe);
         const bool moved = mx > m_run;
@@ -339,15 +383,15 @@ __global__ void __launch_bounds__(kTcThreads, 1)
         // probabilities in the 16-bit format, two keys per 32-bit column
         const float neg_m = -m_safe;
         float sq[4] = {0.f, 0.f, 0.f, 0.f};
-        uint32_t pr[64];
+        uint32_t pr[32];
 #pragma unroll
-        for (int i = 0; i < 64; ++i) {
+        for (int i = 0; i < 32; ++i) {
           const float p0 = ex2_approx(fmaf(sc[2 * i], p.scale_log2, neg_m));
           const float p1 = ex2_approx(fmaf(sc[2 * i + 1], p.scale_log2, neg_m));
           sq[i & 3] += p0 + p1;
           pr[i] = Act16<ACT>::pack(p0, p1);
         }
-        const float sum = (sq[0] + sq[1]) + (sq[2] + sq[3]);
+        l_run += (sq[0] + sq[1]) + (sq[2] + sq[3]);
         // the previous P V must be complete before O is rescaled or P is overwritten (for the
         // first tile of an item the output stage of the item before has waited for it)
         if (j > 0) {
@@ -355,24 +399,17 @@ __global__ void __launch_bounds__(kTcThreads, 1)
           tc_fence_after();
           if (__any_sync(0xffffffffu, moved)) {
 #pragma unroll 1
-            for (int c = 0; c < HD / 32; ++c) {
+            for (int c = 0; c < OC / 32; ++c) {
               uint32_t r[32];
-              tmem_ld_x32(tmem + lane_addr + O_COL + c * 32, r);
+              tmem_ld_x32(tmem + lane_addr + O_COL + half * OC + c * 32, r);
               tmem_wait_ld();
 #pragma unroll
               for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * corr);
-              tmem_st_x32(tmem + lane_addr + O_COL + c * 32, r);
+              tmem_st_x32(tmem + lane_addr + O_COL + half * OC + c * 32, r);
             }
           }
         }
-        {
-          uint32_t lo[32], hi[32];
-#pragma unroll
-          for (int i = 0; i < 32; ++i) { lo[i] = pr[i]; hi[i] = pr[32 + i]; }
-          tmem_st_x32(tmem + lane_addr + P_COL + s * 64, lo);
-          tmem_st_x32(tmem + lane_addr + P_COL + s * 64 + 32, hi);
-        }
-        l_run += sum;
+        tmem_st_x32(tmem + lane_addr + P_COL + s * 64 + half * 32, pr);
         tmem_wait_st();
         tc_fence_before();
         __syncwarp();
@@ -380,16 +417,22 @@ __global__ void __launch_bounds__(kTcThreads, 1)
       }
       if (!alive) break;
       // output: O / l for the rows that exist; then the accumulator is handed back
+      sh.row_sum[half][row] = l_run;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh.sum_bar);
+      if (!tc_wait(&sh.sum_bar, it & 1u, &sh, p.status)) { alive = false; break; }
+      const float l_tot = l_run + sh.row_sum[half ^ 1][row];
       if (!tc_wait(&sh.pv_done, (t + n_kt - 1) & 1u, &sh, p.status)) { alive = false; break; }
       tc_fence_after();
-      const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-      unsigned short* out = static_cast<unsigned short*>(p.out) + (size_t)(seq0 + q_row) * p.ldo + (size_t)h * HD;
+      const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;
+      unsigned short* out = static_cast<unsigned short*>(p.out) + (size_t)(seq0 + q_row) * p.ldo +
+                            (size_t)h * HD + half * OC;
 #pragma unroll 1
-      for (int c = 0; c < HD / 32; ++c) {
+      for (int c = 0; c < OC / 32; ++c) {
         uint32_t r[32];
-        tmem_ld_x32(tmem + lane_addr + O_COL + c * 32, r);
+        tmem_ld_x32(tmem + lane_addr + O_COL + half * OC + c * 32, r);
         tmem_wait_ld();
-        if (c == HD / 32 - 1) {  // every column of this warp's rows is in registers
+        if (c == OC / 32 - 1) {  // every column of this warp's part is in registers
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(&sh.o_empty);
@@ -441,7 +484,7 @@ static EncodeTiledFnA encode_fn_a() {
 
 template <int HD, int ACT>
 static int launch_tc(const CUtensorMap& tm, const TcParams& p, int max_tiles, int H, cudaStream_t s) {
-  const size_t smem = (size_t)5 * kTcTile * HD * 2 + 1024;
+  const size_t smem = (size_t)(1 + kTcKStages + kTcVStages) * kTcTile * HD * 2 + 1024;
   static bool configured[64] = {false};
   int dev = 0;
   cudaGetDevice(&dev);
