@@ -2,7 +2,7 @@
 // tcgen05 tensor cores (Eq. 3: bypassed tokens have no query, key or value here).
 //
 // A work item is 128 consecutive executed tokens (query rows) of one sequence and one
-// head; the grid is persistent (one CTA per SM walks the items, longest first) and an item
+// head; the grid is persistent (one CTA per SM walks the items sequence by sequence) and an item
 // streams that sequence's executed keys / values in tiles of 128:
 //   S = Q K^T     SS MMA, Q and K tiles from 128-byte-swizzled shared memory (TMA),
 //                 fp32 scores in tensor memory, double buffered;
@@ -100,39 +100,37 @@ __device__ __forceinline__ uint64_t v_desc(uint32_t smem_addr, int key16) {
   return d;
 }
 
-// Work items of the persistent grid: (sequence, query tile) pairs sorted by query tile, longest
-// first, each for every head; item i -> pair i / H, head i % H.  CTA c takes items c, c + grid,
-// ... in that order, so its pair rank only grows and the cursor below is advanced, never rewound.
+// Work items of the persistent grid, sequence by sequence; within a sequence by query tile
+// (longest first in even sequences, shortest first in odd ones), each tile for every head.  CTA
+// c takes items c, c + grid, ...  The CTAs running at one time then work on one or two
+// sequences, whose keys and values stay in L2 (with the tiles of all sequences sorted into one
+// list, every sequence's keys were live at once and were re-read from DRAM 3.6 times), and
+// the alternating direction evens out the CTAs' total tile counts.  The cursor only moves forward.
 struct ItemCursor {
-  int lvl;    // query tile index of the pairs being enumerated
-  int base;   // rank of the first pair with this query tile
-  int cnt;    // sequences that have this query tile
+  int seq;    // sequence being enumerated
+  int base;   // index of its first item
+  int nt;     // its query tiles (-1: not counted yet)
 };
 
 __device__ __forceinline__ int seq_tiles(const TcParams& p, int s) {
   return (p.cu_exec[s + 1] - p.cu_exec[s] + kTcTile - 1) / kTcTile;
 }
 
-// pair of rank r (r must not decrease between calls): returns false past the last pair
-__device__ __forceinline__ bool pair_of_rank(const TcParams& p, ItemCursor& c, int r, int& b, int& qt) {
-  while (c.lvl >= 0) {
-    if (c.cnt < 0) {  // count the sequences of this level once
-      c.cnt = 0;
-      for (int s = 0; s < p.B; ++s) c.cnt += seq_tiles(p, s) > c.lvl ? 1 : 0;
+// item i (i must not decrease between calls) -> sequence, head, query tile; false past the end
+__device__ __forceinline__ bool item_at(const TcParams& p, ItemCursor& c, int i, int& b, int& h, int& qt) {
+  while (c.seq < p.B) {
+    if (c.nt < 0) c.nt = seq_tiles(p, c.seq);
+    const int n = c.nt * p.H;
+    if (i < c.base + n) {
+      const int r = i - c.base;
+      b = c.seq;
+      h = r % p.H;
+      qt = (c.seq & 1) ? r / p.H : c.nt - 1 - r / p.H;
+      return true;
     }
-    if (r < c.base + c.cnt) {
-      int k = r - c.base;
-      for (int s = 0; s < p.B; ++s) {
-        if (seq_tiles(p, s) > c.lvl) {
-          if (k == 0) { b = s; qt = c.lvl; return true; }
-          --k;
-        }
-      }
-      return false;
-    }
-    c.base += c.cnt;
-    c.cnt = -1;
-    --c.lvl;
+    c.base += n;
+    c.nt = -1;
+    ++c.seq;
   }
   return false;
 }
@@ -155,12 +153,8 @@ __global__ void __launch_bounds__(kTcThreads, 1)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-  int max_nt = 0, n_pairs = 0;
-  for (int s = 0; s < p.B; ++s) {
-    const int nt = seq_tiles(p, s);
-    max_nt = max(max_nt, nt);
-    n_pairs += nt;
-  }
+  int n_pairs = 0;
+  for (int s = 0; s < p.B; ++s) n_pairs += seq_tiles(p, s);
   const int n_items = n_pairs * p.H;
   if ((int)blockIdx.x >= n_items) return;  // uniform for the CTA: nothing allocated yet
 
@@ -198,18 +192,18 @@ __global__ void __launch_bounds__(kTcThreads, 1)
   // every role walks the same item sequence with its own cursor and its own running counters:
   // t = key tiles so far (ring stage t & 1, phase (t >> 1) & 1), it = items so far
   ItemCursor cur;
-  cur.lvl = max_nt - 1;
+  cur.seq = 0;
   cur.base = 0;
-  cur.cnt = -1;
+  cur.nt = -1;
 
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
     if (lane == 0) {
       uint32_t t = 0, it = 0;
       for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++it) {
-        int b, qt;
-        if (!pair_of_rank(p, cur, item / p.H, b, qt)) break;
-        const int h = item % p.H, hk = h / p.rep;
+        int b, h, qt;
+        if (!item_at(p, cur, item, b, h, qt)) break;
+        const int hk = h / p.rep;
         const int seq0 = p.cu_exec[b];
         if (!tc_wait(&sh.q_empty, (it & 1u) ^ 1u, &sh, p.status)) break;
         mbar_arrive_expect_tx(&sh.q_full, TILE_BYTES);
@@ -235,9 +229,9 @@ __global__ void __launch_bounds__(kTcThreads, 1)
       uint32_t t = 0;
       bool ok = true;
       for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
-        int b, qt;
-        if (!pair_of_rank(p, cur, item / p.H, b, qt)) break;
-        const int hk = (item % p.H) / p.rep;
+        int b, h, qt;
+        if (!item_at(p, cur, item, b, h, qt)) break;
+        const int hk = h / p.rep;
         const int seq0 = p.cu_exec[b];
         for (int j = 0; j <= qt; ++j, ++t) {
           const int s = t % kTcVStages;
@@ -273,8 +267,8 @@ __global__ void __launch_bounds__(kTcThreads, 1)
       uint32_t t = 0, it = 0;
       bool ok = true;
       for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x, ++it) {
-        int b, qt;
-        if (!pair_of_rank(p, cur, item / p.H, b, qt)) break;
+        int b, h, qt;
+        if (!item_at(p, cur, item, b, h, qt)) break;
         const int n_kt = qt + 1;
         if (!tc_wait(&sh.q_full, it & 1u, &sh, p.status)) break;
         ok = issue_qk(t);
@@ -321,9 +315,8 @@ __global__ void __launch_bounds__(kTcThreads, 1)
     uint32_t t = 0, it = 0;
     bool alive = true;
     for (int item = blockIdx.x; alive && item < n_items; item += gridDim.x, ++it) {
-      int b, qt;
-      if (!pair_of_rank(p, cur, item / p.H, b, qt)) break;
-      const int h = item % p.H;
+      int b, h, qt;
+      if (!item_at(p, cur, item, b, h, qt)) break;
       const int seq0 = p.cu_exec[b];
       const int len = p.cu_exec[b + 1] - seq0;
       const int q0 = qt * kTcTile;
@@ -494,7 +487,7 @@ static int launch_tc(const CUtensorMap& tm, const TcParams& p, int max_tiles, in
       return QTALE_ERR_CUDA;
     configured[dev] = true;
   }
-  // persistent grid: one CTA per SM walks the (sequence, query tile, head) items, longest first
+  // persistent grid: one CTA per SM walks the (sequence, query tile, head) items
   (void)max_tiles;
   (void)H;
   attn_prefill_tc_kernel<HD, ACT><<<sm_count(), kTcThreads, smem, s>>>(tm, p);
