@@ -102,6 +102,7 @@ def test_ratio_zero_identity_and_ratio_one_dense(env):
     ("ragged_hd64", inputs.LayerShape(256, 4, 4, 64, 688, 4, 64), 5, 200, 0.3, True),
     ("gqa_hd128", inputs.LayerShape(512, 4, 2, 128, 1024, 4, 128), 3, 300, 0.6, True),
     ("int3_hd128", inputs.LayerShape(512, 4, 4, 128, 1024, 3, 128), 2, 256, 0.7, True),
+    ("many_query_tiles_hd128", inputs.LayerShape(256, 2, 2, 128, 512, 4, 128), 4, 700, 0.9, True),
     ("unfused_swiglu", inputs.LayerShape(256, 4, 4, 64, 688, 4, 64), 2, 128, 0.5, False),
     ("one_token_sequences", inputs.LayerShape(256, 4, 1, 64, 512, 4, 128), 40, 1, 0.5, True),
 ])
