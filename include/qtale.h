@@ -30,7 +30,14 @@
  *    rounding error of a 4096-wide layer inside the max-abs 2e-2 bound (fp16's
  *    range, 65504, must then cover those tensors).  Accumulation is fp32.
  *    Tokens of all sequences are flattened: token t of the call belongs to
- *    sequence b with cu_seqlens[b] <= t < cu_seqlens[b+1].
+ *    sequence b with cu_seqlens[b] <= t < cu_seqlens[b+1].  cu_seqlens (device,
+ *    int32 [B+1]) must satisfy 0 = cu_seqlens[0] <= ... <= cu_seqlens[B] = T
+ *    (empty sequences are fine).  The host cannot see it, so the selection
+ *    kernel checks it: a violation records QTALE_ERR_SHAPE in the device status
+ *    word, tokens outside [cu_seqlens[0], cu_seqlens[B]) never execute, and no
+ *    access leaves the B + 1 entries.
+ *  - Workspaces need not be cleared by the caller, and may be reused between
+ *    calls of different sizes: every kernel initialises what it reads.
  *  - A device-side wait that exceeds its iteration limit ends the kernel
  *    normally and records QTALE_ERR_TIMEOUT in a device status word that
  *    qtale_device_status() reads.
@@ -106,7 +113,7 @@ size_t qtale_router_select_workspace_bytes(int T);
  *
  *   x          [T, d] bf16              w_router  [d] fp32
  *   valid      [T] uint8 or NULL        cu_seqlens [B+1] int32, pos0 [B] or NULL
- * Limits: d % 8 == 0, 1 <= T <= 2^24, 1 <= B <= T.
+ * Limits: d % 8 == 0, 1 <= T <= 2^24, 1 <= B <= T, 0 <= k <= T.
  */
 int qtale_router_select(const void* x, int T, int d, const float* w_router, float bias,
                         const float* scores_override, const uint8_t* valid,
@@ -250,8 +257,10 @@ typedef struct {
   int select_mode;                          /* QTALE_SELECT_*                             */
   float theta;                              /* threshold of Eq. 9 (THRESHOLD)             */
   float ratio;                              /* execution ratio in [0,1] (TOPK): k =
-                                               qtale_topk_count(ratio, T), capped by the
-                                               number of valid tokens                      */
+                                               qtale_topk_count(ratio, number of valid
+                                               tokens); padding does not count (App. B.2);
+                                               with a `valid` mask the count is taken on
+                                               the device                                   */
   int act_dtype;                            /* QTALE_ACT_*: format of the layer's internal
                                                16-bit tensors and of its KV cache          */
 } qtale_layer_config;
@@ -268,7 +277,12 @@ typedef struct {
 } qtale_layer_weights;
 
 /* Per-layer KV cache.  Only executed tokens enter it: a bypassed token does not
- * evaluate f_l (Eq. 3) and therefore produces no key or value at that layer. */
+ * evaluate f_l (Eq. 3) and therefore produces no key or value at that layer.
+ * Capacity: a call appends (executed tokens of sequence b) entries to sequence b
+ * and needs kv_len[b] + that count <= cap.  The lengths live on the device, so
+ * the host cannot check this: entries that do not fit are dropped, kv_len[b]
+ * stays at cap, and QTALE_ERR_CAPACITY is recorded in the device status word
+ * (the layer output of that sequence is then not meaningful). */
 typedef struct {
   void* k;         /* act_dtype [B, cap, n_kv_heads * head_dim], rotary already applied */
   void* v;         /* act_dtype [B, cap, n_kv_heads * head_dim]                         */
@@ -322,12 +336,14 @@ size_t qtale_model_workspace_bytes(const qtale_model_config* cfg, int T_cap, int
  * qtale_layer_forward sharing one theta (Sec. 3.4) or, when per_layer_ratio
  * (HOST float [n_layers]) is given, per-layer top-k at those ratios; final
  * RMSNorm and LM head on the requested rows.
- *   ids [T] int32; hidden_out [T, d] bf16 (final residual stream);
+ *   ids [T] int32; valid [T] uint8 or NULL (0 = padding token, never executed
+ *   at any layer, App. B.2); hidden_out [T, d] bf16 (final residual stream);
  *   logits_out fp32 [n_logit_rows, vocab] or NULL; logit_rows [n_logit_rows]
  *   int32 device; per_layer_n_exec [n_layers] int32 device.
  */
 int qtale_model_prefill(const qtale_model_config* cfg, const qtale_model_weights* w,
                         const int32_t* ids, int T, const int32_t* cu_seqlens, int B,
+                        const uint8_t* valid,
                         const float* per_layer_ratio, void* hidden_out, float* logits_out,
                         const int32_t* logit_rows, int n_logit_rows, int32_t* per_layer_n_exec,
                         void* ws, size_t ws_bytes, void* stream);

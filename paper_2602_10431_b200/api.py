@@ -117,8 +117,8 @@ def lib():
         L.qtale_model_workspace_bytes.argtypes = [C.POINTER(ModelConfig), C.c_int, C.c_int, C.c_int]
         L.qtale_model_prefill.argtypes = [
             C.POINTER(ModelConfig), C.POINTER(ModelWeightsC), C.c_void_p, C.c_int, C.c_void_p,
-            C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p,
-            C.c_void_p, C.c_size_t, C.c_void_p]
+            C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
+            C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
         _lib = L
     return _lib
 
@@ -352,7 +352,7 @@ def model_workspace_bytes(cfg: ModelConfig, T_cap, B_cap, n_logit_rows) -> int:
 
 def model_prefill(cfg: ModelConfig, layers, embed, ids, cu_seqlens, ws, hidden_out,
                   per_layer_ratio=None, final_gamma=None, lm_head=None, logit_rows=None,
-                  logits_out=None, per_layer_n_exec=None):
+                  logits_out=None, per_layer_n_exec=None, valid=None):
     """qtale_model_prefill.  layers: list of LayerWeights."""
     T = int(ids.shape[0])
     B = int(cu_seqlens.shape[0]) - 1
@@ -365,7 +365,7 @@ def model_prefill(cfg: ModelConfig, layers, embed, ids, cu_seqlens, ws, hidden_o
         ratios = (C.c_float * len(layers))(*[float(r) for r in per_layer_ratio])
     n_rows = int(logit_rows.shape[0]) if logit_rows is not None else 0
     check(lib().qtale_model_prefill(
-        C.byref(cfg), C.byref(mw), _ptr(ids), T, _ptr(cu_seqlens), B,
+        C.byref(cfg), C.byref(mw), _ptr(ids), T, _ptr(cu_seqlens), B, _ptr(valid),
         C.cast(ratios, C.c_void_p) if ratios is not None else None, _ptr(hidden_out),
         _ptr(logits_out), _ptr(logit_rows), n_rows, _ptr(per_layer_n_exec), _ptr(ws),
         ws.numel() * ws.element_size(), _stream()), "qtale_model_prefill")

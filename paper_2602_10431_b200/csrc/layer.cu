@@ -3,6 +3,7 @@
 // the router and the residual write-back is sized by the device-side executed
 // token count; the host never reads it.
 #include "attention.cuh"
+#include "router_select.cuh"
 #include "rowops.cuh"
 #include "wq_gemm.cuh"
 
@@ -92,12 +93,17 @@ static int layer_forward_impl(const qtale_layer_config* c, const qtale_layer_wei
     QTALE_TRY(qtale_index_bookkeeping(forced_idx, forced_n, T, cu_seqlens, B, pos0, ws.n_exec,
                                       ws.cu_exec, ws.pos, s));
   } else {
+    // top-k: without a padding mask every token is valid and k is known here; with one the
+    // kernel counts the valid tokens first (the ratio refers to them, App. B.2)
     int k = 0;
-    if (c->select_mode == QTALE_SELECT_TOPK) k = qtale_topk_count((double)c->ratio, T);
-    QTALE_TRY(qtale_router_select(x, T, d, w->router_w, w->router_b, scores_override, valid,
-                                  cu_seqlens, B, pos0, c->select_mode, c->theta, k,
-                                  scores_out ? scores_out : ws.scores, ws.idx, ws.n_exec,
-                                  ws.cu_exec, ws.pos, ws.ticket, 256, s));
+    double ratio = -1.0;
+    if (c->select_mode == QTALE_SELECT_TOPK) {
+      if (valid) ratio = (double)c->ratio; else k = qtale_topk_count((double)c->ratio, T);
+    }
+    QTALE_TRY(router_select_launch(x, T, d, w->router_w, w->router_b, scores_override, valid,
+                                   cu_seqlens, B, pos0, c->select_mode, c->theta, k, ratio,
+                                   scores_out ? scores_out : ws.scores, ws.idx, ws.n_exec,
+                                   ws.cu_exec, ws.pos, ws.ticket, 256, s));
   }
   if (n_exec_out &&
       cudaMemcpyAsync(n_exec_out, ws.n_exec, sizeof(int32_t), cudaMemcpyDeviceToDevice, s) !=
@@ -223,6 +229,7 @@ size_t qtale_model_workspace_bytes(const qtale_model_config* cfg, int T_cap, int
 
 int qtale_model_prefill(const qtale_model_config* cfg, const qtale_model_weights* w,
                         const int32_t* ids, int T, const int32_t* cu_seqlens, int B,
+                        const uint8_t* valid,
                         const float* per_layer_ratio, void* hidden_out, float* logits_out,
                         const int32_t* logit_rows, int n_logit_rows, int32_t* per_layer_n_exec,
                         void* ws, size_t ws_bytes, void* stream) {
@@ -252,7 +259,7 @@ int qtale_model_prefill(const qtale_model_config* cfg, const qtale_model_weights
       return QTALE_ERR_MODE;
     }
     QTALE_TRY(layer_forward_impl(&lc, &w->layers[l], hidden_out, T, cu_seqlens, B, nullptr,
-                                 nullptr, nullptr, nullptr, 0, nullptr, QTALE_PHASE_PREFILL,
+                                 valid, nullptr, nullptr, 0, nullptr, QTALE_PHASE_PREFILL,
                                  per_layer_n_exec ? per_layer_n_exec + l : nullptr, nullptr, lw,
                                  s));
   }

@@ -5,7 +5,7 @@
 // B (the CTA that finishes last, found with a ticket counter): threshold or
 // top-k decision on the fp32 scores and an ordered prefix-sum compaction into
 // the ascending index list, the per-sequence offsets and the positions.
-#include "common.cuh"
+#include "router_select.cuh"
 
 namespace qtale {
 
@@ -25,7 +25,9 @@ struct RouterParams {
   int32_t* cu_exec;
   int32_t* pos;
   unsigned int* ticket;
-  int T, d, B, mode, k;
+  int* status;
+  int T, d, B, mode, k;  // k < 0 (top-k): k = floor(ratio * valid tokens + 0.5), counted here
+  double ratio;
   float bias, theta;
 };
 
@@ -48,7 +50,18 @@ __device__ void select_and_compact(const RouterParams& p, uint32_t* sh_hist, int
   const int lane = tid & 31, wid = tid >> 5, nwarps = nthr >> 5;
   const int T = p.T;
   __shared__ uint32_t s_prefix, s_mask;
-  __shared__ int s_remaining;
+  __shared__ int s_remaining, s_n_valid;
+
+  // cu_seqlens must be 0 = cu[0] <= cu[1] <= ... <= cu[B] = T.  Anything else is reported in the
+  // status word; tokens outside [cu[0], cu[B]) then never execute and every walk below stays
+  // inside the B + 1 entries.
+  const int t_begin = min(max(__ldg(p.cu_seqlens), 0), T);
+  const int t_end = min(max(__ldg(p.cu_seqlens + p.B), t_begin), T);
+  {
+    bool bad = tid == 0 && (__ldg(p.cu_seqlens) != 0 || __ldg(p.cu_seqlens + p.B) != T);
+    for (int q = tid; q < p.B; q += nthr) bad |= __ldg(p.cu_seqlens + q) > __ldg(p.cu_seqlens + q + 1);
+    if (bad) report_device_error(p.status, QTALE_ERR_SHAPE);
+  }
 
   const int seg = ((T + nwarps - 1) / nwarps + 31) & ~31;  // tokens per warp, multiple of 32
   const int w0 = min(T, wid * seg), w1 = min(T, w0 + seg);
@@ -58,7 +71,7 @@ __device__ void select_and_compact(const RouterParams& p, uint32_t* sh_hist, int
   // score and validity of the token of step i (0 and false past the end)
   auto load_one = [&](int i, float& sc, bool& ok) {
     const int t = w0 + 32 * i + lane;
-    ok = t < w1;
+    ok = t < w1 && t >= t_begin && t < t_end;
     sc = 0.f;
     if (ok) {
       sc = __ldcg(p.scores + t);
@@ -79,12 +92,37 @@ __device__ void select_and_compact(const RouterParams& p, uint32_t* sh_hist, int
   uint32_t tau = 0;  // key of the k-th largest score (top-k)
   int need_eq = 0;   // how many tokens with key == tau execute (lowest indices first)
 
-  if (p.mode == QTALE_SELECT_TOPK && p.k > 0) {
+  int k_sel = p.k;
+  if (p.mode == QTALE_SELECT_TOPK && p.k < 0) {
+    // k for a requested ratio of the valid tokens (padding does not count)
+    if (tid == 0) s_n_valid = 0;
+    __syncthreads();
+    int nv = 0;
+    if (keep) {
+      nv = __popc(kok);
+    } else {
+      for (int i = 0; i < n_it; ++i) {
+        float sc;
+        bool ok;
+        load_one(i, sc, ok);
+        nv += ok ? 1 : 0;
+      }
+    }
+    nv = __reduce_add_sync(0xffffffffu, nv);
+    if (lane == 0) atomicAdd(&s_n_valid, nv);
+    __syncthreads();
+    const int n_valid = s_n_valid;
+    double kd = floor(p.ratio * (double)n_valid + 0.5);
+    kd = kd < 0.0 ? 0.0 : (kd > (double)n_valid ? (double)n_valid : kd);
+    k_sel = (int)kd;
+  }
+
+  if (p.mode == QTALE_SELECT_TOPK && k_sel > 0) {
     // MSB-first radix select (four 8-bit digits) of the k-th largest key among valid tokens
     if (tid == 0) {
       s_prefix = 0;
       s_mask = 0;
-      s_remaining = p.k;
+      s_remaining = k_sel;
     }
     for (int pass = 0; pass < 4; ++pass) {
       const int shift = 24 - 8 * pass;
@@ -165,7 +203,7 @@ __device__ void select_and_compact(const RouterParams& p, uint32_t* sh_hist, int
   }
 
   const bool topk = p.mode == QTALE_SELECT_TOPK;
-  const bool none = topk && p.k <= 0;
+  const bool none = topk && k_sel <= 0;
   // (executes for sure, executes if among the first need_eq equal keys)
   auto classify = [&](float sc, bool ok, bool& sure, bool& eq) {
     if (topk) {
@@ -245,7 +283,7 @@ __device__ void select_and_compact(const RouterParams& p, uint32_t* sh_hist, int
     const uint32_t m_take = __ballot_sync(0xffffffffu, take);
     const int my_out = out + __popc(m_take & lt);
     if (t < w1) {
-      while (t >= seq_end) {  // move to the sequence holding t (skips empty ones)
+      while (t >= seq_end && b + 1 < p.B) {  // move to the sequence holding t (skips empty ones)
         ++b;
         seq_start = seq_end;
         seq_end = __ldg(p.cu_seqlens + b + 1);
@@ -410,16 +448,30 @@ int qtale_router_select(const void* x, int T, int d, const float* w_router, floa
                         float theta, int k, float* scores_out, int32_t* idx_out,
                         int32_t* n_exec_out, int32_t* cu_exec_out, int32_t* pos_out, void* ws,
                         size_t ws_bytes, void* stream) {
+  return router_select_launch(x, T, d, w_router, bias, scores_override, valid, cu_seqlens, B, pos0,
+                              mode, theta, k, -1.0, scores_out, idx_out, n_exec_out, cu_exec_out,
+                              pos_out, ws, ws_bytes, static_cast<cudaStream_t>(stream));
+}
+
+}  // extern "C"
+
+namespace qtale {
+
+int router_select_launch(const void* x, int T, int d, const float* w_router, float bias,
+                         const float* scores_override, const uint8_t* valid,
+                         const int32_t* cu_seqlens, int B, const int32_t* pos0, int mode,
+                         float theta, int k, double ratio, float* scores_out, int32_t* idx_out,
+                         int32_t* n_exec_out, int32_t* cu_exec_out, int32_t* pos_out, void* ws,
+                         size_t ws_bytes, cudaStream_t s) {
   if (!scores_out || !idx_out || !n_exec_out || !cu_exec_out || !pos_out || !cu_seqlens || !ws)
     return QTALE_ERR_NULL;
   if (!scores_override && (!x || !w_router)) return QTALE_ERR_NULL;
   if (T < 1 || T > (1 << 24) || B < 1 || B > T) return QTALE_ERR_SHAPE;
   if (!scores_override && (d < 8 || d % 8 != 0 || d > 16384)) return QTALE_ERR_SHAPE;
   if (mode != QTALE_SELECT_THRESHOLD && mode != QTALE_SELECT_TOPK) return QTALE_ERR_MODE;
-  if (mode == QTALE_SELECT_TOPK && (k < 0 || k > T)) return QTALE_ERR_CAPACITY;
+  if (mode == QTALE_SELECT_TOPK && ratio < 0.0 && (k < 0 || k > T)) return QTALE_ERR_CAPACITY;
   if (!aligned16(x) || !aligned16(ws)) return QTALE_ERR_ALIGN;
   if (ws_bytes < qtale_router_select_workspace_bytes(T)) return QTALE_ERR_WORKSPACE;
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
 
   RouterParams p;
   p.x = static_cast<const __nv_bfloat16*>(x);
@@ -434,7 +486,10 @@ int qtale_router_select(const void* x, int T, int d, const float* w_router, floa
   p.cu_exec = cu_exec_out;
   p.pos = pos_out;
   p.ticket = static_cast<unsigned int*>(ws);
-  p.T = T; p.d = d; p.B = B; p.mode = mode; p.k = k;
+  p.status = device_status_ptr();
+  p.T = T; p.d = d; p.B = B; p.mode = mode;
+  p.k = (mode == QTALE_SELECT_TOPK && ratio >= 0.0) ? -1 : k;
+  p.ratio = ratio;
   p.bias = bias; p.theta = theta;
 
   if (cudaMemsetAsync(ws, 0, sizeof(unsigned int), s) != cudaSuccess) return QTALE_ERR_CUDA;
@@ -463,6 +518,10 @@ int qtale_router_select(const void* x, int T, int d, const float* w_router, floa
   router_select_kernel<<<grid, kRouterThreads, smem, s>>>(p);
   return launch_status(cudaGetLastError());
 }
+
+}  // namespace qtale
+
+extern "C" {
 
 // ---- variant for callers that cannot allocate device memory -------------------
 // The kernel's only scratch is its ticket counter; here it lives in a static

@@ -243,24 +243,33 @@ __global__ void __launch_bounds__(kRowThreads)
       if (cu_exec[mid] <= i) lo = mid; else hi = mid;
     }
     const int slot = kv_len[lo] + (i - cu_exec[lo]);
-    if (slot >= cap) continue;  // capacity is validated on the host for the worst case
+    if (slot >= cap) continue;  // cache full: kv_len_update_kernel records QTALE_ERR_CAPACITY
     const size_t dst = ((size_t)lo * cap + slot) * kc + c;
     cache_k[dst] = qkv[(size_t)i * ldc + (q_dim >> 3) + c];
     cache_v[dst] = qkv[(size_t)i * ldc + ((q_dim + kv_dim) >> 3) + c];
   }
 }
 
-__global__ void kv_len_update_kernel(int32_t* kv_len, const int32_t* cu_exec, int B, int cap) {
-  for (int b = blockIdx.x * blockDim.x + threadIdx.x; b < B; b += gridDim.x * blockDim.x)
-    kv_len[b] = min(cap, kv_len[b] + cu_exec[b + 1] - cu_exec[b]);
+// The lengths live on the device, so a full cache can only be detected here: the rows that did
+// not fit are dropped, the length stays at the capacity and the status word reports it.
+__global__ void kv_len_update_kernel(int32_t* kv_len, const int32_t* cu_exec, int B, int cap,
+                                     int* status) {
+  for (int b = blockIdx.x * blockDim.x + threadIdx.x; b < B; b += gridDim.x * blockDim.x) {
+    const int want = kv_len[b] + cu_exec[b + 1] - cu_exec[b];
+    if (want > cap) report_device_error(status, QTALE_ERR_CAPACITY);
+    kv_len[b] = min(cap, want);
+  }
 }
 
-// ---- zero the rows between the executed count and the next multiple of `tile` ----
-// (tiled loads of the attention kernel read whole tiles; rows past the count must be finite)
+// ---- zero the `tile` rows that follow the executed count ----
+// The attention kernel loads key / value tiles of `tile` rows that start at any executed row
+// (a sequence's first row plus a multiple of the tile), so a tile can reach up to tile - 1 rows
+// past the count.  Masked keys get probability 0, but 0 x NaN is NaN in the P V product: those
+// rows must hold finite values whatever the workspace held before.
 __global__ void zero_tail_rows_kernel(uint4* __restrict__ buf, const int32_t* __restrict__ n_exec,
                                       int cap, int ld, int tile) {
   const int n = min(*n_exec, cap);
-  const int end = min(cap, (n + tile - 1) / tile * tile);
+  const int end = min(cap, n + tile);
   const int ldc = ld >> 3;
   const size_t total = (size_t)(end - n) * ldc;
   for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < total;
@@ -381,7 +390,7 @@ int launch_kv_append(const void* qkv, const int32_t* n_exec, int cap_rows, int l
       static_cast<const uint4*>(qkv), n_exec, cap_rows, ld, q_dim, kv_dim, cu_exec, B,
       static_cast<uint4*>(cache_k), static_cast<uint4*>(cache_v), kv_len, cap);
   if (cudaGetLastError() != cudaSuccess) return QTALE_ERR_CUDA;
-  kv_len_update_kernel<<<(B + 255) / 256, 256, 0, s>>>(kv_len, cu_exec, B, cap);
+  kv_len_update_kernel<<<(B + 255) / 256, 256, 0, s>>>(kv_len, cu_exec, B, cap, device_status_ptr());
   return launch_status(cudaGetLastError());
 }
 

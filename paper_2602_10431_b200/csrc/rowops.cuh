@@ -21,7 +21,7 @@ int launch_swiglu(const void* gu, const int32_t* n_exec, int cap, int F, void* a
 int launch_kv_append(const void* qkv, const int32_t* n_exec, int cap_rows, int ld, int q_dim,
                      int kv_dim, const int32_t* cu_exec, int B, void* cache_k, void* cache_v,
                      int32_t* kv_len, int cap, cudaStream_t s);
-// zeroes rows [*n_exec, roundup(*n_exec, tile)) of a 16-bit [cap, ld] tensor
+// zeroes rows [*n_exec, *n_exec + tile) (below cap) of a 16-bit [cap, ld] tensor
 int launch_zero_tail_rows(void* buf, const int32_t* n_exec, int cap, int ld, int tile,
                           cudaStream_t s);
 int launch_embed(const void* embed, const int32_t* ids, int T, int d, int vocab, void* out,

@@ -83,6 +83,31 @@ def test_router_select_padding_override_ties_pos0(env):
         _check_select(api, torch, r, p, oracle.select_topk(p, k, valid), cu, pos0)
 
 
+def test_inconsistent_cu_seqlens_is_reported_not_followed(env):
+    """cu_seqlens lives on the device, so the kernel checks it: offsets that do not end at T
+    (or are not ascending) give QTALE_ERR_SHAPE in the status word, tokens outside
+    [cu[0], cu[B]) never execute, and nothing outside the B + 1 entries is read."""
+    api, torch, dev = env
+    T, d = 256, 256
+    x = inputs.hidden_states(31, T, d)
+    w = inputs.round_bf16((inputs.normal(31, 5, d) * 0.02).astype(np.float32))
+    xd, wd = api.to_device_bf16(x, dev), torch.from_numpy(w).to(dev)
+    p_ref = oracle.router_scores(x, w, 0.0)
+    for cu, lo, hi in [([0, 100, 200], 0, 200), ([10, 100, 256], 10, 256), ([0, 200, 100, 256], 0, 256)]:
+        cud = torch.tensor(cu, dtype=torch.int32, device=dev)
+        r = api.router_select(xd, wd, 0.0, cud, api.SELECT_THRESHOLD, theta=0.0)   # everything executes
+        torch.cuda.synchronize()
+        assert api.device_status() == -3                        # QTALE_ERR_SHAPE
+        n = int(r["n_exec"].item())
+        idx = r["idx"].cpu().numpy()
+        assert n == hi - lo and np.array_equal(idx[:n], np.arange(lo, hi)) and (idx[n:] == -1).all()
+        assert np.abs(r["scores"].cpu().numpy() - p_ref).max() <= 1e-7
+    # a consistent list right afterwards: clean status
+    r = api.router_select(xd, wd, 0.0, torch.tensor([0, 0, 256], dtype=torch.int32, device=dev),
+                          api.SELECT_TOPK, k=17)
+    assert api.device_status() == 0 and int(r["n_exec"].item()) == 17
+
+
 def test_index_bookkeeping(env):
     api, torch, dev = env
     T = 500
@@ -141,6 +166,9 @@ GEMM_CASES = [
     (64, 9600, 128, 4, 128, 37),           # decode kernel, half a row tile per CTA
     (48, 38016, 64, 3, 64, None),          # decode kernel, a whole row tile per CTA, 3-bit
     (33, 256, 704, 4, 64, 33),             # decode kernel, a quarter tile per CTA, four K groups, odd K blocks
+    (64, 512, 4096, 3, 128, 58),           # decode kernel at the 7B-shaped K: 64 K blocks through the ring
+    (64, 256, 11008, 4, 64, 38),           # decode kernel, K of the down projection: 172 K blocks
+    (57, 384, 11008, 3, 128, None),        # the same in 3-bit, token count not a multiple of 8
 ]
 
 
@@ -220,7 +248,9 @@ def test_wq_gemm_epilogues(env, act):
 
 def test_wq_gemm_full_size_sampled(env):
     """7B-sized gate/up projection in the launch configuration the benchmark times
-    (8192-token capacity, device-side count): sampled outputs against the oracle."""
+    (8192-token capacity, device-side count): 66 complete output rows, two from every 256-token
+    tile position of the largest tile width plus the rows around the count, against the oracle
+    (every weight row tile and every K block of those token rows)."""
     api, torch, dev = env
     M, N, K, bits, group = 8192, 22016, 4096, 4, 128
     wq = inputs.quantized_weight(0, 2, N, K, bits, group)
@@ -230,12 +260,11 @@ def test_wq_gemm_full_size_sampled(env):
     md = torch.tensor([m_dev], dtype=torch.int32, device=dev)
     y = api.wq_gemm(api.to_device_act(a, 1, dev), qw, md, api.EPI_STORE_F32)
     assert api.device_status() == 0
-    rows = np.array([0, 1, 255, 256, 4095, 4096, 7000, 7371, 7372])
-    cols = np.unique(np.concatenate([[0, 1, 127, 128, 11007, 11008, 22015],
-                                     inputs.integers(8, 1, 40, N)]))
-    sub = dict(packed=wq["packed"][cols], scales=wq["scales"][cols], zeros=wq["zeros"][cols],
-               N=len(cols), K=K, bits=bits, group=group)
-    ref = oracle.linear(a[rows], round_act(oracle.dequantize_weight(sub), 1))
-    got = y[torch.from_numpy(rows).to(dev)][:, torch.from_numpy(cols).to(dev)].cpu().numpy()
+    off = inputs.integers(8, 1, 64, 256)
+    rows = np.unique(np.concatenate([np.minimum((np.arange(64) // 2) * 256 + off, m_dev - 1),
+                                     [0, 255, 256, 7371, 7372]]))
+    w_hat = round_act(oracle.dequantize_weight(wq), 1)
+    ref = oracle.linear(a[rows], w_hat)
+    got = y[torch.from_numpy(rows).to(dev)].cpu().numpy()
     assert np.abs(got - ref).max() <= 2e-4 * max(1.0, np.abs(ref).max())
     assert not y[m_dev:].any().item()

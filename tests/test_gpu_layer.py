@@ -47,9 +47,10 @@ class Case:
     def cfg(self, mode, act=1, **kw):
         return self.api.layer_config(self.sh, mode, act_dtype=act, **kw)
 
-    def gpu(self, cfg, **kw):
+    def gpu(self, cfg, ws_fill=0, **kw):
         api, torch = self.api, self.torch
-        ws = torch.zeros(api.layer_workspace_bytes(cfg, self.T, self.B), dtype=torch.uint8, device=self.dev)
+        ws = torch.full((api.layer_workspace_bytes(cfg, self.T, self.B),), ws_fill, dtype=torch.uint8,
+                        device=self.dev)
         xd = api.to_device_bf16(self.x, self.dev)
         nex = torch.full((1,), -1, dtype=torch.int32, device=self.dev)
         sc = torch.zeros(self.T, dtype=torch.float32, device=self.dev)
@@ -136,6 +137,65 @@ def test_padding_tokens_never_execute(env):
     assert_layer_close(out, ref, strict=True)
 
 
+def test_topk_ratio_counts_valid_tokens_only(env):
+    """Top-k at a ratio with padding: k is the ratio of the VALID tokens (padding is not part
+    of the workload), counted on the device, and padding never executes."""
+    api, torch, dev = env
+    sh = inputs.LayerShape(256, 4, 4, 64, 512, 4, 64)
+    case = Case(api, torch, dev, sh, [0, 150, 400], seed=13, router_std=0.05)
+    valid = np.ones(case.T, np.uint8)
+    valid[100:150] = 0
+    valid[330:400] = 0                                           # 30 % padding
+    p, m = oracle.route(case.layer, case.x, "topk", ratio=0.5, valid=valid)
+    assert int(m.sum()) == oracle.topk_count(0.5, 280) == 140
+    ref, n_ref = oracle.layer_forward(case.layer, case.x, case.cu, m)
+    out, n, _ = case.gpu(api.layer_config(sh, api.SELECT_TOPK, ratio=0.5),
+                         valid=torch.from_numpy(valid).to(dev))
+    assert n == n_ref == 140
+    assert np.array_equal((out != case.x).any(axis=1), m.astype(bool))
+    assert_layer_close(out, ref, strict=True)
+
+
+@pytest.mark.parametrize("fill", [0xFF, 0x7C])
+def test_workspace_contents_do_not_matter(env, fill):
+    """The caller's workspace is not cleared: every byte 0xFF (fp16 / bf16 NaN patterns) or
+    0x7C (fp16 0x7C7C is a NaN, bf16 a huge number).  The executed count is a multiple of the
+    attention's 128-row tile and the sequences start at ragged rows, so the last key / value
+    tile of a sequence reaches past the executed rows into whatever the workspace held."""
+    api, torch, dev = env
+    sh = inputs.LayerShape(256, 2, 2, 128, 512, 4, 128)
+    case = Case(api, torch, dev, sh, [0, 190, 447, 700], seed=14, router_std=0.05)
+    k = 256
+    p, m = oracle.route(case.layer, case.x, "topk", ratio=k / case.T)
+    assert int(m.sum()) == k
+    ref, _ = oracle.layer_forward(case.layer, case.x, case.cu, m)
+    for act in (0, 1):
+        out, n, _ = case.gpu(case.cfg(api.SELECT_TOPK, act, ratio=k / case.T), ws_fill=fill)
+        assert n == k and np.isfinite(out).all()
+        assert_layer_close(out, ref, strict=True)
+
+
+def test_full_kv_cache_is_reported(env):
+    """A decode step on a cache that is already full cannot append: the step reports
+    QTALE_ERR_CAPACITY through the device status word instead of silently attending without
+    the new token."""
+    api, torch, dev = env
+    sh = inputs.LayerShape(256, 2, 2, 128, 512, 4, 64)
+    B, cap = 3, 16
+    case = Case(api, torch, dev, sh, inputs.cu_seqlens_uniform(B, 1), seed=15)
+    kv = api.KvCache(B, cap, sh.kv_dim, dev, act_dtype=1)
+    kv.kv_len.copy_(torch.tensor([cap, 3, cap - 1], dtype=torch.int32, device=dev))
+    cfg = case.cfg(api.SELECT_THRESHOLD, 1, theta=0.0)          # every sequence executes
+    ws = torch.zeros(api.layer_workspace_bytes(cfg, B, B), dtype=torch.uint8, device=dev)
+    xd = api.to_device_bf16(case.x, dev)
+    nex = torch.zeros(1, dtype=torch.int32, device=dev)
+    api.layer_forward(cfg, case.lw, xd, case.cud, ws, nex, pos0=kv.kv_len.clone(), kv=kv,
+                      phase=api.PHASE_DECODE)
+    assert api.device_status() == -7                             # QTALE_ERR_CAPACITY
+    assert api.device_status() == 0                              # reading clears the word
+    assert kv.kv_len.cpu().numpy().tolist() == [cap, 4, cap]
+
+
 @pytest.mark.parametrize("bits,group,Hkv,act", [(3, 128, 4, 1), (4, 64, 2, 0), (4, 64, 2, 1)])
 def test_decode_step_with_executed_only_cache(env, bits, group, Hkv, act):
     """Prefill fills the per-layer cache with executed tokens only; a decode step
@@ -189,7 +249,6 @@ def test_decode_step_with_executed_only_cache(env, bits, group, Hkv, act):
     assert_layer_close(out_new, ref_new, strict=True)
 
 
-@pytest.mark.timeout(120)
 def test_decode_step_ragged_cache_lengths(env):
     """Decode against caches whose lengths differ per sequence and leave every remainder
     modulo the key-loop stride of the decode attention (1 key, a stride plus one, ...):
@@ -270,7 +329,10 @@ def test_model_prefill_teacher_forced(env):
         out = api.to_host_f32(xd)
         got_mask = (out != x_in).any(axis=1)
         assert_selection_matches(np.nonzero(got_mask)[0], int(got_mask.sum()), p, m, theta)
-        if int(nex.item()) == n_ref:
+        # the count may differ from the oracle's only by tokens inside the excluded band
+        band = np.abs(p.astype(np.float64) - theta) <= 1e-6
+        assert abs(int(nex.item()) - n_ref) <= int(band.sum())
+        if not (got_mask != m.astype(bool)).any():
             assert_layer_close(out, ref, strict=True)
         counts.append(int(nex.item()))
     assert api.device_status() == 0
@@ -298,12 +360,37 @@ def test_model_prefill_teacher_forced(env):
     assert per_layer.cpu().numpy().tolist() == [oracle.topk_count(r, T) for r in (0.75, 0.5, 0.25)]
 
 
+_C2 = {}
+
+
+def _c2_case(env):
+    """The 7B-shaped layer of the benchmark (weights generated once per test run)."""
+    if "case" not in _C2:
+        api, torch, dev = env
+        c = inputs.CONFIG_SHAPES["c2"]
+        _C2["case"] = Case(api, torch, dev, c["shape"], inputs.cu_seqlens_uniform(c["B"], c["S"]), seed=0)
+    return _C2["case"]
+
+
+def _assert_c2_close(out, ref, act, inside=0.9995):
+    """`inside`: share of elements that must meet the plain 2e-2 bound (the rest, outputs
+    of magnitude 8 and more, are held to one bf16 ulp)."""
+    if act == 1:
+        assert_layer_close(out, ref, strict=False)
+        assert float((np.abs(out - ref) <= 2e-2).mean()) >= inside
+    else:
+        assert rel_fro(out, ref) <= 1e-2
+        assert np.abs(out - ref).max() <= 0.15
+
+
 @pytest.mark.parametrize("act", [1, 0])
-def test_config2_full_size_layer_prefix_parity(env, act):
+def test_config2_full_size_layer_parity(env, act):
     """The benchmark's configuration (7B-shaped layer, int4 g128, 4 x 2048 tokens,
-    top-k ratio 0.5).  Causal attention makes a prefix of each sequence
-    self-contained, so the oracle is run on the first 96 tokens of every sequence
-    with the full-size run's mask; all bypassed rows must be bit-identical.
+    top-k ratio 0.5), in the launch configuration the benchmark times.  Sequences are
+    independent and causal attention makes a prefix self-contained, so the oracle is run
+    on ALL 2048 tokens of sequence 0 (every query tile, key tile and head of that
+    sequence; about a thousand executed tokens) and on the first 96 tokens of the other
+    three, with the full-size run's mask; all bypassed rows must be bit-identical.
 
     fp16 internal tensors: max-abs 2e-2, widened only to one bf16 ulp of the output
     where |x| >= 8 (half an ulp of the bf16 residual stream alone is 3.1e-2 there).
@@ -312,9 +399,8 @@ def test_config2_full_size_layer_prefix_parity(env, act):
     accumulates to an rms error of about 1.7e-2 at this width, so only the relative
     Frobenius bound can hold; max-abs is checked against 0.15."""
     api, torch, dev = env
-    c = inputs.CONFIG_SHAPES["c2"]
-    sh, B, S = c["shape"], c["B"], c["S"]
-    case = Case(api, torch, dev, sh, inputs.cu_seqlens_uniform(B, S), seed=0)
+    case = _c2_case(env)
+    B, S = case.B, case.T // case.B
     p, m = oracle.route(case.layer, case.x, "topk", ratio=0.5)
     out, n, sc = case.gpu(case.cfg(api.SELECT_TOPK, act, ratio=0.5))
     assert n == 4096 == int(m.sum())
@@ -322,11 +408,84 @@ def test_config2_full_size_layer_prefix_parity(env, act):
     changed = (out != case.x).any(axis=1)
     assert np.array_equal(changed, m.astype(bool))               # bit-exact selection, identity elsewhere
     P = 96
-    rows = np.concatenate([np.arange(b * S, b * S + P) for b in range(B)])
-    ref, _ = oracle.layer_forward(case.layer, case.x[rows], inputs.cu_seqlens_uniform(B, P), m[rows])
-    if act == 1:
-        assert_layer_close(out[rows], ref, strict=False)
-        assert float((np.abs(out[rows] - ref) <= 2e-2).mean()) >= 0.9995
-    else:
-        assert rel_fro(out[rows], ref) <= 1e-2
-        assert np.abs(out[rows] - ref).max() <= 0.15
+    lens = [S] + [P] * (B - 1)
+    rows = np.concatenate([np.arange(b * S, b * S + lens[b]) for b in range(B)])
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    ref, _ = oracle.layer_forward(case.layer, case.x[rows], cu, m[rows])
+    _assert_c2_close(out[rows], ref, act)
+
+
+def test_config2_ratio_one_whole_sequence(env):
+    """Same layer at ratio 1.0 on one 2048-token sequence: sixteen key tiles per query
+    tile and head, every token tile of the GEMMs, the whole output against the oracle."""
+    api, torch, dev = env
+    case = _c2_case(env)
+    S = case.T // case.B
+    x = case.x[S:2 * S]                                          # sequence 1 of the batch
+    cu = np.array([0, S], np.int32)
+    ref, n_ref = oracle.layer_forward(case.layer, x, cu, np.ones(S, np.uint8))
+    cfg = case.cfg(api.SELECT_TOPK, 1, ratio=1.0)
+    ws = torch.full((api.layer_workspace_bytes(cfg, S, 1),), 0xFF, dtype=torch.uint8, device=dev)
+    xd = api.to_device_bf16(x, dev)
+    nex = torch.zeros(1, dtype=torch.int32, device=dev)
+    api.layer_forward(cfg, case.lw, xd, torch.from_numpy(cu).to(dev), ws, nex)
+    assert api.device_status() == 0 and int(nex.item()) == n_ref == S
+    _assert_c2_close(api.to_host_f32(xd), ref, 1)
+
+
+@pytest.mark.parametrize("cfg_name,ratio", [("c3_int3", 0.9), ("c3_int4g64", 0.6)])
+def test_config3_decode_step_parity(env, cfg_name, ratio):
+    """Decode step at the benchmark's width (hidden 4096, 32 heads, FFN 11008; int3 g128 and
+    int4 g64): 64 sequences with one new token each against per-sequence caches of about
+    2048 entries (ragged: 2040 .. 2052), router logits ~ N(0,1) with the threshold between
+    the k-th and (k+1)-th score.  The oracle only pays for the executed sequences' caches,
+    so eight of the 64 sequences (executed and bypassed ones) carry real N(0,1) keys and
+    values of that length and are compared; the others have short caches."""
+    api, torch, dev = env
+    c = inputs.CONFIG_SHAPES[cfg_name]
+    sh, B = c["shape"], c["B"]
+    cap = 2056
+    case = Case(api, torch, dev, sh, inputs.cu_seqlens_uniform(B, 1), seed=21)
+    logits = inputs.normal(21, 2001, B)
+    scores = (1.0 / (1.0 + np.exp(-logits))).astype(np.float32)
+    k = oracle.topk_count(ratio, B)
+    order = np.sort(scores)[::-1]
+    theta = float((order[k - 1] + order[k]) / 2)
+    m = oracle.select_threshold(scores, theta)
+    assert int(m.sum()) == k
+    long_seqs = np.concatenate([np.nonzero(m)[0][:6], np.nonzero(m == 0)[0][:2]])
+    kl = (3 + inputs.integers(21, 2002, B, 40)).astype(np.int32)      # short caches
+    kl[long_seqs] = 2040 + np.arange(len(long_seqs), dtype=np.int32) * 2 - 1
+    kvd = sh.kv_dim
+    ck = np.zeros((B, cap, kvd), np.float32)
+    cv = np.zeros((B, cap, kvd), np.float32)
+    kv = api.KvCache(B, cap, kvd, dev, act_dtype=1)
+    for b in range(B):
+        n = int(kl[b])
+        ck[b, :n] = inputs.activations(21, 3000 + b, n, kvd)
+        cv[b, :n] = inputs.activations(21, 4000 + b, n, kvd)
+        kv.k[b, :n].copy_(torch.from_numpy(ck[b, :n]).to(dev).to(kv.k.dtype))   # bf16-valued normals
+        kv.v[b, :n].copy_(torch.from_numpy(cv[b, :n]).to(dev).to(kv.v.dtype))   # are exact in fp16
+    kv.kv_len.copy_(torch.from_numpy(kl))
+    pos0 = kl.copy()
+    kl_ref = kl.copy()
+    ref, n_ref = oracle.layer_forward(case.layer, case.x, case.cu, m, pos0=pos0, cache_k=ck, cache_v=cv,
+                                      kv_len=kl_ref)
+    cfg = case.cfg(api.SELECT_THRESHOLD, 1, theta=theta)
+    ws = torch.full((api.layer_workspace_bytes(cfg, B, B),), 0xFF, dtype=torch.uint8, device=dev)
+    xd = api.to_device_bf16(case.x, dev)
+    nex = torch.zeros(1, dtype=torch.int32, device=dev)
+    api.layer_forward(cfg, case.lw, xd, case.cud, ws, nex, pos0=torch.from_numpy(pos0).to(dev),
+                      scores_override=torch.from_numpy(scores).to(dev), kv=kv, phase=api.PHASE_DECODE)
+    assert api.device_status() == 0
+    assert int(nex.item()) == n_ref == k
+    assert np.array_equal(kv.kv_len.cpu().numpy(), kl_ref)       # bypassed sequences append nothing
+    out = api.to_host_f32(xd)
+    assert np.array_equal(out[m == 0], case.x[m == 0])
+    _assert_c2_close(out, ref, 1, inside=0.999)
+    # the appended key / value rows of the compared sequences
+    gk, gv = api.to_host_f32(kv.k), api.to_host_f32(kv.v)
+    for b in long_seqs:
+        if m[b]:
+            n = int(kl[b])
+            assert rel_fro(gk[b, n], ck[b, n]) <= 5e-3 and rel_fro(gv[b, n], cv[b, n]) <= 5e-3
