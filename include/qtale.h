@@ -86,6 +86,8 @@ int qtale_device_status(void* stream);
  * clamped to [0, n].  Host function. */
 int qtale_topk_count(double ratio, int n_valid);
 
+/* Scratch of qtale_router_select for a call of T tokens: 16 KB of counters plus
+ * 8 bytes per token (candidate list of the top-k selection). */
 size_t qtale_router_select_workspace_bytes(int T);
 
 /*
@@ -131,21 +133,25 @@ int qtale_router_select(const void* x, int T, int d, const float* w_router, floa
  * a real-time or safety-checked loop that forbids allocator calls after start-up,
  * or a caller that simply has no buffer left to lend as `ws`.  Same arguments,
  * results and limits as qtale_router_select, minus the workspace: the kernel's
- * scratch (its 4-byte ticket counter, 256 bytes reserved) sits in an array that
- * is part of the library's device image, so every GPU that loads the library
- * holds those 256 bytes until the process exits.  The call itself performs no
- * cudaMalloc / cudaFree and uses no allocating library routine.
+ * scratch (counters, histogram, per-CTA counts, top-k candidate list) sits in an
+ * array that is part of the library's device image, sized for
+ * QTALE_ROUTER_STATIC_MAX_TOKENS tokens (16 KB + 8 bytes per token = 528 KB), so
+ * every GPU that loads the library holds that much until the process exits.  The
+ * call itself performs no cudaMalloc / cudaFree and uses no allocating library
+ * routine.
  *
- *  - Limit: T whose scratch need (qtale_router_select_workspace_bytes(T))
- *    exceeds the 256 built-in bytes is refused with QTALE_ERR_CAPACITY.
+ *  - Limit: T > QTALE_ROUTER_STATIC_MAX_TOKENS is refused with
+ *    QTALE_ERR_CAPACITY (nothing is launched); use qtale_router_select with a
+ *    workspace of your own for larger calls.
  *  - The first call on each device looks up the array's device address (one
- *    cudaGetSymbolAddress, result cached per device); make that first call
- *    outside any stream capture.
- *  - All calls on a device share the one array.  The counter is cleared on the
+ *    cudaGetSymbolAddress, result cached per device ordinal; the cache does not
+ *    survive a cudaDeviceReset); make that first call outside any stream capture.
+ *  - All calls on a device share the one array.  Its counters are cleared on the
  *    stream before every launch, so leftovers of the previous call are harmless,
  *    but two calls whose kernels overlap on the GPU (different streams) race on
  *    it: keep calls to this entry point on one stream, or order them yourself.
  */
+#define QTALE_ROUTER_STATIC_MAX_TOKENS 65536
 int qtale_router_select_static(const void* x, int T, int d, const float* w_router, float bias,
                                const float* scores_override, const uint8_t* valid,
                                const int32_t* cu_seqlens, int B, const int32_t* pos0, int mode,

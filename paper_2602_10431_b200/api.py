@@ -152,6 +152,13 @@ def topk_count(ratio: float, n_valid: int) -> int:
 # selection
 # ---------------------------------------------------------------------------------
 
+ROUTER_STATIC_MAX_TOKENS = 65536
+
+
+def router_select_workspace_bytes(T: int) -> int:
+    return int(lib().qtale_router_select_workspace_bytes(int(T)))
+
+
 def router_select(x, w_router, bias, cu_seqlens, mode, theta=0.5, k=0, scores_override=None,
                   valid=None, pos0=None, out=None):
     """qtale_router_select.  x bf16 [T, d]; w_router fp32 [d]; cu_seqlens int32 [B+1].
@@ -168,7 +175,8 @@ def router_select(x, w_router, bias, cu_seqlens, mode, theta=0.5, k=0, scores_ov
     pos = o.get("pos") if "pos" in o else torch.full((T,), -1, dtype=torch.int32, device=dev)
     n_exec = o.get("n_exec") if "n_exec" in o else torch.zeros(1, dtype=torch.int32, device=dev)
     cu_exec = o.get("cu_exec") if "cu_exec" in o else torch.zeros(B + 1, dtype=torch.int32, device=dev)
-    ws = o.get("ws") if "ws" in o else torch.zeros(256, dtype=torch.uint8, device=dev)
+    ws = o.get("ws") if "ws" in o else torch.empty(router_select_workspace_bytes(T), dtype=torch.uint8,
+                                                   device=dev)
     check(lib().qtale_router_select(
         _ptr(x), T, d, _ptr(w_router), float(bias), _ptr(scores_override), _ptr(valid),
         _ptr(cu_seqlens), B, _ptr(pos0), int(mode), float(theta), int(k), _ptr(scores), _ptr(idx),

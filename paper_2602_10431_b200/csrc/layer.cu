@@ -12,7 +12,8 @@ namespace qtale {
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 struct LayerWs {
-  unsigned char* ticket;
+  unsigned char* router_ws;  // scratch of the selection kernel
+  size_t router_ws_bytes;
   float* scores;
   int32_t* idx;
   int32_t* pos;
@@ -39,7 +40,8 @@ static LayerWs carve(const qtale_layer_config* c, int T, int B, void* base) {
   };
   const size_t t = (size_t)T;
   const int qd = c->n_heads * c->head_dim, kvd = c->n_kv_heads * c->head_dim;
-  w.ticket = take(256);
+  w.router_ws_bytes = qtale_router_select_workspace_bytes(T);
+  w.router_ws = take(w.router_ws_bytes);
   w.scores = reinterpret_cast<float*>(take(t * 4));
   w.idx = reinterpret_cast<int32_t*>(take(t * 4));
   w.pos = reinterpret_cast<int32_t*>(take(t * 4));
@@ -103,7 +105,7 @@ static int layer_forward_impl(const qtale_layer_config* c, const qtale_layer_wei
     QTALE_TRY(router_select_launch(x, T, d, w->router_w, w->router_b, scores_override, valid,
                                    cu_seqlens, B, pos0, c->select_mode, c->theta, k, ratio,
                                    scores_out ? scores_out : ws.scores, ws.idx, ws.n_exec,
-                                   ws.cu_exec, ws.pos, ws.ticket, 256, s));
+                                   ws.cu_exec, ws.pos, ws.router_ws, ws.router_ws_bytes, s));
   }
   if (n_exec_out &&
       cudaMemcpyAsync(n_exec_out, ws.n_exec, sizeof(int32_t), cudaMemcpyDeviceToDevice, s) !=

@@ -11,6 +11,23 @@ namespace qtale {
 
 constexpr int kRouterThreads = 512;  // 16 warps
 constexpr int kRowsPerWarp = 2;
+constexpr int kBins = 2048;          // first-level histogram of the top-k selection
+constexpr int kScoreSmem = 4096;     // a CTA keeps its tokens' scores in shared memory up to this many
+constexpr int kCandSmem = 1024;      // candidates ranked in shared memory (more: radix select by one CTA)
+constexpr int kMaxGrid = 1024;
+constexpr uint32_t kSpinLimit = 1u << 20;  // polls of a global word before a wait gives up
+
+// Scratch in the caller's workspace (32-bit words).  The first kZeroWords(grid) words are
+// cleared on the stream before every launch; the candidate list needs no clearing.
+constexpr int kWsBarrier = 0;      // grid barrier arrivals
+constexpr int kWsValid = 1;        // valid tokens of the call
+constexpr int kWsCand = 2;         // candidates appended so far
+constexpr int kWsCutKey = 3;       // cut-off of the top-k selection (published by CTA 0 when the
+constexpr int kWsCutTok = 4;       //   candidates do not fit shared memory)
+constexpr int kWsHist = 16;        // kBins counters
+constexpr int kWsCount = kWsHist + kBins;  // one word per CTA: executed tokens of its chunk | 2^31
+constexpr size_t kWsHeaderBytes = 16384;   // candidates (key, ~token) follow
+static_assert((kWsCount + kMaxGrid) * 4 <= (int)kWsHeaderBytes, "scratch header");
 
 struct RouterParams {
   const __nv_bfloat16* x;
@@ -24,9 +41,10 @@ struct RouterParams {
   int32_t* n_exec;
   int32_t* cu_exec;
   int32_t* pos;
-  unsigned int* ticket;
+  uint32_t* ws;
   int* status;
   int T, d, B, mode, k;  // k < 0 (top-k): k = floor(ratio * valid tokens + 0.5), counted here
+  int chunk;             // consecutive tokens per CTA
   double ratio;
   float bias, theta;
 };
@@ -35,315 +53,114 @@ __device__ __forceinline__ uint32_t score_key(float s) {
   uint32_t b = __float_as_uint(s);
   return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
 }
+// first-level bin of a score: uniform over [0, 1) (scores are probabilities), monotone for any input
+__device__ __forceinline__ int score_bin(float s) {
+  return s <= 0.f ? 0 : (s >= 1.f ? kBins - 1 : min(kBins - 1, (int)(s * (float)kBins)));
+}
+__device__ __forceinline__ uint32_t ld_acquire(const uint32_t* p) {
+  uint32_t v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_release(uint32_t* p, uint32_t v) {
+  asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
 
-// ---- phase B: decision + compaction, executed by one CTA ----------------------
-// Every sweep over the scores is warp-cooperative and coalesced: warp w owns the
-// contiguous token segment [w * seg, (w + 1) * seg) and walks it 32 tokens at a
-// time (token = segment start + 32 i + lane), so ballots give each selected
-// token its rank in token order.  When a lane's share is at most kKeep scores
-// they are read once and kept in registers for all sweeps.
-constexpr int kKeep = 16;
+// Barrier over the whole (co-resident) grid: arrival number `target` completes it.  Bounded.
+__device__ bool grid_barrier(const RouterParams& p, uint32_t target, int* s_abort) {
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    atomicAdd(p.ws + kWsBarrier, 1u);
+    uint32_t it = 0;
+    while (ld_acquire(p.ws + kWsBarrier) < target) {
+      if (++it > kSpinLimit) {
+        *s_abort = 1;
+        report_device_error(p.status, QTALE_ERR_TIMEOUT);
+        break;
+      }
+    }
+  }
+  __syncthreads();
+  return *s_abort == 0;
+}
 
-__device__ void select_and_compact(const RouterParams& p, uint32_t* sh_hist, int* sh_scan) {
-  const int tid = threadIdx.x;
-  const int nthr = blockDim.x;
+// inclusive prefix sum over the CTA's threads in thread order (s_w: one word per warp)
+__device__ __forceinline__ int block_inclusive_scan(int v, int* s_w, int& total) {
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  int inc = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int n = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += n;
+  }
+  __syncthreads();  // s_w may still be read from the previous use
+  if (lane == 31) s_w[wid] = inc;
+  __syncthreads();
+  int before = 0, tot = 0;
+  for (int w = 0; w < nw; ++w) {
+    const int c = s_w[w];
+    if (w < wid) before += c;
+    tot += c;
+  }
+  total = tot;
+  return inc + before;
+}
+
+// ---- the fused kernel -------------------------------------------------------
+// CTA c owns the consecutive tokens [c * chunk, (c + 1) * chunk).
+//   1. scores of its tokens (bandwidth-bound sweep of their rows of x, fp64 accumulation);
+//   2. top-k only: a histogram of all scores over kBins uniform bins is accumulated in global
+//      memory; after a grid barrier every CTA finds the bin holding the k-th largest score, the
+//      (few) tokens of that bin are appended to a candidate list, and after a second barrier
+//      every CTA ranks the candidates by (score descending, token ascending) to get the cut-off;
+//   3. each CTA counts its executed tokens, publishes the count, adds up the counts of the CTAs
+//      before it (they publish as soon as they know theirs) and writes its part of the ascending
+//      index list, the positions and the per-sequence offsets.
+// Launched cooperatively, so all CTAs are resident while they wait for each other.
+__global__ void __launch_bounds__(kRouterThreads, 2) router_select_kernel(const RouterParams p) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  __shared__ float s_sc[kScoreSmem];
+  __shared__ uint2 s_cand[kCandSmem];
+  __shared__ int s_w[32];
+  __shared__ uint32_t s_hist[256];
+  __shared__ int s_abort, s_bstar, s_rank, s_nvalid;
+  __shared__ uint32_t s_cut_key, s_cut_tok, s_prefix_hi, s_prefix_lo;
+
+  const int tid = threadIdx.x, nthr = blockDim.x;
   const int lane = tid & 31, wid = tid >> 5, nwarps = nthr >> 5;
-  const int T = p.T;
-  __shared__ uint32_t s_prefix, s_mask;
-  __shared__ int s_remaining, s_n_valid;
+  const int T = p.T, G = gridDim.x, cta = blockIdx.x;
+  const int c0 = min(T, cta * p.chunk), c1 = min(T, c0 + p.chunk);
+  const int n_own = c1 - c0;
+  const bool in_smem = p.chunk <= kScoreSmem;
+  if (tid == 0) s_abort = 0;
 
   // cu_seqlens must be 0 = cu[0] <= cu[1] <= ... <= cu[B] = T.  Anything else is reported in the
   // status word; tokens outside [cu[0], cu[B]) then never execute and every walk below stays
   // inside the B + 1 entries.
   const int t_begin = min(max(__ldg(p.cu_seqlens), 0), T);
   const int t_end = min(max(__ldg(p.cu_seqlens + p.B), t_begin), T);
-  {
+  if (cta == 0) {
     bool bad = tid == 0 && (__ldg(p.cu_seqlens) != 0 || __ldg(p.cu_seqlens + p.B) != T);
     for (int q = tid; q < p.B; q += nthr) bad |= __ldg(p.cu_seqlens + q) > __ldg(p.cu_seqlens + q + 1);
     if (bad) report_device_error(p.status, QTALE_ERR_SHAPE);
   }
 
-  const int seg = ((T + nwarps - 1) / nwarps + 31) & ~31;  // tokens per warp, multiple of 32
-  const int w0 = min(T, wid * seg), w1 = min(T, w0 + seg);
-  const int n_it = (w1 - w0 + 31) >> 5;                    // 32-token steps of this warp
-  const bool keep = seg <= 32 * kKeep;                     // uniform over the CTA
-
-  // score and validity of the token of step i (0 and false past the end)
-  auto load_one = [&](int i, float& sc, bool& ok) {
-    const int t = w0 + 32 * i + lane;
-    ok = t < w1 && t >= t_begin && t < t_end;
-    sc = 0.f;
-    if (ok) {
-      sc = __ldcg(p.scores + t);
-      if (p.valid) ok = p.valid[t] != 0;
-    }
-  };
-  float ksc[kKeep];
-  uint32_t kok = 0;  // bit i: token of step i is valid
-  if (keep) {
-#pragma unroll
-    for (int i = 0; i < kKeep; ++i) {
-      bool ok;
-      load_one(i, ksc[i], ok);
-      kok |= (ok ? 1u : 0u) << i;
-    }
-  }
-
-  uint32_t tau = 0;  // key of the k-th largest score (top-k)
-  int need_eq = 0;   // how many tokens with key == tau execute (lowest indices first)
-
-  int k_sel = p.k;
-  if (p.mode == QTALE_SELECT_TOPK && p.k < 0) {
-    // k for a requested ratio of the valid tokens (padding does not count)
-    if (tid == 0) s_n_valid = 0;
-    __syncthreads();
-    int nv = 0;
-    if (keep) {
-      nv = __popc(kok);
-    } else {
-      for (int i = 0; i < n_it; ++i) {
-        float sc;
-        bool ok;
-        load_one(i, sc, ok);
-        nv += ok ? 1 : 0;
-      }
-    }
-    nv = __reduce_add_sync(0xffffffffu, nv);
-    if (lane == 0) atomicAdd(&s_n_valid, nv);
-    __syncthreads();
-    const int n_valid = s_n_valid;
-    double kd = floor(p.ratio * (double)n_valid + 0.5);
-    kd = kd < 0.0 ? 0.0 : (kd > (double)n_valid ? (double)n_valid : kd);
-    k_sel = (int)kd;
-  }
-
-  if (p.mode == QTALE_SELECT_TOPK && k_sel > 0) {
-    // MSB-first radix select (four 8-bit digits) of the k-th largest key among valid tokens
-    if (tid == 0) {
-      s_prefix = 0;
-      s_mask = 0;
-      s_remaining = k_sel;
-    }
-    for (int pass = 0; pass < 4; ++pass) {
-      const int shift = 24 - 8 * pass;
-      for (int i = tid; i < 256; i += nthr) sh_hist[i] = 0;
-      __syncthreads();
-      const uint32_t prefix = s_prefix, mask = s_mask;
-      auto count_key = [&](float sc, bool ok) {
-        const uint32_t key = score_key(sc);
-        const bool in = ok && (key & mask) == prefix;
-        const uint32_t bucket = (key >> shift) & 0xFFu;
-        // scores cluster in few buckets of the leading digits: one atomic when the warp agrees
-        const uint32_t members = __ballot_sync(0xffffffffu, in);
-        if (members == 0) return;
-        const int first = __ffs(members) - 1;
-        const uint32_t b0 = __shfl_sync(0xffffffffu, bucket, first);
-        if (__all_sync(0xffffffffu, !in || bucket == b0)) {
-          if (lane == first) atomicAdd(&sh_hist[b0], (uint32_t)__popc(members));
-        } else if (in) {
-          atomicAdd(&sh_hist[bucket], 1u);
-        }
-      };
-      if (keep) {
-#pragma unroll
-        for (int i = 0; i < kKeep; ++i) count_key(ksc[i], (kok >> i) & 1u);
-      } else {
-        for (int i0 = 0; i0 < n_it; i0 += 8) {
-          float sc[8];
-          bool ok[8];
-#pragma unroll
-          for (int j = 0; j < 8; ++j) load_one(i0 + j, sc[j], ok[j]);
-#pragma unroll
-          for (int j = 0; j < 8; ++j) count_key(sc[j], ok[j]);
-        }
-      }
-      __syncthreads();
-      // bucket holding the target rank: warp 0 scans the 256 counts from the top, 8 per lane
-      if (wid == 0) {
-        int c[8], sum = 0;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          c[j] = (int)sh_hist[255 - (lane * 8 + j)];
-          sum += c[j];
-        }
-        int inc = sum;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-          const int n = __shfl_up_sync(0xffffffffu, inc, o);
-          if (lane >= o) inc += n;
-        }
-        const int rem = s_remaining;
-        int before = inc - sum;  // keys in buckets above this lane's eight
-        int found = -1, new_rem = 0;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          if (found < 0 && before + c[j] >= rem && before < rem) {
-            found = 255 - (lane * 8 + j);
-            new_rem = rem - before;
-          }
-          before += c[j];
-        }
-        const uint32_t owner = __ballot_sync(0xffffffffu, found >= 0);
-        if (owner == 0) {
-          // k exceeds the number of valid tokens: everything valid executes (lowest bucket)
-          if (lane == 0) {
-            s_prefix = prefix;
-            s_mask = mask | (0xFFu << shift);
-          }
-        } else if (lane == __ffs(owner) - 1) {
-          s_remaining = new_rem;  // rank of the target inside the bucket (1-based)
-          s_prefix = prefix | ((uint32_t)found << shift);
-          s_mask = mask | (0xFFu << shift);
-        }
-      }
-      __syncthreads();
-    }
-    tau = s_prefix;
-    need_eq = s_remaining;
-  }
-
-  const bool topk = p.mode == QTALE_SELECT_TOPK;
-  const bool none = topk && k_sel <= 0;
-  // (executes for sure, executes if among the first need_eq equal keys)
-  auto classify = [&](float sc, bool ok, bool& sure, bool& eq) {
-    if (topk) {
-      const uint32_t key = score_key(sc);
-      sure = ok && !none && key > tau;
-      eq = ok && !none && key == tau;
-    } else {
-      sure = ok && sc >= p.theta;
-      eq = false;
-    }
-  };
-
-  // sweep 1: executed tokens and tied tokens of each warp's segment
-  int n_sure = 0, n_eq = 0;
-  if (keep) {
-#pragma unroll
-    for (int i = 0; i < kKeep; ++i) {
-      bool sure, eq;
-      classify(ksc[i], (kok >> i) & 1u, sure, eq);
-      n_sure += __popc(__ballot_sync(0xffffffffu, sure));
-      n_eq += __popc(__ballot_sync(0xffffffffu, eq));
-    }
-  } else {
-    for (int i0 = 0; i0 < n_it; i0 += 8) {
-      float sc[8];
-      bool ok[8];
-#pragma unroll
-      for (int j = 0; j < 8; ++j) load_one(i0 + j, sc[j], ok[j]);
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        bool sure, eq;
-        classify(sc[j], ok[j], sure, eq);
-        n_sure += __popc(__ballot_sync(0xffffffffu, sure));
-        n_eq += __popc(__ballot_sync(0xffffffffu, eq));
-      }
-    }
-  }
-  // exclusive scans over the warps (at most 32 of them): sh_scan[0..31] sure, [32..63] tied
-  if (lane == 0) {
-    sh_scan[wid] = n_sure;
-    sh_scan[32 + wid] = n_eq;
-  }
-  __syncthreads();
-  int eq_before = 0, sure_before = 0, tot_eq = 0, tot_sure = 0;
-  for (int w = 0; w < nwarps; ++w) {
-    const int a = sh_scan[w], b = sh_scan[32 + w];
-    if (w < wid) {
-      sure_before += a;
-      eq_before += b;
-    }
-    tot_sure += a;
-    tot_eq += b;
-  }
-  const int total = tot_sure + min(tot_eq, need_eq);
-  int out = sure_before + min(eq_before, need_eq);
-
-  // sweep 2: ordered write of idx / pos, and cu_exec at every sequence start.
-  // b = sequence holding the lane's current token (largest b with cu_seqlens[b] <= t).
-  int b = 0;
-  {
-    const int t = min(w0 + lane, T - 1);
-    int lo = 0, hi = p.B;  // cu[lo] <= t < cu[hi]
-    while (hi - lo > 1) {
-      const int mid = (lo + hi) >> 1;
-      if (__ldg(p.cu_seqlens + mid) <= t) lo = mid; else hi = mid;
-    }
-    b = lo;
-  }
-  int seq_start = __ldg(p.cu_seqlens + b), seq_end = __ldg(p.cu_seqlens + b + 1);
-  const uint32_t lt = (1u << lane) - 1u;
-  auto emit = [&](int i, float sc, bool ok) {
-    const int t = w0 + 32 * i + lane;
-    bool sure, eq;
-    classify(sc, ok, sure, eq);
-    const uint32_t m_eq = __ballot_sync(0xffffffffu, eq);
-    const bool take = sure || (eq && eq_before + __popc(m_eq & lt) < need_eq);
-    const uint32_t m_take = __ballot_sync(0xffffffffu, take);
-    const int my_out = out + __popc(m_take & lt);
-    if (t < w1) {
-      while (t >= seq_end && b + 1 < p.B) {  // move to the sequence holding t (skips empty ones)
-        ++b;
-        seq_start = seq_end;
-        seq_end = __ldg(p.cu_seqlens + b + 1);
-      }
-      if (t == seq_start) {  // first token of sequence b and of the empty sequences before it
-        for (int q = b; q >= 0 && __ldg(p.cu_seqlens + q) == t; --q) p.cu_exec[q] = my_out;
-      }
-      if (take) {
-        p.idx[my_out] = t;
-        p.pos[my_out] = t - seq_start + (p.pos0 ? __ldg(p.pos0 + b) : 0);
-      }
-    }
-    out += __popc(m_take);
-    eq_before += __popc(m_eq);
-  };
-  if (keep) {
-#pragma unroll
-    for (int i = 0; i < kKeep; ++i) emit(i, ksc[i], (kok >> i) & 1u);
-  } else {
-    for (int i0 = 0; i0 < n_it; i0 += 8) {
-      float sc[8];
-      bool ok[8];
-#pragma unroll
-      for (int j = 0; j < 8; ++j) load_one(i0 + j, sc[j], ok[j]);
-#pragma unroll
-      for (int j = 0; j < 8; ++j) emit(i0 + j, sc[j], ok[j]);
-    }
-  }
-  if (tid == 0) *p.n_exec = total;
-  for (int qq = tid; qq <= p.B; qq += nthr)
-    if (p.cu_seqlens[qq] >= T) p.cu_exec[qq] = total;
-}
-
-// ---- the fused kernel -------------------------------------------------------
-__global__ void __launch_bounds__(kRouterThreads)
-    router_select_kernel(const RouterParams p) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  __shared__ uint32_t sh_hist[256];
-  __shared__ int sh_scan[64];
-  __shared__ int s_is_last;
-
-  const int tid = threadIdx.x;
+  // ---- 1. scores ----
   if (p.scores_override == nullptr) {
-    // phase A: router GEMV.  Router weights staged in shared memory as fp32, laid out
-    // [iteration][lane][8] so a lane's eight weights are two 16-byte loads.  Each 16-byte
-    // load of x (8 bf16) is reduced with fp32 FMAs into a block sum, and the block sums
-    // are accumulated in fp64: conversions and fp64 adds are one per 8 elements, which
-    // keeps the sweep bandwidth bound, and the result stays within about 1e-8 of the
-    // all-fp64 dot product.
+    // Router weights staged in shared memory as fp32, laid out [iteration][lane][8] so a lane's
+    // eight weights are two 16-byte loads.  Each 16-byte load of x (8 bf16) is reduced with fp32
+    // FMAs into a block sum, and the block sums are accumulated in fp64: conversions and fp64
+    // adds are one per 8 elements, which keeps the sweep bandwidth bound, and the result stays
+    // within about 1e-8 of the all-fp64 dot product.
     float* w_s = reinterpret_cast<float*>(smem_raw);
     const int d = p.d;
     const int n_it = (d + 255) / 256;
-    for (int i = tid; i < n_it * 256; i += blockDim.x) w_s[i] = (i < d) ? p.w[i] : 0.f;
+    for (int i = tid; i < n_it * 256; i += nthr) w_s[i] = (i < d) ? p.w[i] : 0.f;
     __syncthreads();
-    const int lane = tid & 31;
-    const int warp = tid >> 5;
-    const int warps_per_cta = blockDim.x >> 5;
-    const int n_groups = (p.T + kRowsPerWarp - 1) / kRowsPerWarp;
-    for (int g = blockIdx.x * warps_per_cta + warp; g < n_groups; g += gridDim.x * warps_per_cta) {
-      const int r0 = g * kRowsPerWarp;
+    const int n_groups = (n_own + kRowsPerWarp - 1) / kRowsPerWarp;
+    for (int g = wid; g < n_groups; g += nwarps) {
+      const int r0 = c0 + g * kRowsPerWarp;
       double acc[kRowsPerWarp];
 #pragma unroll
       for (int r = 0; r < kRowsPerWarp; ++r) acc[r] = 0.0;
@@ -355,7 +172,7 @@ __global__ void __launch_bounds__(kRouterThreads)
           const int col = (it0 + u) * 256 + lane * 8;
 #pragma unroll
           for (int r = 0; r < kRowsPerWarp; ++r) {
-            const int row = min(r0 + r, p.T - 1);
+            const int row = min(r0 + r, c1 - 1);
             v[u][r] = (it0 + u < n_it && col < d) ? ld_nc_16(p.x + (size_t)row * d + col)
                                                   : make_uint4(0, 0, 0, 0);
           }
@@ -382,26 +199,236 @@ __global__ void __launch_bounds__(kRouterThreads)
 #pragma unroll
       for (int r = 0; r < kRowsPerWarp; ++r) {
         const double z = warp_sum(acc[r]) + (double)p.bias;
-        if (lane == 0 && r0 + r < p.T) p.scores[r0 + r] = (float)(1.0 / (1.0 + exp(-z)));
+        if (lane == 0 && r0 + r < c1) {
+          const float sc = (float)(1.0 / (1.0 + exp(-z)));
+          p.scores[r0 + r] = sc;
+          if (in_smem) s_sc[r0 + r - c0] = sc;
+        }
       }
     }
   } else {
-    for (int t = blockIdx.x * blockDim.x + tid; t < p.T; t += gridDim.x * blockDim.x)
-      p.scores[t] = p.scores_override[t];
+    for (int i = tid; i < n_own; i += nthr) {
+      const float sc = p.scores_override[c0 + i];
+      p.scores[c0 + i] = sc;
+      if (in_smem) s_sc[i] = sc;
+    }
+  }
+  __syncthreads();  // the CTA's scores are in shared memory (or, for huge chunks, in p.scores)
+
+  auto score_at = [&](int i) { return in_smem ? s_sc[i] : p.scores[c0 + i]; };
+  auto ok_at = [&](int i) {
+    const int t = c0 + i;
+    return i < n_own && t >= t_begin && t < t_end && (p.valid == nullptr || p.valid[t] != 0);
+  };
+  const int n_slab = (n_own + nthr - 1) / nthr;
+
+  // ---- 2. top-k: cut-off = k-th largest (score, lower token first) among the valid tokens ----
+  const bool topk = p.mode == QTALE_SELECT_TOPK;
+  bool none = false;                        // top-k with k = 0 (or no valid token)
+  int bstar = 0;                            // bin of the k-th score
+  uint64_t cut = 0;                         // (key << 32 | ~token) of the k-th token
+  if (topk) {
+    uint32_t step = 0;  // grid barriers passed
+    int nv = 0;
+    for (int sl = 0; sl < n_slab; ++sl) {
+      const int i = sl * nthr + tid;
+      if (ok_at(i)) {
+        ++nv;
+        atomicAdd(p.ws + kWsHist + score_bin(score_at(i)), 1u);
+      }
+    }
+    nv = __reduce_add_sync(0xffffffffu, nv);
+    if (lane == 0 && nv) atomicAdd(p.ws + kWsValid, (uint32_t)nv);
+    if (!grid_barrier(p, ++step * G, &s_abort)) return;
+
+    const int n_valid = (int)__ldcg(p.ws + kWsValid);
+    int k = p.k;
+    if (k < 0) {  // k for a requested ratio of the valid tokens (padding does not count)
+      double kd = floor(p.ratio * (double)n_valid + 0.5);
+      k = kd < 0.0 ? 0 : (kd > (double)n_valid ? n_valid : (int)kd);
+    }
+    k = min(k, n_valid);
+    none = k <= 0;
+    if (!none) {
+      // thread j reads bins from the top: tid 0 owns the four highest.  With `above` = valid
+      // tokens in higher bins, the k-th sits in the bin where above < k <= above + count.
+      constexpr int PER = kBins / kRouterThreads;
+      const int hi_bin = kBins - 1 - tid * PER;
+      uint32_t h[PER];
+      int v = 0;
+#pragma unroll
+      for (int e = 0; e < PER; ++e) {
+        h[e] = __ldcg(p.ws + kWsHist + hi_bin - e);
+        v += (int)h[e];
+      }
+      int total;
+      int above = block_inclusive_scan(v, s_w, total) - v;
+#pragma unroll
+      for (int e = 0; e < PER; ++e) {
+        if (above < k && k <= above + (int)h[e]) {
+          s_bstar = hi_bin - e;
+          s_rank = k - above;       // 1-based rank of the k-th inside its bin
+          s_nvalid = (int)h[e];     // tokens in that bin
+        }
+        above += (int)h[e];
+      }
+      __syncthreads();
+      bstar = s_bstar;
+      const int r = s_rank, c = s_nvalid;
+      uint2* cand = reinterpret_cast<uint2*>(reinterpret_cast<unsigned char*>(p.ws) + kWsHeaderBytes);
+      for (int sl = 0; sl < n_slab; ++sl) {
+        const int i = sl * nthr + tid;
+        if (ok_at(i)) {
+          const float sc = score_at(i);
+          if (score_bin(sc) == bstar) {
+            const uint32_t slot = atomicAdd(p.ws + kWsCand, 1u);
+            if (slot < (uint32_t)T) cand[slot] = make_uint2(score_key(sc), ~(uint32_t)(c0 + i));
+          }
+        }
+      }
+      if (!grid_barrier(p, ++step * G, &s_abort)) return;
+      if (c <= kCandSmem) {
+        // every CTA ranks the candidates itself: the r-th in the order is the cut-off
+        for (int i = tid; i < c; i += nthr) s_cand[i] = __ldcg(cand + i);
+        __syncthreads();
+        for (int i = tid; i < c; i += nthr) {
+          const uint64_t me = ((uint64_t)s_cand[i].x << 32) | s_cand[i].y;
+          int before = 0;
+          for (int j = 0; j < c; ++j)
+            before += ((((uint64_t)s_cand[j].x << 32) | s_cand[j].y) > me) ? 1 : 0;
+          if (before == r - 1) {
+            s_cut_key = s_cand[i].x;
+            s_cut_tok = s_cand[i].y;
+          }
+        }
+        __syncthreads();
+      } else {
+        // many equal or close scores: CTA 0 finds the r-th largest 64-bit (key, ~token) by an
+        // MSB-first radix select over the list in global memory and publishes it
+        if (cta == 0) {
+          if (tid == 0) {
+            s_prefix_hi = 0;
+            s_prefix_lo = 0;
+            s_rank = r;
+          }
+          for (int pass = 0; pass < 8; ++pass) {
+            const int shift = 56 - 8 * pass;
+            for (int i = tid; i < 256; i += nthr) s_hist[i] = 0;
+            __syncthreads();
+            const uint64_t prefix = ((uint64_t)s_prefix_hi << 32) | s_prefix_lo;
+            const uint64_t mask = pass == 0 ? 0ull : ~0ull << (shift + 8);
+            for (int i = tid; i < c; i += nthr) {
+              const uint2 e = __ldcg(cand + i);
+              const uint64_t v64 = ((uint64_t)e.x << 32) | e.y;
+              if ((v64 & mask) == prefix) atomicAdd(&s_hist[(uint32_t)(v64 >> shift) & 0xFFu], 1u);
+            }
+            __syncthreads();
+            if (tid == 0) {
+              int rem = s_rank, digit = 0;
+              for (int b = 255; b >= 0; --b) {
+                const int cnt = (int)s_hist[b];
+                if (rem <= cnt) { digit = b; break; }
+                rem -= cnt;
+              }
+              const uint64_t np = prefix | ((uint64_t)digit << shift);
+              s_prefix_hi = (uint32_t)(np >> 32);
+              s_prefix_lo = (uint32_t)np;
+              s_rank = rem;
+            }
+            __syncthreads();
+          }
+          if (tid == 0) {
+            p.ws[kWsCutKey] = s_prefix_hi;
+            p.ws[kWsCutTok] = s_prefix_lo;
+          }
+        }
+        if (!grid_barrier(p, ++step * G, &s_abort)) return;
+        if (tid == 0) {
+          s_cut_key = __ldcg(p.ws + kWsCutKey);
+          s_cut_tok = __ldcg(p.ws + kWsCutTok);
+        }
+        __syncthreads();
+      }
+      cut = ((uint64_t)s_cut_key << 32) | s_cut_tok;
+    }
   }
 
-  // ticket: the CTA that arrives last runs the selection
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) {
-    const unsigned int t = atomicAdd(p.ticket, 1u);
-    s_is_last = (t == gridDim.x - 1);
+  // execute / bypass decision of the CTA's token i
+  auto decide = [&](int i) {
+    if (!ok_at(i)) return false;
+    const float sc = score_at(i);
+    if (!topk) return sc >= p.theta;
+    if (none) return false;
+    const int b = score_bin(sc);
+    if (b != bstar) return b > bstar;
+    return (((uint64_t)score_key(sc) << 32) | ~(uint32_t)(c0 + i)) >= cut;
+  };
+
+  // ---- 3. ordered compaction ----
+  int own = 0;
+  for (int sl = 0; sl < n_slab; ++sl) own += __syncthreads_count(decide(sl * nthr + tid) ? 1 : 0);
+  if (tid == 0) st_release(p.ws + kWsCount + cta, (uint32_t)own | 0x80000000u);
+  // executed tokens of the CTAs before this one
+  int before = 0;
+  for (int j = tid; j < cta; j += nthr) {
+    uint32_t v, it = 0;
+    while (((v = ld_acquire(p.ws + kWsCount + j)) & 0x80000000u) == 0) {
+      if (++it > kSpinLimit) {
+        s_abort = 1;
+        report_device_error(p.status, QTALE_ERR_TIMEOUT);
+        break;
+      }
+    }
+    before += (int)(v & 0x7FFFFFFFu);
+  }
+  {
+    int total;
+    block_inclusive_scan(before, s_w, total);
+    before = total;
   }
   __syncthreads();
-  if (!s_is_last) return;
-  __threadfence();
-  select_and_compact(p, sh_hist, sh_scan);
-  if (tid == 0) *p.ticket = 0;  // leave the counter ready for the next launch
+  if (s_abort) return;
+
+  const uint32_t lt = (1u << lane) - 1u;
+  int run = before;  // executed tokens before the current slab
+  for (int sl = 0; sl < n_slab; ++sl) {
+    const int i = sl * nthr + tid;
+    const int t = c0 + i;
+    const bool take = decide(i);
+    const uint32_t m_take = __ballot_sync(0xffffffffu, take);
+    __syncthreads();
+    if (lane == 0) s_w[wid] = __popc(m_take);
+    __syncthreads();
+    int wbase = 0, slab_total = 0;
+    for (int w = 0; w < nwarps; ++w) {
+      const int c = s_w[w];
+      if (w < wid) wbase += c;
+      slab_total += c;
+    }
+    const int my_out = run + wbase + __popc(m_take & lt);  // executed tokens before token t
+    if (i < n_own) {
+      // b = sequence holding t (largest b with cu_seqlens[b] <= t)
+      int lo = 0, hi = p.B;
+      while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (__ldg(p.cu_seqlens + mid) <= t) lo = mid; else hi = mid;
+      }
+      const int seq_start = __ldg(p.cu_seqlens + lo);
+      if (t == seq_start) {  // first token of sequence lo and of the empty sequences before it
+        for (int q = lo; q >= 0 && __ldg(p.cu_seqlens + q) == t; --q) p.cu_exec[q] = my_out;
+      }
+      if (take) {
+        p.idx[my_out] = t;
+        p.pos[my_out] = t - seq_start + (p.pos0 ? __ldg(p.pos0 + lo) : 0);
+      }
+    }
+    run += slab_total;
+  }
+  if (cta == G - 1) {
+    if (tid == 0) *p.n_exec = run;
+    for (int q = tid; q <= p.B; q += nthr)
+      if (__ldg(p.cu_seqlens + q) >= T) p.cu_exec[q] = run;
+  }
 }
 
 // ---- bookkeeping for a caller-supplied index list ----------------------------
@@ -438,8 +465,9 @@ using namespace qtale;
 extern "C" {
 
 size_t qtale_router_select_workspace_bytes(int T) {
-  (void)T;
-  return 256;  // ticket counter (kept zero between launches)
+  // counters, histogram and per-CTA counts, then one (key, token) pair per token for the
+  // candidates of the top-k selection (all of them when every score is the same)
+  return kWsHeaderBytes + (size_t)(T > 0 ? T : 0) * 8;
 }
 
 int qtale_router_select(const void* x, int T, int d, const float* w_router, float bias,
@@ -485,38 +513,47 @@ int router_select_launch(const void* x, int T, int d, const float* w_router, flo
   p.n_exec = n_exec_out;
   p.cu_exec = cu_exec_out;
   p.pos = pos_out;
-  p.ticket = static_cast<unsigned int*>(ws);
+  p.ws = static_cast<uint32_t*>(ws);
   p.status = device_status_ptr();
   p.T = T; p.d = d; p.B = B; p.mode = mode;
   p.k = (mode == QTALE_SELECT_TOPK && ratio >= 0.0) ? -1 : k;
   p.ratio = ratio;
   p.bias = bias; p.theta = theta;
 
-  if (cudaMemsetAsync(ws, 0, sizeof(unsigned int), s) != cudaSuccess) return QTALE_ERR_CUDA;
-  int grid;
-  size_t smem = 0;
-  if (scores_override) {
-    // copy of the supplied scores: enough CTAs that each thread moves a few elements
-    grid = (T + kRouterThreads * 4 - 1) / (kRouterThreads * 4);
-    if (grid > sm_count()) grid = sm_count();
-    if (grid < 1) grid = 1;
-  } else {
-    const int n_it = (d + 255) / 256;
-    smem = (size_t)n_it * 256 * sizeof(float);
-    const int warps = kRouterThreads / 32;
-    const int n_groups = (T + kRowsPerWarp - 1) / kRowsPerWarp;
-    grid = (n_groups + warps - 1) / warps;
-    const int cap = sm_count() * 2;
-    if (grid > cap) grid = cap;
-    if (grid < 1) grid = 1;
-    if (smem > 48 * 1024) {
-      if (cudaFuncSetAttribute(router_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                               (int)smem) != cudaSuccess)
-        return QTALE_ERR_CUDA;
-    }
+  const size_t smem = scores_override ? 0 : (size_t)((d + 255) / 256) * 256 * sizeof(float);
+  // The CTAs wait for each other, so the grid must fit the device at once: at most what the
+  // occupancy calculator allows, at least 32 tokens per CTA (two per warp), an even chunk.
+  static int cached_dev = -1, cached_per_sm = 0;
+  static size_t cached_smem = 0;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return QTALE_ERR_CUDA;
+  if (dev != cached_dev || smem != cached_smem) {
+    if (smem > 20 * 1024 &&  // static + dynamic shared memory beyond the default 48 KB
+        cudaFuncSetAttribute(router_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)smem) != cudaSuccess)
+      return QTALE_ERR_CUDA;
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, router_select_kernel, kRouterThreads,
+                                                      smem) != cudaSuccess || per_sm < 1)
+      return QTALE_ERR_CUDA;
+    cached_per_sm = per_sm > 2 ? 2 : per_sm;
+    cached_dev = dev;
+    cached_smem = smem;
   }
-  router_select_kernel<<<grid, kRouterThreads, smem, s>>>(p);
-  return launch_status(cudaGetLastError());
+  int grid = sm_count() * cached_per_sm;
+  if (grid > kMaxGrid) grid = kMaxGrid;
+  const int want = (T + 31) / 32;
+  if (grid > want) grid = want;
+  int chunk = (T + grid - 1) / grid;
+  chunk = (chunk + 1) & ~1;
+  grid = (T + chunk - 1) / chunk;
+  p.chunk = chunk;
+
+  if (cudaMemsetAsync(ws, 0, (size_t)(kWsCount + grid) * sizeof(uint32_t), s) != cudaSuccess)
+    return QTALE_ERR_CUDA;
+  void* args[] = {&p};
+  return launch_status(cudaLaunchCooperativeKernel(router_select_kernel, dim3(grid),
+                                                   dim3(kRouterThreads), args, smem, s));
 }
 
 }  // namespace qtale
@@ -524,9 +561,12 @@ int router_select_launch(const void* x, int T, int d, const float* w_router, flo
 extern "C" {
 
 // ---- variant for callers that cannot allocate device memory -------------------
-// The kernel's only scratch is its ticket counter; here it lives in a static
-// device array that every GPU loading the library carries until exit.
-#define QTALE_ROUTER_STATIC_SCRATCH_BYTES 256
+// The kernel's scratch (counters, histogram, per-CTA counts and the candidate list of the
+// top-k selection) lives in a static device array, sized for QTALE_ROUTER_STATIC_MAX_TOKENS
+// tokens, that every GPU loading the library carries until exit.
+#define QTALE_ROUTER_STATIC_SCRATCH_BYTES (16384 + 8 * QTALE_ROUTER_STATIC_MAX_TOKENS)
+static_assert(QTALE_ROUTER_STATIC_SCRATCH_BYTES >= kWsHeaderBytes + 8 * (size_t)QTALE_ROUTER_STATIC_MAX_TOKENS,
+              "static scratch must cover the workspace of the largest accepted call");
 static __device__ __align__(256) unsigned char g_router_static_scratch[QTALE_ROUTER_STATIC_SCRATCH_BYTES];
 
 int qtale_router_select_static(const void* x, int T, int d, const float* w_router, float bias,
@@ -548,8 +588,8 @@ int qtale_router_select_static(const void* x, int T, int d, const float* w_route
       return QTALE_ERR_CUDA;
     scratch_of_device[dev] = ptr;
   }
-  // The shared entry point zeroes the ticket word (cudaMemsetAsync on the stream)
-  // before the launch, so whatever the previous call left behind does not matter.
+  // The shared entry point clears the counters (cudaMemsetAsync on the stream) before
+  // the launch, so whatever the previous call left behind does not matter.
   return qtale_router_select(x, T, d, w_router, bias, scores_override, valid, cu_seqlens, B, pos0,
                              mode, theta, k, scores_out, idx_out, n_exec_out, cu_exec_out, pos_out,
                              scratch_of_device[dev], QTALE_ROUTER_STATIC_SCRATCH_BYTES, stream);

@@ -83,6 +83,56 @@ def test_router_select_padding_override_ties_pos0(env):
         _check_select(api, torch, r, p, oracle.select_topk(p, k, valid), cu, pos0)
 
 
+def _select_case(api, torch, dev, p, cu, mode, k=0, theta=0.5, valid=None):
+    pd = torch.from_numpy(p).to(dev)
+    vd = None if valid is None else torch.from_numpy(valid).to(dev)
+    r = api.router_select(None, None, 0.0, torch.from_numpy(cu).to(dev), mode, theta=theta, k=k,
+                          scores_override=pd, valid=vd)
+    m = oracle.select_topk(p, k, valid) if mode == api.SELECT_TOPK else oracle.select_threshold(p, theta, valid)
+    _check_select(api, torch, r, p, m, cu, threshold=None if mode == api.SELECT_TOPK else theta)
+    return int(r["n_exec"].item())
+
+
+def test_topk_selection_with_many_equal_scores(env):
+    """Equal scores are ordered by token index.  All scores equal, or a block of more equal
+    scores than the in-kernel candidate buffer holds (1024), takes the radix-select path of
+    the cut-off; a few equal scores take the ranking path; both across several CTAs."""
+    api, torch, dev = env
+    T = 5000
+    cu = np.array([0, 1200, 1200, 3100, 5000], np.int32)
+    same = np.full(T, 0.625, np.float32)
+    for k in [1, 1234, 4999, 5000]:
+        assert _select_case(api, torch, dev, same, cu, api.SELECT_TOPK, k=k) == k
+    p = inputs.beta22(41, 1, T).astype(np.float32)
+    p[700:2900] = p[10]                                         # 2200 equal scores in the middle
+    valid = (inputs.uniform(41, 2, T) > 0.1).astype(np.uint8)
+    above = int(((p > p[10]) & (valid == 1)).sum())
+    for k in [above, above + 1, above + 1500, above + int(((p == p[10]) & (valid == 1)).sum()), above + 2300]:
+        _select_case(api, torch, dev, p, cu, api.SELECT_TOPK, k=k, valid=valid)
+    p = inputs.beta22(41, 3, T).astype(np.float32)
+    p[::7] = p[3]                                               # 715 equal scores, interleaved
+    for k in [int((p > p[3]).sum()) + 100, 2500]:
+        _select_case(api, torch, dev, p, cu, api.SELECT_TOPK, k=k)
+    # scores outside [0, 1) fall into the end bins of the histogram and are still ordered exactly
+    p = (inputs.normal(41, 4, T) * 2).astype(np.float32)
+    for k in [17, 2500, 4000]:
+        _select_case(api, torch, dev, p, cu, api.SELECT_TOPK, k=k)
+
+
+@pytest.mark.parametrize("T,B", [(65536, 16), (200000, 5), (1300000, 3)])
+def test_selection_at_scale(env, T, B):
+    """65536 tokens in 16 sequences with Beta(2,2) scores is the 13B-shaped stack's selection
+    (threshold from the closed-form quantile and top-k at ratio 0.7); the larger cases give a CTA
+    more tokens than threads, and more than it keeps in shared memory."""
+    api, torch, dev = env
+    p = inputs.beta22(43, 1, T).astype(np.float32)
+    cu = (np.arange(B + 1, dtype=np.int64) * T // B).astype(np.int32)
+    n = _select_case(api, torch, dev, p, cu, api.SELECT_THRESHOLD, theta=0.3)
+    assert abs(n / T - (1 - (3 * 0.3 ** 2 - 2 * 0.3 ** 3))) < 0.01   # Beta(2,2) tail above 0.3
+    k = api.topk_count(0.7, T) if T == 65536 else 500
+    assert _select_case(api, torch, dev, p, cu, api.SELECT_TOPK, k=k) == k
+
+
 def test_inconsistent_cu_seqlens_is_reported_not_followed(env):
     """cu_seqlens lives on the device, so the kernel checks it: offsets that do not end at T
     (or are not ascending) give QTALE_ERR_SHAPE in the status word, tokens outside
