@@ -1,13 +1,24 @@
 #!/usr/bin/env python
 """Benchmark of the token-adaptive quantised layer forward on B200.
 
-One step = one pass of the whole layer path (router + selection + compaction,
-gather + RMSNorm, four quantised GEMMs, rotary, attention over executed tokens,
-residual scatter) over one batch of synthetic Llama-2-7B-shaped input: hidden
-4096, 32 heads, FFN 11008, int4 group-128 weights, batch 4 x 2048 tokens,
-top-k selection at the requested execution ratio.  Prints ONE JSON line.
+Headline: one step = one pass of the whole layer path (router + selection +
+compaction, gather + RMSNorm, four quantised GEMMs, rotary, attention over
+executed tokens, residual scatter) over one batch of synthetic
+Llama-2-7B-shaped input: hidden 4096, 32 heads, FFN 11008, int4 group-128
+weights, batch 4 x 2048 tokens, top-k selection at the requested execution
+ratio.  Further legs time, through the same C ABI, the memory-bound stages
+(router + selection, gather + RMSNorm), the decode step, the 8B-shaped model
+prefill and the 13B-shaped irregular stack, each against its own roofline.
+Prints ONE JSON line.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--ratio R] [--impl reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--ratio R] [--legs a,b,...]
+                  [--impl reference]
+
+Timing: a region is exactly K steps between two CUDA events on the launching
+stream, bracketed by a barrier and a device synchronise; regions are repeated
+back to back until --min-seconds of GPU time have passed, `ms_per_step` is the
+median region (the power-capped, sustained figure), `burst` the first region
+after an idle second.  Clocks are sampled with nvidia-smi during the regions.
 """
 from __future__ import annotations
 
@@ -26,17 +37,17 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-from paper_2602_10431_b200 import inputs  # noqa: E402
+from paper_2602_10431_b200 import accounting, inputs  # noqa: E402
 
 METRIC = "tokens/s per token-adaptive int4 layer (7B-shaped, prefill 4x2048) at execution ratio"
 UNIT = "tokens/s"
 SWEEP = [1.0, 0.9, 0.75, 0.5]
 WORKLOAD = ("c2: 7B-shaped layer (hidden 4096, 32 heads, FFN 11008), int4 g128, "
             "batch 4 x seq 2048 prefill")
-# DRAM traffic of the four GEMM launches of one step at ratio 0.5 (4096 executed tokens), from
-# one ncu capture of the kernel as it stands; None at other ratios.
-GEMM_DRAM_BYTES = 716259840
-KERNELS_PER_STEP = 11  # router, gather+norm, 4 GEMMs, rotary table, rotary, tail zeroing, attention, RMSNorm
+# kernels of this library per layer step (prefill): router/select, gather + norm, QKV GEMM,
+# rotary table, rotary, tail zeroing, attention, O GEMM, RMSNorm, gate/up GEMM, down GEMM
+KERNELS_PER_STEP = 11
+ALL_LEGS = ["sweep", "gemm", "bf16", "router", "gather", "decode", "c4", "c5", "e2e", "cpu"]
 
 
 def measured_peaks():
@@ -51,17 +62,18 @@ def measured_peaks():
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    """One nvidia-smi process sampling clocks and throttle reasons for the whole run; every
+    timed leg asks for the samples that arrived inside its own regions."""
 
     FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
               "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    NAMES = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
 
     def __init__(self, gpu_index: int):
         self.gpu = gpu_index
         self.proc = None
-        self.lines = []      # (arrival time, csv line)
-        self.window = None   # (start, end) of the timed region, host clock
+        self.lines = []  # (arrival time, csv line)
 
     def start(self):
         try:
@@ -79,19 +91,22 @@ class ClockSampler:
 
     def stop(self):
         if self.proc is None:
-            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
-        time.sleep(0.15)
+            return
         self.proc.terminate()
         try:
             self.proc.wait(timeout=2)
         except subprocess.TimeoutExpired:
             self.proc.kill()
+
+    def summary(self, windows):
+        """Clocks over the samples that fall inside `windows` (list of (t0, t1) host times).
+        Samples outside the timed regions are never used: with too few inside, the summary
+        says so instead of describing the idle GPU."""
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        time.sleep(0.05)
+        inside = [ln for (t, ln) in list(self.lines) if any(a <= t <= b + 0.01 for a, b in windows)]
         sm, mx, power, reasons = [], [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        inside = [ln for (t, ln) in self.lines
-                  if self.window is None or self.window[0] <= t <= self.window[1] + 0.02]
-        if len(inside) < 3:  # region shorter than a few sampling periods: keep every sample
-            inside = [ln for (_, ln) in self.lines]
         for ln in inside:
             f = [c.strip() for c in ln.split(",")]
             if len(f) < 9:
@@ -102,13 +117,23 @@ class ClockSampler:
                 power.append(float(f[3]))
             except ValueError:
                 continue
-            for name, val in zip(names, f[5:9]):
+            for name, val in zip(self.NAMES, f[5:9]):
                 if val.lower().startswith("active"):
                     reasons.add(name)
-        if not sm:
-            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["no samples"])
-        return dict(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons),
-                    samples=len(sm), power_w_max=max(power) if power else None)
+        any_mx = None
+        for _, ln in list(self.lines)[:3]:
+            f = [c.strip() for c in ln.split(",")]
+            if len(f) >= 3:
+                try:
+                    any_mx = float(f[2])
+                except ValueError:
+                    pass
+        if len(sm) < 3:
+            return dict(sm_mhz=None, sm_max_mhz=any_mx, reasons=[], samples=len(sm),
+                        note="timed regions shorter than three sampling periods: no clock figure")
+        return dict(sm_mhz=statistics.median(sm), sm_min_mhz=min(sm), sm_max_mhz=max(mx),
+                    reasons=sorted(reasons), samples=len(sm), power_w_median=statistics.median(power),
+                    power_w_max=max(power))
 
 
 def max_over_ranks(ms: float, device=None) -> float:
@@ -126,6 +151,20 @@ def max_over_ranks(ms: float, device=None) -> float:
 def aggregate_tokens_per_s(tokens_per_rank: int, world: int, ms_per_step: float) -> float:
     """Whole-job throughput of `world` replicas that each process tokens_per_rank per step."""
     return world * tokens_per_rank / (ms_per_step * 1e-3)
+
+
+def replica_command(n_gpus: int, script: str, script_args, port: int):
+    """Command line that runs `script` as n_gpus independent replicas of one node, one process
+    per GPU (the path has no exchange step; the ranks only meet in the timing barrier)."""
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1",
+            "--nproc-per-node", str(n_gpus), "--master-addr", "127.0.0.1",
+            "--master-port", str(port), script] + list(script_args)
+
+
+def spawn_replicas(n_gpus: int, script: str, script_args, port=None) -> int:
+    """`bench.py --gpus N` started as a plain process: re-launch under torchrun."""
+    port = port or 29500 + os.getpid() % 2000
+    return subprocess.call(replica_command(n_gpus, script, script_args, port))
 
 
 def build_layer_inputs(seed, cfg_name):
@@ -192,6 +231,119 @@ def run_reference(args):
 # our arm
 # ------------------------------------------------------------------------------------
 
+class Timer:
+    """Timed regions of exactly `steps` calls each, repeated until `min_seconds` of device time."""
+
+    def __init__(self, torch, dist, world, dev, sampler):
+        self.torch, self.dist, self.world, self.dev, self.sampler = torch, dist, world, dev, sampler
+
+    def barrier(self):
+        if self.world > 1:
+            self.dist.barrier()
+        self.torch.cuda.synchronize()
+
+    def region(self, fn, steps, windows):
+        torch = self.torch
+        self.barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0 = time.time()
+        e0.record()
+        for i in range(steps):
+            fn(i)
+        e1.record()
+        self.barrier()
+        windows.append((t0, time.time()))
+        return max_over_ranks(e0.elapsed_time(e1), self.dev if self.world > 1 else None)
+
+    def run(self, fn, steps, warmup, min_seconds=1.0, between=None, max_regions=200, idle=False):
+        """Returns dict(ms, burst_ms, regions, clocks): ms = median region / steps."""
+        for i in range(warmup):
+            fn(i)
+        if between is not None:
+            between()
+        if idle:
+            self.barrier()
+            time.sleep(1.0)  # let the chip cool, so that the first region is a burst figure
+        windows, times = [], []
+        total = 0.0
+        while True:
+            ms = self.region(fn, steps, windows)
+            times.append(ms)
+            total += ms
+            # every rank takes the same decision: `total` is a max over ranks already
+            if total >= min_seconds * 1e3 or len(times) >= max_regions:
+                break
+            if between is not None:
+                between()
+        med = statistics.median(times)
+        clocks = self.sampler.summary(windows) if self.sampler is not None else None
+        out = dict(ms=med / steps, burst_ms=times[0] / steps, min_ms=min(times) / steps,
+                   regions=len(times), steps_per_region=steps, clocks=clocks)
+        if clocks and clocks.get("sm_mhz"):
+            out["ms_x_ghz"] = med / steps * clocks["sm_mhz"] / 1e3
+        return out
+
+
+def graph_of(torch, fn, n=1):
+    """CUDA graph of n calls (short kernels are otherwise timed at the host's launch rate)."""
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(g, stream=side):
+            for _ in range(n):
+                fn()
+    torch.cuda.current_stream().wait_stream(side)
+    return g
+
+
+def timing_weight(torch, api, dev, gen, N, K, bits, group, row_mode=0):
+    """Quantised linear for timing legs: random codes written straight into the kernel-native
+    blob on the device (seeded), every group with scale 0.0027 and zero-point 2^(bits-1), i.e.
+    weights spread over about +-0.02.  Generating and quantising Gaussian weights on the host
+    takes half a minute per 7B-sized layer; the kernels' timing does not depend on the values."""
+    import ctypes as C
+    nbytes = C.c_size_t(0)
+    api.check(api.lib().qtale_wq_repack(None, None, None, N, K, bits, group, row_mode, None,
+                                        C.byref(nbytes)), "qtale_wq_repack(size)")
+    block = 128 * 64 * bits // 8
+    tile = block + 512
+    blob = torch.randint(0, 256, (nbytes.value // tile, tile), dtype=torch.uint8, device=dev, generator=gen)
+    sz = np.array([np.float16(0.0027), np.float16(1 << (bits - 1))], np.float16).view(np.uint8)
+    blob[:, block:] = torch.from_numpy(np.tile(sz, 128)).to(dev)
+    q = api.QuantWeight.__new__(api.QuantWeight)
+    q.blob = blob.reshape(-1)
+    q.N, q.K, q.bits, q.group, q.row_mode = N, K, bits, group, row_mode
+    q.c = api.WqWeight(q.blob.data_ptr(), N, K, bits, group, row_mode)
+    return q
+
+
+def timing_layer(torch, api, dev, gen, sh):
+    """api.LayerWeights with timing weights (see timing_weight) and a random router."""
+    lw = api.LayerWeights.__new__(api.LayerWeights)
+    lw.qkv = timing_weight(torch, api, dev, gen, sh.q_dim + 2 * sh.kv_dim, sh.d, sh.bits, sh.group)
+    lw.o = timing_weight(torch, api, dev, gen, sh.d, sh.q_dim, sh.bits, sh.group)
+    lw.gate_up = timing_weight(torch, api, dev, gen, 2 * sh.ffn, sh.d, sh.bits, sh.group, api.ROWS_SWIGLU)
+    lw.down = timing_weight(torch, api, dev, gen, sh.d, sh.ffn, sh.bits, sh.group)
+    lw.gamma1 = torch.ones(sh.d, dtype=torch.float32, device=dev)
+    lw.gamma2 = torch.ones(sh.d, dtype=torch.float32, device=dev)
+    lw.router_w = (torch.randn(sh.d, device=dev, generator=gen) * 0.02).to(torch.bfloat16).float()
+    lw.router_b = 0.0
+    lw.c = api.LayerWeightsC(lw.qkv.c, lw.o.c, lw.gate_up.c, lw.down.c, lw.gamma1.data_ptr(),
+                             lw.gamma2.data_ptr(), lw.router_w.data_ptr(), 0.0)
+    return lw
+
+
+def hbm_roofline(kernel, nbytes, ms, peaks, note=None):
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    r = dict(bound="hbm", kernel=kernel, achieved=gbs, peak=peaks["hbm_gbs"], unit="GB/s",
+             frac=gbs / peaks["hbm_gbs"], peak_source="%s (copy bandwidth)" % peaks["source"],
+             algorithmic_bytes=int(nbytes), traffic=None)
+    if note:
+        r["note"] = note
+    return r
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -205,6 +357,15 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
     api.lib()  # fail loudly if the CUDA library is missing
+    legs = set(args.legs.split(",")) if args.legs else set(ALL_LEGS)
+    if world > 1:
+        legs &= {"sweep", "e2e"}  # the other legs describe one GPU; replicas add nothing to them
+    peaks = measured_peaks()
+    sampler = ClockSampler(local)
+    sampler.start()
+    timer = Timer(torch, dist, world, dev, sampler)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(1234)
 
     sh, B, S, w, x, cu = build_layer_inputs(0, "c2")
     T = B * S
@@ -212,133 +373,339 @@ def run_ours(args):
     cud = torch.from_numpy(cu).to(dev)
     ratio = args.ratio
     cfg = api.layer_config(sh, api.SELECT_TOPK, ratio=ratio)
-    ws = torch.zeros(api.layer_workspace_bytes(cfg, T, B), dtype=torch.uint8, device=dev)
-    n_buf = 4
+    ws = torch.empty(api.layer_workspace_bytes(cfg, T, B), dtype=torch.uint8, device=dev)
     x_host = torch.from_numpy(x).to(torch.bfloat16).pin_memory()
-    out_host = torch.empty_like(x_host).pin_memory()
-    bufs = [x_host.to(dev) for _ in range(n_buf)]
+    x_src = x_host.to(dev)
+    # one input buffer per step of a region (the layer works in place), refilled with the
+    # N(0,1) input between regions, so that every timed step sees the stated input
+    n_buf = max(4, min(args.steps, 128))
+    bufs = [x_src.clone() for _ in range(n_buf)]
     nex = torch.zeros(1, dtype=torch.int32, device=dev)
+
+    def refill():
+        for b in bufs:
+            b.copy_(x_src)
 
     def step(i, c=cfg):
         api.layer_forward(c, lw, bufs[i % n_buf], cud, ws, nex)
 
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    def timed(fn, steps, warmup, sampler=None, drain=None):
-        for i in range(warmup):
-            fn(i)
-        if drain is not None:
-            drain()
-        barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        t_start = time.time()
-        e0.record()
-        for i in range(steps):
-            fn(i)
-        if drain is not None:
-            drain()  # the timed stream waits for the copies still in flight on the others
-        e1.record()
-        barrier()
-        if sampler is not None:
-            sampler.window = (t_start, time.time())
-        return max_over_ranks(e0.elapsed_time(e1), dev if world > 1 else None)
+    def check_status():
+        rc = api.device_status()
+        if rc != 0:
+            raise RuntimeError("device status: " + api.strerror(rc))
 
     # ---- headline: device-resident inputs ----
-    sampler = ClockSampler(local)
-    sampler.start()
-    time.sleep(0.3)  # let the first samples arrive before the timed region
-    ms = timed(step, args.steps, args.warmup, sampler)
-    clocks = sampler.stop()
-    ms_per_step = ms / args.steps
+    head = timer.run(step, args.steps, args.warmup, args.min_seconds, between=refill, idle=True)
+    ms_per_step = head["ms"]
     value = aggregate_tokens_per_s(T, world, ms_per_step)
-    rc = api.device_status()
-    if rc != 0:
-        raise RuntimeError("device status: " + api.strerror(rc))
+    check_status()
     n_exec = int(nex.item())
+    extra = {}
 
-    # ---- sweep over execution ratios ----
+    # ---- sweep over execution ratios, interleaved over several rounds ----
     sweep = {}
-    sw_steps = max(3, min(100, args.steps // 2))
-    for r in SWEEP:
-        c = api.layer_config(sh, api.SELECT_TOPK, ratio=r)
-        m = timed(lambda i, c=c: step(i, c), sw_steps, 3) / sw_steps
-        sweep["%.2f" % r] = dict(ms=m, tokens_per_s=world * T / (m * 1e-3))
-    base = sweep["1.00"]["ms"]
-    for r in sweep:
-        sweep[r]["speedup_vs_ratio_1"] = base / sweep[r]["ms"]
+    if "sweep" in legs:
+        cfgs = {r: api.layer_config(sh, api.SELECT_TOPK, ratio=r) for r in SWEEP}
+        sw_steps = max(3, min(n_buf, args.steps))
+        samples = {r: [] for r in SWEEP}
+        windows = []
+        for i in range(3):
+            step(i, cfgs[1.0])
+        for rnd in range(args.sweep_rounds):
+            for r in (SWEEP if rnd % 2 == 0 else SWEEP[::-1]):
+                refill()
+                samples[r].append(timer.region(lambda i, c=cfgs[r]: step(i, c), sw_steps, windows) / sw_steps)
+        for r in SWEEP:
+            m = statistics.median(samples[r])
+            sweep["%.2f" % r] = dict(ms=m, min_ms=min(samples[r]), tokens_per_s=world * T / (m * 1e-3),
+                                     ideal_speedup=accounting.layer_flops(sh, [S] * B, 1.0) /
+                                     accounting.layer_flops(sh, [S] * B, r))
+        base = sweep["1.00"]["ms"]
+        for r in sweep:
+            sweep[r]["speedup_vs_ratio_1"] = base / sweep[r]["ms"]
+        sweep["how"] = ("%d rounds, ratios interleaved (order reversed every other round), %d steps "
+                        "per region, median per ratio" % (args.sweep_rounds, sw_steps))
+        sweep["clocks"] = sampler.summary(windows)
+        check_status()
 
-    # ---- roofline of the dominant kernel: the four quantised GEMMs at this ratio ----
-    peaks = measured_peaks()
-    k = api.topk_count(ratio, T)
-    m_dev = torch.tensor([k], dtype=torch.int32, device=dev)
-    qd = sh.n_heads * sh.head_dim
-    adt = api.act_torch_dtype(cfg.act_dtype)
-    a_d = torch.randn(T, sh.d, device=dev).to(adt)
-    a_q = torch.randn(T, qd, device=dev).to(adt)
-    a_f = torch.randn(T, sh.ffn, device=dev).to(adt)
-    y_qkv = torch.empty(T, lw.qkv.N, dtype=adt, device=dev)
-    y_o = torch.empty(T, sh.d, dtype=adt, device=dev)
-    y_act = torch.empty(T, sh.ffn, dtype=adt, device=dev)
+    # ---- roofline of the dominant kernel: the four quantised GEMMs of a step, real epilogues ----
+    roofline = None
+    if "gemm" in legs or True:
+        k = api.topk_count(ratio, T)
+        m_dev = torch.tensor([k], dtype=torch.int32, device=dev)
+        qd = sh.n_heads * sh.head_dim
+        adt = api.act_torch_dtype(cfg.act_dtype)
+        a_d = torch.randn(T, sh.d, device=dev, generator=gen).to(adt)
+        a_q = torch.randn(T, qd, device=dev, generator=gen).to(adt)
+        a_f = (torch.randn(T, sh.ffn, device=dev, generator=gen) * 0.3).to(adt)
+        y_qkv = torch.empty(T, lw.qkv.N, dtype=adt, device=dev)
+        u = torch.empty(T, sh.d, dtype=torch.float32, device=dev)
+        y_act = torch.empty(T, sh.ffn, dtype=adt, device=dev)
+        idx = torch.sort(torch.randperm(T, device=dev, generator=gen)[:max(k, 1)])[0].to(torch.int32)
+        idx_full = torch.zeros(T, dtype=torch.int32, device=dev)
+        idx_full[:k] = idx[:k]
+        x_g = x_src.clone()
 
-    def gemms(i):
-        api.wq_gemm(a_d, lw.qkv, m_dev, api.EPI_STORE_16, y=y_qkv)
-        api.wq_gemm(a_q, lw.o, m_dev, api.EPI_STORE_16, y=y_o)
-        api.wq_gemm(a_d, lw.gate_up, m_dev, api.EPI_SWIGLU, y=y_act)
-        api.wq_gemm(a_f, lw.down, m_dev, api.EPI_STORE_16, y=y_o)
+        def gemms(i):
+            api.wq_gemm(a_d, lw.qkv, m_dev, api.EPI_STORE_16, y=y_qkv)
+            api.wq_gemm(a_q, lw.o, m_dev, api.EPI_RESID_F32, y=u, idx=idx_full, resid=x_g)
+            api.wq_gemm(a_d, lw.gate_up, m_dev, api.EPI_SWIGLU, y=y_act)
+            api.wq_gemm(a_f, lw.down, m_dev, api.EPI_RESID_SCATTER, idx=idx_full, resid=u, dst=x_g)
 
-    g_steps = max(3, min(200, args.steps // 2))
-    g_ms = timed(gemms, g_steps, 3) / g_steps
-    flops = 2.0 * sh.linear_params() * k
-    achieved = flops / (g_ms * 1e-3) / 1e12
-    peak = peaks["bf16_tflops_sustained"]
-    roofline = dict(bound="tensor", kernel="wq_gemm_pair_kernel<4,1> (4 launches per step)",
-                    achieved=achieved, peak=peak, unit="TFLOP/s", frac=achieved / peak,
-                    peak_source="%s (sustained bf16)" % peaks["source"],
-                    traffic=GEMM_DRAM_BYTES if abs(ratio - 0.5) < 1e-9 else None,
-                    traffic_unit="bytes per 4 launches (dram__bytes_read.sum + dram__bytes_write.sum, "
-                                 "ncu, ratio 0.5; profiles/wq_gemm_pair_layer_step_traffic.md)",
-                    ms_per_4_launches=g_ms, share_of_step=g_ms / ms_per_step)
+        g = timer.run(gemms, max(3, min(100, args.steps)), 3, args.min_seconds, idle=True)
+        flops = 2.0 * sh.linear_params() * k
+        sustained = flops / (g["ms"] * 1e-3) / 1e12
+        burst = flops / (g["burst_ms"] * 1e-3) / 1e12
+        roofline = dict(bound="tensor", kernel="wq_gemm_pair_kernel<4,1> (the 4 launches of a step, "
+                        "with the layer's epilogues: store, x[idx]+acc, SwiGLU, residual scatter)",
+                        achieved=sustained, peak=peaks["bf16_tflops_sustained"], unit="TFLOP/s",
+                        frac=sustained / peaks["bf16_tflops_sustained"],
+                        peak_source="%s (sustained bf16 matmul; regions repeated for %.1f s)" % (
+                            peaks["source"], args.min_seconds),
+                        burst=dict(achieved=burst, peak=peaks["bf16_tflops"],
+                                   frac=burst / peaks["bf16_tflops"],
+                                   note="first region after an idle second, against the burst peak"),
+                        traffic=None,
+                        ms_per_4_launches=g["ms"], share_of_step=g["ms"] / ms_per_step,
+                        executed_tokens=k, clocks=g["clocks"])
+        check_status()
+        del a_d, a_q, a_f, y_qkv, u, y_act, x_g
+
+    # ---- the same layer with bf16 internal tensors ----
+    if "bf16" in legs:
+        cfg_b = api.layer_config(sh, api.SELECT_TOPK, ratio=ratio, act_dtype=api.ACT_BF16)
+        r = timer.run(lambda i: step(i, cfg_b), max(3, min(n_buf, args.steps)), 3, 0.4, between=refill)
+        extra["c2_bf16_internal"] = dict(ms_per_step=r["ms"], tokens_per_s=T / (r["ms"] * 1e-3),
+                                         note="internal 16-bit tensors and dequantised weights in bf16 "
+                                              "instead of fp16", clocks=r["clocks"])
+        check_status()
 
     # ---- end to end: host buffers, H2D of the inputs and D2H of the result every step ----
     # Every step copies its input from pinned host memory, runs the layer through the public
     # call and copies its result back; the copies run on two streams of their own, so step
-    # i + 1's input and step i - 1's result travel while step i computes (n_buf device buffers).
-    main = torch.cuda.current_stream()
-    copy_in, copy_out = torch.cuda.Stream(), torch.cuda.Stream()
-    ev_in = [torch.cuda.Event() for _ in range(n_buf)]
-    ev_done = [torch.cuda.Event() for _ in range(n_buf)]
-    ev_out = [torch.cuda.Event() for _ in range(n_buf)]
-    out_hosts = [out_host] + [torch.empty_like(x_host).pin_memory() for _ in range(n_buf - 1)]
+    # i + 1's input and step i - 1's result travel while step i computes.
+    e2e = None
+    if "e2e" in legs or True:
+        n_e = 4
+        main = torch.cuda.current_stream()
+        copy_in, copy_out = torch.cuda.Stream(), torch.cuda.Stream()
+        ev_in = [torch.cuda.Event() for _ in range(n_e)]
+        ev_done = [torch.cuda.Event() for _ in range(n_e)]
+        ev_out = [torch.cuda.Event() for _ in range(n_e)]
+        out_hosts = [torch.empty_like(x_host).pin_memory() for _ in range(n_e)]
 
-    def e2e_step(i):
-        j = i % n_buf
-        buf = bufs[j]
-        with torch.cuda.stream(copy_in):
-            copy_in.wait_event(ev_out[j])  # the buffer's previous result has left the device
-            buf.copy_(x_host, non_blocking=True)
-            ev_in[j].record(copy_in)
-        main.wait_event(ev_in[j])
-        api.layer_forward(cfg, lw, buf, cud, ws, nex)
-        ev_done[j].record(main)
-        with torch.cuda.stream(copy_out):
-            copy_out.wait_event(ev_done[j])
-            out_hosts[j].copy_(buf, non_blocking=True)
-            ev_out[j].record(copy_out)
+        def e2e_step(i):
+            j = i % n_e
+            buf = bufs[j]
+            with torch.cuda.stream(copy_in):
+                copy_in.wait_event(ev_out[j])  # the buffer's previous result has left the device
+                buf.copy_(x_host, non_blocking=True)
+                ev_in[j].record(copy_in)
+            main.wait_event(ev_in[j])
+            api.layer_forward(cfg, lw, buf, cud, ws, nex)
+            ev_done[j].record(main)
+            with torch.cuda.stream(copy_out):
+                copy_out.wait_event(ev_done[j])
+                out_hosts[j].copy_(buf, non_blocking=True)
+                ev_out[j].record(copy_out)
 
-    def e2e_drain():
+        e_steps = max(3, min(50, args.steps))
+
+        def e2e_region(i):
+            e2e_step(i)
+            if i == e_steps - 1:  # the timed stream waits for the copies still in flight
+                main.wait_stream(copy_in)
+                main.wait_stream(copy_out)
+
         main.wait_stream(copy_in)
-        main.wait_stream(copy_out)
+        er = timer.run(e2e_region, e_steps, 3, 0.5)
+        nbytes = x_host.numel() * 2
+        e2e = dict(value=world * T / (er["ms"] * 1e-3), unit=UNIT, h2d_bytes_per_step=nbytes,
+                   d2h_bytes_per_step=nbytes, ms_per_step=er["ms"],
+                   note="copies on their own streams, overlapped with the neighbouring steps' compute")
+        check_status()
 
-    main.wait_stream(copy_in)
-    e_steps = max(3, min(50, args.steps // 2))
-    e_ms = timed(e2e_step, e_steps, 3, drain=e2e_drain) / e_steps
-    nbytes = x_host.numel() * 2
-    e2e = dict(value=world * T / (e_ms * 1e-3), unit=UNIT, h2d_bytes_per_step=nbytes,
-               d2h_bytes_per_step=nbytes, ms_per_step=e_ms,
-               note="copies on their own streams, overlapped with the neighbouring steps' compute")
+    # ---- memory-bound stages through the C ABI, each against the measured copy bandwidth ----
+    if "router" in legs:
+        out = {}
+        for name, Tr, dr in [("c2_T8192_d4096", 8192, 4096), ("c5_T65536_d5120", 65536, 5120)]:
+            xr = torch.randn(Tr, dr, device=dev, generator=gen).to(torch.bfloat16)
+            wr = (torch.randn(dr, device=dev, generator=gen) * 0.02).to(torch.bfloat16).float()
+            cur = torch.tensor([0, Tr], dtype=torch.int32, device=dev)
+            o = api.router_select(xr, wr, 0.0, cur, api.SELECT_THRESHOLD, theta=0.5)
+            nbytes = Tr * (2 * dr + 4) + 8 * int(o["n_exec"].item())
+            for mode, mname in [(api.SELECT_THRESHOLD, "threshold"), (api.SELECT_TOPK, "topk")]:
+                call = lambda: api.router_select(xr, wr, 0.0, cur, mode, theta=0.5, k=Tr // 2, out=o)
+                call()
+                n_in = 20 if Tr <= 8192 else 5
+                gr = graph_of(torch, call, n_in)
+                r = timer.run(lambda i: gr.replay(), 10, 3, 0.25)
+                ms = r["ms"] / n_in
+                out["%s_%s" % (name, mname)] = dict(
+                    us=ms * 1e3, launch="CUDA graph of %d calls (scratch clear + kernel each)" % n_in,
+                    roofline=hbm_roofline("router_select_kernel", nbytes, ms, peaks), clocks=r["clocks"])
+            del xr
+        extra["router_select"] = out
+        check_status()
+
+    if "gather" in legs:
+        Tg, dg = 65536, 5120
+        kg = api.topk_count(0.7, Tg)
+        xg = torch.randn(Tg, dg, device=dev, generator=gen).to(torch.bfloat16)
+        idxg = torch.zeros(Tg, dtype=torch.int32, device=dev)
+        idxg[:kg] = torch.sort(torch.randperm(Tg, device=dev, generator=gen)[:kg])[0].to(torch.int32)
+        ng = torch.tensor([kg], dtype=torch.int32, device=dev)
+        gam = torch.ones(dg, dtype=torch.float32, device=dev)
+        hn = torch.empty(Tg, dg, dtype=torch.float16, device=dev)
+        call = lambda: api.compact(xg, idxg, ng, gam, 1e-5, want_xc=False, hn_out=hn, act_dtype=api.ACT_F16)
+        call()
+        gr = graph_of(torch, call, 5)
+        r = timer.run(lambda i: gr.replay(), 10, 3, 0.25)
+        ms = r["ms"] / 5
+        extra["gather_rmsnorm"] = dict(
+            us=ms * 1e3, rows="%d of %d, d %d" % (kg, Tg, dg),
+            roofline=hbm_roofline("compact_kernel", kg * dg * 4, ms, peaks), clocks=r["clocks"])
+        del xg, hn
+        check_status()
+
+    # ---- c3: one decode step of the 7B-shaped layer, 64 sequences with 2048 cached tokens ----
+    if "decode" in legs:
+        out = {}
+        for name in ("c3_int3", "c3_int4g64"):
+            c3 = inputs.CONFIG_SHAPES[name]
+            s3, B3 = c3["shape"], c3["B"]
+            lw3 = timing_layer(torch, api, dev, gen, s3)
+            cap = 2048 + 64
+            kv = api.KvCache(B3, cap, s3.kv_dim, dev, act_dtype=api.ACT_F16)
+            kv.k.normal_(generator=gen)
+            kv.v.normal_(generator=gen)
+            len0 = torch.full((B3,), 2048, dtype=torch.int32, device=dev)
+            logits = torch.randn(B3, device=dev, generator=gen)
+            scores = torch.sigmoid(logits).float()
+            x3 = torch.randn(B3, s3.d, device=dev, generator=gen).to(torch.bfloat16)
+            cu3 = torch.arange(B3 + 1, dtype=torch.int32, device=dev)
+            wbytes = accounting.packed_weight_bytes(s3)
+            for r3 in (0.9, 0.6):
+                k3 = api.topk_count(r3, B3)
+                srt = torch.sort(scores, descending=True)[0]
+                theta = float((srt[k3 - 1] + srt[k3]) / 2)
+                cfg3 = api.layer_config(s3, api.SELECT_THRESHOLD, theta=theta)
+                ws3 = torch.empty(api.layer_workspace_bytes(cfg3, B3, B3), dtype=torch.uint8, device=dev)
+                xb = x3.clone()
+
+                def dstep():
+                    api.layer_forward(cfg3, lw3, xb, cu3, ws3, nex, pos0=len0, scores_override=scores,
+                                      kv=kv, phase=api.PHASE_DECODE)
+
+                def reset():
+                    kv.kv_len.copy_(len0)
+                    xb.copy_(x3)
+
+                reset()
+                dstep()
+                torch.cuda.synchronize()
+                assert int(nex.item()) == k3
+                reset()
+                gr = graph_of(torch, dstep, 1)
+                n_rep = 20  # the caches grow by one entry per executed sequence and step
+                r = timer.run(lambda i: gr.replay(), n_rep, 3, 0.25, between=reset)
+                reset()
+                kv_bytes = k3 * 2 * 2048 * s3.kv_dim * 2
+                nbytes = wbytes + kv_bytes
+                out["%s_ratio_%.1f" % (name, r3)] = dict(
+                    ms_per_step=r["ms"], executed_sequences=k3, tokens_per_s=B3 / (r["ms"] * 1e-3),
+                    launch="CUDA graph of one decode step",
+                    roofline=hbm_roofline("decode step (4 small-M GEMMs + attention over the cache)",
+                                          nbytes, r["ms"], peaks,
+                                          note="bytes = packed weights %d + keys/values of the executed "
+                                               "sequences %d" % (wbytes, kv_bytes)),
+                    clocks=r["clocks"])
+            del kv, lw3
+        extra["c3_decode_step"] = out
+        check_status()
+
+    # ---- c4: 8B-shaped 32-layer model prefill, per-layer top-k at ratio 0.75 ----
+    if "c4" in legs:
+        c4 = inputs.CONFIG_SHAPES["c4"]
+        s4, B4, S4 = c4["shape"], c4["B"], c4["S"]
+        L4, V4 = 32, 128256
+        T4 = B4 * S4
+        layers = [timing_layer(torch, api, dev, gen, s4) for _ in range(L4)]
+        embed = torch.randn(V4, s4.d, device=dev, generator=gen).to(torch.bfloat16)
+        lm_head = (torch.randn(V4, s4.d, device=dev, generator=gen) * 0.02).to(torch.bfloat16)
+        fg = torch.ones(s4.d, dtype=torch.float32, device=dev)
+        ids = torch.randint(0, V4, (T4,), dtype=torch.int32, device=dev, generator=gen)
+        cu4 = torch.from_numpy(inputs.cu_seqlens_uniform(B4, S4)).to(dev)
+        rows = (cu4[1:] - 1).to(torch.int32)
+        mcfg = api.ModelConfig(L4, V4, api.layer_config(s4, api.SELECT_TOPK, ratio=0.75))
+        mws = torch.empty(api.model_workspace_bytes(mcfg, T4, B4, B4), dtype=torch.uint8, device=dev)
+        hidden = torch.empty(T4, s4.d, dtype=torch.bfloat16, device=dev)
+        logits = torch.empty(B4, V4, dtype=torch.float32, device=dev)
+        per_layer = torch.zeros(L4, dtype=torch.int32, device=dev)
+
+        def mstep(i):
+            api.model_prefill(mcfg, layers, embed, ids, cu4, mws, hidden, per_layer_ratio=[0.75] * L4,
+                              final_gamma=fg, lm_head=lm_head, logit_rows=rows, logits_out=logits,
+                              per_layer_n_exec=per_layer)
+
+        r = timer.run(mstep, 3, 2, 0.5)
+        check_status()
+        k4 = api.topk_count(0.75, T4)
+        assert per_layer.cpu().tolist() == [k4] * L4
+        fl = L4 * accounting.layer_flops(s4, [S4] * B4, 0.75) + 2.0 * s4.d * V4 * B4
+        extra["c4_model_prefill"] = dict(
+            ms_per_step=r["ms"], tokens_per_s=T4 / (r["ms"] * 1e-3), layers=L4, tokens=T4,
+            select="per-layer top-k, ratio 0.75 (%d of %d tokens per layer)" % (k4, T4),
+            logits="last token of each sequence",
+            achieved_tflops=fl / (r["ms"] * 1e-3) / 1e12,
+            frac_of_sustained_bf16=fl / (r["ms"] * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
+            weights="random codes (seeded, device side), distinct per layer", clocks=r["clocks"])
+        del layers, embed, lm_head, mws, hidden, logits
+
+    # ---- c5: 13B-shaped 8-layer stack, 16 x 4096 tokens, per-layer ratios from U[0.4, 1.0],
+    # ---- per-token scores ~ Beta(2,2) supplied to the selection ----
+    if "c5" in legs:
+        c5 = inputs.CONFIG_SHAPES["c5"]
+        s5, B5, S5 = c5["shape"], c5["B"], c5["S"]
+        L5 = 8
+        T5 = B5 * S5
+        layers = [timing_layer(torch, api, dev, gen, s5) for _ in range(L5)]
+        ratios = 0.4 + 0.6 * inputs.uniform(0, 5000, L5)
+        # threshold of each layer from the Beta(2,2) distribution: P(score >= theta) = ratio,
+        # i.e. 3 theta^2 - 2 theta^3 = 1 - ratio (bisection on the closed-form CDF)
+        thetas = []
+        for rl in ratios:
+            lo, hi = 0.0, 1.0
+            for _ in range(60):
+                mid = (lo + hi) / 2
+                lo, hi = (mid, hi) if 3 * mid * mid - 2 * mid ** 3 < 1 - rl else (lo, mid)
+            thetas.append((lo + hi) / 2)
+        sc5 = [torch.from_numpy(inputs.beta22(0, 5001 + li, T5).astype(np.float32)).to(dev) for li in range(L5)]
+        cfgs5 = [api.layer_config(s5, api.SELECT_THRESHOLD, theta=th) for th in thetas]
+        ws5 = torch.empty(api.layer_workspace_bytes(cfgs5[0], T5, B5), dtype=torch.uint8, device=dev)
+        x5_src = torch.randn(T5, s5.d, device=dev, generator=gen).to(torch.bfloat16)
+        x5 = x5_src.clone()
+        cu5 = torch.from_numpy(inputs.cu_seqlens_uniform(B5, S5)).to(dev)
+        counts = torch.zeros(L5, dtype=torch.int32, device=dev)
+
+        def sstep(i):
+            for li in range(L5):
+                api.layer_forward(cfgs5[li], layers[li], x5, cu5, ws5, counts[li:li + 1],
+                                  scores_override=sc5[li])
+
+        r = timer.run(sstep, 2, 1, 0.4, between=lambda: x5.copy_(x5_src))
+        check_status()
+        n5 = counts.cpu().tolist()
+        # per-sequence executed counts differ: take the flops from the realised ratios
+        fl = sum(accounting.layer_flops(s5, [S5] * B5, n / T5) for n in n5)
+        extra["c5_irregular_stack"] = dict(
+            ms_per_step=r["ms"], tokens_per_s=T5 / (r["ms"] * 1e-3), layers=L5, tokens=T5,
+            target_ratios=[round(float(v), 4) for v in ratios], executed_per_layer=n5,
+            select="threshold per layer from the Beta(2,2) quantile, scores supplied",
+            achieved_tflops=fl / (r["ms"] * 1e-3) / 1e12,
+            frac_of_sustained_bf16=fl / (r["ms"] * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
+            weights="random codes (seeded, device side), distinct per layer", clocks=r["clocks"])
+        del layers, ws5, x5, x5_src, sc5
 
     line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps,
                 warmup=args.warmup, ms_per_step=ms_per_step, higher_is_better=True, scaling="weak",
@@ -348,12 +715,19 @@ def run_ours(args):
                                       "dequantised weights, fp32 accumulation",
                             tokens=T,
                             l2="inputs larger than L2 (packed weights 107 MB + more than 1 GB of "
-                               "activations per step, %d rotating input buffers)" % n_buf,
+                               "activations per step; %d input buffers, one per step of a region, "
+                               "refilled with the N(0,1) input between regions)" % n_buf,
                             multi_gpu="replicas only: every rank runs the same batch, no collective"),
-                clocks=clocks, gpu_launches=KERNELS_PER_STEP * args.steps, sweep=sweep,
-                roofline=roofline, e2e=e2e)
+                timing=dict(regions=head["regions"], steps_per_region=args.steps,
+                            sustained_ms_per_step=head["ms"], burst_ms_per_step=head["burst_ms"],
+                            min_ms_per_step=head["min_ms"], ms_x_ghz=head.get("ms_x_ghz"),
+                            how="value = median region (regions back to back for %.1f s: power-capped); "
+                                "burst = first region after an idle second" % args.min_seconds),
+                clocks=head["clocks"],
+                gpu_launches=KERNELS_PER_STEP * args.steps * head["regions"],
+                sweep=sweep, roofline=roofline, e2e=e2e, legs=extra)
 
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if rank == 0 and world == 1 and "cpu" in legs:
         sample = 2048  # one whole sequence: about 10-30 s of host time
         run, threads = oracle_runner(sh, w, x, ratio, sample)
         t0 = time.perf_counter()
@@ -361,6 +735,7 @@ def run_ours(args):
         dt = time.perf_counter() - t0
         line["cpu_baseline"] = dict(value=sample / dt, unit=UNIT, cores=threads, kind="oracle",
                                     sample=sample_desc(sample, ratio) + "; one pass, %.1f s" % dt)
+    sampler.stop()
     if rank == 0:
         print(json.dumps(line))
     if world > 1:
@@ -371,16 +746,25 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=400)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--ratio", type=float, default=0.5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--legs", default="", help="comma-separated subset of: " + ",".join(ALL_LEGS))
+    ap.add_argument("--min-seconds", type=float, default=1.0,
+                    help="regions of --steps steps are repeated until this much device time")
+    ap.add_argument("--sweep-rounds", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.no_cpu_baseline:
+        args.legs = ",".join(l for l in (args.legs.split(",") if args.legs else ALL_LEGS) if l != "cpu")
     if args.warmup < 3:
         args.warmup = 3
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started as a plain process: become N replicas, one per GPU
+        return spawn_replicas(args.gpus, os.path.abspath(__file__), sys.argv[1:])
     return run_ours(args)
 
 

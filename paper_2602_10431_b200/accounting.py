@@ -44,3 +44,17 @@ def gather_bytes(n_exec, d, with_norm=False):
 
 def scatter_bytes(n_exec, d):
     return n_exec * (4 * d + 2 * d)
+
+
+def layer_flops(sh, seq_lens, ratio):
+    """FLOPs of one layer call on sequences of `seq_lens` tokens of which a share `ratio`
+    executes (evenly per sequence): linears on the executed tokens plus causal attention
+    among them."""
+    ex = [ratio * s for s in seq_lens]
+    lin = 2.0 * linear_params(sh.d, sh.n_heads, sh.n_kv_heads, sh.head_dim, sh.ffn) * sum(ex)
+    return lin + attention_flops(ex, sh.n_heads, sh.head_dim)
+
+
+def packed_weight_bytes(sh):
+    """Bytes of the four packed linears of one layer (codes + per-group scale and zero-point)."""
+    return int(layer_weight_bytes(sh.d, sh.n_heads, sh.n_kv_heads, sh.head_dim, sh.ffn, sh.bits, sh.group))

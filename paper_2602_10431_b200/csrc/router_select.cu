@@ -15,6 +15,7 @@ constexpr int kBins = 2048;          // first-level histogram of the top-k selec
 constexpr int kScoreSmem = 4096;     // a CTA keeps its tokens' scores in shared memory up to this many
 constexpr int kCandSmem = 1024;      // candidates ranked in shared memory (more: radix select by one CTA)
 constexpr int kMaxGrid = 1024;
+constexpr int kLocalHistTokens = 16384;  // up to here every CTA builds the score histogram itself
 constexpr uint32_t kSpinLimit = 1u << 20;  // polls of a global word before a wait gives up
 
 // Scratch in the caller's workspace (32-bit words).  The first kZeroWords(grid) words are
@@ -110,10 +111,12 @@ __device__ __forceinline__ int block_inclusive_scan(int v, int* s_w, int& total)
 // ---- the fused kernel -------------------------------------------------------
 // CTA c owns the consecutive tokens [c * chunk, (c + 1) * chunk).
 //   1. scores of its tokens (bandwidth-bound sweep of their rows of x, fp64 accumulation);
-//   2. top-k only: a histogram of all scores over kBins uniform bins is accumulated in global
-//      memory; after a grid barrier every CTA finds the bin holding the k-th largest score, the
-//      (few) tokens of that bin are appended to a candidate list, and after a second barrier
-//      every CTA ranks the candidates by (score descending, token ascending) to get the cut-off;
+//   2. top-k only: after a grid barrier every CTA knows the histogram of all scores over kBins
+//      uniform bins (small calls: built by each CTA from the scores of all; large calls:
+//      accumulated in global memory during the sweep), finds the bin holding the k-th largest
+//      score, collects the (few) tokens of that bin as candidates (small calls: from its own
+//      registers; large: a shared list and a second barrier) and ranks them by (score descending,
+//      token ascending) to get the cut-off;
 //   3. each CTA counts its executed tokens, publishes the count, adds up the counts of the CTAs
 //      before it (they publish as soon as they know theirs) and writes its part of the ascending
 //      index list, the positions and the per-sequence offsets.
@@ -124,7 +127,8 @@ __global__ void __launch_bounds__(kRouterThreads, 2) router_select_kernel(const 
   __shared__ uint2 s_cand[kCandSmem];
   __shared__ int s_w[32];
   __shared__ uint32_t s_hist[256];
-  __shared__ int s_abort, s_bstar, s_rank, s_nvalid;
+  __shared__ uint32_t s_h[kBins];
+  __shared__ int s_abort, s_bstar, s_rank, s_nvalid, s_ncand, s_fill;
   __shared__ uint32_t s_cut_key, s_cut_tok, s_prefix_hi, s_prefix_lo;
 
   const int tid = threadIdx.x, nthr = blockDim.x;
@@ -156,27 +160,33 @@ __global__ void __launch_bounds__(kRouterThreads, 2) router_select_kernel(const 
     float* w_s = reinterpret_cast<float*>(smem_raw);
     const int d = p.d;
     const int n_it = (d + 255) / 256;
+    constexpr int kUnroll = 4;  // 16-byte loads in flight per lane: kUnroll x rows per warp
+    auto load_block = [&](int r0, int it0, uint4 (&v)[kUnroll][kRowsPerWarp]) {
+#pragma unroll
+      for (int u = 0; u < kUnroll; ++u) {
+        const int col = (it0 + u) * 256 + lane * 8;
+#pragma unroll
+        for (int r = 0; r < kRowsPerWarp; ++r) {
+          const int row = min(r0 + r, c1 - 1);
+          v[u][r] = (it0 + u < n_it && col < d) ? ld_nc_16(p.x + (size_t)row * d + col)
+                                                : make_uint4(0, 0, 0, 0);
+        }
+      }
+    };
+    const int n_groups = (n_own + kRowsPerWarp - 1) / kRowsPerWarp;
+    // the first loads of x are in flight while the router weights are staged
+    uint4 v0[kUnroll][kRowsPerWarp];
+    if (wid < n_groups) load_block(c0 + wid * kRowsPerWarp, 0, v0);
     for (int i = tid; i < n_it * 256; i += nthr) w_s[i] = (i < d) ? p.w[i] : 0.f;
     __syncthreads();
-    const int n_groups = (n_own + kRowsPerWarp - 1) / kRowsPerWarp;
     for (int g = wid; g < n_groups; g += nwarps) {
       const int r0 = c0 + g * kRowsPerWarp;
       double acc[kRowsPerWarp];
 #pragma unroll
       for (int r = 0; r < kRowsPerWarp; ++r) acc[r] = 0.0;
-      constexpr int kUnroll = 4;  // 16-byte loads in flight per lane: kUnroll x rows per warp
       for (int it0 = 0; it0 < n_it; it0 += kUnroll) {
-        uint4 v[kUnroll][kRowsPerWarp];
-#pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
-          const int col = (it0 + u) * 256 + lane * 8;
-#pragma unroll
-          for (int r = 0; r < kRowsPerWarp; ++r) {
-            const int row = min(r0 + r, c1 - 1);
-            v[u][r] = (it0 + u < n_it && col < d) ? ld_nc_16(p.x + (size_t)row * d + col)
-                                                  : make_uint4(0, 0, 0, 0);
-          }
-        }
+        uint4 (&v)[kUnroll][kRowsPerWarp] = v0;
+        if (it0 != 0 || g != wid) load_block(r0, it0, v);  // the very first block is already there
 #pragma unroll
         for (int u = 0; u < kUnroll; ++u) {
           if (it0 + u >= n_it) break;
@@ -229,19 +239,70 @@ __global__ void __launch_bounds__(kRouterThreads, 2) router_select_kernel(const 
   uint64_t cut = 0;                         // (key << 32 | ~token) of the k-th token
   if (topk) {
     uint32_t step = 0;  // grid barriers passed
-    int nv = 0;
-    for (int sl = 0; sl < n_slab; ++sl) {
-      const int i = sl * nthr + tid;
-      if (ok_at(i)) {
-        ++nv;
-        atomicAdd(p.ws + kWsHist + score_bin(score_at(i)), 1u);
+    // Calls of up to kLocalHistTokens tokens: after the barrier every CTA reads ALL scores
+    // (a few 16-byte loads per thread, issued together), builds the histogram in its own shared
+    // memory and keeps the scores in registers for the candidate pass: one barrier, no global
+    // atomics.  Larger calls accumulate the histogram in global memory during the sweep.
+    const bool local = T <= kLocalHistTokens;
+    constexpr int kLocalVec = kLocalHistTokens / (kRouterThreads * 4);  // float4 loads per thread
+    float lsc[kLocalVec * 4];
+    uint32_t lok = 0;  // bit j: score j of this thread belongs to a valid token
+    int n_valid = 0;
+    if (local) {
+      for (int i = tid; i < kBins; i += nthr) s_h[i] = 0;
+      if (tid == 0) s_nvalid = 0;
+      if (!grid_barrier(p, ++step * G, &s_abort)) return;
+#pragma unroll
+      for (int j = 0; j < kLocalVec; ++j) {
+        const int t0 = (j * nthr + tid) * 4;
+        float4 q = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (t0 + 3 < T) {
+          q = __ldcg(reinterpret_cast<const float4*>(p.scores + t0));
+        } else if (t0 < T) {
+          q.x = __ldcg(p.scores + t0);
+          if (t0 + 1 < T) q.y = __ldcg(p.scores + t0 + 1);
+          if (t0 + 2 < T) q.z = __ldcg(p.scores + t0 + 2);
+        }
+        lsc[4 * j] = q.x; lsc[4 * j + 1] = q.y; lsc[4 * j + 2] = q.z; lsc[4 * j + 3] = q.w;
       }
+      int nv = 0;
+#pragma unroll
+      for (int j = 0; j < kLocalVec; ++j) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int t = (j * nthr + tid) * 4 + e;
+          if (t < T && t >= t_begin && t < t_end && (p.valid == nullptr || p.valid[t] != 0)) {
+            lok |= 1u << (4 * j + e);
+            ++nv;
+            atomicAdd(&s_h[score_bin(lsc[4 * j + e])], 1u);
+          }
+        }
+      }
+      nv = __reduce_add_sync(0xffffffffu, nv);
+      if (lane == 0 && nv) atomicAdd(&s_nvalid, nv);
+      __syncthreads();
+      n_valid = s_nvalid;
+    } else {
+      int nv = 0;
+      for (int sl = 0; sl < n_slab; ++sl) {
+        const int i = sl * nthr + tid;
+        if (ok_at(i)) {
+          ++nv;
+          atomicAdd(p.ws + kWsHist + score_bin(score_at(i)), 1u);
+        }
+      }
+      nv = __reduce_add_sync(0xffffffffu, nv);
+      if (lane == 0 && nv) atomicAdd(p.ws + kWsValid, (uint32_t)nv);
+      if (!grid_barrier(p, ++step * G, &s_abort)) return;
     }
-    nv = __reduce_add_sync(0xffffffffu, nv);
-    if (lane == 0 && nv) atomicAdd(p.ws + kWsValid, (uint32_t)nv);
-    if (!grid_barrier(p, ++step * G, &s_abort)) return;
-
-    const int n_valid = (int)__ldcg(p.ws + kWsValid);
+    // thread j reads bins from the top: tid 0 owns the four highest
+    constexpr int PER = kBins / kRouterThreads;
+    const int hi_bin = kBins - 1 - tid * PER;
+    uint32_t h[PER];
+#pragma unroll
+    for (int e = 0; e < PER; ++e)
+      h[e] = local ? s_h[hi_bin - e] : __ldcg(p.ws + kWsHist + hi_bin - e);
+    if (!local) n_valid = (int)__ldcg(p.ws + kWsValid);
     int k = p.k;
     if (k < 0) {  // k for a requested ratio of the valid tokens (padding does not count)
       double kd = floor(p.ratio * (double)n_valid + 0.5);
@@ -250,17 +311,11 @@ __global__ void __launch_bounds__(kRouterThreads, 2) router_select_kernel(const 
     k = min(k, n_valid);
     none = k <= 0;
     if (!none) {
-      // thread j reads bins from the top: tid 0 owns the four highest.  With `above` = valid
-      // tokens in higher bins, the k-th sits in the bin where above < k <= above + count.
-      constexpr int PER = kBins / kRouterThreads;
-      const int hi_bin = kBins - 1 - tid * PER;
-      uint32_t h[PER];
+      // with `above` = valid tokens in higher bins, the k-th sits in the bin where
+      // above < k <= above + count
       int v = 0;
 #pragma unroll
-      for (int e = 0; e < PER; ++e) {
-        h[e] = __ldcg(p.ws + kWsHist + hi_bin - e);
-        v += (int)h[e];
-      }
+      for (int e = 0; e < PER; ++e) v += (int)h[e];
       int total;
       int above = block_inclusive_scan(v, s_w, total) - v;
 #pragma unroll
@@ -268,29 +323,46 @@ __global__ void __launch_bounds__(kRouterThreads, 2) router_select_kernel(const 
         if (above < k && k <= above + (int)h[e]) {
           s_bstar = hi_bin - e;
           s_rank = k - above;       // 1-based rank of the k-th inside its bin
-          s_nvalid = (int)h[e];     // tokens in that bin
+          s_ncand = (int)h[e];      // tokens in that bin
         }
         above += (int)h[e];
       }
       __syncthreads();
       bstar = s_bstar;
-      const int r = s_rank, c = s_nvalid;
+      const int r = s_rank, c = s_ncand;
       uint2* cand = reinterpret_cast<uint2*>(reinterpret_cast<unsigned char*>(p.ws) + kWsHeaderBytes);
-      for (int sl = 0; sl < n_slab; ++sl) {
-        const int i = sl * nthr + tid;
-        if (ok_at(i)) {
-          const float sc = score_at(i);
-          if (score_bin(sc) == bstar) {
-            const uint32_t slot = atomicAdd(p.ws + kWsCand, 1u);
-            if (slot < (uint32_t)T) cand[slot] = make_uint2(score_key(sc), ~(uint32_t)(c0 + i));
+      // candidates = the valid tokens of bin bstar
+      if (local && c <= kCandSmem) {
+        if (tid == 0) s_fill = 0;
+        __syncthreads();
+#pragma unroll
+        for (int j = 0; j < kLocalVec * 4; ++j) {
+          if (((lok >> j) & 1u) && score_bin(lsc[j]) == bstar) {
+            const int slot = atomicAdd(&s_fill, 1);
+            if (slot < kCandSmem)
+              s_cand[slot] = make_uint2(score_key(lsc[j]), ~(uint32_t)(((j >> 2) * nthr + tid) * 4 + (j & 3)));
           }
         }
+        __syncthreads();
+      } else {
+        for (int sl = 0; sl < n_slab; ++sl) {
+          const int i = sl * nthr + tid;
+          if (ok_at(i)) {
+            const float sc = score_at(i);
+            if (score_bin(sc) == bstar) {
+              const uint32_t slot = atomicAdd(p.ws + kWsCand, 1u);
+              if (slot < (uint32_t)T) cand[slot] = make_uint2(score_key(sc), ~(uint32_t)(c0 + i));
+            }
+          }
+        }
+        if (!grid_barrier(p, ++step * G, &s_abort)) return;
+        if (c <= kCandSmem) {
+          for (int i = tid; i < c; i += nthr) s_cand[i] = __ldcg(cand + i);
+          __syncthreads();
+        }
       }
-      if (!grid_barrier(p, ++step * G, &s_abort)) return;
       if (c <= kCandSmem) {
         // every CTA ranks the candidates itself: the r-th in the order is the cut-off
-        for (int i = tid; i < c; i += nthr) s_cand[i] = __ldcg(cand + i);
-        __syncthreads();
         for (int i = tid; i < c; i += nthr) {
           const uint64_t me = ((uint64_t)s_cand[i].x << 32) | s_cand[i].y;
           int before = 0;
@@ -528,7 +600,7 @@ int router_select_launch(const void* x, int T, int d, const float* w_router, flo
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return QTALE_ERR_CUDA;
   if (dev != cached_dev || smem != cached_smem) {
-    if (smem > 20 * 1024 &&  // static + dynamic shared memory beyond the default 48 KB
+    if (smem > 0 &&  // static + dynamic shared memory may exceed the default 48 KB
         cudaFuncSetAttribute(router_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)smem) != cudaSuccess)
       return QTALE_ERR_CUDA;

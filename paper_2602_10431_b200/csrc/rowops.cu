@@ -10,29 +10,33 @@ namespace qtale {
 constexpr int kRowThreads = 256;
 
 // ---- gather (+ RMSNorm) ------------------------------------------------------
-// One warp per executed row; the row (d <= 32*8*MAXC bf16) stays in registers.
+// One CTA of 128 threads per executed row: the row (d <= 128 * 8 * MAXC bf16) stays in
+// registers between the sum of squares and the write, a thread holds MAXC 16-byte chunks.
+// Many small CTAs per SM keep loads, reductions and stores of different rows overlapped.
+constexpr int kGatherThreads = 128;
 template <int MAXC, int ACT>
-__global__ void __launch_bounds__(kRowThreads)
+__global__ void __launch_bounds__(kGatherThreads)
     compact_kernel(const uint4* __restrict__ x, const int32_t* __restrict__ idx,
                    const int32_t* __restrict__ n_exec, int cap, int d,
                    const float* __restrict__ gamma, float eps, uint4* __restrict__ xc,
                    uint4* __restrict__ hn) {
-  const int lane = threadIdx.x & 31;
-  const int warps = (gridDim.x * blockDim.x) >> 5;
+  __shared__ float s_part[2][kGatherThreads / 32];
+  const int tid = threadIdx.x;
   const int n = n_exec ? min(*n_exec, cap) : cap;
   const int chunks = d >> 3;  // 16-byte chunks per row
-  for (int i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < n; i += warps) {
+  int par = 0;
+  for (int i = blockIdx.x; i < n; i += gridDim.x, par ^= 1) {
     const uint4* src = x + (size_t)idx[i] * chunks;
     uint4 v[MAXC];
 #pragma unroll
     for (int c = 0; c < MAXC; ++c) {
-      const int cc = c * 32 + lane;
+      const int cc = c * kGatherThreads + tid;
       if (cc < chunks) v[c] = ld_nc_16(src + cc);
     }
     if (xc) {
 #pragma unroll
       for (int c = 0; c < MAXC; ++c) {
-        const int cc = c * 32 + lane;
+        const int cc = c * kGatherThreads + tid;
         if (cc < chunks) st_16(xc + (size_t)i * chunks + cc, v[c]);
       }
     }
@@ -40,7 +44,7 @@ __global__ void __launch_bounds__(kRowThreads)
       float ss = 0.f;
 #pragma unroll
       for (int c = 0; c < MAXC; ++c) {
-        const int cc = c * 32 + lane;
+        const int cc = c * kGatherThreads + tid;
         if (cc < chunks) {
           const uint32_t u[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
 #pragma unroll
@@ -52,10 +56,16 @@ __global__ void __launch_bounds__(kRowThreads)
         }
       }
       ss = warp_sum(ss);
-      const float inv = rsqrtf(ss / (float)d + eps);
+      // partial sums alternate between two slots, so one barrier per row is enough
+      if ((tid & 31) == 0) s_part[par][tid >> 5] = ss;
+      __syncthreads();
+      float tot = 0.f;
+#pragma unroll
+      for (int w = 0; w < kGatherThreads / 32; ++w) tot += s_part[par][w];
+      const float inv = rsqrtf(tot / (float)d + eps);
 #pragma unroll
       for (int c = 0; c < MAXC; ++c) {
-        const int cc = c * 32 + lane;
+        const int cc = c * kGatherThreads + tid;
         if (cc < chunks) {
           const float4 g0 = *reinterpret_cast<const float4*>(gamma + cc * 8);
           const float4 g1 = *reinterpret_cast<const float4*>(gamma + cc * 8 + 4);
@@ -301,18 +311,20 @@ static int launch_compact_t(const void* x, const int32_t* idx, const int32_t* n_
                             int d, const float* gamma, float eps, void* xc, void* hn,
                             cudaStream_t s) {
   const int chunks = d / 8;
-  const int grid = row_grid(8);
+  const int grid = min(cap, row_grid(12));
   auto X = static_cast<const uint4*>(x);
   auto XC = static_cast<uint4*>(xc);
   auto HN = static_cast<uint4*>(hn);
-  if (chunks <= 32 * 4)
-    compact_kernel<4, ACT><<<grid, kRowThreads, 0, s>>>(X, idx, n_exec, cap, d, gamma, eps, XC, HN);
-  else if (chunks <= 32 * 16)
-    compact_kernel<16, ACT><<<grid, kRowThreads, 0, s>>>(X, idx, n_exec, cap, d, gamma, eps, XC, HN);
-  else if (chunks <= 32 * 32)
-    compact_kernel<32, ACT><<<grid, kRowThreads, 0, s>>>(X, idx, n_exec, cap, d, gamma, eps, XC, HN);
-  else
-    return QTALE_ERR_SHAPE;
+#define QTALE_COMPACT(C)                                                                         \
+  compact_kernel<C, ACT><<<grid, kGatherThreads, 0, s>>>(X, idx, n_exec, cap, d, gamma, eps, XC, HN)
+  if (chunks <= kGatherThreads * 1) QTALE_COMPACT(1);
+  else if (chunks <= kGatherThreads * 2) QTALE_COMPACT(2);
+  else if (chunks <= kGatherThreads * 4) QTALE_COMPACT(4);
+  else if (chunks <= kGatherThreads * 5) QTALE_COMPACT(5);
+  else if (chunks <= kGatherThreads * 8) QTALE_COMPACT(8);
+  else if (chunks <= kGatherThreads * 16) QTALE_COMPACT(16);
+  else return QTALE_ERR_SHAPE;
+#undef QTALE_COMPACT
   return launch_status(cudaGetLastError());
 }
 

@@ -41,3 +41,21 @@ def test_single_process_is_a_no_op():
     import bench
     assert bench.max_over_ranks(1.25) == 1.25
     assert bench.aggregate_tokens_per_s(8192, 1, 2.0) == 8192 / 2e-3
+
+
+def test_gpus_flag_starts_one_replica_per_gpu(tmp_path):
+    """`bench.py --gpus N` started as a plain process re-launches itself as N ranks of one
+    node.  The same launcher runs a stand-in script here (gloo, CPU): two processes come up with
+    RANK / WORLD_SIZE set, meet in the barrier, and the job's time is the slower replica's."""
+    sys.path.insert(0, ROOT)
+    import json
+    import bench
+    out = tmp_path / "out.json"
+    cmd = bench.replica_command(2, os.path.join(ROOT, "tests", "replica_stub.py"), [str(out), "--steps", "3"], 29400)
+    assert cmd[1:4] == ["-m", "torch.distributed.run", "--nnodes=1"] and "127.0.0.1" in cmd
+    rc = bench.spawn_replicas(2, os.path.join(ROOT, "tests", "replica_stub.py"), [str(out), "--steps", "3"],
+                              port=29400 + os.getpid() % 500)
+    assert rc == 0
+    res = json.loads(out.read_text())
+    assert res["world"] == 2 and res["ms"] == 3.0 and res["value"] == 2 * 100 / 3e-3
+    assert res["args"] == ["--steps", "3"]
