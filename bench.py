@@ -44,9 +44,10 @@ UNIT = "tokens/s"
 SWEEP = [1.0, 0.9, 0.75, 0.5]
 WORKLOAD = ("c2: 7B-shaped layer (hidden 4096, 32 heads, FFN 11008), int4 g128, "
             "batch 4 x seq 2048 prefill")
-# kernels of this library per layer step (prefill): router/select, gather + norm, QKV GEMM,
-# rotary table, rotary, tail zeroing, attention, O GEMM, RMSNorm, gate/up GEMM, down GEMM
-KERNELS_PER_STEP = 11
+# kernels of this library per layer step (prefill): router/select, gather + norm (+ rotary
+# table), QKV GEMM (+ rotary), attention, O GEMM, RMSNorm, gate/up GEMM (+ SwiGLU), down GEMM
+# (+ residual scatter)
+KERNELS_PER_STEP = 8
 ALL_LEGS = ["sweep", "gemm", "bf16", "router", "gather", "decode", "c4", "c5", "e2e", "cpu"]
 
 
@@ -321,7 +322,8 @@ def timing_weight(torch, api, dev, gen, N, K, bits, group, row_mode=0):
 def timing_layer(torch, api, dev, gen, sh):
     """api.LayerWeights with timing weights (see timing_weight) and a random router."""
     lw = api.LayerWeights.__new__(api.LayerWeights)
-    lw.qkv = timing_weight(torch, api, dev, gen, sh.q_dim + 2 * sh.kv_dim, sh.d, sh.bits, sh.group)
+    lw.qkv = timing_weight(torch, api, dev, gen, sh.q_dim + 2 * sh.kv_dim, sh.d, sh.bits, sh.group,
+                           api.ROWS_ROPE64 if sh.head_dim == 64 else api.ROWS_ROPE128)
     lw.o = timing_weight(torch, api, dev, gen, sh.d, sh.q_dim, sh.bits, sh.group)
     lw.gate_up = timing_weight(torch, api, dev, gen, 2 * sh.ffn, sh.d, sh.bits, sh.group, api.ROWS_SWIGLU)
     lw.down = timing_weight(torch, api, dev, gen, sh.d, sh.ffn, sh.bits, sh.group)
@@ -439,6 +441,7 @@ def run_ours(args):
         a_q = torch.randn(T, qd, device=dev, generator=gen).to(adt)
         a_f = (torch.randn(T, sh.ffn, device=dev, generator=gen) * 0.3).to(adt)
         y_qkv = torch.empty(T, lw.qkv.N, dtype=adt, device=dev)
+        cs_t = torch.rand(T, sh.head_dim // 2, 2, device=dev, generator=gen)
         u = torch.empty(T, sh.d, dtype=torch.float32, device=dev)
         y_act = torch.empty(T, sh.ffn, dtype=adt, device=dev)
         idx = torch.sort(torch.randperm(T, device=dev, generator=gen)[:max(k, 1)])[0].to(torch.int32)
@@ -447,7 +450,7 @@ def run_ours(args):
         x_g = x_src.clone()
 
         def gemms(i):
-            api.wq_gemm(a_d, lw.qkv, m_dev, api.EPI_STORE_16, y=y_qkv)
+            api.wq_gemm(a_d, lw.qkv, m_dev, api.EPI_ROPE, y=y_qkv, rope_cs=cs_t, rope_features=qd + sh.kv_dim)
             api.wq_gemm(a_q, lw.o, m_dev, api.EPI_RESID_F32, y=u, idx=idx_full, resid=x_g)
             api.wq_gemm(a_d, lw.gate_up, m_dev, api.EPI_SWIGLU, y=y_act)
             api.wq_gemm(a_f, lw.down, m_dev, api.EPI_RESID_SCATTER, idx=idx_full, resid=u, dst=x_g)
@@ -457,7 +460,7 @@ def run_ours(args):
         sustained = flops / (g["ms"] * 1e-3) / 1e12
         burst = flops / (g["burst_ms"] * 1e-3) / 1e12
         roofline = dict(bound="tensor", kernel="wq_gemm_pair_kernel<4,1> (the 4 launches of a step, "
-                        "with the layer's epilogues: store, x[idx]+acc, SwiGLU, residual scatter)",
+                        "with the layer's epilogues: rotary, x[idx]+acc, SwiGLU, residual scatter)",
                         achieved=sustained, peak=peaks["bf16_tflops_sustained"], unit="TFLOP/s",
                         frac=sustained / peaks["bf16_tflops_sustained"],
                         peak_source="%s (sustained bf16 matmul; regions repeated for %.1f s)" % (

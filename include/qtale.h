@@ -210,6 +210,9 @@ typedef struct {
 #define QTALE_WQ_ROWS_PLAIN 0  /* output feature n sits in tile n / 128, lane n % 128       */
 #define QTALE_WQ_ROWS_SWIGLU 1 /* W = [gate; up] (N = 2F): each 128-row tile holds 64 gate
                                   rows and the matching 64 up rows, needed by EPI_SWIGLU   */
+#define QTALE_WQ_ROWS_ROPE64 2  /* W = [Wq; Wk; Wv] with heads of 64 / 128 features: inside a  */
+#define QTALE_WQ_ROWS_ROPE128 3 /* tile every feature sits next to its rotary partner half a
+                                  head further (N % head_dim == 0), needed by EPI_ROPE      */
 
 /*
  * Offline repack, HOST pointers.  Input is the interface layout: codes
@@ -229,6 +232,11 @@ int qtale_wq_repack(const uint8_t* codes, const uint16_t* scales, const uint16_t
 #define QTALE_EPI_RESID_SCATTER 3 /* dst[idx[m],n] = bf16(resid_f32[m,n] + acc)    (Eq. 3) */
 #define QTALE_EPI_SWIGLU 4        /* y[m,j] = act_dtype(silu(acc[m,j]) * acc[m,F+j]), N = 2F;
                                      needs QTALE_WQ_ROWS_SWIGLU weights                   */
+#define QTALE_EPI_ROPE 5          /* y[m,:] = act_dtype(acc[m,:]) with the rotary embedding applied
+                                     to the features below rope_features (query and key heads):
+                                     (x_j, x_{j+hd/2}) -> (x_j c - x_{j+hd/2} s, x_{j+hd/2} c + x_j s)
+                                     with (c, s) = rope_cs[m, j]; one rounding of the fp32 result;
+                                     needs QTALE_WQ_ROWS_ROPE* weights                    */
 
 typedef struct {
   const int32_t* idx;    /* [M_cap] row indices (RESID_F32, RESID_SCATTER) */
@@ -237,6 +245,8 @@ typedef struct {
   int ld_resid;          /* elements */
   void* dst;             /* RESID_SCATTER: bf16 [T, ld_dst], rows idx[m] written */
   int ld_dst;
+  const void* rope_cs;   /* ROPE: float2 (cos, sin) [M_cap, head_dim / 2] of each row's position */
+  int rope_features;     /* ROPE: features [0, rope_features) are rotated, a multiple of head_dim */
 } qtale_epilogue_args;
 
 /*

@@ -18,9 +18,9 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libqtale.so")
 
 SELECT_THRESHOLD, SELECT_TOPK, SELECT_FORCED = 0, 1, 2
-EPI_STORE_16, EPI_STORE_F32, EPI_RESID_F32, EPI_RESID_SCATTER, EPI_SWIGLU = 0, 1, 2, 3, 4
+EPI_STORE_16, EPI_STORE_F32, EPI_RESID_F32, EPI_RESID_SCATTER, EPI_SWIGLU, EPI_ROPE = 0, 1, 2, 3, 4, 5
 ACT_BF16, ACT_F16 = 0, 1
-ROWS_PLAIN, ROWS_SWIGLU = 0, 1
+ROWS_PLAIN, ROWS_SWIGLU, ROWS_ROPE64, ROWS_ROPE128 = 0, 1, 2, 3
 PHASE_PREFILL, PHASE_DECODE = 0, 1
 
 EXPORTS = [
@@ -44,7 +44,8 @@ class WqWeight(C.Structure):
 
 class EpilogueArgs(C.Structure):
     _fields_ = [("idx", C.c_void_p), ("resid", C.c_void_p), ("ld_resid", C.c_int),
-                ("dst", C.c_void_p), ("ld_dst", C.c_int)]
+                ("dst", C.c_void_p), ("ld_dst", C.c_int), ("rope_cs", C.c_void_p),
+                ("rope_features", C.c_int)]
 
 
 class LayerConfig(C.Structure):
@@ -273,7 +274,7 @@ class QuantWeight:
 
 
 def wq_gemm(a, w: QuantWeight, m_dev=None, epilogue=EPI_STORE_16, y=None, idx=None, resid=None,
-            dst=None):
+            dst=None, rope_cs=None, rope_features=0):
     """qtale_wq_gemm.  a bf16 or fp16 [M_cap, K] (its dtype is the act_dtype); returns y
     (or dst for RESID_SCATTER)."""
     M_cap, lda = int(a.shape[0]), int(a.stride(0))
@@ -282,10 +283,12 @@ def wq_gemm(a, w: QuantWeight, m_dev=None, epilogue=EPI_STORE_16, y=None, idx=No
     if epilogue in (EPI_RESID_F32, EPI_RESID_SCATTER):
         epi = EpilogueArgs(idx.data_ptr(), resid.data_ptr(), int(resid.stride(0)),
                            dst.data_ptr() if dst is not None else None,
-                           int(dst.stride(0)) if dst is not None else 0)
+                           int(dst.stride(0)) if dst is not None else 0, None, 0)
+    if epilogue == EPI_ROPE:
+        epi = EpilogueArgs(None, None, 0, None, 0, rope_cs.data_ptr(), int(rope_features))
     if y is None and epilogue != EPI_RESID_SCATTER:
         n_out = w.N // 2 if epilogue == EPI_SWIGLU else w.N
-        dt = a.dtype if epilogue in (EPI_STORE_16, EPI_SWIGLU) else torch.float32
+        dt = a.dtype if epilogue in (EPI_STORE_16, EPI_SWIGLU, EPI_ROPE) else torch.float32
         y = torch.zeros(M_cap, n_out, dtype=dt, device=a.device)
     check(lib().qtale_wq_gemm(_ptr(a), lda, _ptr(m_dev), M_cap, C.byref(w.c), act_dtype, int(epilogue),
                               C.byref(epi) if epi is not None else None, _ptr(y),
@@ -307,8 +310,15 @@ def layer_config(sh, select_mode=SELECT_THRESHOLD, theta=0.5, ratio=1.0,
 class LayerWeights:
     """Device-resident weights of one layer (from inputs.layer_weights)."""
 
-    def __init__(self, w: dict, device="cuda", fuse_swiglu=True):
-        self.qkv = QuantWeight(w["qkv"], device)
+    def __init__(self, w: dict, device="cuda", fuse_swiglu=True, fuse_rope=True, head_dim=None):
+        # head_dim is needed for the rotary row layout of the QKV matrix
+        rope_mode = ROWS_PLAIN
+        if fuse_rope:
+            head_dim = head_dim or w.get("head_dim")
+            if head_dim not in (64, 128):
+                raise QtaleError("LayerWeights(fuse_rope=True) needs head_dim (64 or 128)")
+            rope_mode = ROWS_ROPE64 if head_dim == 64 else ROWS_ROPE128
+        self.qkv = QuantWeight(w["qkv"], device, rope_mode)
         self.o = QuantWeight(w["o"], device)
         self.gate_up = QuantWeight(w["gate_up"], device, ROWS_SWIGLU if fuse_swiglu else ROWS_PLAIN)
         self.down = QuantWeight(w["down"], device)

@@ -2,6 +2,8 @@
 // a stack of them, composed from the library's kernels.  Everything between
 // the router and the residual write-back is sized by the device-side executed
 // token count; the host never reads it.
+#include <string.h>
+
 #include "attention.cuh"
 #include "router_select.cuh"
 #include "rowops.cuh"
@@ -112,14 +114,33 @@ static int layer_forward_impl(const qtale_layer_config* c, const qtale_layer_wei
           cudaSuccess)
     return QTALE_ERR_CUDA;
 
-  // 2. gather the executed tokens and apply the first RMSNorm
-  QTALE_TRY(launch_compact(x, idx, ws.n_exec, T, d, w->gamma1, c->rms_eps, act, nullptr, ws.hn, s));
-  // 3. q, k, v projections
-  QTALE_TRY(wq_gemm_launch(ws.hn, d, ws.n_exec, T, &w->qkv, act, QTALE_EPI_STORE_16, nullptr, ws.qkv,
-                           nqkv, s));
-  // 4. rotary embedding at the original positions
-  QTALE_TRY(launch_rope_table(ws.pos, ws.n_exec, T, hd, c->rope_theta, ws.cs, s));
-  QTALE_TRY(launch_rope(ws.qkv, ws.n_exec, T, nqkv, H + Hkv, hd, ws.cs, act, s));
+  // 2. gather the executed tokens and apply the first RMSNorm; the same launch writes the
+  //    rotary table of their (original) positions and, for the prefill attention's tiled loads,
+  //    clears the value columns of the 128 rows after the executed count
+  const bool fused_rope = w->qkv.row_mode != QTALE_WQ_ROWS_PLAIN;
+  GatherExtras gx;
+  gx.pos = ws.pos;
+  gx.cs = reinterpret_cast<float2*>(ws.cs);
+  gx.half = hd / 2;
+  gx.rope_base = c->rope_theta;
+  gx.tail = phase == QTALE_PHASE_DECODE ? nullptr : static_cast<uint4*>(ws.qkv);
+  gx.tail_ld = nqkv;
+  gx.tail_col0 = qd + kvd;
+  gx.tail_cols = kvd;
+  gx.tail_rows = 128;
+  QTALE_TRY(launch_compact(x, idx, ws.n_exec, T, d, w->gamma1, c->rms_eps, act, nullptr, ws.hn, s, &gx));
+  // 3. q, k, v projections, rotary embedding at the original positions in the epilogue
+  if (fused_rope) {
+    qtale_epilogue_args er;
+    memset(&er, 0, sizeof(er));
+    er.rope_cs = ws.cs;
+    er.rope_features = qd + kvd;
+    QTALE_TRY(wq_gemm_launch(ws.hn, d, ws.n_exec, T, &w->qkv, act, QTALE_EPI_ROPE, &er, ws.qkv, nqkv, s));
+  } else {
+    QTALE_TRY(wq_gemm_launch(ws.hn, d, ws.n_exec, T, &w->qkv, act, QTALE_EPI_STORE_16, nullptr, ws.qkv,
+                             nqkv, s));
+    QTALE_TRY(launch_rope(ws.qkv, ws.n_exec, T, nqkv, H + Hkv, hd, ws.cs, act, s));
+  }
   // 5. attention among executed tokens (+ cache)
   if (kv) {
     QTALE_TRY(launch_kv_append(ws.qkv, ws.n_exec, T, nqkv, qd, kvd, ws.cu_exec, B, kv->k, kv->v,
@@ -129,11 +150,11 @@ static int layer_forward_impl(const qtale_layer_config* c, const qtale_layer_wei
     QTALE_TRY(launch_attn_decode(ws.qkv, nqkv, H, Hkv, hd, act, idx, ws.n_exec, T, kv->k, kv->v,
                                  kv->kv_len, kv->cap, ws.ao, qd, s));
   } else {
-    QTALE_TRY(launch_zero_tail_rows(ws.qkv, ws.n_exec, T, nqkv, 128, s));
     QTALE_TRY(launch_attn_prefill(ws.qkv, nqkv, H, Hkv, hd, act, ws.cu_exec, B, T, ws.ao, qd, s));
   }
   // 6. output projection + residual: u = x[idx] + attention branch (fp32)
   qtale_epilogue_args e;
+  memset(&e, 0, sizeof(e));
   e.idx = idx;
   e.resid = x;
   e.ld_resid = d;
@@ -176,8 +197,9 @@ static int check_weights(const qtale_layer_config* c, const qtale_layer_weights*
     if (q->group != c->group) return QTALE_ERR_GROUP;
     if (!aligned16(q->packed)) return QTALE_ERR_ALIGN;
   }
-  if (w->qkv.row_mode != QTALE_WQ_ROWS_PLAIN || w->o.row_mode != QTALE_WQ_ROWS_PLAIN ||
-      w->down.row_mode != QTALE_WQ_ROWS_PLAIN)
+  const int rope_mode = c->head_dim == 64 ? QTALE_WQ_ROWS_ROPE64 : QTALE_WQ_ROWS_ROPE128;
+  if ((w->qkv.row_mode != QTALE_WQ_ROWS_PLAIN && w->qkv.row_mode != rope_mode) ||
+      w->o.row_mode != QTALE_WQ_ROWS_PLAIN || w->down.row_mode != QTALE_WQ_ROWS_PLAIN)
     return QTALE_ERR_MODE;
   return QTALE_OK;
 }

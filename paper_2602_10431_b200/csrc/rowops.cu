@@ -3,6 +3,8 @@
 // append, embedding gather.  All move 16 bytes per thread per access, keep a
 // row's data in registers between the reduction and the write, and read the
 // executed-token count from device memory.
+#include <string.h>
+
 #include "rowops.cuh"
 
 namespace qtale {
@@ -19,14 +21,37 @@ __global__ void __launch_bounds__(kGatherThreads)
     compact_kernel(const uint4* __restrict__ x, const int32_t* __restrict__ idx,
                    const int32_t* __restrict__ n_exec, int cap, int d,
                    const float* __restrict__ gamma, float eps, uint4* __restrict__ xc,
-                   uint4* __restrict__ hn) {
+                   uint4* __restrict__ hn, const GatherExtras ex) {
   __shared__ float s_part[2][kGatherThreads / 32];
   const int tid = threadIdx.x;
   const int n = n_exec ? min(*n_exec, cap) : cap;
   const int chunks = d >> 3;  // 16-byte chunks per row
+  // Riding along (the kernel is bandwidth bound, its arithmetic units idle):
+  //  * the rotary table of the executed tokens, cs[i][j] = (cos, sin)(pos[i] * base^(-2j/hd)) in
+  //    fp64 arithmetic, read by the epilogue of the QKV projection;
+  //  * zeroes in the value columns of the `tail_rows` rows that follow the executed count: the
+  //    attention kernel loads key / value tiles that start at any executed row, so a tile can
+  //    reach that far past the count; masked keys get probability 0, but 0 x NaN is NaN in the
+  //    P V product, so those rows must be finite whatever the workspace held before.
+  double inv_freq = 0.0;
+  if (ex.cs && tid < ex.half) inv_freq = pow((double)ex.rope_base, -(double)tid / (double)ex.half);
+  if (ex.tail) {
+    const int end = min(cap, n + ex.tail_rows);
+    const int cpr = ex.tail_cols >> 3;  // 16-byte chunks per row to clear
+    const int total = max(end - n, 0) * cpr;
+    for (int e = blockIdx.x * kGatherThreads + tid; e < total; e += gridDim.x * kGatherThreads) {
+      const int r = e / cpr, c = e % cpr;
+      ex.tail[(size_t)(n + r) * (ex.tail_ld >> 3) + (ex.tail_col0 >> 3) + c] = make_uint4(0, 0, 0, 0);
+    }
+  }
   int par = 0;
   for (int i = blockIdx.x; i < n; i += gridDim.x, par ^= 1) {
     const uint4* src = x + (size_t)idx[i] * chunks;
+    if (ex.cs && tid < ex.half) {
+      double sn, cn;
+      sincos((double)ex.pos[i] * inv_freq, &sn, &cn);
+      ex.cs[(size_t)i * ex.half + tid] = make_float2((float)cn, (float)sn);
+    }
     uint4 v[MAXC];
 #pragma unroll
     for (int c = 0; c < MAXC; ++c) {
@@ -154,25 +179,10 @@ __global__ void __launch_bounds__(kRowThreads)
   }
 }
 
-// ---- rotary table: cs[i][j] = (cos, sin)(pos[i] * base^(-2j/hd)), fp64 math ----
-__global__ void rope_table_kernel(const int32_t* __restrict__ pos,
-                                  const int32_t* __restrict__ n_exec, int cap, int half,
-                                  float base, float2* __restrict__ cs) {
-  const int n = min(*n_exec, cap);
-  const size_t total = (size_t)n * half;
-  for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < total;
-       e += (size_t)gridDim.x * blockDim.x) {
-    const int i = (int)(e / half), j = (int)(e % half);
-    const double inv_freq = pow((double)base, -(double)j / (double)half);
-    double s, c;
-    sincos((double)pos[i] * inv_freq, &s, &c);
-    cs[e] = make_float2((float)c, (float)s);
-  }
-}
-
 // ---- rotary embedding on the q and k heads of the fused qkv tensor -------------
 // qkv: [n, ld] bf16; heads 0 .. n_rot-1 (q heads then k heads) are rotated in place,
-// pairing element j with j + hd/2.
+// pairing element j with j + hd/2.  Only used when the QKV weights are in the plain row
+// layout; with the rotary layout the rotation happens in the projection's epilogue.
 template <int ACT>
 __global__ void __launch_bounds__(kRowThreads)
     rope_kernel(uint4* __restrict__ qkv, const int32_t* __restrict__ n_exec, int cap, int ld,
@@ -271,22 +281,6 @@ __global__ void kv_len_update_kernel(int32_t* kv_len, const int32_t* cu_exec, in
   }
 }
 
-// ---- zero the `tile` rows that follow the executed count ----
-// The attention kernel loads key / value tiles of `tile` rows that start at any executed row
-// (a sequence's first row plus a multiple of the tile), so a tile can reach up to tile - 1 rows
-// past the count.  Masked keys get probability 0, but 0 x NaN is NaN in the P V product: those
-// rows must hold finite values whatever the workspace held before.
-__global__ void zero_tail_rows_kernel(uint4* __restrict__ buf, const int32_t* __restrict__ n_exec,
-                                      int cap, int ld, int tile) {
-  const int n = min(*n_exec, cap);
-  const int end = min(cap, n + tile);
-  const int ldc = ld >> 3;
-  const size_t total = (size_t)(end - n) * ldc;
-  for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < total;
-       e += (size_t)gridDim.x * blockDim.x)
-    buf[(size_t)n * ldc + e] = make_uint4(0, 0, 0, 0);
-}
-
 // ---- embedding gather ------------------------------------------------------------
 __global__ void __launch_bounds__(kRowThreads)
     embed_kernel(const uint4* __restrict__ embed, const int32_t* __restrict__ ids, int T, int d,
@@ -309,14 +303,14 @@ static int row_grid(int per_sm) { return sm_count() * per_sm; }
 template <int ACT>
 static int launch_compact_t(const void* x, const int32_t* idx, const int32_t* n_exec, int cap,
                             int d, const float* gamma, float eps, void* xc, void* hn,
-                            cudaStream_t s) {
+                            const GatherExtras& ex, cudaStream_t s) {
   const int chunks = d / 8;
   const int grid = min(cap, row_grid(12));
   auto X = static_cast<const uint4*>(x);
   auto XC = static_cast<uint4*>(xc);
   auto HN = static_cast<uint4*>(hn);
 #define QTALE_COMPACT(C)                                                                         \
-  compact_kernel<C, ACT><<<grid, kGatherThreads, 0, s>>>(X, idx, n_exec, cap, d, gamma, eps, XC, HN)
+  compact_kernel<C, ACT><<<grid, kGatherThreads, 0, s>>>(X, idx, n_exec, cap, d, gamma, eps, XC, HN, ex)
   if (chunks <= kGatherThreads * 1) QTALE_COMPACT(1);
   else if (chunks <= kGatherThreads * 2) QTALE_COMPACT(2);
   else if (chunks <= kGatherThreads * 4) QTALE_COMPACT(4);
@@ -329,9 +323,14 @@ static int launch_compact_t(const void* x, const int32_t* idx, const int32_t* n_
 }
 
 int launch_compact(const void* x, const int32_t* idx, const int32_t* n_exec, int cap, int d,
-                   const float* gamma, float eps, int act, void* xc, void* hn, cudaStream_t s) {
-  return act == QTALE_ACT_F16 ? launch_compact_t<1>(x, idx, n_exec, cap, d, gamma, eps, xc, hn, s)
-                              : launch_compact_t<0>(x, idx, n_exec, cap, d, gamma, eps, xc, hn, s);
+                   const float* gamma, float eps, int act, void* xc, void* hn, cudaStream_t s,
+                   const GatherExtras* extras) {
+  GatherExtras ex;
+  memset(&ex, 0, sizeof(ex));
+  if (extras) ex = *extras;
+  if (ex.cs && (ex.half > kGatherThreads || ex.half < 1)) return QTALE_ERR_SHAPE;
+  return act == QTALE_ACT_F16 ? launch_compact_t<1>(x, idx, n_exec, cap, d, gamma, eps, xc, hn, ex, s)
+                              : launch_compact_t<0>(x, idx, n_exec, cap, d, gamma, eps, xc, hn, ex, s);
 }
 
 int launch_scatter_add(void* x, const void* xc, const float* f, const int32_t* idx,
@@ -366,13 +365,6 @@ int launch_rmsnorm_f32(const float* u, const int32_t* n_rows, int cap, int d, co
                               : launch_rmsnorm_f32_t<0>(u, n_rows, cap, d, gamma, eps, out, s);
 }
 
-int launch_rope_table(const int32_t* pos, const int32_t* n_exec, int cap, int hd, float base,
-                      float* cs, cudaStream_t s) {
-  rope_table_kernel<<<row_grid(4), 256, 0, s>>>(pos, n_exec, cap, hd / 2, base,
-                                                reinterpret_cast<float2*>(cs));
-  return launch_status(cudaGetLastError());
-}
-
 int launch_rope(void* qkv, const int32_t* n_exec, int cap, int ld, int n_rot, int hd,
                 const float* cs, int act, cudaStream_t s) {
   if (act == QTALE_ACT_F16)
@@ -403,12 +395,6 @@ int launch_kv_append(const void* qkv, const int32_t* n_exec, int cap_rows, int l
       static_cast<uint4*>(cache_k), static_cast<uint4*>(cache_v), kv_len, cap);
   if (cudaGetLastError() != cudaSuccess) return QTALE_ERR_CUDA;
   kv_len_update_kernel<<<(B + 255) / 256, 256, 0, s>>>(kv_len, cu_exec, B, cap, device_status_ptr());
-  return launch_status(cudaGetLastError());
-}
-
-int launch_zero_tail_rows(void* buf, const int32_t* n_exec, int cap, int ld, int tile,
-                          cudaStream_t s) {
-  zero_tail_rows_kernel<<<64, 256, 0, s>>>(static_cast<uint4*>(buf), n_exec, cap, ld, tile);
   return launch_status(cudaGetLastError());
 }
 

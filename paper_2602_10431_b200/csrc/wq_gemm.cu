@@ -44,6 +44,8 @@ namespace qtale {
 using namespace ptx;
 
 constexpr int kGemmThreads = 640;
+constexpr int kPairThreads = 640;
+constexpr int kPairFirstDq = 4;    // first dequantiser warp of the CTA-pair kernel
 constexpr int kDequantWarps = 16;
 constexpr int kTileRows = 128;           // weight rows per tile (MMA M)
 constexpr int kKB = 64;                  // K elements per pipeline step (128 B of 16-bit data)
@@ -103,6 +105,9 @@ struct GemmParams {
   int ld_resid;
   void* dst;
   int ld_dst;
+  const float2* rope_cs;   // ROPE epilogue: (cos, sin) [M_cap, rope_hd / 2]
+  int rope_hd;             // head dim of the rotary layout (ROPE row modes), else 0
+  int rope_limit;          // output features below this are rotated (query and key heads)
   int* status;
 };
 
@@ -136,6 +141,14 @@ __device__ __forceinline__ int tile_row_to_n(const GemmParams& p, int nt, int L)
     const int j = nt * 64 + q * 16 + (r & 15);
     if (j >= p.F) return -1;
     return (r < 16) ? j : p.F + j;
+  }
+  if (p.rope_hd) {
+    // rotary layout: a lane quadrant holds 16 features of the first half of a head (lanes 0-15)
+    // and their partners half a head further (lanes 16-31)
+    const int q = L >> 5, r = L & 31, half = p.rope_hd >> 1;
+    const int e = q * 16 + (r & 15);
+    const int n = nt * kTileRows + (e / half) * p.rope_hd + (e % half) + (r < 16 ? 0 : half);
+    return n < p.N ? n : -1;
   }
   const int n = nt * kTileRows + L;
   return n < p.N ? n : -1;
@@ -211,75 +224,156 @@ struct Ring {
 // `stage` holds the chunk transposed: stage[m * kEpiRowWords + lane_n] = D[lane_n, m].
 // Each lane then owns 8 consecutive output features of one token row, so global
 // accesses are 16 bytes per lane and 64 or 128 contiguous bytes per row.
-template <int ACT>
+//
+// What an epilogue reads from global memory (residual rows, rotary table, token indices) is
+// fetched by epilogue_fetch into an EpiOperands, separately from epilogue_chunk which uses it,
+// so that a kernel can issue the loads before it waits for the accumulator columns.  (Fetching
+// one whole chunk ahead measured the same: the epilogue is bound by instruction issue.)
+constexpr int kRowGroups = kEpiCols / 8;
+struct EpiOperands {
+  uint4 q[4];            // ROPE: (cos, sin) x 8; RESID_F32: bf16 rows of both row groups (q[0], q[1]);
+                         // RESID_SCATTER: fp32 rows, two 16-byte halves per row group
+  int tok[kRowGroups];   // token index of the lane's row in each row group (RESID epilogues)
+};
+
+// EPI template argument of the epilogue helpers: the epilogue if the kernel is compiled for one
+// (the CTA-pair kernel: the unused branches and their registers disappear), -1 to read p.epilogue
+template <int EPI>
+__device__ __forceinline__ int epilogue_kind(const GemmParams& p) {
+  return EPI >= 0 ? EPI : p.epilogue;
+}
+template <int EPI>
+__device__ __forceinline__ bool epilogue_gathers(const GemmParams& p) {
+  return epilogue_kind<EPI>(p) == QTALE_EPI_RESID_F32 || epilogue_kind<EPI>(p) == QTALE_EPI_RESID_SCATTER;
+}
+// first output feature of the lane's eight in the plain / residual epilogues (-1: padding)
+__device__ __forceinline__ int epilogue_n0(const GemmParams& p, int lane, int nt, int quad) {
+  return tile_row_to_n(p, nt, quad * 32 + (lane & 3) * 8);
+}
+// token indices of the lane's rows of the chunk starting at m0 (RESID epilogues)
+template <int EPI>
+__device__ __forceinline__ void epilogue_fetch_tok(const GemmParams& p, int lane, int m0, int M,
+                                                   EpiOperands& o) {
+  if (!epilogue_gathers<EPI>(p)) return;  // uniform over the warp: the shuffles below need all lanes
+  int my_row = 0;
+  if (lane < kEpiCols && m0 + lane < M) my_row = __ldg(p.idx + m0 + lane);
+#pragma unroll
+  for (int i = 0; i < kRowGroups; ++i) o.tok[i] = __shfl_sync(0xffffffffu, my_row, i * 8 + (lane >> 2));
+}
+// the operands themselves (o.tok must be there already)
+template <int EPI>
+__device__ __forceinline__ void epilogue_fetch(const GemmParams& p, int lane, int nt, int quad, int m0,
+                                               int M, EpiOperands& o) {
+  const int epi = epilogue_kind<EPI>(p);
+  if (epi == QTALE_EPI_ROPE) {
+    const int half = p.rope_hd >> 1;
+    const int e0 = quad * 16 + (lane & 1) * 8;
+    const int f_lo = nt * kTileRows + (e0 / half) * p.rope_hd + (e0 % half);
+    const int m = m0 + (lane >> 1);
+    if (f_lo < p.N && f_lo < p.rope_limit && m < M) {
+      const uint4* t = reinterpret_cast<const uint4*>(p.rope_cs + (size_t)m * half + (e0 % half));
+#pragma unroll
+      for (int e = 0; e < 4; ++e) o.q[e] = __ldg(t + e);  // (c, s) x 8
+    }
+    return;
+  }
+  if (!epilogue_gathers<EPI>(p)) return;
+  const int n0 = epilogue_n0(p, lane, nt, quad);
+  if (n0 < 0) return;
+#pragma unroll
+  for (int i = 0; i < kRowGroups; ++i) {
+    const int m = m0 + i * 8 + (lane >> 2);
+    if (m >= M) continue;
+    if (epi == QTALE_EPI_RESID_F32) {
+      o.q[i] = ld_nc_16(static_cast<const unsigned short*>(p.resid) + (size_t)o.tok[i] * p.ld_resid + n0);
+    } else {
+      const uint4* r = reinterpret_cast<const uint4*>(static_cast<const float*>(p.resid) +
+                                                      (size_t)m * p.ld_resid + n0);
+      o.q[2 * i] = __ldg(r);
+      o.q[2 * i + 1] = __ldg(r + 1);
+    }
+  }
+}
+
+template <int ACT, int EPI>
 __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const float* stage, int lane,
-                                               int nt, int quad, int m0, int M) {
-  if (p.epilogue == QTALE_EPI_SWIGLU) {
+                                               int nt, int quad, int m0, int M, const EpiOperands& o) {
+  const int epi = epilogue_kind<EPI>(p);
+  if (epi == QTALE_EPI_SWIGLU) {
     // lanes n = 0..15 of the chunk are gate rows, n = 16..31 the matching up rows
     const int jc = (lane & 1) * 8;
     const int j0 = nt * 64 + quad * 16 + jc;
     if (j0 >= p.F) return;
-    {
-      const int row = lane >> 1;
-      const int m = m0 + row;
-      if (m >= M) return;
-      const float4 g0 = *reinterpret_cast<const float4*>(stage + row * kEpiRowWords + jc);
-      const float4 g1 = *reinterpret_cast<const float4*>(stage + row * kEpiRowWords + jc + 4);
-      const float4 u0 = *reinterpret_cast<const float4*>(stage + row * kEpiRowWords + 16 + jc);
-      const float4 u1 = *reinterpret_cast<const float4*>(stage + row * kEpiRowWords + 16 + jc + 4);
-      const float g[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
-      const float u[8] = {u0.x, u0.y, u0.z, u0.w, u1.x, u1.y, u1.z, u1.w};
-      uint32_t o[4];
+    const int row = lane >> 1;
+    const int m = m0 + row;
+    if (m >= M) return;
+    const float4 g0 = *reinterpret_cast<const float4*>(stage + row * kEpiRowWords + jc);
+    const float4 g1 = *reinterpret_cast<const float4*>(stage + row * kEpiRowWords + jc + 4);
+    const float4 u0 = *reinterpret_cast<const float4*>(stage + row * kEpiRowWords + 16 + jc);
+    const float4 u1 = *reinterpret_cast<const float4*>(stage + row * kEpiRowWords + 16 + jc + 4);
+    const float g[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+    const float u[8] = {u0.x, u0.y, u0.z, u0.w, u1.x, u1.y, u1.z, u1.w};
+    uint32_t w[4];
 #pragma unroll
-      for (int e = 0; e < 4; ++e)
-        o[e] = Act16<ACT>::pack(g[2 * e] / (1.f + __expf(-g[2 * e])) * u[2 * e],
-                                g[2 * e + 1] / (1.f + __expf(-g[2 * e + 1])) * u[2 * e + 1]);
-      st_16(static_cast<unsigned short*>(p.y) + (size_t)m * p.ldy + j0,
-            make_uint4(o[0], o[1], o[2], o[3]));
+    for (int e = 0; e < 4; ++e)
+      w[e] = Act16<ACT>::pack(g[2 * e] / (1.f + __expf(-g[2 * e])) * u[2 * e],
+                              g[2 * e + 1] / (1.f + __expf(-g[2 * e + 1])) * u[2 * e + 1]);
+    st_16(static_cast<unsigned short*>(p.y) + (size_t)m * p.ldy + j0, make_uint4(w[0], w[1], w[2], w[3]));
+    return;
+  }
+  if (epi == QTALE_EPI_ROPE) {
+    // lanes n = 0..15 of the chunk hold features of the first half of a head, n = 16..31 their
+    // partners: (x1, x2) -> (x1 cos - x2 sin, x2 cos + x1 sin) at the token's position, formed
+    // from the fp32 accumulators and rounded once; value heads are stored as they are
+    const int jc = (lane & 1) * 8;
+    const int half = p.rope_hd >> 1;
+    const int e0 = quad * 16 + jc;
+    const int f_lo = nt * kTileRows + (e0 / half) * p.rope_hd + (e0 % half);
+    const int row = lane >> 1;
+    const int m = m0 + row;
+    if (f_lo >= p.N || m >= M) return;
+    const float4 a0 = *reinterpret_cast<const float4*>(stage + row * kEpiRowWords + jc);
+    const float4 a1 = *reinterpret_cast<const float4*>(stage + row * kEpiRowWords + jc + 4);
+    const float4 b0 = *reinterpret_cast<const float4*>(stage + row * kEpiRowWords + 16 + jc);
+    const float4 b1 = *reinterpret_cast<const float4*>(stage + row * kEpiRowWords + 16 + jc + 4);
+    float x1[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+    float x2[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+    if (f_lo < p.rope_limit) {
+      const uint32_t t[16] = {o.q[0].x, o.q[0].y, o.q[0].z, o.q[0].w, o.q[1].x, o.q[1].y, o.q[1].z, o.q[1].w,
+                              o.q[2].x, o.q[2].y, o.q[2].z, o.q[2].w, o.q[3].x, o.q[3].y, o.q[3].z, o.q[3].w};
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const float c = __uint_as_float(t[2 * e]), sn = __uint_as_float(t[2 * e + 1]);
+        const float u = x1[e], v = x2[e];
+        x1[e] = u * c - v * sn;
+        x2[e] = v * c + u * sn;
+      }
     }
+    unsigned short* y = static_cast<unsigned short*>(p.y) + (size_t)m * p.ldy + f_lo;
+    st_16(y, make_uint4(Act16<ACT>::pack(x1[0], x1[1]), Act16<ACT>::pack(x1[2], x1[3]),
+                        Act16<ACT>::pack(x1[4], x1[5]), Act16<ACT>::pack(x1[6], x1[7])));
+    st_16(y + half, make_uint4(Act16<ACT>::pack(x2[0], x2[1]), Act16<ACT>::pack(x2[2], x2[3]),
+                               Act16<ACT>::pack(x2[4], x2[5]), Act16<ACT>::pack(x2[6], x2[7])));
     return;
   }
   const int nc = (lane & 3) * 8;
-  const int n0 = tile_row_to_n(p, nt, quad * 32 + nc);  // 8 consecutive features, all valid or none
-  const bool n_ok = n0 >= 0;  // no early return: the shuffles below need the whole warp
-  const bool gathers = p.epilogue == QTALE_EPI_RESID_F32 || p.epilogue == QTALE_EPI_RESID_SCATTER;
-  int my_row = 0;
-  if (gathers && lane < kEpiCols && m0 + lane < M) my_row = __ldg(p.idx + m0 + lane);
-  // residual operands of both row groups are requested before the first use
-  constexpr int kRowGroups = kEpiCols / 8;
-  uint4 rb[kRowGroups];
-  float4 rf[kRowGroups][2];
-  int tok[kRowGroups];
+  const int n0 = epilogue_n0(p, lane, nt, quad);  // 8 consecutive features, all valid or none
+  if (n0 < 0) return;
 #pragma unroll
   for (int i = 0; i < kRowGroups; ++i) {
     const int row = i * 8 + (lane >> 2);
     const int m = m0 + row;
-    tok[i] = __shfl_sync(0xffffffffu, my_row, row);
-    if (m < M && n_ok) {
-      if (p.epilogue == QTALE_EPI_RESID_F32) {
-        rb[i] = ld_nc_16(static_cast<const unsigned short*>(p.resid) + (size_t)tok[i] * p.ld_resid + n0);
-      } else if (p.epilogue == QTALE_EPI_RESID_SCATTER) {
-        const float* r = static_cast<const float*>(p.resid) + (size_t)m * p.ld_resid + n0;
-        rf[i][0] = __ldg(reinterpret_cast<const float4*>(r));
-        rf[i][1] = __ldg(reinterpret_cast<const float4*>(r) + 1);
-      }
-    }
-  }
-#pragma unroll
-  for (int i = 0; i < kRowGroups; ++i) {
-    const int row = i * 8 + (lane >> 2);
-    const int m = m0 + row;
-    if (m >= M || !n_ok) continue;
+    if (m >= M) continue;
     const float4 a0 = *reinterpret_cast<const float4*>(stage + row * kEpiRowWords + nc);
     const float4 a1 = *reinterpret_cast<const float4*>(stage + row * kEpiRowWords + nc + 4);
     float v[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
-    if (p.epilogue == QTALE_EPI_STORE_16) {
+    if (epi == QTALE_EPI_STORE_16) {
       st_16(static_cast<unsigned short*>(p.y) + (size_t)m * p.ldy + n0,
             make_uint4(Act16<ACT>::pack(v[0], v[1]), Act16<ACT>::pack(v[2], v[3]),
                        Act16<ACT>::pack(v[4], v[5]), Act16<ACT>::pack(v[6], v[7])));
-    } else if (p.epilogue == QTALE_EPI_STORE_F32 || p.epilogue == QTALE_EPI_RESID_F32) {
-      if (p.epilogue == QTALE_EPI_RESID_F32) {
-        const uint32_t w[4] = {rb[i].x, rb[i].y, rb[i].z, rb[i].w};
+    } else if (epi == QTALE_EPI_STORE_F32 || epi == QTALE_EPI_RESID_F32) {
+      if (epi == QTALE_EPI_RESID_F32) {
+        const uint32_t w[4] = {o.q[i].x, o.q[i].y, o.q[i].z, o.q[i].w};
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
           v[2 * e] += bf16_lo(w[e]);
@@ -292,9 +386,11 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const float*
       st_16(y + 4, make_uint4(__float_as_uint(v[4]), __float_as_uint(v[5]), __float_as_uint(v[6]),
                               __float_as_uint(v[7])));
     } else {  // QTALE_EPI_RESID_SCATTER: x[idx[m]] = bf16(u + acc)   (Eq. 3)
-      const float r[8] = {rf[i][0].x, rf[i][0].y, rf[i][0].z, rf[i][0].w,
-                          rf[i][1].x, rf[i][1].y, rf[i][1].z, rf[i][1].w};
-      st_16(static_cast<unsigned short*>(p.dst) + (size_t)tok[i] * p.ld_dst + n0,
+      const uint4 r0 = o.q[2 * i], r1 = o.q[2 * i + 1];
+      const float r[8] = {__uint_as_float(r0.x), __uint_as_float(r0.y), __uint_as_float(r0.z),
+                          __uint_as_float(r0.w), __uint_as_float(r1.x), __uint_as_float(r1.y),
+                          __uint_as_float(r1.z), __uint_as_float(r1.w)};
+      st_16(static_cast<unsigned short*>(p.dst) + (size_t)o.tok[i] * p.ld_dst + n0,
             make_uint4(pack_bf16x2(v[0] + r[0], v[1] + r[1]), pack_bf16x2(v[2] + r[2], v[3] + r[3]),
                        pack_bf16x2(v[4] + r[4], v[5] + r[5]), pack_bf16x2(v[6] + r[6], v[7] + r[7])));
     }
@@ -582,7 +678,10 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
           __syncwarp();
           // the next chunk's accumulator read overlaps this chunk's global traffic
           if (c0 + 2 * kEpiCols < TW && m0 + 2 * kEpiCols < M) tmem_ld_x16(d_taddr + c0 + 2 * kEpiCols, r);
-          epilogue_chunk<ACT>(p, stage, lane, nt, quad, m0, M);
+          EpiOperands eo;
+          epilogue_fetch_tok<-1>(p, lane, m0, M, eo);
+          epilogue_fetch<-1>(p, lane, nt, quad, m0, M, eo);
+          epilogue_chunk<ACT, -1>(p, stage, lane, nt, quad, m0, M, eo);
           __syncwarp();
         }
         tmem_wait_ld();
@@ -679,8 +778,8 @@ __device__ __forceinline__ bool pair_wait(uint64_t* bar, uint32_t parity, PairSh
   return false;
 }
 
-template <int BITS, int ACT>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
+template <int BITS, int ACT, int EPI>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
     wq_gemm_pair_kernel(const __grid_constant__ PairTmapSet tmaps_x, const GemmParams p) {
   using Cfg = PairCfg<BITS>;
   constexpr int S = kPairStages;
@@ -826,12 +925,14 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
       }
     mma_done:;
     }
-  } else if (warp >= 4) {
+  } else if (warp >= kPairFirstDq) {
     // ---------------- dequantisers, then epilogue ----------------
+    // (a warp reaches the tensor-memory lanes 32 (warp % 4) .. + 31; any four consecutive warps
+    // cover the four quadrants)
     const int quad = warp & 3;
     const int L = quad * 32 + lane;
-    const int set = (warp - 4) >> 2;
-    float* stage = epi_base + (size_t)(warp - 4) * (kEpiWarpBytes / 4);
+    const int set = (warp - kPairFirstDq) >> 2;
+    float* stage = epi_base + (size_t)(warp - kPairFirstDq) * (kEpiWarpBytes / 4);
     const uint32_t ready_leader = map_to_cta(smem_u32(&sh.ready[0]), 0);
     const uint32_t d_empty_leader = map_to_cta(smem_u32(&sh.d_empty), 0);
     const uint32_t a_taddr0 =
@@ -941,12 +1042,16 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
         for (int c0 = set * kEpiCols; c0 < TW; c0 += 4 * kEpiCols) {
           const int m0 = m_base + c0;
           if (m0 >= M) break;
+          // what the chunk reads from global memory is requested before the wait for its accumulator columns
+          EpiOperands eo;
+          epilogue_fetch_tok<EPI>(p, lane, m0, M, eo);
+          epilogue_fetch<EPI>(p, lane, nt, quad, m0, M, eo);
           tmem_wait_ld();
 #pragma unroll
           for (int c = 0; c < kEpiCols; ++c) stage[c * kEpiRowWords + lane] = __uint_as_float(r[c]);
           __syncwarp();
           if (c0 + 4 * kEpiCols < TW && m0 + 4 * kEpiCols < M) tmem_ld_x16(d_taddr + c0 + 4 * kEpiCols, r);
-          epilogue_chunk<ACT>(p, stage, lane, nt, quad, m0, M);
+          epilogue_chunk<ACT, EPI>(p, stage, lane, nt, quad, m0, M, eo);
           __syncwarp();
         }
         tmem_wait_ld();
@@ -1206,9 +1311,13 @@ __global__ void __launch_bounds__(kSmallThreads, 2)
   for (int unit = warp; unit < Cfg::kQuads * (kSmallTokens / kEpiCols); unit += kSmallMmaWarps) {
     const int ql = unit % Cfg::kQuads, chunk = unit / Cfg::kQuads;
     const int m0 = chunk * kEpiCols;
-    if (m0 < M)
-      epilogue_chunk<ACT>(p, out + (ql * kSmallTokens + m0) * kEpiRowWords, lane, nt,
-                          slice * Cfg::kQuads + ql, m0, M);
+    if (m0 < M) {
+      EpiOperands eo;
+      epilogue_fetch_tok<-1>(p, lane, m0, M, eo);
+      epilogue_fetch<-1>(p, lane, nt, slice * Cfg::kQuads + ql, m0, M, eo);
+      epilogue_chunk<ACT, -1>(p, out + (ql * kSmallTokens + m0) * kEpiRowWords, lane, nt,
+                          slice * Cfg::kQuads + ql, m0, M, eo);
+    }
   }
 }
 
@@ -1290,22 +1399,22 @@ static int dispatch_tn(const TmapSet& tx, const CUtensorMap& tw, const GemmParam
 }
 
 // ---- CTA-pair kernel ----
-template <int BITS, int ACT>
-static int launch_pair(const PairTmapSet& tx, const GemmParams& p, cudaStream_t s) {
+template <int BITS, int ACT, int EPI>
+static int launch_pair_epi(const PairTmapSet& tx, const GemmParams& p, cudaStream_t s) {
   using Cfg = PairCfg<BITS>;
   static int clusters_of_device[64] = {0};
   int dev = 0;
   cudaGetDevice(&dev);
   if (dev < 0 || dev >= 64) return QTALE_ERR_CUDA;
   if (clusters_of_device[dev] == 0) {
-    if (cudaFuncSetAttribute(wq_gemm_pair_kernel<BITS, ACT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    if (cudaFuncSetAttribute(wq_gemm_pair_kernel<BITS, ACT, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)Cfg::kSmemBytes) != cudaSuccess)
       return QTALE_ERR_CUDA;
     // how many CTA pairs the device can hold at once: the persistent grid is sized to it
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3((unsigned)sm_count() & ~1u);
-    cfg.blockDim = dim3(kGemmThreads);
+    cfg.blockDim = dim3(kPairThreads);
     cfg.dynamicSmemBytes = Cfg::kSmemBytes;
     cudaLaunchAttribute attr;
     attr.id = cudaLaunchAttributeClusterDimension;
@@ -1315,7 +1424,7 @@ static int launch_pair(const PairTmapSet& tx, const GemmParams& p, cudaStream_t 
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, wq_gemm_pair_kernel<BITS, ACT>, &cfg) != cudaSuccess || n < 1) {
+    if (cudaOccupancyMaxActiveClusters(&n, wq_gemm_pair_kernel<BITS, ACT, EPI>, &cfg) != cudaSuccess || n < 1) {
       cudaGetLastError();
       n = sm_count() / 2;
     }
@@ -1325,8 +1434,22 @@ static int launch_pair(const PairTmapSet& tx, const GemmParams& p, cudaStream_t 
   int clusters = clusters_of_device[dev];
   if (clusters > max_tiles) clusters = max_tiles;
   if (clusters < 1) clusters = 1;
-  wq_gemm_pair_kernel<BITS, ACT><<<2 * clusters, kGemmThreads, Cfg::kSmemBytes, s>>>(tx, p);
+  wq_gemm_pair_kernel<BITS, ACT, EPI><<<2 * clusters, kPairThreads, Cfg::kSmemBytes, s>>>(tx, p);
   return launch_status(cudaGetLastError());
+}
+
+// one instantiation per epilogue: each carries only its own epilogue code and registers
+template <int BITS, int ACT>
+static int launch_pair(const PairTmapSet& tx, const GemmParams& p, cudaStream_t s) {
+  switch (p.epilogue) {
+    case QTALE_EPI_STORE_16: return launch_pair_epi<BITS, ACT, QTALE_EPI_STORE_16>(tx, p, s);
+    case QTALE_EPI_STORE_F32: return launch_pair_epi<BITS, ACT, QTALE_EPI_STORE_F32>(tx, p, s);
+    case QTALE_EPI_RESID_F32: return launch_pair_epi<BITS, ACT, QTALE_EPI_RESID_F32>(tx, p, s);
+    case QTALE_EPI_RESID_SCATTER: return launch_pair_epi<BITS, ACT, QTALE_EPI_RESID_SCATTER>(tx, p, s);
+    case QTALE_EPI_SWIGLU: return launch_pair_epi<BITS, ACT, QTALE_EPI_SWIGLU>(tx, p, s);
+    case QTALE_EPI_ROPE: return launch_pair_epi<BITS, ACT, QTALE_EPI_ROPE>(tx, p, s);
+  }
+  return QTALE_ERR_MODE;
 }
 
 static int make_pair_tmaps(PairTmapSet* set, const void* base, int rows, int cols, int ld, int act) {
@@ -1414,6 +1537,11 @@ int wq_gemm_launch(const void* a, int lda, const int32_t* m_dev, int M_cap,
     p.dst = epi->dst;
     p.ld_dst = epi->ld_dst;
   }
+  p.rope_hd = w->row_mode == QTALE_WQ_ROWS_ROPE64 ? 64 : (w->row_mode == QTALE_WQ_ROWS_ROPE128 ? 128 : 0);
+  if (epilogue == QTALE_EPI_ROPE) {
+    p.rope_cs = static_cast<const float2*>(epi->rope_cs);
+    p.rope_limit = epi->rope_features;
+  }
   p.status = device_status_ptr();
   if (M_cap >= kPairMinTokens) {
     PairTmapSet px;
@@ -1497,8 +1625,10 @@ int qtale_wq_repack(const uint8_t* codes, const uint16_t* scales, const uint16_t
   if (bits != 3 && bits != 4) return QTALE_ERR_BITS;
   if (group != 64 && group != 128) return QTALE_ERR_GROUP;
   if (N < 1 || K < 1) return QTALE_ERR_SHAPE;
-  if (row_mode != QTALE_WQ_ROWS_PLAIN && row_mode != QTALE_WQ_ROWS_SWIGLU) return QTALE_ERR_MODE;
+  if (row_mode < QTALE_WQ_ROWS_PLAIN || row_mode > QTALE_WQ_ROWS_ROPE128) return QTALE_ERR_MODE;
   if (row_mode == QTALE_WQ_ROWS_SWIGLU && (N % 2) != 0) return QTALE_ERR_SHAPE;
+  if (row_mode == QTALE_WQ_ROWS_ROPE64 && (N % 64) != 0) return QTALE_ERR_SHAPE;
+  if (row_mode == QTALE_WQ_ROWS_ROPE128 && (N % 128) != 0) return QTALE_ERR_SHAPE;
   WqGeometry g;
   const size_t total = wq_blob_bytes(N, K, bits, group, row_mode, &g);
   if (!packed_out) {
@@ -1520,6 +1650,12 @@ int qtale_wq_repack(const uint8_t* codes, const uint16_t* scales, const uint16_t
         const int q = L >> 5, r = L & 31;
         const int j = nt * 64 + q * 16 + (r & 15);
         n = (j < F) ? ((r < 16) ? j : F + j) : -1;
+      } else if (row_mode == QTALE_WQ_ROWS_ROPE64 || row_mode == QTALE_WQ_ROWS_ROPE128) {
+        const int hd = row_mode == QTALE_WQ_ROWS_ROPE64 ? 64 : 128, half = hd / 2;
+        const int q = L >> 5, r = L & 31;
+        const int e = q * 16 + (r & 15);
+        n = nt * kTileRows + (e / half) * hd + (e % half) + (r < 16 ? 0 : half);
+        if (n >= N) n = -1;
       } else {
         n = nt * kTileRows + L;
         if (n >= N) n = -1;
@@ -1597,8 +1733,16 @@ int qtale_wq_gemm(const void* a, int lda, const int32_t* m_dev, int M_cap, const
   if (w->bits != 3 && w->bits != 4) return QTALE_ERR_BITS;
   if (w->group != 64 && w->group != 128) return QTALE_ERR_GROUP;
   if (M_cap < 1 || w->N < 1 || w->K < 1 || lda < w->K) return QTALE_ERR_SHAPE;
-  if (epilogue < QTALE_EPI_STORE_16 || epilogue > QTALE_EPI_SWIGLU) return QTALE_ERR_MODE;
+  if (epilogue < QTALE_EPI_STORE_16 || epilogue > QTALE_EPI_ROPE) return QTALE_ERR_MODE;
   if (epilogue == QTALE_EPI_SWIGLU && w->row_mode != QTALE_WQ_ROWS_SWIGLU) return QTALE_ERR_MODE;
+  if (epilogue == QTALE_EPI_ROPE) {
+    if (w->row_mode != QTALE_WQ_ROWS_ROPE64 && w->row_mode != QTALE_WQ_ROWS_ROPE128) return QTALE_ERR_MODE;
+    if (!epi || !epi->rope_cs) return QTALE_ERR_NULL;
+    const int hd = w->row_mode == QTALE_WQ_ROWS_ROPE64 ? 64 : 128;
+    if (epi->rope_features < 0 || epi->rope_features > w->N || epi->rope_features % hd != 0)
+      return QTALE_ERR_SHAPE;
+    if (!aligned16(epi->rope_cs)) return QTALE_ERR_ALIGN;
+  }
   if (epilogue == QTALE_EPI_RESID_F32 || epilogue == QTALE_EPI_RESID_SCATTER) {
     if (!epi || !epi->idx || !epi->resid) return QTALE_ERR_NULL;
     if (epilogue == QTALE_EPI_RESID_SCATTER && !epi->dst) return QTALE_ERR_NULL;

@@ -264,6 +264,7 @@ def layer_weights(seed: int, layer: int, sh: LayerShape):
         "gamma2": np.ones(d, dtype=np.float32),
         "router_w": round_bf16((normal(seed, b + 4, d) * 0.02).astype(np.float32)),
         "router_b": 0.0,
+        "head_dim": sh.head_dim,
     }
     return w
 

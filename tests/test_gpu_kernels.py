@@ -296,6 +296,41 @@ def test_wq_gemm_epilogues(env, act):
     assert api.device_status() == 0
 
 
+@pytest.mark.parametrize("hd,H,Hkv,M,m_dev", [(128, 3, 1, 200, 177), (64, 3, 2, 40, None), (64, 4, 1, 300, 299)])
+@pytest.mark.parametrize("act", [0, 1])
+def test_wq_gemm_rotary_epilogue(env, hd, H, Hkv, M, m_dev, act):
+    """QKV projection with the rotary embedding applied in the epilogue (query and key heads
+    rotated at each row's position, value heads stored as they are), against the oracle's
+    linear + rope.  Covers both head sizes, a head count that leaves half a row tile empty and
+    all three GEMM kernels (CTA pair, single CTA, small-M)."""
+    api, torch, dev = env
+    d, bits, group, base = 256, 4, 64, 10000.0
+    N = (H + 2 * Hkv) * hd
+    a = inputs.activations(50 + hd, 11, M, d)
+    wq = inputs.quantized_weight(51 + hd, 12, N, d, bits, group)
+    w_hat = round_act(oracle.dequantize_weight(wq), act)
+    mm = M if m_dev is None else m_dev
+    pos = inputs.integers(52, 1, M, 5000)
+    j = np.arange(hd // 2, dtype=np.float64)
+    ang = pos[:, None].astype(np.float64) * base ** (-j / (hd // 2))
+    cs = np.stack([np.cos(ang), np.sin(ang)], axis=-1).astype(np.float32)        # the table is an input here
+    y_ref = oracle.linear(a[:mm], w_hat)
+    qk = oracle.rope(y_ref[:, :(H + Hkv) * hd], H + Hkv, hd, pos[:mm], base)
+    ref = np.concatenate([qk, y_ref[:, (H + Hkv) * hd:]], axis=1)
+    qw = api.QuantWeight(wq, dev, api.ROWS_ROPE64 if hd == 64 else api.ROWS_ROPE128)
+    md = None if m_dev is None else torch.tensor([m_dev], dtype=torch.int32, device=dev)
+    y = api.wq_gemm(api.to_device_act(a, act, dev), qw, md, api.EPI_ROPE,
+                    rope_cs=torch.from_numpy(cs).to(dev), rope_features=(H + Hkv) * hd)
+    assert api.device_status() == 0
+    got = api.to_host_f32(y)
+    assert got.shape == (M, N) and not got[mm:].any()
+    # fp32 rotation of fp32 accumulators, one rounding to the activation format
+    assert np.all(np.abs(got[:mm] - ref) <= np.abs(ref) * 2 * act_eps(act) + 2e-4 * max(1.0, np.abs(ref).max()))
+    # the plain epilogue on the same (permuted) weights still gives the logical column order
+    plain = api.wq_gemm(api.to_device_act(a, act, dev), qw, md, api.EPI_STORE_F32).cpu().numpy()
+    assert np.abs(plain[:mm] - y_ref).max() <= 1e-4 * max(1.0, np.abs(y_ref).max())
+
+
 def test_wq_gemm_full_size_sampled(env):
     """7B-sized gate/up projection in the launch configuration the benchmark times
     (8192-token capacity, device-side count): 66 complete output rows, two from every 256-token

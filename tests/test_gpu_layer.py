@@ -41,7 +41,7 @@ class Case:
         self.w["gamma2"] = (1 + 0.1 * inputs.normal(seed, 91, sh.d)).astype(np.float32)
         self.x = inputs.hidden_states(seed, self.T, sh.d)
         self.layer = oracle.DenseLayer(sh, self.w)
-        self.lw = api.LayerWeights(self.w, dev, fuse_swiglu=fuse)
+        self.lw = api.LayerWeights(self.w, dev, fuse_swiglu=fuse, fuse_rope=fuse)
         self.cud = torch.from_numpy(self.cu).to(dev)
 
     def cfg(self, mode, act=1, **kw):
@@ -104,7 +104,9 @@ def test_ratio_zero_identity_and_ratio_one_dense(env):
     ("gqa_hd128", inputs.LayerShape(512, 4, 2, 128, 1024, 4, 128), 3, 300, 0.6, True),
     ("int3_hd128", inputs.LayerShape(512, 4, 4, 128, 1024, 3, 128), 2, 256, 0.7, True),
     ("many_query_tiles_hd128", inputs.LayerShape(256, 2, 2, 128, 512, 4, 128), 4, 700, 0.9, True),
-    ("unfused_swiglu", inputs.LayerShape(256, 4, 4, 64, 688, 4, 64), 2, 128, 0.5, False),
+    ("unfused_swiglu_rope", inputs.LayerShape(256, 4, 4, 64, 688, 4, 64), 2, 128, 0.5, False),
+    ("unfused_hd128_gqa", inputs.LayerShape(512, 4, 2, 128, 1024, 4, 128), 3, 200, 0.6, False),
+    ("odd_heads_hd64", inputs.LayerShape(192, 3, 1, 64, 512, 4, 64), 3, 150, 0.7, True),
     ("one_token_sequences", inputs.LayerShape(256, 4, 1, 64, 512, 4, 128), 40, 1, 0.5, True),
 ])
 @pytest.mark.parametrize("act", [0, 1])
