@@ -663,6 +663,29 @@ def run_ours(args):
             achieved_tflops=fl / (r["ms"] * 1e-3) / 1e12,
             frac_of_sustained_bf16=fl / (r["ms"] * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
             weights="random codes (seeded, device side), distinct per layer", clocks=r["clocks"])
+        # (ii) the paper's mechanism: ONE global theta for all layers, found for R_avg = 0.75 by
+        # the ratio-targeted search (untimed), then the same prefill in threshold mode
+        from paper_2602_10431_b200 import calibrate
+        theta, r_avg, hist = calibrate.calibrate_model_theta(api, mcfg, layers, embed, ids, cu4, mws, hidden,
+                                                             0.75)
+        mcfg.layer.select_mode = api.SELECT_THRESHOLD
+        mcfg.layer.theta = float(theta)
+
+        def tstep(i):
+            api.model_prefill(mcfg, layers, embed, ids, cu4, mws, hidden, final_gamma=fg, lm_head=lm_head,
+                              logit_rows=rows, logits_out=logits, per_layer_n_exec=per_layer)
+
+        r = timer.run(tstep, 3, 2, 0.5)
+        check_status()
+        n4 = per_layer.cpu().tolist()
+        fl = sum(accounting.layer_flops(s4, [S4] * B4, n / T4) for n in n4) + 2.0 * s4.d * V4 * B4
+        extra["c4_model_prefill_global_theta"] = dict(
+            ms_per_step=r["ms"], tokens_per_s=T4 / (r["ms"] * 1e-3), theta=theta, r_avg=sum(n4) / (L4 * T4),
+            search_runs=len(hist), executed_per_layer_min_max=[min(n4), max(n4)],
+            achieved_tflops=fl / (r["ms"] * 1e-3) / 1e12,
+            frac_of_sustained_bf16=fl / (r["ms"] * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
+            select="one global theta for all layers (Eq. 9), found on the device for R_avg 0.75",
+            clocks=r["clocks"])
         del layers, embed, lm_head, mws, hidden, logits
 
     # ---- c5: 13B-shaped 8-layer stack, 16 x 4096 tokens, per-layer ratios from U[0.4, 1.0],

@@ -159,6 +159,25 @@ int qtale_router_select_static(const void* x, int T, int d, const float* w_route
                                int32_t* n_exec_out, int32_t* cu_exec_out, int32_t* pos_out,
                                void* stream);
 
+/*
+ * Threshold for a requested execution ratio (Sec. 3.4, Eq. 9: one global theta
+ * controls the ratio after training; App. A.1 searches it on a grid).  Given
+ * the router scores of a calibration batch pooled over all layers, returns the
+ * theta for which the share of valid scores with score >= theta is `ratio`:
+ * theta = the k-th largest valid score, k = floor(ratio * n_valid + 0.5) (the
+ * exact quantile, no histogram approximation); k = 0 gives theta = 2 (above
+ * every probability).  *count_out = number of valid scores >= theta (k, or more
+ * when scores tie at theta).  The accuracy-driven half of the paper's search
+ * needs task data and is not part of this library.
+ *   scores [n] fp32 device; valid [n] uint8 or NULL; theta_out [1] fp32 and
+ *   count_out [1] int32 on the device; ws of qtale_theta_workspace_bytes().
+ * Limits: 1 <= n <= 2^31, 0 <= ratio <= 1, scores must not be NaN.
+ */
+size_t qtale_theta_workspace_bytes(void);
+int qtale_theta_for_ratio(const float* scores, const uint8_t* valid, size_t n, double ratio,
+                          float* theta_out, int32_t* count_out, void* ws, size_t ws_bytes,
+                          void* stream);
+
 /* Bookkeeping for a caller-supplied ascending index list (QTALE_SELECT_FORCED):
  * fills n_exec_out, cu_exec_out and pos_out as qtale_router_select does.
  * idx [n] int32 device, 0 <= n <= T. */
@@ -355,14 +374,16 @@ size_t qtale_model_workspace_bytes(const qtale_model_config* cfg, int T_cap, int
  *   ids [T] int32; valid [T] uint8 or NULL (0 = padding token, never executed
  *   at any layer, App. B.2); hidden_out [T, d] bf16 (final residual stream);
  *   logits_out fp32 [n_logit_rows, vocab] or NULL; logit_rows [n_logit_rows]
- *   int32 device; per_layer_n_exec [n_layers] int32 device.
+ *   int32 device; per_layer_n_exec [n_layers] int32 device; layer_scores_out
+ *   fp32 [n_layers, T] or NULL: every layer's router scores (the input of
+ *   qtale_theta_for_ratio when theta is calibrated for a ratio).
  */
 int qtale_model_prefill(const qtale_model_config* cfg, const qtale_model_weights* w,
                         const int32_t* ids, int T, const int32_t* cu_seqlens, int B,
                         const uint8_t* valid,
                         const float* per_layer_ratio, void* hidden_out, float* logits_out,
                         const int32_t* logit_rows, int n_logit_rows, int32_t* per_layer_n_exec,
-                        void* ws, size_t ws_bytes, void* stream);
+                        float* layer_scores_out, void* ws, size_t ws_bytes, void* stream);
 
 #ifdef __cplusplus
 }

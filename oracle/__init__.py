@@ -46,6 +46,9 @@ def lib():
         _lib.orc_layer_forward.restype = C.c_int
         _lib.orc_get_threads.restype = C.c_int
         _lib.orc_row_bytes.restype = C.c_int
+        _lib.orc_theta_for_ratio.restype = C.c_float
+        _lib.orc_theta_for_ratio.argtypes = [C.POINTER(C.c_float), C.POINTER(C.c_uint8), C.c_long,
+                                             C.c_double, C.POINTER(C.c_long)]
         set_threads(os.cpu_count() or 1)
     return _lib
 
@@ -126,6 +129,15 @@ def select_topk(p, k, valid=None):
     m = np.empty(p.shape[0], dtype=np.uint8)
     lib().orc_select_topk(_p(p, C.c_float), _p(v, C.c_uint8), p.shape[0], int(k), _p(m, C.c_uint8))
     return m
+
+
+def theta_for_ratio(p, ratio, valid=None):
+    """Global threshold for a requested execution ratio (Sec. 3.4): returns (theta, count)."""
+    p = _f32(p).reshape(-1)
+    v = None if valid is None else _u8(valid).reshape(-1)
+    c = C.c_long(0)
+    th = lib().orc_theta_for_ratio(_p(p, C.c_float), _p(v, C.c_uint8), p.shape[0], float(ratio), C.byref(c))
+    return float(th), int(c.value)
 
 
 def compact_indices(mask, cu_seqlens):
@@ -333,16 +345,18 @@ def route(layer: DenseLayer, x, mode, theta=0.5, ratio=None, valid=None):
 
 
 def model_prefill(layers, embed, ids, cu_seqlens, theta=None, ratios=None, final_gamma=None,
-                  lm_head=None, logit_rows=None, eps=1e-5):
+                  lm_head=None, logit_rows=None, eps=1e-5, valid=None, scores_out=None):
     """Embedding gather, L token-adaptive layers sharing one theta (or per-layer
     top-k ratios), final RMSNorm, LM head on the requested rows."""
     x = _f32(embed)[np.asarray(ids, dtype=np.int64)]
     counts = []
     for li, layer in enumerate(layers):
         if ratios is not None:
-            _, m = route(layer, x, "topk", ratio=ratios[li])
+            p, m = route(layer, x, "topk", ratio=ratios[li], valid=valid)
         else:
-            _, m = route(layer, x, "threshold", theta=theta)
+            p, m = route(layer, x, "threshold", theta=theta, valid=valid)
+        if scores_out is not None:
+            scores_out.append(p)
         x, n = layer_forward(layer, x, cu_seqlens, m)
         counts.append(n)
     logits = None

@@ -161,6 +161,38 @@ void orc_select_topk(const float* p, const uint8_t* valid, int T, int k, uint8_t
   }
 }
 
+/* Threshold for a requested execution ratio (Sec. 3.4: one global theta sets the
+ * ratio after training; lowering it executes more).  Given pooled router scores
+ * of a calibration batch, the theta for which a share `ratio` of the valid
+ * scores satisfies p >= theta (Eq. 9) is the k-th largest valid score with
+ * k = floor(ratio * n_valid + 0.5): written out as a full descending sort.
+ * k = 0: theta = 2, above every probability.  Returns theta, *count = number of
+ * valid scores >= theta (more than k only when scores tie at theta). */
+static int cmp_float_desc(const void* a, const void* b) {
+  const float x = *(const float*)a, y = *(const float*)b;
+  return (x < y) - (x > y);
+}
+float orc_theta_for_ratio(const float* p, const uint8_t* valid, long n, double ratio, long* count) {
+  float* v = (float*)malloc(sizeof(float) * (size_t)(n > 0 ? n : 1));
+  long nv = 0;
+  for (long i = 0; i < n; ++i)
+    if (!valid || valid[i]) v[nv++] = p[i];
+  double kd = floor(ratio * (double)nv + 0.5);
+  if (kd < 0) kd = 0;
+  if (kd > (double)nv) kd = (double)nv;
+  const long k = (long)kd;
+  float theta = 2.0f;
+  long c = 0;
+  if (k > 0) {
+    qsort(v, (size_t)nv, sizeof(float), cmp_float_desc);
+    theta = v[k - 1];
+    for (long i = 0; i < nv; ++i) c += v[i] >= theta;
+  }
+  free(v);
+  if (count) *count = c;
+  return theta;
+}
+
 /* Active-token gather bookkeeping (App. B.2): ascending index list, count,
  * per-sequence offsets of executed tokens and each executed token's position
  * inside its own sequence. */

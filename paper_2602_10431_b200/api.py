@@ -29,7 +29,7 @@ EXPORTS = [
     "qtale_index_bookkeeping",
     "qtale_compact", "qtale_scatter_add", "qtale_wq_repack", "qtale_wq_gemm",
     "qtale_layer_workspace_bytes", "qtale_layer_forward", "qtale_model_workspace_bytes",
-    "qtale_model_prefill",
+    "qtale_model_prefill", "qtale_theta_workspace_bytes", "qtale_theta_for_ratio",
 ]
 
 
@@ -119,7 +119,11 @@ def lib():
         L.qtale_model_prefill.argtypes = [
             C.POINTER(ModelConfig), C.POINTER(ModelWeightsC), C.c_void_p, C.c_int, C.c_void_p,
             C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
-            C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+            C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+        L.qtale_theta_workspace_bytes.restype = C.c_size_t
+        L.qtale_theta_workspace_bytes.argtypes = []
+        L.qtale_theta_for_ratio.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t, C.c_double, C.c_void_p,
+                                            C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
         _lib = L
     return _lib
 
@@ -200,6 +204,21 @@ def router_select_static(x, w_router, bias, cu_seqlens, mode, out, theta=0.5, k=
         _ptr(out["idx"]), _ptr(out["n_exec"]), _ptr(out["cu_exec"]), _ptr(out["pos"]), _stream()),
         "qtale_router_select_static")
     return out
+
+
+def theta_for_ratio(scores, ratio, valid=None, out=None):
+    """qtale_theta_for_ratio on a flat fp32 device tensor of pooled router scores.
+    Returns (theta, count) as one-element device tensors (no host read-back here)."""
+    dev = scores.device
+    o = out or {}
+    theta = o.get("theta") if "theta" in o else torch.zeros(1, dtype=torch.float32, device=dev)
+    count = o.get("count") if "count" in o else torch.zeros(1, dtype=torch.int32, device=dev)
+    ws = o.get("ws") if "ws" in o else torch.empty(int(lib().qtale_theta_workspace_bytes()),
+                                                   dtype=torch.uint8, device=dev)
+    check(lib().qtale_theta_for_ratio(_ptr(scores), _ptr(valid), int(scores.numel()), float(ratio),
+                                      _ptr(theta), _ptr(count), _ptr(ws), ws.numel(), _stream()),
+          "qtale_theta_for_ratio")
+    return theta, count
 
 
 def index_bookkeeping(idx, n, T, cu_seqlens, pos0=None):
@@ -370,7 +389,7 @@ def model_workspace_bytes(cfg: ModelConfig, T_cap, B_cap, n_logit_rows) -> int:
 
 def model_prefill(cfg: ModelConfig, layers, embed, ids, cu_seqlens, ws, hidden_out,
                   per_layer_ratio=None, final_gamma=None, lm_head=None, logit_rows=None,
-                  logits_out=None, per_layer_n_exec=None, valid=None):
+                  logits_out=None, per_layer_n_exec=None, valid=None, layer_scores_out=None):
     """qtale_model_prefill.  layers: list of LayerWeights."""
     T = int(ids.shape[0])
     B = int(cu_seqlens.shape[0]) - 1
@@ -385,7 +404,7 @@ def model_prefill(cfg: ModelConfig, layers, embed, ids, cu_seqlens, ws, hidden_o
     check(lib().qtale_model_prefill(
         C.byref(cfg), C.byref(mw), _ptr(ids), T, _ptr(cu_seqlens), B, _ptr(valid),
         C.cast(ratios, C.c_void_p) if ratios is not None else None, _ptr(hidden_out),
-        _ptr(logits_out), _ptr(logit_rows), n_rows, _ptr(per_layer_n_exec), _ptr(ws),
+        _ptr(logits_out), _ptr(logit_rows), n_rows, _ptr(per_layer_n_exec), _ptr(layer_scores_out), _ptr(ws),
         ws.numel() * ws.element_size(), _stream()), "qtale_model_prefill")
     return hidden_out
 

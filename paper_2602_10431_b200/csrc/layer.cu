@@ -256,7 +256,7 @@ int qtale_model_prefill(const qtale_model_config* cfg, const qtale_model_weights
                         const uint8_t* valid,
                         const float* per_layer_ratio, void* hidden_out, float* logits_out,
                         const int32_t* logit_rows, int n_logit_rows, int32_t* per_layer_n_exec,
-                        void* ws, size_t ws_bytes, void* stream) {
+                        float* layer_scores_out, void* ws, size_t ws_bytes, void* stream) {
   if (!cfg || !w || !ids || !cu_seqlens || !hidden_out || !ws || !w->embed || !w->layers)
     return QTALE_ERR_NULL;
   QTALE_TRY(check_config(&cfg->layer));
@@ -284,7 +284,8 @@ int qtale_model_prefill(const qtale_model_config* cfg, const qtale_model_weights
     }
     QTALE_TRY(layer_forward_impl(&lc, &w->layers[l], hidden_out, T, cu_seqlens, B, nullptr,
                                  valid, nullptr, nullptr, 0, nullptr, QTALE_PHASE_PREFILL,
-                                 per_layer_n_exec ? per_layer_n_exec + l : nullptr, nullptr, lw,
+                                 per_layer_n_exec ? per_layer_n_exec + l : nullptr,
+                                 layer_scores_out ? layer_scores_out + (size_t)l * T : nullptr, lw,
                                  s));
   }
   if (logits_out) {

@@ -133,6 +133,32 @@ def test_selection_at_scale(env, T, B):
     assert _select_case(api, torch, dev, p, cu, api.SELECT_TOPK, k=k) == k
 
 
+@pytest.mark.parametrize("n", [1, 777, 262144, 1500000])
+def test_theta_for_ratio_matches_the_sorted_quantile(env, n):
+    """The device-side quantile is a selection, so theta and the count must equal the oracle's
+    sort-based ones bit for bit: padding, ties at the cut, ratios 0 and 1, 32 layers x 8192
+    pooled scores (the model-prefill calibration size) and a case of many CTAs."""
+    api, torch, dev = env
+    p = inputs.beta22(61, 1, n).astype(np.float32)
+    if n > 700:
+        p[100:700] = p[3]
+    valid = (inputs.uniform(61, 2, n) > 0.15).astype(np.uint8)
+    pd, vd = torch.from_numpy(p).to(dev), torch.from_numpy(valid).to(dev)
+    for ratio in [0.0, 0.3, 0.75, 1.0]:
+        for v_np, v_d in [(None, None), (valid, vd)]:
+            if v_np is not None and v_np.sum() == 0:
+                continue
+            th_ref, c_ref = oracle.theta_for_ratio(p, ratio, v_np)
+            th, c = api.theta_for_ratio(pd, ratio, valid=v_d)
+            assert api.device_status() == 0
+            assert float(th.item()) == np.float32(th_ref) and int(c.item()) == c_ref
+    # Eq. 9 with that theta executes the requested share
+    th, c = api.theta_for_ratio(pd, 0.5)
+    r = api.router_select(None, None, 0.0, torch.tensor([0, n], dtype=torch.int32, device=dev),
+                          api.SELECT_THRESHOLD, theta=float(th.item()), scores_override=pd)
+    assert int(r["n_exec"].item()) == int(c.item()) >= api.topk_count(0.5, n)
+
+
 def test_inconsistent_cu_seqlens_is_reported_not_followed(env):
     """cu_seqlens lives on the device, so the kernel checks it: offsets that do not end at T
     (or are not ascending) give QTALE_ERR_SHAPE in the status word, tokens outside

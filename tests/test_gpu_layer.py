@@ -362,6 +362,53 @@ def test_model_prefill_teacher_forced(env):
     assert per_layer.cpu().numpy().tolist() == [oracle.topk_count(r, T) for r in (0.75, 0.5, 0.25)]
 
 
+def test_global_theta_for_a_target_ratio(env):
+    """One theta for all layers (Sec. 3.4) found for a target average execution ratio: the
+    search runs the stack, pools every layer's router scores and takes their quantile on the
+    device until R_avg is within 0.005 of the target.  Checked against the oracle teacher-forced:
+    with the found theta, every layer's selection on the GPU's own input equals the oracle's."""
+    api, torch, dev = env
+    from paper_2602_10431_b200 import calibrate
+    sh = inputs.LayerShape(256, 4, 2, 64, 512, 4, 128)
+    L, V, B, S = 4, 500, 4, 300
+    cu = inputs.ragged_seqlens(19, B, S)
+    T = int(cu[-1])
+    dense, lws = [], []
+    for li in range(L):
+        w = inputs.layer_weights(19, li, sh)
+        w["router_w"] = inputs.round_bf16((inputs.normal(19, 500 + li, sh.d) * 0.05).astype(np.float32))
+        w["router_b"] = 0.3 * (li - 1.5)                          # layers with different ratios
+        dense.append(oracle.DenseLayer(sh, w))
+        lws.append(api.LayerWeights(w, dev))
+    embed = inputs.activations(19, 600, V, sh.d)
+    ids = inputs.integers(19, 603, T, V)
+    valid = (inputs.uniform(19, 604, T) > 0.1).astype(np.uint8)
+    cud, idd = torch.from_numpy(cu).to(dev), torch.from_numpy(ids).to(dev)
+    vd, ed = torch.from_numpy(valid).to(dev), api.to_device_bf16(embed, dev)
+    mcfg = api.ModelConfig(L, V, api.layer_config(sh, api.SELECT_THRESHOLD, theta=0.5))
+    mws = torch.empty(api.model_workspace_bytes(mcfg, T, B, 0), dtype=torch.uint8, device=dev)
+    hidden = torch.zeros(T, sh.d, dtype=torch.bfloat16, device=dev)
+    target = 0.62
+    theta, r_avg, hist = calibrate.calibrate_model_theta(api, mcfg, lws, ed, idd, cud, mws, hidden, target,
+                                                         valid=vd)
+    assert api.device_status() == 0
+    assert abs(r_avg - target) <= 0.005 and len(hist) <= 8
+    # the found theta through the plain entry point, layer by layer against the oracle
+    cfg = api.layer_config(sh, api.SELECT_THRESHOLD, theta=theta)
+    xd = api.to_device_bf16(embed[ids], dev)
+    wsb = torch.empty(api.layer_workspace_bytes(cfg, T, B), dtype=torch.uint8, device=dev)
+    total = 0
+    for li in range(L):
+        x_in = api.to_host_f32(xd)
+        p, m = oracle.route(dense[li], x_in, "threshold", theta=theta, valid=valid)
+        nex = torch.zeros(1, dtype=torch.int32, device=dev)
+        api.layer_forward(cfg, lws[li], xd, cud, wsb, nex, valid=vd)
+        got = (api.to_host_f32(xd) != x_in).any(axis=1)
+        assert_selection_matches(np.nonzero(got)[0], int(got.sum()), p, m, theta)
+        total += int(nex.item())
+    assert abs(total / (L * int(valid.sum())) - r_avg) < 1e-9    # the search's last run, reproduced
+
+
 _C2 = {}
 
 

@@ -425,3 +425,51 @@ def test_model_shares_one_theta_and_reports_counts():
     assert c_none == [0, 0, 0] and np.array_equal(x_none, embed[ids])
     _, _, c_k = oracle.model_prefill(layers, embed, ids, cu, ratios=[0.75, 0.5, 0.25])
     assert c_k == [18, 12, 6]
+
+
+def test_theta_for_ratio_is_the_exact_quantile():
+    """Sec. 3.4: one theta sets the ratio.  For distinct scores the theta of ratio r is the
+    k-th largest with k = round(r n): exactly k scores pass p >= theta (Eq. 9), one more as soon as
+    theta drops to the next score; closed form on an arithmetic grid; padding is left out; r = 0
+    gives a theta nothing passes; ties at theta can only add to the count."""
+    n = 1000
+    p = (np.arange(1, n + 1, dtype=np.float32) / np.float32(n + 1))        # i / (n + 1), ascending
+    perm = np.argsort(inputs.uniform(11, 1, n))
+    for r in [0.0, 0.001, 0.25, 0.5, 0.731, 1.0]:
+        th, c = oracle.theta_for_ratio(p[perm], r)
+        k = oracle.topk_count(r, n)
+        if k == 0:
+            assert th > 1.0 and c == 0 and oracle.select_threshold(p, th).sum() == 0
+            continue
+        assert th == p[n - k] and c == k                                   # closed form on the grid
+        assert oracle.select_threshold(p[perm], th).sum() == k            # Eq. 9 with that theta
+        assert oracle.select_threshold(p[perm], np.nextafter(np.float32(th), np.float32(2))).sum() == k - 1
+        assert np.array_equal(oracle.select_threshold(p[perm], th), oracle.select_topk(p[perm], k))
+    # brute force against numpy's sort on random scores with padding and planted ties
+    q = inputs.beta22(12, 1, 5000).astype(np.float32)
+    q[100:160] = q[7]
+    valid = (inputs.uniform(12, 2, 5000) > 0.2).astype(np.uint8)
+    for r in [0.1, 0.5, 0.9]:
+        th, c = oracle.theta_for_ratio(q, r, valid)
+        srt = np.sort(q[valid == 1])[::-1]
+        k = oracle.topk_count(r, len(srt))
+        assert th == srt[k - 1] and c == int((q[valid == 1] >= th).sum()) >= k
+    # monotone: a higher ratio never raises theta (lowering theta raises the ratio, Sec. 3.4)
+    ths = [oracle.theta_for_ratio(q, r, valid)[0] for r in np.linspace(0.05, 1.0, 20)]
+    assert all(a >= b for a, b in zip(ths, ths[1:]))
+
+
+def test_theta_search_loop_converges_and_falls_back_to_bisection():
+    """Host logic of the ratio-targeted search on made-up response curves (no GPU)."""
+    from paper_2602_10431_b200 import calibrate
+    # a consistent world: the suggested theta is the right one -> two runs
+    resp = lambda th: min(1.0, max(0.0, 1.2 - 1.5 * th))                  # ratio falls with theta
+    inv = lambda r: (1.2 - r) / 1.5
+    th, r, hist = calibrate.search_theta(lambda t: (resp(t), inv(0.75)), 0.75)
+    assert abs(r - 0.75) <= 0.005 and len(hist) == 2
+    # a misleading suggestion (always far too low): the bracket takes over and bisects
+    th, r, hist = calibrate.search_theta(lambda t: (resp(t), 0.01), 0.6, max_iters=30)
+    assert abs(r - 0.6) <= 0.005 and abs(th - inv(0.6)) < 0.01
+    # unreachable target: returns the closest run seen
+    th, r, hist = calibrate.search_theta(lambda t: (0.3, 0.4), 0.9, max_iters=5)
+    assert r == 0.3 and len(hist) == 5
