@@ -329,7 +329,9 @@ def timing_layer(torch, api, dev, gen, sh):
     lw.down = timing_weight(torch, api, dev, gen, sh.d, sh.ffn, sh.bits, sh.group)
     lw.gamma1 = torch.ones(sh.d, dtype=torch.float32, device=dev)
     lw.gamma2 = torch.ones(sh.d, dtype=torch.float32, device=dev)
-    lw.router_w = (torch.randn(sh.d, device=dev, generator=gen) * 0.02).to(torch.bfloat16).float()
+    # router logits of order one at every depth of a random-init stack (the residual stream grows
+    # from layer to layer): weights ~ N(0, (0.25 / sqrt(d))^2), so no score saturates to 0 or 1
+    lw.router_w = (torch.randn(sh.d, device=dev, generator=gen) * (0.25 / sh.d ** 0.5)).to(torch.bfloat16).float()
     lw.router_b = 0.0
     lw.c = api.LayerWeightsC(lw.qkv.c, lw.o.c, lw.gate_up.c, lw.down.c, lw.gamma1.data_ptr(),
                              lw.gamma2.data_ptr(), lw.router_w.data_ptr(), 0.0)
