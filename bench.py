@@ -48,7 +48,7 @@ WORKLOAD = ("c2: 7B-shaped layer (hidden 4096, 32 heads, FFN 11008), int4 g128, 
 # table), QKV GEMM (+ rotary), attention, O GEMM, RMSNorm, gate/up GEMM (+ SwiGLU), down GEMM
 # (+ residual scatter)
 KERNELS_PER_STEP = 8
-ALL_LEGS = ["sweep", "gemm", "bf16", "router", "gather", "decode", "c4", "c5", "e2e", "cpu"]
+ALL_LEGS = ["sweep", "gemm", "bf16", "router", "gather", "decode", "decode_loop", "c4", "c5", "e2e", "cpu"]
 
 
 def measured_peaks():
@@ -627,6 +627,86 @@ def run_ours(args):
                     clocks=r["clocks"])
             del kv, lw3
         extra["c3_decode_step"] = out
+        check_status()
+
+    # ---- multi-step decode: 8 layers of the 7B shape, 64 sequences from 2048 cached tokens, 64
+    # ---- steps with the greedy next token; per-layer executed-only caches drift apart ----
+    if "decode_loop" in legs:
+        out = {}
+        Ld, Vd, Bd, steps_d, len0_d = 8, 32000, 64, 64, 2048
+        for name in ("c3_int3", "c3_int4g64"):
+            s3 = inputs.CONFIG_SHAPES[name]["shape"]
+            layers = [timing_layer(torch, api, dev, gen, s3) for _ in range(Ld)]
+            embed = torch.randn(Vd, s3.d, device=dev, generator=gen).to(torch.bfloat16)
+            lm_head = (torch.randn(Vd, s3.d, device=dev, generator=gen) * 0.02).to(torch.bfloat16)
+            fg = torch.ones(s3.d, dtype=torch.float32, device=dev)
+            cap = len0_d + 2 * steps_d + 8
+            caches = [api.KvCache(Bd, cap, s3.kv_dim, dev, act_dtype=api.ACT_F16) for _ in range(Ld)]
+            for c in caches:
+                c.k.normal_(generator=gen)
+                c.v.normal_(generator=gen)
+            ids0 = torch.randint(0, Vd, (Bd,), dtype=torch.int32, device=dev, generator=gen)
+            mcfg = api.ModelConfig(Ld, Vd, api.layer_config(s3, api.SELECT_THRESHOLD, theta=0.5))
+            dws = torch.empty(api.model_decode_workspace_bytes(mcfg, Bd), dtype=torch.uint8, device=dev)
+            hid = torch.empty(Bd, s3.d, dtype=torch.bfloat16, device=dev)
+            logits = torch.empty(Bd, Vd, dtype=torch.float32, device=dev)
+            ids_a, ids_b = ids0.clone(), torch.zeros_like(ids0)
+            posd = torch.zeros(Bd, dtype=torch.int32, device=dev)
+            counts = torch.zeros(Ld, dtype=torch.int32, device=dev)
+            acc = torch.zeros(Ld, dtype=torch.int64, device=dev)
+            sc = torch.empty(steps_d, Ld, Bd, dtype=torch.float32, device=dev)
+            wbytes = accounting.packed_weight_bytes(s3)
+
+            def reset():
+                for c in caches:
+                    c.kv_len.fill_(len0_d)
+                posd.fill_(len0_d)
+                ids_a.copy_(ids0)
+                acc.zero_()
+
+            def loop(n, scores=None):
+                a, b = ids_a, ids_b
+                for i in range(n):
+                    api.model_decode_step(mcfg, layers, embed, a, posd, caches, dws, hid, final_gamma=fg,
+                                          lm_head=lm_head, logits_out=logits, next_ids_out=b,
+                                          per_layer_n_exec=counts,
+                                          layer_scores_out=None if scores is None else scores[i])
+                    acc.add_(counts)
+                    a, b = b, a
+
+            from paper_2602_10431_b200 import calibrate
+            for r3 in (0.9, 0.6):
+                # one theta for all layers and steps, searched for the target R_avg over the whole
+                # 64-step run (untimed): run, pool all router scores, take their quantile, repeat
+                def trial(theta):
+                    mcfg.layer.theta = float(theta)
+                    reset()
+                    loop(steps_d, sc)
+                    th, _ = api.theta_for_ratio(sc.view(-1), r3)
+                    return float(acc.sum().item()) / (Ld * Bd * steps_d), float(th.item())
+
+                theta, _, hist = calibrate.search_theta(trial, r3, tol=0.01)
+                mcfg.layer.theta = float(theta)
+                reset()
+                r = timer.run(lambda i: loop(steps_d), 1, 0, 0.3, between=reset, max_regions=3)
+                executed = acc.cpu().numpy().astype(float)
+                r_avg = float(executed.sum() / (Ld * Bd * steps_d))
+                lens = torch.stack([c.kv_len for c in caches]).cpu().numpy()
+                ms_step = r["ms"] / steps_d
+                kv_bytes = float(executed.sum() / steps_d) * 2 * (len0_d + steps_d / 2 * r_avg) * s3.kv_dim * 2
+                nbytes = Ld * wbytes + kv_bytes + Vd * s3.d * 2
+                out["%s_ratio_%.1f" % (name, r3)] = dict(
+                    ms_per_step=ms_step, tokens_per_s=Bd / (ms_step * 1e-3), steps=steps_d, layers=Ld,
+                    sequences=Bd, theta=mcfg.layer.theta, r_avg=r_avg, theta_search_runs=len(hist),
+                    cache_len_min_max=[int(lens.min()), int(lens.max())],
+                    roofline=hbm_roofline("decode step of the stack (per layer: 4 small-M GEMMs + attention "
+                                          "over the cache; bf16 LM head)", nbytes, ms_step, peaks,
+                                          note="bytes per step = packed weights of 8 layers + keys/values "
+                                               "of the executed (sequence, layer) pairs + LM head"),
+                    launch="host loop of %d qtale_model_decode_step calls" % steps_d, clocks=r["clocks"])
+                reset()
+            del caches, layers, embed, lm_head
+        extra["decode_loop"] = out
         check_status()
 
     # ---- c4: 8B-shaped 32-layer model prefill, per-layer top-k at ratio 0.75 ----

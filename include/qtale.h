@@ -372,7 +372,8 @@ size_t qtale_model_workspace_bytes(const qtale_model_config* cfg, int T_cap, int
  * (HOST float [n_layers]) is given, per-layer top-k at those ratios; final
  * RMSNorm and LM head on the requested rows.
  *   ids [T] int32; valid [T] uint8 or NULL (0 = padding token, never executed
- *   at any layer, App. B.2); hidden_out [T, d] bf16 (final residual stream);
+ *   at any layer, App. B.2); caches: HOST array [n_layers] of empty per-layer
+ *   caches to fill with the executed tokens' keys / values, or NULL; hidden_out [T, d] bf16 (final residual stream);
  *   logits_out fp32 [n_logit_rows, vocab] or NULL; logit_rows [n_logit_rows]
  *   int32 device; per_layer_n_exec [n_layers] int32 device; layer_scores_out
  *   fp32 [n_layers, T] or NULL: every layer's router scores (the input of
@@ -380,10 +381,38 @@ size_t qtale_model_workspace_bytes(const qtale_model_config* cfg, int T_cap, int
  */
 int qtale_model_prefill(const qtale_model_config* cfg, const qtale_model_weights* w,
                         const int32_t* ids, int T, const int32_t* cu_seqlens, int B,
-                        const uint8_t* valid,
+                        const uint8_t* valid, const qtale_kv_cache* caches,
                         const float* per_layer_ratio, void* hidden_out, float* logits_out,
                         const int32_t* logit_rows, int n_logit_rows, int32_t* per_layer_n_exec,
                         float* layer_scores_out, void* ws, size_t ws_bytes, void* stream);
+
+size_t qtale_model_decode_workspace_bytes(const qtale_model_config* cfg, int B_cap);
+
+/*
+ * One decode step of a stack of token-adaptive layers: every sequence brings one
+ * new token, each layer decides per sequence whether that token executes
+ * (Eq. 9, one theta for all layers, Sec. 3.4) and only then appends its key /
+ * value to that layer's cache (Eq. 3: a bypassed token does not evaluate f_l).
+ * Over many steps the cache lengths therefore diverge between sequences and
+ * between layers; this is the regime where weight-only quantisation pays
+ * (Sec. 2.3: the step is bound by the weight and cache streams).
+ *
+ *   ids [B] int32 (the new tokens); pos [B] int32 device: position of each new
+ *   token in its sequence (rotary position; counts bypassed tokens too), advanced
+ *   by one for every valid sequence when the step is done; valid [B] uint8 or
+ *   NULL (0 = finished sequence: never executes, position kept); caches: HOST
+ *   array [n_layers], each [B, cap, n_kv_heads * head_dim] with its own kv_len;
+ *   hidden_out [B, d] bf16; logits_out fp32 [B, vocab] or NULL; next_ids_out [B]
+ *   int32 or NULL: greedy choice (largest logit, lowest index among equal ones);
+ *   per_layer_n_exec [n_layers] or NULL: sequences executed by each layer in
+ *   this step; layer_scores_out fp32 [n_layers, B] or NULL.
+ * Top-k selection works as in qtale_layer_forward (ratio of the valid sequences).
+ */
+int qtale_model_decode_step(const qtale_model_config* cfg, const qtale_model_weights* w,
+                            const int32_t* ids, int B, int32_t* pos, const uint8_t* valid,
+                            const qtale_kv_cache* caches, void* hidden_out, float* logits_out,
+                            int32_t* next_ids_out, int32_t* per_layer_n_exec,
+                            float* layer_scores_out, void* ws, size_t ws_bytes, void* stream);
 
 #ifdef __cplusplus
 }

@@ -30,6 +30,7 @@ EXPORTS = [
     "qtale_compact", "qtale_scatter_add", "qtale_wq_repack", "qtale_wq_gemm",
     "qtale_layer_workspace_bytes", "qtale_layer_forward", "qtale_model_workspace_bytes",
     "qtale_model_prefill", "qtale_theta_workspace_bytes", "qtale_theta_for_ratio",
+    "qtale_model_decode_workspace_bytes", "qtale_model_decode_step",
 ]
 
 
@@ -118,8 +119,14 @@ def lib():
         L.qtale_model_workspace_bytes.argtypes = [C.POINTER(ModelConfig), C.c_int, C.c_int, C.c_int]
         L.qtale_model_prefill.argtypes = [
             C.POINTER(ModelConfig), C.POINTER(ModelWeightsC), C.c_void_p, C.c_int, C.c_void_p,
-            C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
+            C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
             C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+        L.qtale_model_decode_workspace_bytes.restype = C.c_size_t
+        L.qtale_model_decode_workspace_bytes.argtypes = [C.POINTER(ModelConfig), C.c_int]
+        L.qtale_model_decode_step.argtypes = [
+            C.POINTER(ModelConfig), C.POINTER(ModelWeightsC), C.c_void_p, C.c_int, C.c_void_p,
+            C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+            C.c_void_p, C.c_size_t, C.c_void_p]
         L.qtale_theta_workspace_bytes.restype = C.c_size_t
         L.qtale_theta_workspace_bytes.argtypes = []
         L.qtale_theta_for_ratio.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t, C.c_double, C.c_void_p,
@@ -389,7 +396,8 @@ def model_workspace_bytes(cfg: ModelConfig, T_cap, B_cap, n_logit_rows) -> int:
 
 def model_prefill(cfg: ModelConfig, layers, embed, ids, cu_seqlens, ws, hidden_out,
                   per_layer_ratio=None, final_gamma=None, lm_head=None, logit_rows=None,
-                  logits_out=None, per_layer_n_exec=None, valid=None, layer_scores_out=None):
+                  logits_out=None, per_layer_n_exec=None, valid=None, layer_scores_out=None,
+                  caches=None):
     """qtale_model_prefill.  layers: list of LayerWeights."""
     T = int(ids.shape[0])
     B = int(cu_seqlens.shape[0]) - 1
@@ -403,9 +411,37 @@ def model_prefill(cfg: ModelConfig, layers, embed, ids, cu_seqlens, ws, hidden_o
     n_rows = int(logit_rows.shape[0]) if logit_rows is not None else 0
     check(lib().qtale_model_prefill(
         C.byref(cfg), C.byref(mw), _ptr(ids), T, _ptr(cu_seqlens), B, _ptr(valid),
+        C.cast(_cache_array(caches), C.c_void_p) if caches is not None else None,
         C.cast(ratios, C.c_void_p) if ratios is not None else None, _ptr(hidden_out),
         _ptr(logits_out), _ptr(logit_rows), n_rows, _ptr(per_layer_n_exec), _ptr(layer_scores_out), _ptr(ws),
         ws.numel() * ws.element_size(), _stream()), "qtale_model_prefill")
+    return hidden_out
+
+
+def _cache_array(caches):
+    return (KvCacheC * len(caches))(*[c.c for c in caches])
+
+
+def model_decode_workspace_bytes(cfg: ModelConfig, B_cap) -> int:
+    return int(lib().qtale_model_decode_workspace_bytes(C.byref(cfg), int(B_cap)))
+
+
+def model_decode_step(cfg: ModelConfig, layers, embed, ids, pos, caches, ws, hidden_out, valid=None,
+                      final_gamma=None, lm_head=None, logits_out=None, next_ids_out=None,
+                      per_layer_n_exec=None, layer_scores_out=None):
+    """qtale_model_decode_step.  layers: list of LayerWeights; caches: list of KvCache (one per
+    layer); pos is advanced in place."""
+    B = int(ids.shape[0])
+    arr = (LayerWeightsC * len(layers))(*[l.c for l in layers])
+    carr = _cache_array(caches)
+    mw = ModelWeightsC(embed.data_ptr(), arr,
+                       final_gamma.data_ptr() if final_gamma is not None else None,
+                       lm_head.data_ptr() if lm_head is not None else None)
+    check(lib().qtale_model_decode_step(
+        C.byref(cfg), C.byref(mw), _ptr(ids), B, _ptr(pos), _ptr(valid), C.cast(carr, C.c_void_p),
+        _ptr(hidden_out), _ptr(logits_out), _ptr(next_ids_out), _ptr(per_layer_n_exec),
+        _ptr(layer_scores_out), _ptr(ws), ws.numel() * ws.element_size(), _stream()),
+        "qtale_model_decode_step")
     return hidden_out
 
 

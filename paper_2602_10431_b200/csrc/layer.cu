@@ -253,7 +253,7 @@ size_t qtale_model_workspace_bytes(const qtale_model_config* cfg, int T_cap, int
 
 int qtale_model_prefill(const qtale_model_config* cfg, const qtale_model_weights* w,
                         const int32_t* ids, int T, const int32_t* cu_seqlens, int B,
-                        const uint8_t* valid,
+                        const uint8_t* valid, const qtale_kv_cache* caches,
                         const float* per_layer_ratio, void* hidden_out, float* logits_out,
                         const int32_t* logit_rows, int n_logit_rows, int32_t* per_layer_n_exec,
                         float* layer_scores_out, void* ws, size_t ws_bytes, void* stream) {
@@ -282,8 +282,11 @@ int qtale_model_prefill(const qtale_model_config* cfg, const qtale_model_weights
     } else if (lc.select_mode == QTALE_SELECT_FORCED) {
       return QTALE_ERR_MODE;
     }
+    if (caches && (!caches[l].k || !caches[l].v || !caches[l].kv_len || caches[l].cap < 1))
+      return QTALE_ERR_NULL;
     QTALE_TRY(layer_forward_impl(&lc, &w->layers[l], hidden_out, T, cu_seqlens, B, nullptr,
-                                 valid, nullptr, nullptr, 0, nullptr, QTALE_PHASE_PREFILL,
+                                 valid, nullptr, nullptr, 0, caches ? &caches[l] : nullptr,
+                                 QTALE_PHASE_PREFILL,
                                  per_layer_n_exec ? per_layer_n_exec + l : nullptr,
                                  layer_scores_out ? layer_scores_out + (size_t)l * T : nullptr, lw,
                                  s));
@@ -295,6 +298,56 @@ int qtale_model_prefill(const qtale_model_config* cfg, const qtale_model_weights
                                logits_out, cfg->vocab, s));
   }
   return QTALE_OK;
+}
+
+size_t qtale_model_decode_workspace_bytes(const qtale_model_config* cfg, int B_cap) {
+  if (!cfg || B_cap < 1) return 0;
+  const size_t layer = qtale_layer_workspace_bytes(&cfg->layer, B_cap, B_cap);
+  if (layer == 0) return 0;
+  return layer + align_up((size_t)B_cap * cfg->layer.d * 2, 256) + align_up((size_t)(B_cap + 1) * 4, 256);
+}
+
+int qtale_model_decode_step(const qtale_model_config* cfg, const qtale_model_weights* w,
+                            const int32_t* ids, int B, int32_t* pos, const uint8_t* valid,
+                            const qtale_kv_cache* caches, void* hidden_out, float* logits_out,
+                            int32_t* next_ids_out, int32_t* per_layer_n_exec,
+                            float* layer_scores_out, void* ws, size_t ws_bytes, void* stream) {
+  if (!cfg || !w || !ids || !pos || !caches || !hidden_out || !ws || !w->embed || !w->layers)
+    return QTALE_ERR_NULL;
+  QTALE_TRY(check_config(&cfg->layer));
+  if (cfg->n_layers < 1 || cfg->vocab < 1 || B < 1) return QTALE_ERR_SHAPE;
+  if (cfg->layer.select_mode == QTALE_SELECT_FORCED) return QTALE_ERR_MODE;
+  if ((logits_out || next_ids_out) && (!w->lm_head || !w->final_gamma)) return QTALE_ERR_NULL;
+  if (next_ids_out && !logits_out) return QTALE_ERR_NULL;
+  for (int l = 0; l < cfg->n_layers; ++l) {
+    QTALE_TRY(check_weights(&cfg->layer, &w->layers[l]));
+    if (!caches[l].k || !caches[l].v || !caches[l].kv_len || caches[l].cap < 1) return QTALE_ERR_NULL;
+  }
+  if (!aligned16(hidden_out) || !aligned16(ws) || !aligned16(w->embed)) return QTALE_ERR_ALIGN;
+  if (ws_bytes < qtale_model_decode_workspace_bytes(cfg, B)) return QTALE_ERR_WORKSPACE;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const int d = cfg->layer.d;
+  const LayerWs lw = carve(&cfg->layer, B, B, ws);
+  unsigned char* base = static_cast<unsigned char*>(ws) + lw.total;
+  void* hrows = base;
+  int32_t* cu = reinterpret_cast<int32_t*>(base + align_up((size_t)B * d * 2, 256));
+
+  QTALE_TRY(launch_iota(cu, B + 1, s));  // one new token per sequence: cu_seqlens = 0, 1, ..., B
+  QTALE_TRY(launch_embed(w->embed, ids, B, d, cfg->vocab, hidden_out, s));
+  for (int l = 0; l < cfg->n_layers; ++l) {
+    QTALE_TRY(layer_forward_impl(&cfg->layer, &w->layers[l], hidden_out, B, cu, B, pos, valid, nullptr,
+                                 nullptr, 0, &caches[l], QTALE_PHASE_DECODE,
+                                 per_layer_n_exec ? per_layer_n_exec + l : nullptr,
+                                 layer_scores_out ? layer_scores_out + (size_t)l * B : nullptr, lw, s));
+  }
+  if (logits_out) {
+    QTALE_TRY(launch_compact(hidden_out, cu, nullptr, B, d, w->final_gamma, cfg->layer.rms_eps,
+                             QTALE_ACT_BF16, nullptr, hrows, s));
+    QTALE_TRY(bf16_gemm_launch(hrows, d, nullptr, B, w->lm_head, cfg->vocab, d, d, logits_out,
+                               cfg->vocab, s));
+    if (next_ids_out) QTALE_TRY(launch_argmax_rows(logits_out, B, cfg->vocab, next_ids_out, s));
+  }
+  return launch_advance_pos(pos, valid, B, s);
 }
 
 }  // extern "C"

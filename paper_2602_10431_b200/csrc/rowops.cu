@@ -296,6 +296,43 @@ __global__ void __launch_bounds__(kRowThreads)
   }
 }
 
+// ---- decode-loop helpers ------------------------------------------------------------
+// cu[b] = b for b = 0 .. B: one new token per sequence
+__global__ void iota_kernel(int32_t* __restrict__ cu, int n) {
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) cu[i] = i;
+}
+// the next token of a sequence sits one position further (finished sequences stay where they are)
+__global__ void advance_pos_kernel(int32_t* __restrict__ pos, const uint8_t* __restrict__ valid, int B) {
+  for (int b = blockIdx.x * blockDim.x + threadIdx.x; b < B; b += gridDim.x * blockDim.x)
+    if (!valid || valid[b]) pos[b] += 1;
+}
+// greedy choice: index of the largest logit of each row, the lowest index among equal ones
+__global__ void __launch_bounds__(kRowThreads)
+    argmax_rows_kernel(const float* __restrict__ logits, int V, int32_t* __restrict__ out) {
+  __shared__ float s_v[kRowThreads / 32];
+  __shared__ int s_i[kRowThreads / 32];
+  const float* row = logits + (size_t)blockIdx.x * V;
+  float best = -INFINITY;
+  int bi = 0x7FFFFFFF;
+  for (int j = threadIdx.x; j < V; j += kRowThreads) {
+    const float v = row[j];
+    if (v > best || (v == best && j < bi)) { best = v; bi = j; }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float ov = __shfl_xor_sync(0xffffffffu, best, o);
+    const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+    if (ov > best || (ov == best && oi < bi)) { best = ov; bi = oi; }
+  }
+  if ((threadIdx.x & 31) == 0) { s_v[threadIdx.x >> 5] = best; s_i[threadIdx.x >> 5] = bi; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < kRowThreads / 32; ++w)
+      if (s_v[w] > best || (s_v[w] == best && s_i[w] < bi)) { best = s_v[w]; bi = s_i[w]; }
+    out[blockIdx.x] = bi == 0x7FFFFFFF ? 0 : bi;
+  }
+}
+
 // ---- host launchers ----------------------------------------------------------------
 
 static int row_grid(int per_sm) { return sm_count() * per_sm; }
@@ -395,6 +432,21 @@ int launch_kv_append(const void* qkv, const int32_t* n_exec, int cap_rows, int l
       static_cast<uint4*>(cache_k), static_cast<uint4*>(cache_v), kv_len, cap);
   if (cudaGetLastError() != cudaSuccess) return QTALE_ERR_CUDA;
   kv_len_update_kernel<<<(B + 255) / 256, 256, 0, s>>>(kv_len, cu_exec, B, cap, device_status_ptr());
+  return launch_status(cudaGetLastError());
+}
+
+int launch_iota(int32_t* cu, int n, cudaStream_t s) {
+  iota_kernel<<<(n + 255) / 256, 256, 0, s>>>(cu, n);
+  return launch_status(cudaGetLastError());
+}
+
+int launch_advance_pos(int32_t* pos, const uint8_t* valid, int B, cudaStream_t s) {
+  advance_pos_kernel<<<(B + 255) / 256, 256, 0, s>>>(pos, valid, B);
+  return launch_status(cudaGetLastError());
+}
+
+int launch_argmax_rows(const float* logits, int rows, int V, int32_t* out, cudaStream_t s) {
+  argmax_rows_kernel<<<rows, kRowThreads, 0, s>>>(logits, V, out);
   return launch_status(cudaGetLastError());
 }
 

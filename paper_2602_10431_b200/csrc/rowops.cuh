@@ -29,6 +29,9 @@ int launch_swiglu(const void* gu, const int32_t* n_exec, int cap, int F, void* a
 int launch_kv_append(const void* qkv, const int32_t* n_exec, int cap_rows, int ld, int q_dim,
                      int kv_dim, const int32_t* cu_exec, int B, void* cache_k, void* cache_v,
                      int32_t* kv_len, int cap, cudaStream_t s);
+int launch_iota(int32_t* cu, int n, cudaStream_t s);
+int launch_advance_pos(int32_t* pos, const uint8_t* valid, int B, cudaStream_t s);
+int launch_argmax_rows(const float* logits, int rows, int V, int32_t* out, cudaStream_t s);
 int launch_embed(const void* embed, const int32_t* ids, int T, int d, int vocab, void* out,
                  cudaStream_t s);
 

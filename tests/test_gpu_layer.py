@@ -362,6 +362,126 @@ def test_model_prefill_teacher_forced(env):
     assert per_layer.cpu().numpy().tolist() == [oracle.topk_count(r, T) for r in (0.75, 0.5, 0.25)]
 
 
+def test_decode_loop_with_diverging_per_layer_caches(env):
+    """Prefill of ragged prompts, then 64 decode steps of a 3-layer stack with one theta: each
+    layer's cache holds executed tokens only, so its lengths drift apart between sequences and
+    layers.  Teacher-forced per layer and step (the oracle gets the GPU's input of that layer):
+    selection bit-exact, output within the layer tolerance, cache lengths equal at every step.
+    Then the one-call entry points (model prefill with caches, model decode step with the
+    greedy next token) must reproduce the layer-by-layer hidden states bit for bit; the logits
+    are checked against the oracle's final norm + linear on the GPU's hidden state and the
+    chosen ids against the argmax of the GPU's own logits (first maximum)."""
+    api, torch, dev = env
+    sh = inputs.LayerShape(256, 4, 2, 64, 512, 4, 128)
+    L, V, B, cap, steps = 3, 400, 6, 128, 64
+    theta = 0.45
+    cu = np.array([0, 5, 30, 31, 71, 90, 120], np.int32)            # prompts of 5, 25, 1, 40, 19, 30 tokens
+    T = int(cu[-1])
+    dense, lws = [], []
+    for li in range(L):
+        w = inputs.layer_weights(23, li, sh)
+        w["router_w"] = inputs.round_bf16((inputs.normal(23, 500 + li, sh.d) * 0.05).astype(np.float32))
+        w["router_b"] = 0.2 * (1 - li)
+        dense.append(oracle.DenseLayer(sh, w))
+        lws.append(api.LayerWeights(w, dev))
+    embed = inputs.activations(23, 600, V, sh.d)
+    lm_head = inputs.activations(23, 601, V, sh.d, 0.05)
+    fgam = (1 + 0.1 * inputs.normal(23, 602, sh.d)).astype(np.float32)
+    prompt = inputs.integers(23, 603, T, V)
+    ed, lmd, fgd = api.to_device_bf16(embed, dev), api.to_device_bf16(lm_head, dev), torch.from_numpy(fgam).to(dev)
+    cfg = api.layer_config(sh, api.SELECT_THRESHOLD, theta=theta)
+    mcfg = api.ModelConfig(L, V, cfg)
+    kvd = sh.kv_dim
+    cud = torch.from_numpy(cu).to(dev)
+
+    def fresh_caches():
+        return [api.KvCache(B, cap, kvd, dev, act_dtype=1) for _ in range(L)]
+
+    # ---- layer by layer, teacher forced: prefill ----
+    gc = fresh_caches()
+    ock = [np.zeros((B, cap, kvd), np.float32) for _ in range(L)]
+    ocv = [np.zeros((B, cap, kvd), np.float32) for _ in range(L)]
+    okl = [np.zeros(B, np.int32) for _ in range(L)]
+    wsb = torch.empty(api.layer_workspace_bytes(cfg, T, B), dtype=torch.uint8, device=dev)
+    xd = api.to_device_bf16(embed[prompt], dev)
+    for li in range(L):
+        x_in = api.to_host_f32(xd)
+        p, m = oracle.route(dense[li], x_in, "threshold", theta=theta)
+        ref, _ = oracle.layer_forward(dense[li], x_in, cu, m, cache_k=ock[li], cache_v=ocv[li], kv_len=okl[li])
+        api.layer_forward(cfg, lws[li], xd, cud, wsb, kv=gc[li], phase=api.PHASE_PREFILL)
+        out = api.to_host_f32(xd)
+        got = (out != x_in).any(axis=1)
+        assert_selection_matches(np.nonzero(got)[0], int(got.sum()), p, m, theta)
+        assert_layer_close(out, ref, strict=True)
+        assert np.array_equal(gc[li].kv_len.cpu().numpy(), okl[li])
+    hidden_prefill = xd.clone()
+    len_after_prefill = [c.kv_len.clone() for c in gc]
+
+    # ---- layer by layer, teacher forced: 64 decode steps (ids given by the GPU's greedy choice) ----
+    cu1 = inputs.cu_seqlens_uniform(B, 1)
+    cu1d = torch.from_numpy(cu1).to(dev)
+    ws1 = torch.empty(api.layer_workspace_bytes(cfg, B, B), dtype=torch.uint8, device=dev)
+    pos = (cu[1:] - cu[:-1]).astype(np.int32)                        # next position = prompt length
+    last_rows = (cu[1:] - 1).astype(np.int64)
+    h_last = api.to_host_f32(hidden_prefill)[last_rows]
+    ids = np.argmax(oracle.linear(oracle.rmsnorm(h_last, fgam, sh.rms_eps), lm_head), axis=1).astype(np.int32)
+    first_ids = ids.copy()
+    trace_hidden, trace_ids, ratios = [], [], np.zeros(L)
+    for st in range(steps):
+        xd = api.to_device_bf16(embed[ids], dev)
+        pd = torch.from_numpy(pos).to(dev)
+        for li in range(L):
+            x_in = api.to_host_f32(xd)
+            p, m = oracle.route(dense[li], x_in, "threshold", theta=theta)
+            ref, _ = oracle.layer_forward(dense[li], x_in, cu1, m, pos0=pos, cache_k=ock[li], cache_v=ocv[li],
+                                          kv_len=okl[li])
+            api.layer_forward(cfg, lws[li], xd, cu1d, ws1, pos0=pd, kv=gc[li], phase=api.PHASE_DECODE)
+            out = api.to_host_f32(xd)
+            got = (out != x_in).any(axis=1)
+            assert_selection_matches(np.nonzero(got)[0], int(got.sum()), p, m, theta)
+            assert_layer_close(out, ref, strict=True)
+            assert np.array_equal(gc[li].kv_len.cpu().numpy(), okl[li]), (st, li)
+            ratios[li] += m.mean() / steps
+        trace_hidden.append(xd.clone())
+        h = api.to_host_f32(xd)
+        ids = np.argmax(oracle.linear(oracle.rmsnorm(h, fgam, sh.rms_eps), lm_head), axis=1).astype(np.int32)
+        trace_ids.append(ids.copy())
+        pos = pos + 1
+    assert api.device_status() == 0
+    lens = np.stack([k for k in okl])                                 # [L, B]
+    assert len(np.unique(lens)) > B                                   # lengths diverged across sequences and layers
+    assert 0.2 < ratios.min() and ratios.max() < 0.95 and np.ptp(ratios) > 0.05
+
+    # ---- the one-call entry points reproduce it ----
+    mc = fresh_caches()
+    mws = torch.empty(api.model_workspace_bytes(mcfg, T, B, 0), dtype=torch.uint8, device=dev)
+    hidden = torch.zeros(T, sh.d, dtype=torch.bfloat16, device=dev)
+    api.model_prefill(mcfg, lws, ed, torch.from_numpy(prompt).to(dev), cud, mws, hidden, caches=mc)
+    assert torch.equal(hidden, hidden_prefill)
+    for li in range(L):
+        assert torch.equal(mc[li].kv_len, len_after_prefill[li])
+    dws = torch.empty(api.model_decode_workspace_bytes(mcfg, B), dtype=torch.uint8, device=dev)
+    hid = torch.zeros(B, sh.d, dtype=torch.bfloat16, device=dev)
+    logits = torch.zeros(B, V, dtype=torch.float32, device=dev)
+    cur = torch.from_numpy(first_ids).to(dev)
+    nxt = torch.zeros(B, dtype=torch.int32, device=dev)
+    posd = torch.from_numpy((cu[1:] - cu[:-1]).astype(np.int32)).to(dev)
+    counts = torch.zeros(L, dtype=torch.int32, device=dev)
+    for st in range(steps):
+        api.model_decode_step(mcfg, lws, ed, cur, posd, mc, dws, hid, final_gamma=fgd, lm_head=lmd,
+                              logits_out=logits, next_ids_out=nxt, per_layer_n_exec=counts)
+        assert torch.equal(hid, trace_hidden[st]), st
+        lg = logits.cpu().numpy()
+        ref_lg = oracle.linear(oracle.rmsnorm(api.to_host_f32(hid), fgam, sh.rms_eps), lm_head)
+        assert rel_fro(lg, ref_lg) <= 5e-3
+        assert np.array_equal(nxt.cpu().numpy(), np.argmax(lg, axis=1))       # first maximum of the GPU's logits
+        cur = torch.from_numpy(trace_ids[st]).to(dev)                          # stay on the checked trajectory
+    assert api.device_status() == 0
+    for li in range(L):
+        assert np.array_equal(mc[li].kv_len.cpu().numpy(), okl[li])
+    assert np.array_equal(posd.cpu().numpy(), cu[1:] - cu[:-1] + steps)
+
+
 def test_global_theta_for_a_target_ratio(env):
     """One theta for all layers (Sec. 3.4) found for a target average execution ratio: the
     search runs the stack, pools every layer's router scores and takes their quantile on the
