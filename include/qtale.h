@@ -125,6 +125,23 @@ int qtale_router_select(const void* x, int T, int d, const float* w_router, floa
                         size_t ws_bytes, void* stream);
 
 /*
+ * Router as a small MLP (Eq. 2: "a lightweight MLP" produces the two class
+ * logits; Eq. 9: the execute probability is their softmax):
+ *   u = W1 x + b1,  a = max(u, 0),  (g0, g1) = W2 a + b2,  score = softmax(g)[0]
+ *         = 1 / (1 + exp(-((W2[0] - W2[1]) . a + b2_execute - b2_bypass))).
+ * The paper states neither the hidden width nor the activation; ReLU is this
+ * library's reading.  The hidden layer runs on the tensor cores with fp64
+ * accumulation across 64-feature chunks, so the scores agree with an fp64
+ * evaluation to about 1e-7.  Feed scores_out to qtale_router_select as
+ * scores_override (qtale_layer_forward does that when router_h > 0).
+ *   x [T, d] bf16; w1 [h, d] bf16; b1 [h] fp32; w2 [2, h] fp32 (row 0 execute,
+ *   row 1 bypass); scores_out [T] fp32.  Limits: d % 8 == 0, 1 <= h <= 64.
+ */
+int qtale_router_mlp_scores(const void* x, int T, int d, const void* w1, const float* b1,
+                            const float* w2, int h, float b2_execute, float b2_bypass,
+                            float* scores_out, void* stream);
+
+/*
  * qtale_router_select for callers that must not allocate device memory.
  * (No counterpart in the paper: this is a packaging variant of the call above.)
  *
@@ -309,6 +326,12 @@ typedef struct {
   const float* gamma2;     /* [d] fp32, pre-MLP RMSNorm gain                   */
   const float* router_w;   /* [d] fp32, execute-minus-bypass logit weights     */
   float router_b;
+  int router_h;            /* 0: the linear router above; > 0: MLP router with this
+                              many hidden units (see qtale_router_mlp_scores)   */
+  const void* router_w1;   /* [router_h, d] bf16                               */
+  const float* router_b1;  /* [router_h] fp32                                  */
+  const float* router_w2;  /* [2, router_h] fp32                               */
+  float router_b2[2];      /* execute, bypass                                  */
 } qtale_layer_weights;
 
 /* Per-layer KV cache.  Only executed tokens enter it: a bypassed token does not

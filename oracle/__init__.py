@@ -102,6 +102,19 @@ def router_scores(x, w, bias, return_logits=False):
     return (p, z) if return_logits else p
 
 
+def router_mlp_scores(x, w1, b1, w2, b2, return_logits=False):
+    """MLP router: w1 [h, d], b1 [h], w2 [2, h], b2 [2]; returns p0 (and g0 - g1)."""
+    x, w1, b1, w2, b2 = _f32(x), _f32(w1), _f32(b1), _f32(w2), _f32(b2)
+    T, d = x.shape
+    h = w1.shape[0]
+    assert w1.shape == (h, d) and b1.shape == (h,) and w2.shape == (2, h) and b2.shape == (2,)
+    p = np.empty(T, dtype=np.float32)
+    z = np.empty(T, dtype=np.float64)
+    lib().orc_router_mlp_scores(_p(x, C.c_float), T, d, _p(w1, C.c_float), _p(b1, C.c_float), h,
+                                _p(w2, C.c_float), _p(b2, C.c_float), _p(p, C.c_float), _p(z, C.c_double))
+    return (p, z) if return_logits else p
+
+
 def softmax2_p0(g0, g1):
     g0 = np.ascontiguousarray(g0, dtype=np.float64)
     g1 = np.ascontiguousarray(g1, dtype=np.float64)

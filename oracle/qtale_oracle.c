@@ -118,6 +118,31 @@ void orc_router_scores(const float* x, int T, int d, const float* w, float bias,
   }
 }
 
+/* Router as a small MLP (Eq. 2: "a lightweight MLP" emits the two class logits):
+ * u = W1 x + b1 (hidden units), a = max(u, 0), (g0, g1) = W2 a + b2, and
+ * p0 = softmax([g0, g1])[0] (Eq. 9).  The paper gives neither the width nor the
+ * activation; ReLU is this library's reading ("parity unpinned" by the paper).
+ * w1 [h, d], b1 [h], w2 [2, h] (row 0: execute logit, row 1: bypass logit), b2 [2]. */
+void orc_router_mlp_scores(const float* x, int T, int d, const float* w1, const float* b1, int h,
+                           const float* w2, const float* b2, float* p_out, double* z_out) {
+#pragma omp parallel for schedule(static)
+  for (int t = 0; t < T; ++t) {
+    double g0 = (double)b2[0], g1 = (double)b2[1];
+    for (int j = 0; j < h; ++j) {
+      double u = 0.0;
+      for (int k = 0; k < d; ++k) u += (double)x[(size_t)t * d + k] * (double)w1[(size_t)j * d + k];
+      u += (double)b1[j];
+      const double a = u > 0.0 ? u : 0.0;
+      g0 += (double)w2[j] * a;
+      g1 += (double)w2[(size_t)h + j] * a;
+    }
+    const double m = g0 > g1 ? g0 : g1;
+    const double e0 = exp(g0 - m), e1 = exp(g1 - m);
+    if (z_out) z_out[t] = g0 - g1;
+    p_out[t] = (float)(e0 / (e0 + e1));
+  }
+}
+
 /* General two-logit form of Eq. 9: p = softmax([g0, g1]); returns p[0]. */
 void orc_softmax2_p0(const double* g0, const double* g1, int T, float* p_out) {
   for (int t = 0; t < T; ++t) {

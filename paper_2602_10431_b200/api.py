@@ -30,7 +30,7 @@ EXPORTS = [
     "qtale_compact", "qtale_scatter_add", "qtale_wq_repack", "qtale_wq_gemm",
     "qtale_layer_workspace_bytes", "qtale_layer_forward", "qtale_model_workspace_bytes",
     "qtale_model_prefill", "qtale_theta_workspace_bytes", "qtale_theta_for_ratio",
-    "qtale_model_decode_workspace_bytes", "qtale_model_decode_step",
+    "qtale_model_decode_workspace_bytes", "qtale_model_decode_step", "qtale_router_mlp_scores",
 ]
 
 
@@ -59,7 +59,8 @@ class LayerConfig(C.Structure):
 class LayerWeightsC(C.Structure):
     _fields_ = [("qkv", WqWeight), ("o", WqWeight), ("gate_up", WqWeight), ("down", WqWeight),
                 ("gamma1", C.c_void_p), ("gamma2", C.c_void_p), ("router_w", C.c_void_p),
-                ("router_b", C.c_float)]
+                ("router_b", C.c_float), ("router_h", C.c_int), ("router_w1", C.c_void_p),
+                ("router_b1", C.c_void_p), ("router_w2", C.c_void_p), ("router_b2", C.c_float * 2)]
 
 
 class KvCacheC(C.Structure):
@@ -127,6 +128,9 @@ def lib():
             C.POINTER(ModelConfig), C.POINTER(ModelWeightsC), C.c_void_p, C.c_int, C.c_void_p,
             C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
             C.c_void_p, C.c_size_t, C.c_void_p]
+        L.qtale_router_mlp_scores.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p,
+                                              C.c_void_p, C.c_int, C.c_float, C.c_float, C.c_void_p,
+                                              C.c_void_p]
         L.qtale_theta_workspace_bytes.restype = C.c_size_t
         L.qtale_theta_workspace_bytes.argtypes = []
         L.qtale_theta_for_ratio.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t, C.c_double, C.c_void_p,
@@ -211,6 +215,18 @@ def router_select_static(x, w_router, bias, cu_seqlens, mode, out, theta=0.5, k=
         _ptr(out["idx"]), _ptr(out["n_exec"]), _ptr(out["cu_exec"]), _ptr(out["pos"]), _stream()),
         "qtale_router_select_static")
     return out
+
+
+def router_mlp_scores(x, w1, b1, w2, b2, scores_out=None):
+    """qtale_router_mlp_scores.  x bf16 [T, d]; w1 bf16 [h, d]; b1 fp32 [h]; w2 fp32 [2, h];
+    b2 = (execute, bypass)."""
+    T, d = int(x.shape[0]), int(x.shape[1])
+    if scores_out is None:
+        scores_out = torch.empty(T, dtype=torch.float32, device=x.device)
+    check(lib().qtale_router_mlp_scores(_ptr(x), T, d, _ptr(w1), _ptr(b1), _ptr(w2), int(w1.shape[0]),
+                                        float(b2[0]), float(b2[1]), _ptr(scores_out), _stream()),
+          "qtale_router_mlp_scores")
+    return scores_out
 
 
 def theta_for_ratio(scores, ratio, valid=None, out=None):
@@ -355,6 +371,16 @@ class LayerWeights:
         self.c = LayerWeightsC(self.qkv.c, self.o.c, self.gate_up.c, self.down.c,
                                self.gamma1.data_ptr(), self.gamma2.data_ptr(),
                                self.router_w.data_ptr(), self.router_b)
+        mlp = w.get("router_mlp")  # dict(w1 [h, d], b1 [h], w2 [2, h], b2 [2]) -> MLP router
+        if mlp is not None:
+            self.router_w1 = to_device_bf16(mlp["w1"], device)
+            self.router_b1 = torch.from_numpy(np.ascontiguousarray(mlp["b1"], np.float32)).to(device)
+            self.router_w2 = torch.from_numpy(np.ascontiguousarray(mlp["w2"], np.float32)).to(device)
+            self.c.router_h = int(mlp["w1"].shape[0])
+            self.c.router_w1 = self.router_w1.data_ptr()
+            self.c.router_b1 = self.router_b1.data_ptr()
+            self.c.router_w2 = self.router_w2.data_ptr()
+            self.c.router_b2 = (C.c_float * 2)(float(mlp["b2"][0]), float(mlp["b2"][1]))
 
     def set_router_bias(self, b: float):
         self.router_b = float(b)

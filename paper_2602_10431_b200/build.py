@@ -14,7 +14,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libqtale.so")
-SOURCES = ["runtime.cu", "router_select.cu", "rowops.cu", "wq_gemm.cu", "attention.cu", "attention_tc.cu", "layer.cu", "calibrate.cu"]
+SOURCES = ["runtime.cu", "router_select.cu", "rowops.cu", "wq_gemm.cu", "attention.cu", "attention_tc.cu", "layer.cu", "calibrate.cu", "router_mlp.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 

@@ -104,6 +104,13 @@ static int layer_forward_impl(const qtale_layer_config* c, const qtale_layer_wei
     if (c->select_mode == QTALE_SELECT_TOPK) {
       if (valid) ratio = (double)c->ratio; else k = qtale_topk_count((double)c->ratio, T);
     }
+    float* sc_buf = scores_out ? scores_out : ws.scores;
+    if (!scores_override && w->router_h > 0) {
+      // MLP router: its scores come from a kernel of their own and enter the selection as given
+      QTALE_TRY(router_mlp_launch(x, T, d, w->router_w1, w->router_b1, w->router_w2, w->router_h,
+                                  w->router_b2[0], w->router_b2[1], sc_buf, s));
+      scores_override = sc_buf;
+    }
     QTALE_TRY(router_select_launch(x, T, d, w->router_w, w->router_b, scores_override, valid,
                                    cu_seqlens, B, pos0, c->select_mode, c->theta, k, ratio,
                                    scores_out ? scores_out : ws.scores, ws.idx, ws.n_exec,
@@ -232,8 +239,10 @@ int qtale_layer_forward(const qtale_layer_config* cfg, const qtale_layer_weights
   if (cfg->select_mode == QTALE_SELECT_FORCED) {
     if (forced_n < 0 || forced_n > T) return QTALE_ERR_CAPACITY;
     if (forced_n > 0 && !forced_idx) return QTALE_ERR_NULL;
-  } else if (!scores_override && !w->router_w) {
-    return QTALE_ERR_NULL;
+  } else if (!scores_override) {
+    if (w->router_h < 0 || w->router_h > 64) return QTALE_ERR_SHAPE;
+    if (w->router_h == 0 && !w->router_w) return QTALE_ERR_NULL;
+    if (w->router_h > 0 && (!w->router_w1 || !w->router_b1 || !w->router_w2)) return QTALE_ERR_NULL;
   }
   if (ws_bytes < qtale_layer_workspace_bytes(cfg, T, B)) return QTALE_ERR_WORKSPACE;
   const LayerWs lw = carve(cfg, T, B, ws);

@@ -14,4 +14,8 @@ int router_select_launch(const void* x, int T, int d, const float* w_router, flo
                          int32_t* n_exec_out, int32_t* cu_exec_out, int32_t* pos_out, void* ws,
                          size_t ws_bytes, cudaStream_t s);
 
+// MLP router scores (arguments as qtale_router_mlp_scores, already validated)
+int router_mlp_launch(const void* x, int T, int d, const void* w1, const float* b1, const float* w2,
+                      int h, float b2_execute, float b2_bypass, float* scores, cudaStream_t s);
+
 }  // namespace qtale

@@ -133,6 +133,33 @@ def test_selection_at_scale(env, T, B):
     assert _select_case(api, torch, dev, p, cu, api.SELECT_TOPK, k=k) == k
 
 
+@pytest.mark.parametrize("T,d,h", [(100, 256, 8), (777, 1000, 5), (2100, 4096, 64), (33, 64, 17)])
+def test_router_mlp_scores(env, T, d, h):
+    """MLP router (Eq. 2) against the oracle's fp64 evaluation: the hidden layer runs on the
+    tensor cores with fp64 accumulation across 64-feature chunks, so the probabilities agree to
+    1e-6 and a threshold decision on them is the oracle's outside the 1e-6 band.  Covers a
+    feature count that is not a multiple of the chunk, hidden widths that are not multiples of 8
+    and a partial last row block."""
+    api, torch, dev = env
+    x = inputs.hidden_states(80 + h, T, d)
+    w1 = inputs.round_bf16((inputs.normal(81, 1, h * d) * 0.05).astype(np.float32)).reshape(h, d)
+    b1 = (inputs.normal(81, 2, h) * 0.5).astype(np.float32)
+    w2 = (inputs.normal(81, 3, 2 * h) * 0.5).astype(np.float32).reshape(2, h)
+    b2 = np.array([0.2, -0.1], np.float32)
+    p_ref = oracle.router_mlp_scores(x, w1, b1, w2, b2)
+    sc = api.router_mlp_scores(api.to_device_bf16(x, dev), api.to_device_bf16(w1, dev),
+                               torch.from_numpy(b1).to(dev), torch.from_numpy(w2).to(dev), b2)
+    got = sc.cpu().numpy()
+    assert api.device_status() == 0
+    assert np.abs(got - p_ref).max() <= 1e-6
+    assert 0.05 < p_ref.mean() < 0.95
+    cu = np.array([0, T // 3, T], np.int32)
+    theta = float(np.median(p_ref))
+    r = api.router_select(None, None, 0.0, torch.from_numpy(cu).to(dev), api.SELECT_THRESHOLD, theta=theta,
+                          scores_override=sc)
+    _check_select(api, torch, r, p_ref, oracle.select_threshold(p_ref, theta), cu, threshold=theta)
+
+
 @pytest.mark.parametrize("n", [1, 777, 262144, 1500000])
 def test_theta_for_ratio_matches_the_sorted_quantile(env, n):
     """The device-side quantile is a selection, so theta and the count must equal the oracle's

@@ -362,6 +362,43 @@ def test_model_prefill_teacher_forced(env):
     assert per_layer.cpu().numpy().tolist() == [oracle.topk_count(r, T) for r in (0.75, 0.5, 0.25)]
 
 
+def test_layer_with_mlp_router(env):
+    """The layer with the router as a small MLP (Eq. 2) instead of the linear map: selection
+    against the oracle's MLP scores, output with the oracle's mask."""
+    api, torch, dev = env
+    sh = inputs.LayerShape(256, 4, 4, 64, 512, 4, 64)
+    h = 16
+    case = Case.__new__(Case)
+    case.api, case.torch, case.dev, case.sh = api, torch, dev, sh
+    case.cu = inputs.ragged_seqlens(27, 3, 160)
+    case.T, case.B = int(case.cu[-1]), 3
+    case.w = inputs.layer_weights(27, 0, sh)
+    mlp = dict(w1=inputs.round_bf16((inputs.normal(27, 70, h * sh.d) * 0.05).astype(np.float32)).reshape(h, sh.d),
+               b1=(inputs.normal(27, 71, h) * 0.3).astype(np.float32),
+               w2=(inputs.normal(27, 72, 2 * h) * 0.7).astype(np.float32).reshape(2, h),
+               b2=np.array([0.1, 0.0], np.float32))
+    case.w["router_mlp"] = mlp
+    case.x = inputs.hidden_states(27, case.T, sh.d)
+    case.layer = oracle.DenseLayer(sh, case.w)
+    case.lw = api.LayerWeights(case.w, dev)
+    case.cud = torch.from_numpy(case.cu).to(dev)
+    p = oracle.router_mlp_scores(case.x, mlp["w1"], mlp["b1"], mlp["w2"], mlp["b2"])
+    theta = float(np.quantile(p, 0.4))
+    m = oracle.select_threshold(p, theta)
+    ref, n_ref = oracle.layer_forward(case.layer, case.x, case.cu, m)
+    out, n, sc = case.gpu(case.cfg(api.SELECT_THRESHOLD, 1, theta=theta))
+    assert np.abs(sc - p).max() <= 1e-6
+    got = (out != case.x).any(axis=1)
+    assert_selection_matches(np.nonzero(got)[0], int(got.sum()), p, m, theta)
+    assert n == n_ref and 0.5 < n / case.T < 0.7
+    assert_layer_close(out, ref, strict=True)
+    # top-k on the MLP scores
+    k = oracle.topk_count(0.3, case.T)
+    mk = oracle.select_topk(p, k)
+    out, n, _ = case.gpu(case.cfg(api.SELECT_TOPK, 1, ratio=0.3))
+    assert n == k and np.array_equal((out != case.x).any(axis=1), mk.astype(bool))
+
+
 def test_decode_loop_with_diverging_per_layer_caches(env):
     """Prefill of ragged prompts, then 64 decode steps of a 3-layer stack with one theta: each
     layer's cache holds executed tokens only, so its lengths drift apart between sequences and

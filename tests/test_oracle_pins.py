@@ -473,3 +473,40 @@ def test_theta_search_loop_converges_and_falls_back_to_bisection():
     # unreachable target: returns the closest run seen
     th, r, hist = calibrate.search_theta(lambda t: (0.3, 0.4), 0.9, max_iters=5)
     assert r == 0.3 and len(hist) == 5
+
+
+def test_router_mlp_reduces_to_the_linear_router_and_matches_numpy():
+    """Eq. 2 / Eq. 9 with an MLP router.  (a) Hidden units (w, -w) with output weights (+1, -1)
+    on the execute logit rebuild the linear router exactly: max(u, 0) - max(-u, 0) = u, so the
+    scores must be bit-identical to orc_router_scores.  (b) Only the logit difference matters:
+    adding a constant to both logits, or moving weight between the two output rows, leaves p0
+    unchanged.  (c) A numpy fp64 restatement (matrix form) agrees to rounding.  (d) A hidden unit
+    that is never active (large negative bias) contributes nothing."""
+    T, d, h = 50, 96, 5
+    x = inputs.hidden_states(71, T, d)
+    w = inputs.round_bf16((inputs.normal(71, 2, d) * 0.1).astype(np.float32))
+    p_lin, z_lin = oracle.router_scores(x, w, 0.25, return_logits=True)
+    w1 = np.stack([w, -w])
+    p, z = oracle.router_mlp_scores(x, w1, np.zeros(2, np.float32), np.array([[1, -1], [0, 0]], np.float32),
+                                    np.array([0.25, 0.0], np.float32), return_logits=True)
+    assert np.array_equal(p, p_lin) and np.array_equal(z, z_lin)
+    w1 = inputs.round_bf16((inputs.normal(71, 3, h * d) * 0.1).astype(np.float32)).reshape(h, d)
+    b1 = (inputs.normal(71, 4, h) * 0.3).astype(np.float32)
+    w2 = inputs.normal(71, 5, 2 * h).astype(np.float32).reshape(2, h)
+    b2 = np.array([0.1, -0.2], np.float32)
+    p, z = oracle.router_mlp_scores(x, w1, b1, w2, b2, return_logits=True)
+    a = np.maximum(x.astype(np.float64) @ w1.astype(np.float64).T + b1, 0)
+    g = a @ w2.astype(np.float64).T + b2
+    assert np.allclose(z, g[:, 0] - g[:, 1], rtol=1e-12, atol=1e-12)
+    assert np.allclose(p, np.exp(g[:, 0]) / np.exp(g).sum(axis=1), atol=1e-7)
+    p_shift = oracle.router_mlp_scores(x, w1, b1, w2, b2 + np.float32(3.0))
+    assert np.abs(p_shift - p).max() <= 1e-7
+    w2d = np.stack([w2[0] - w2[1], np.zeros(h, np.float32)]).astype(np.float32)
+    p_diff = oracle.router_mlp_scores(x, w1, b1, w2d, np.array([b2[0] - b2[1], 0], np.float32))
+    assert np.abs(p_diff - p).max() <= 1e-6
+    b1_dead = b1.copy()
+    b1_dead[2] = -1e6
+    w2_zero = w2.copy()
+    w2_zero[:, 2] = 0
+    assert np.array_equal(oracle.router_mlp_scores(x, w1, b1_dead, w2, b2),
+                          oracle.router_mlp_scores(x, w1, b1, w2_zero, b2))
