@@ -581,7 +581,7 @@ def run_ours(args):
             s3, B3 = c3["shape"], c3["B"]
             lw3 = timing_layer(torch, api, dev, gen, s3)
             cap = 2048 + 64
-            kv = api.KvCache(B3, cap, s3.kv_dim, dev, act_dtype=api.ACT_F16)
+            kv = api.KvCache(B3, cap, s3.kv_dim, dev, act_dtype=api.ACT_F16, head_dim=s3.head_dim)
             kv.k.normal_(generator=gen)
             kv.v.normal_(generator=gen)
             len0 = torch.full((B3,), 2048, dtype=torch.int32, device=dev)
@@ -641,7 +641,7 @@ def run_ours(args):
             lm_head = (torch.randn(Vd, s3.d, device=dev, generator=gen) * 0.02).to(torch.bfloat16)
             fg = torch.ones(s3.d, dtype=torch.float32, device=dev)
             cap = len0_d + 2 * steps_d + 8
-            caches = [api.KvCache(Bd, cap, s3.kv_dim, dev, act_dtype=api.ACT_F16) for _ in range(Ld)]
+            caches = [api.KvCache(Bd, cap, s3.kv_dim, dev, act_dtype=api.ACT_F16, head_dim=s3.head_dim) for _ in range(Ld)]
             for c in caches:
                 c.k.normal_(generator=gen)
                 c.v.normal_(generator=gen)

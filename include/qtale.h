@@ -293,10 +293,16 @@ typedef struct {
  * The packed weights are dequantised inside the kernel to the 16-bit format of
  * `a` (exact (code - zero) * scale in fp32, one rounding) and accumulated in
  * fp32.
+ * ws / ws_bytes: optional scratch of qtale_wq_gemm_workspace_bytes() (NULL / 0:
+ * none).  With it, products of at most 64 token rows (a decode step) run with
+ * the input dimension split over the SMs, the partial sums meeting in the
+ * scratch (added in a fixed order: results do not depend on timing); without it
+ * they run on a kernel that needs no scratch.  Larger products never use it.
  */
+size_t qtale_wq_gemm_workspace_bytes(void);
 int qtale_wq_gemm(const void* a, int lda, const int32_t* m_dev, int M_cap, const qtale_wq_weight* w,
                   int act_dtype, int epilogue, const qtale_epilogue_args* epi, void* y, int ldy,
-                  void* stream);
+                  void* ws, size_t ws_bytes, void* stream);
 
 /* ------------------------------------------------------------------------- */
 /* Layer and model                                                             */
@@ -342,8 +348,10 @@ typedef struct {
  * stays at cap, and QTALE_ERR_CAPACITY is recorded in the device status word
  * (the layer output of that sequence is then not meaningful). */
 typedef struct {
-  void* k;         /* act_dtype [B, cap, n_kv_heads * head_dim], rotary already applied */
-  void* v;         /* act_dtype [B, cap, n_kv_heads * head_dim]                         */
+  void* k;         /* act_dtype [B, n_kv_heads, cap, head_dim], rotary already applied: the
+                      entries of one (sequence, head) are contiguous, so the decode
+                      attention streams them at full memory bandwidth                   */
+  void* v;         /* act_dtype [B, n_kv_heads, cap, head_dim]                          */
   int32_t* kv_len; /* int32 [B], entries in use per sequence (updated)             */
   int cap;
 } qtale_kv_cache;
@@ -424,7 +432,7 @@ size_t qtale_model_decode_workspace_bytes(const qtale_model_config* cfg, int B_c
  *   token in its sequence (rotary position; counts bypassed tokens too), advanced
  *   by one for every valid sequence when the step is done; valid [B] uint8 or
  *   NULL (0 = finished sequence: never executes, position kept); caches: HOST
- *   array [n_layers], each [B, cap, n_kv_heads * head_dim] with its own kv_len;
+ *   array [n_layers], each [B, n_kv_heads, cap, head_dim] with its own kv_len;
  *   hidden_out [B, d] bf16; logits_out fp32 [B, vocab] or NULL; next_ids_out [B]
  *   int32 or NULL: greedy choice (largest logit, lowest index among equal ones);
  *   per_layer_n_exec [n_layers] or NULL: sequences executed by each layer in

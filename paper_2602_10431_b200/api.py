@@ -28,6 +28,7 @@ EXPORTS = [
     "qtale_router_select_workspace_bytes", "qtale_router_select", "qtale_router_select_static",
     "qtale_index_bookkeeping",
     "qtale_compact", "qtale_scatter_add", "qtale_wq_repack", "qtale_wq_gemm",
+    "qtale_wq_gemm_workspace_bytes",
     "qtale_layer_workspace_bytes", "qtale_layer_forward", "qtale_model_workspace_bytes",
     "qtale_model_prefill", "qtale_theta_workspace_bytes", "qtale_theta_for_ratio",
     "qtale_model_decode_workspace_bytes", "qtale_model_decode_step", "qtale_router_mlp_scores",
@@ -109,7 +110,9 @@ def lib():
                                       C.c_int, C.c_int, C.c_void_p, C.POINTER(C.c_size_t)]
         L.qtale_wq_gemm.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.POINTER(WqWeight),
                                     C.c_int, C.c_int, C.POINTER(EpilogueArgs), C.c_void_p, C.c_int,
-                                    C.c_void_p]
+                                    C.c_void_p, C.c_size_t, C.c_void_p]
+        L.qtale_wq_gemm_workspace_bytes.restype = C.c_size_t
+        L.qtale_wq_gemm_workspace_bytes.argtypes = []
         L.qtale_layer_workspace_bytes.restype = C.c_size_t
         L.qtale_layer_workspace_bytes.argtypes = [C.POINTER(LayerConfig), C.c_int, C.c_int]
         L.qtale_layer_forward.argtypes = [
@@ -315,8 +318,12 @@ class QuantWeight:
         self.c = WqWeight(self.blob.data_ptr(), self.N, self.K, self.bits, self.group, row_mode)
 
 
+def wq_gemm_workspace_bytes() -> int:
+    return int(lib().qtale_wq_gemm_workspace_bytes())
+
+
 def wq_gemm(a, w: QuantWeight, m_dev=None, epilogue=EPI_STORE_16, y=None, idx=None, resid=None,
-            dst=None, rope_cs=None, rope_features=0):
+            dst=None, rope_cs=None, rope_features=0, ws=None):
     """qtale_wq_gemm.  a bf16 or fp16 [M_cap, K] (its dtype is the act_dtype); returns y
     (or dst for RESID_SCATTER)."""
     M_cap, lda = int(a.shape[0]), int(a.stride(0))
@@ -334,7 +341,9 @@ def wq_gemm(a, w: QuantWeight, m_dev=None, epilogue=EPI_STORE_16, y=None, idx=No
         y = torch.zeros(M_cap, n_out, dtype=dt, device=a.device)
     check(lib().qtale_wq_gemm(_ptr(a), lda, _ptr(m_dev), M_cap, C.byref(w.c), act_dtype, int(epilogue),
                               C.byref(epi) if epi is not None else None, _ptr(y),
-                              int(y.stride(0)) if y is not None else 0, _stream()), "qtale_wq_gemm")
+                              int(y.stride(0)) if y is not None else 0, _ptr(ws),
+                              ws.numel() * ws.element_size() if ws is not None else 0, _stream()),
+          "qtale_wq_gemm")
     return dst if epilogue == EPI_RESID_SCATTER else y
 
 
@@ -388,13 +397,29 @@ class LayerWeights:
 
 
 class KvCache:
-    def __init__(self, B, cap, kv_dim, device="cuda", act_dtype=ACT_F16):
+    """Per-layer cache of the executed tokens' keys / values, [B, n_kv_heads, cap, head_dim]."""
+
+    def __init__(self, B, cap, kv_dim, device="cuda", act_dtype=ACT_F16, head_dim=128):
         dt = act_torch_dtype(act_dtype)
-        self.k = torch.zeros(B, cap, kv_dim, dtype=dt, device=device)
-        self.v = torch.zeros(B, cap, kv_dim, dtype=dt, device=device)
+        self.B, self.cap, self.head_dim, self.n_kv_heads = B, cap, head_dim, kv_dim // head_dim
+        self.k = torch.zeros(B, self.n_kv_heads, cap, head_dim, dtype=dt, device=device)
+        self.v = torch.zeros(B, self.n_kv_heads, cap, head_dim, dtype=dt, device=device)
         self.kv_len = torch.zeros(B, dtype=torch.int32, device=device)
-        self.cap = cap
         self.c = KvCacheC(self.k.data_ptr(), self.v.data_ptr(), self.kv_len.data_ptr(), cap)
+
+    def k_view(self):
+        """Keys as a [B, cap, n_kv_heads, head_dim] view (entry-major, for filling / inspecting)."""
+        return self.k.permute(0, 2, 1, 3)
+
+    def v_view(self):
+        return self.v.permute(0, 2, 1, 3)
+
+    def k_rows(self):
+        """Keys as a [B, cap, n_kv_heads * head_dim] copy: one row per cached token."""
+        return self.k_view().reshape(self.B, self.cap, -1)
+
+    def v_rows(self):
+        return self.v_view().reshape(self.B, self.cap, -1)
 
 
 def layer_workspace_bytes(cfg: LayerConfig, T_cap: int, B_cap: int) -> int:

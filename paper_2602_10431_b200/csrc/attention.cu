@@ -53,9 +53,10 @@ __global__ void __launch_bounds__(kDecThreads)
 #pragma unroll
     for (int e = 0; e < 8; ++e) acc[r][e] = 0.f;
   }
-  const size_t row_stride = (size_t)Hkv * HD;
-  const __nv_bfloat16* kb = cache_k + ((size_t)b * cap) * row_stride + (size_t)hk * HD + sub * 8;
-  const __nv_bfloat16* vb = cache_v + ((size_t)b * cap) * row_stride + (size_t)hk * HD + sub * 8;
+  // cache layout [B, Hkv, cap, HD]: the keys of this (sequence, head) are one contiguous stream
+  const size_t row_stride = HD;
+  const __nv_bfloat16* kb = cache_k + (((size_t)b * Hkv + hk) * cap) * HD + sub * 8;
+  const __nv_bfloat16* vb = cache_v + (((size_t)b * Hkv + hk) * cap) * HD + sub * 8;
   constexpr int UNROLL = 4;
   // the trip count is the same for every lane (the shuffles below name the whole warp); keys
   // past the end are masked by `ok`

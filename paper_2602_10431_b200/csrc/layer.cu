@@ -28,6 +28,8 @@ struct LayerWs {
   float* u;     // fp32 [T, d]            x + attention branch
   void* gu;     // bf16 [T, 2 F]          gate | up (only when SwiGLU is not fused)
   void* act;    // bf16 [T, F]
+  void* splitk; // scratch of the split-K GEMMs of a decode step
+  size_t splitk_bytes;
   size_t total;
 };
 
@@ -56,6 +58,8 @@ static LayerWs carve(const qtale_layer_config* c, int T, int B, void* base) {
   w.u = reinterpret_cast<float*>(take(t * c->d * 4));
   w.gu = take(t * 2 * c->ffn * 2);
   w.act = take(t * c->ffn * 2);
+  w.splitk_bytes = wq_splitk_workspace_bytes();
+  w.splitk = take(w.splitk_bytes);
   w.total = off;
   return w;
 }
@@ -114,12 +118,21 @@ static int layer_forward_impl(const qtale_layer_config* c, const qtale_layer_wei
     QTALE_TRY(router_select_launch(x, T, d, w->router_w, w->router_b, scores_override, valid,
                                    cu_seqlens, B, pos0, c->select_mode, c->theta, k, ratio,
                                    scores_out ? scores_out : ws.scores, ws.idx, ws.n_exec,
-                                   ws.cu_exec, ws.pos, ws.router_ws, ws.router_ws_bytes, s));
+                                   ws.cu_exec, ws.pos, ws.router_ws, ws.router_ws_bytes, s,
+                                   n_exec_out));
   }
-  if (n_exec_out &&
+  if (n_exec_out && c->select_mode == QTALE_SELECT_FORCED &&
       cudaMemcpyAsync(n_exec_out, ws.n_exec, sizeof(int32_t), cudaMemcpyDeviceToDevice, s) !=
           cudaSuccess)
     return QTALE_ERR_CUDA;
+
+  // decode steps: the linears run with the K dimension split over the SMs (ticket words zeroed)
+  void* sk = nullptr;
+  if (phase == QTALE_PHASE_DECODE && T <= 64) {
+    sk = ws.splitk;
+    if (cudaMemsetAsync(sk, 0, wq_splitk_ticket_bytes(), s) != cudaSuccess) return QTALE_ERR_CUDA;
+  }
+  const size_t skb = ws.splitk_bytes;
 
   // 2. gather the executed tokens and apply the first RMSNorm; the same launch writes the
   //    rotary table of their (original) positions and, for the prefill attention's tiled loads,
@@ -142,15 +155,15 @@ static int layer_forward_impl(const qtale_layer_config* c, const qtale_layer_wei
     memset(&er, 0, sizeof(er));
     er.rope_cs = ws.cs;
     er.rope_features = qd + kvd;
-    QTALE_TRY(wq_gemm_launch(ws.hn, d, ws.n_exec, T, &w->qkv, act, QTALE_EPI_ROPE, &er, ws.qkv, nqkv, s));
+    QTALE_TRY(wq_gemm_launch(ws.hn, d, ws.n_exec, T, &w->qkv, act, QTALE_EPI_ROPE, &er, ws.qkv, nqkv, s, sk, skb, 0));
   } else {
     QTALE_TRY(wq_gemm_launch(ws.hn, d, ws.n_exec, T, &w->qkv, act, QTALE_EPI_STORE_16, nullptr, ws.qkv,
-                             nqkv, s));
+                             nqkv, s, sk, skb, 0));
     QTALE_TRY(launch_rope(ws.qkv, ws.n_exec, T, nqkv, H + Hkv, hd, ws.cs, act, s));
   }
   // 5. attention among executed tokens (+ cache)
   if (kv) {
-    QTALE_TRY(launch_kv_append(ws.qkv, ws.n_exec, T, nqkv, qd, kvd, ws.cu_exec, B, kv->k, kv->v,
+    QTALE_TRY(launch_kv_append(ws.qkv, ws.n_exec, T, nqkv, qd, kvd, hd, ws.cu_exec, B, kv->k, kv->v,
                                kv->kv_len, kv->cap, s));
   }
   if (phase == QTALE_PHASE_DECODE) {
@@ -167,16 +180,16 @@ static int layer_forward_impl(const qtale_layer_config* c, const qtale_layer_wei
   e.ld_resid = d;
   e.dst = nullptr;
   e.ld_dst = 0;
-  QTALE_TRY(wq_gemm_launch(ws.ao, qd, ws.n_exec, T, &w->o, act, QTALE_EPI_RESID_F32, &e, ws.u, d, s));
+  QTALE_TRY(wq_gemm_launch(ws.ao, qd, ws.n_exec, T, &w->o, act, QTALE_EPI_RESID_F32, &e, ws.u, d, s, sk, skb, 1));
   // 7. second RMSNorm
   QTALE_TRY(launch_rmsnorm_f32(ws.u, ws.n_exec, T, d, w->gamma2, c->rms_eps, act, ws.hn, s));
   // 8. gate / up projections and SwiGLU
   if (w->gate_up.row_mode == QTALE_WQ_ROWS_SWIGLU) {
     QTALE_TRY(wq_gemm_launch(ws.hn, d, ws.n_exec, T, &w->gate_up, act, QTALE_EPI_SWIGLU, nullptr, ws.act,
-                             F, s));
+                             F, s, sk, skb, 2));
   } else {
     QTALE_TRY(wq_gemm_launch(ws.hn, d, ws.n_exec, T, &w->gate_up, act, QTALE_EPI_STORE_16, nullptr,
-                             ws.gu, 2 * F, s));
+                             ws.gu, 2 * F, s, sk, skb, 2));
     QTALE_TRY(launch_swiglu(ws.gu, ws.n_exec, T, F, ws.act, act, s));
   }
   // 9. down projection + residual scatter: x[idx] = bf16(u + MLP branch)   (Eq. 3)
@@ -185,7 +198,7 @@ static int layer_forward_impl(const qtale_layer_config* c, const qtale_layer_wei
   e.dst = x;
   e.ld_dst = d;
   QTALE_TRY(wq_gemm_launch(ws.act, F, ws.n_exec, T, &w->down, act, QTALE_EPI_RESID_SCATTER, &e, nullptr,
-                           0, s));
+                           0, s, sk, skb, 3));
   return QTALE_OK;
 }
 

@@ -40,6 +40,7 @@ struct RouterParams {
   float* scores;
   int32_t* idx;
   int32_t* n_exec;
+  int32_t* n_exec_copy;  // optional second destination of the count
   int32_t* cu_exec;
   int32_t* pos;
   uint32_t* ws;
@@ -70,6 +71,7 @@ __device__ __forceinline__ void st_release(uint32_t* p, uint32_t v) {
 // Barrier over the whole (co-resident) grid: arrival number `target` completes it.  Bounded.
 __device__ bool grid_barrier(const RouterParams& p, uint32_t target, int* s_abort) {
   __syncthreads();
+  if (gridDim.x == 1) return true;  // a single CTA: nothing to wait for, no counter touched
   if (threadIdx.x == 0) {
     __threadfence();
     atomicAdd(p.ws + kWsBarrier, 1u);
@@ -497,7 +499,10 @@ __global__ void __launch_bounds__(kRouterThreads, 2) router_select_kernel(const 
     run += slab_total;
   }
   if (cta == G - 1) {
-    if (tid == 0) *p.n_exec = run;
+    if (tid == 0) {
+      *p.n_exec = run;
+      if (p.n_exec_copy) *p.n_exec_copy = run;
+    }
     for (int q = tid; q <= p.B; q += nthr)
       if (__ldg(p.cu_seqlens + q) >= T) p.cu_exec[q] = run;
   }
@@ -562,7 +567,7 @@ int router_select_launch(const void* x, int T, int d, const float* w_router, flo
                          const int32_t* cu_seqlens, int B, const int32_t* pos0, int mode,
                          float theta, int k, double ratio, float* scores_out, int32_t* idx_out,
                          int32_t* n_exec_out, int32_t* cu_exec_out, int32_t* pos_out, void* ws,
-                         size_t ws_bytes, cudaStream_t s) {
+                         size_t ws_bytes, cudaStream_t s, int32_t* n_exec_copy) {
   if (!scores_out || !idx_out || !n_exec_out || !cu_exec_out || !pos_out || !cu_seqlens || !ws)
     return QTALE_ERR_NULL;
   if (!scores_override && (!x || !w_router)) return QTALE_ERR_NULL;
@@ -583,6 +588,7 @@ int router_select_launch(const void* x, int T, int d, const float* w_router, flo
   p.scores = scores_out;
   p.idx = idx_out;
   p.n_exec = n_exec_out;
+  p.n_exec_copy = n_exec_copy;
   p.cu_exec = cu_exec_out;
   p.pos = pos_out;
   p.ws = static_cast<uint32_t*>(ws);
@@ -621,7 +627,9 @@ int router_select_launch(const void* x, int T, int d, const float* w_router, flo
   grid = (T + chunk - 1) / chunk;
   p.chunk = chunk;
 
-  if (cudaMemsetAsync(ws, 0, (size_t)(kWsCount + grid) * sizeof(uint32_t), s) != cudaSuccess)
+  // a single CTA (decode steps, small calls) neither waits nor counts: nothing to clear
+  if (grid > 1 &&
+      cudaMemsetAsync(ws, 0, (size_t)(kWsCount + grid) * sizeof(uint32_t), s) != cudaSuccess)
     return QTALE_ERR_CUDA;
   void* args[] = {&p};
   return launch_status(cudaLaunchCooperativeKernel(router_select_kernel, dim3(grid),

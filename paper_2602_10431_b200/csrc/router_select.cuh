@@ -12,7 +12,7 @@ int router_select_launch(const void* x, int T, int d, const float* w_router, flo
                          const int32_t* cu_seqlens, int B, const int32_t* pos0, int mode,
                          float theta, int k, double ratio, float* scores_out, int32_t* idx_out,
                          int32_t* n_exec_out, int32_t* cu_exec_out, int32_t* pos_out, void* ws,
-                         size_t ws_bytes, cudaStream_t s);
+                         size_t ws_bytes, cudaStream_t s, int32_t* n_exec_copy = nullptr);
 
 // MLP router scores (arguments as qtale_router_mlp_scores, already validated)
 int router_mlp_launch(const void* x, int T, int d, const void* w1, const float* b1, const float* w2,

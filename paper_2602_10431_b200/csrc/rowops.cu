@@ -247,7 +247,7 @@ __global__ void __launch_bounds__(kRowThreads)
 // ---- KV-cache append of the executed tokens' K (rotated) and V ------------------
 __global__ void __launch_bounds__(kRowThreads)
     kv_append_kernel(const uint4* __restrict__ qkv, const int32_t* __restrict__ n_exec, int cap_rows,
-                     int ld, int q_dim, int kv_dim, const int32_t* __restrict__ cu_exec, int B,
+                     int ld, int q_dim, int kv_dim, int hd, const int32_t* __restrict__ cu_exec, int B,
                      uint4* __restrict__ cache_k, uint4* __restrict__ cache_v,
                      const int32_t* __restrict__ kv_len, int cap) {
   const int n = min(*n_exec, cap_rows);
@@ -264,7 +264,9 @@ __global__ void __launch_bounds__(kRowThreads)
     }
     const int slot = kv_len[lo] + (i - cu_exec[lo]);
     if (slot >= cap) continue;  // cache full: kv_len_update_kernel records QTALE_ERR_CAPACITY
-    const size_t dst = ((size_t)lo * cap + slot) * kc + c;
+    // cache layout [B, Hkv, cap, hd]
+    const int hc = hd >> 3, head = c / hc, within = c % hc;
+    const size_t dst = (((size_t)lo * (kv_dim / hd) + head) * cap + slot) * hc + within;
     cache_k[dst] = qkv[(size_t)i * ldc + (q_dim >> 3) + c];
     cache_v[dst] = qkv[(size_t)i * ldc + ((q_dim + kv_dim) >> 3) + c];
   }
@@ -425,10 +427,10 @@ int launch_swiglu(const void* gu, const int32_t* n_exec, int cap, int F, void* a
 }
 
 int launch_kv_append(const void* qkv, const int32_t* n_exec, int cap_rows, int ld, int q_dim,
-                     int kv_dim, const int32_t* cu_exec, int B, void* cache_k, void* cache_v,
+                     int kv_dim, int hd, const int32_t* cu_exec, int B, void* cache_k, void* cache_v,
                      int32_t* kv_len, int cap, cudaStream_t s) {
   kv_append_kernel<<<row_grid(4), kRowThreads, 0, s>>>(
-      static_cast<const uint4*>(qkv), n_exec, cap_rows, ld, q_dim, kv_dim, cu_exec, B,
+      static_cast<const uint4*>(qkv), n_exec, cap_rows, ld, q_dim, kv_dim, hd, cu_exec, B,
       static_cast<uint4*>(cache_k), static_cast<uint4*>(cache_v), kv_len, cap);
   if (cudaGetLastError() != cudaSuccess) return QTALE_ERR_CUDA;
   kv_len_update_kernel<<<(B + 255) / 256, 256, 0, s>>>(kv_len, cu_exec, B, cap, device_status_ptr());

@@ -27,7 +27,7 @@ int launch_rope(void* qkv, const int32_t* n_exec, int cap, int ld, int n_rot, in
 int launch_swiglu(const void* gu, const int32_t* n_exec, int cap, int F, void* act, int act_dtype,
                   cudaStream_t s);
 int launch_kv_append(const void* qkv, const int32_t* n_exec, int cap_rows, int ld, int q_dim,
-                     int kv_dim, const int32_t* cu_exec, int B, void* cache_k, void* cache_v,
+                     int kv_dim, int hd, const int32_t* cu_exec, int B, void* cache_k, void* cache_v,
                      int32_t* kv_len, int cap, cudaStream_t s);
 int launch_iota(int32_t* cu, int n, cudaStream_t s);
 int launch_advance_pos(int32_t* pos, const uint8_t* valid, int B, cudaStream_t s);

@@ -56,6 +56,7 @@ constexpr int kAColsPerSlot = kKB / 2;   // two 16-bit values per 32-bit TMEM co
 constexpr int kEpiCols = 16;             // tokens per epilogue chunk
 constexpr int kEpiRowWords = 36;         // padded row (32 fp32 + 4) of the epilogue staging tile
 constexpr int kEpiWarpBytes = kEpiCols * kEpiRowWords * 4;
+constexpr size_t kSplitTileBytes = (size_t)2 * 128 * 64 * 4;  // one fp32 partial tile: 256 rows x 64 tokens
 
 template <int TN, int BITS>
 struct GemmCfg {
@@ -108,6 +109,9 @@ struct GemmParams {
   const float2* rope_cs;   // ROPE epilogue: (cos, sin) [M_cap, rope_hd / 2]
   int rope_hd;             // head dim of the rotary layout (ROPE row modes), else 0
   int rope_limit;          // output features below this are rotated (query and key heads)
+  int split_k;             // single-CTA kernel: K slices per output tile (1: none)
+  float* partial;          // split_k > 1: fp32 partial tiles [tile][slice][256 rows][TN tokens]
+  int* tickets;            // split_k > 1: one counter per output tile, zero at launch
   int* status;
 };
 
@@ -118,6 +122,7 @@ struct __align__(8) GemmShared {
   uint64_t d_full[2], d_empty[2];        // the accumulators, per row tile
   uint32_t tmem_base;
   volatile int abort_flag;
+  uint64_t part_bar;  // split K: all warps have written their part of the partial tile
 };
 
 // Bounded wait: gives up after kWaitSlices suspended tests, records a timeout and raises
@@ -397,7 +402,40 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const float*
   }
 }
 
-template <int TN, int BITS, int ACT>
+// Split K: sum of the S partial tiles' 16 columns of one row (slice order, so the result does not
+// depend on timing), written transposed into the warp's staging tile.  Four slices (sixteen
+// 16-byte loads) are requested at a time.
+__device__ __forceinline__ void splitk_sum_to_stage(const float* part, int S, size_t slice_stride,
+                                                 float* stage, int lane) {
+  float acc[kEpiCols];
+#pragma unroll
+  for (int c = 0; c < kEpiCols; ++c) acc[c] = 0.f;
+  constexpr int kBatch = 4;
+#pragma unroll 1
+  for (int sl0 = 0; sl0 < S; sl0 += kBatch) {
+    float4 v[kBatch][kEpiCols / 4];
+#pragma unroll
+    for (int b = 0; b < kBatch; ++b) {
+      const float4* src = reinterpret_cast<const float4*>(part + (size_t)min(sl0 + b, S - 1) * slice_stride);
+#pragma unroll
+      for (int q4 = 0; q4 < kEpiCols / 4; ++q4) v[b][q4] = __ldcg(src + q4);
+    }
+#pragma unroll
+    for (int b = 0; b < kBatch; ++b) {
+      if (sl0 + b < S) {
+#pragma unroll
+        for (int q4 = 0; q4 < kEpiCols / 4; ++q4) {
+          acc[4 * q4] += v[b][q4].x; acc[4 * q4 + 1] += v[b][q4].y;
+          acc[4 * q4 + 2] += v[b][q4].z; acc[4 * q4 + 3] += v[b][q4].w;
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int c = 0; c < kEpiCols; ++c) stage[c * kEpiRowWords + lane] = acc[c];
+}
+
+template <int TN, int BITS, int ACT, bool SPLIT>
 __global__ void __launch_bounds__(kGemmThreads, 1)
     wq_gemm_kernel(const __grid_constant__ TmapSet tmaps_x,
                    const __grid_constant__ CUtensorMap tmap_w, const GemmParams p) {
@@ -431,6 +469,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
       mbar_init(&sh.d_full[r], 1);
       mbar_init(&sh.d_empty[r], 8);
     }
+    mbar_init(&sh.part_bar, kDequantWarps);
     sh.abort_flag = 0;
     fence_barrier_init();
   }
@@ -466,11 +505,24 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
       if (best < 0 || cost < best) { best = cost; TW = w; }
     }
   }
+  if (SPLIT) TW = TN;  // partial tiles are laid out for one full-width token tile
   const CUtensorMap* tmap_x = &tmaps_x.m[TW / 32 - 1];
   // tile index = mt * n_rp + rp: CTAs running at the same time share a few token tiles and
   // sweep the (small, L2-resident) packed weights, so activations stream from HBM once
   const int n_mt = (M + TW - 1) / TW;
-  const int total_tiles = n_mt * n_rp;
+  // Split K (token counts of a decode step): a tile is (token tile, K slice, row-tile group);
+  // every slice leaves an fp32 partial tile in global memory and counts itself in; when a CTA
+  // has done all its tiles it sums its share of each output tile it took part in.
+  const int S = SPLIT ? max(p.split_k, 1) : 1;
+  const int total_tiles = n_mt * n_rp * S;
+  auto tile_coords = [&](int tile, int& rp, int& mt, int& ks, int& kb0, int& kb1) {
+    rp = tile % n_rp;
+    const int q = tile / n_rp;
+    ks = q % S;
+    mt = q / S;
+    kb0 = (int)((long)ks * nkb / S);
+    kb1 = (int)((long)(ks + 1) * nkb / S);
+  };
   const uint32_t x_stage_tx = (uint32_t)TW * 128u + (BITS == 16 ? kTileRows * 128 : 0);
 
   if (warp == 0 || warp == 2) {
@@ -480,8 +532,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
       Ring rx, rw;
       int count = 0;
       for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
-        const int rp = tile % n_rp, mt = tile / n_rp;
-        for (int kb = 0; kb < nkb; ++kb, ++count) {
+        int rp, mt, ks, kb0, kb1;
+        tile_coords(tile, rp, mt, ks, kb0, kb1);
+        for (int kb = kb0; kb < kb1; ++kb, ++count) {
           if ((count & 1) == parity) {
             if (BITS != 16) {
               // one contiguous chunk per (row-tile pair, K block): both tiles' codes, each
@@ -517,12 +570,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
       Ring rx, ra;
       uint32_t dph = 0;
       for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
-        const int rp = tile % n_rp;
+        int rp, mt_, ks_, kb0, kb1;
+        tile_coords(tile, rp, mt_, ks_, kb0, kb1);
         const bool has_tile = r < RT && rp * RT + r < p.n_tiles;
         // the accumulator is free once the previous tile has been drained
         if (!wait_or_abort(&sh.d_empty[r], dph ^ 1u, &sh, p.status)) goto mma_done;
         tc_fence_after();
-        for (int kb = 0; kb < nkb; ++kb) {
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (!wait_or_abort(&sh.full_x[rx.s], rx.ph, &sh, p.status)) goto mma_done;
           if (BITS != 16) {
             if (!wait_or_abort(&sh.a_full[r][ra.s], ra.ph, &sh, p.status)) goto mma_done;
@@ -533,7 +587,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
             const uint64_t b_desc = smem_desc_sw128(smem_u32(st));
 #pragma unroll
             for (int j = 0; j < kKB / 16; ++j) {
-              const uint32_t acc = (kb | j) != 0 ? 1u : 0u;
+              const uint32_t acc = (kb != kb0 || j != 0) ? 1u : 0u;
               if (BITS == 16) {
                 const uint64_t a_desc = smem_desc_sw128(smem_u32(st + Cfg::kXBytes));
                 mma_ss(d_tmem, a_desc + 2u * j, b_desc + 2u * j, idesc, acc);
@@ -569,11 +623,12 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
     uint32_t dph = 0;
     int count = 0;  // running K block number, as in the producers
     for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
-      const int rp = tile % n_rp, mt = tile / n_rp;
+      int rp, mt, ks, kb0, kb1;
+      tile_coords(tile, rp, mt, ks, kb0, kb1);
       const int nt = rp * RT + g;
       const bool has_tile = g < RT && nt < p.n_tiles;
       if (BITS != 16) {
-        for (int kb = 0; kb < nkb; ++kb, ++count) {
+        for (int kb = kb0; kb < kb1; ++kb, ++count) {
           if ((count & 1) != h) {  // the other set's block (ring slots alternate with the parity)
             rw.advance(SW);
             ra.advance(SA);
@@ -663,33 +718,116 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
       // ---- accumulator g, one lane quadrant per warp ----
       if (!wait_or_abort(&sh.d_full[g], dph, &sh, p.status)) goto role_done;
       tc_fence_after();
-      if (has_tile) {
-        const int m_base = mt * TW;
-        const uint32_t d_taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + g * Cfg::kDCols;
-        uint32_t r[kEpiCols];
-        if (m_base + h * kEpiCols < M) tmem_ld_x16(d_taddr + h * kEpiCols, r);
+      if (!SPLIT) {
+        if (has_tile) {
+          const int m_base = mt * TW;
+          const uint32_t d_taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + g * Cfg::kDCols;
+          uint32_t r[kEpiCols];
+          if (m_base + h * kEpiCols < M) tmem_ld_x16(d_taddr + h * kEpiCols, r);
 #pragma unroll 1
-        for (int c0 = h * kEpiCols; c0 < TW; c0 += 2 * kEpiCols) {
-          const int m0 = m_base + c0;
-          if (m0 >= M) break;
-          tmem_wait_ld();
+          for (int c0 = h * kEpiCols; c0 < TW; c0 += 2 * kEpiCols) {
+            const int m0 = m_base + c0;
+            if (m0 >= M) break;
+            tmem_wait_ld();
 #pragma unroll
-          for (int c = 0; c < kEpiCols; ++c) stage[c * kEpiRowWords + lane] = __uint_as_float(r[c]);
-          __syncwarp();
-          // the next chunk's accumulator read overlaps this chunk's global traffic
-          if (c0 + 2 * kEpiCols < TW && m0 + 2 * kEpiCols < M) tmem_ld_x16(d_taddr + c0 + 2 * kEpiCols, r);
+            for (int c = 0; c < kEpiCols; ++c) stage[c * kEpiRowWords + lane] = __uint_as_float(r[c]);
+            __syncwarp();
+            // the next chunk's accumulator read overlaps this chunk's global traffic
+            if (c0 + 2 * kEpiCols < TW && m0 + 2 * kEpiCols < M) tmem_ld_x16(d_taddr + c0 + 2 * kEpiCols, r);
+            EpiOperands eo;
+            epilogue_fetch_tok<-1>(p, lane, m0, M, eo);
+            epilogue_fetch<-1>(p, lane, nt, quad, m0, M, eo);
+            epilogue_chunk<ACT, -1>(p, stage, lane, nt, quad, m0, M, eo);
+            __syncwarp();
+          }
+          tmem_wait_ld();
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh.d_empty[g]);
+      } else {
+        // split K: the raw accumulator goes to this slice's partial tile (row L of row tile g,
+        // TN tokens per row), then the accumulator is handed back at once
+        const int m_base = mt * TW;
+        const int out_tile = mt * n_rp + rp;
+        float* part = p.partial + ((size_t)out_tile * S) * (2 * kTileRows * TN) +
+                      (size_t)(g * kTileRows + L) * TN;
+        if (has_tile) {
+          const uint32_t d_taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + g * Cfg::kDCols;
+          for (int c0 = h * kEpiCols; c0 < TW; c0 += 2 * kEpiCols) {
+            if (m_base + c0 >= M) break;
+            uint32_t r[kEpiCols];
+            tmem_ld_x16(d_taddr + c0, r);
+            tmem_wait_ld();
+            float4* dst = reinterpret_cast<float4*>(part + (size_t)ks * (2 * kTileRows * TN) + c0);
+#pragma unroll
+            for (int q4 = 0; q4 < kEpiCols / 4; ++q4)
+              dst[q4] = make_float4(__uint_as_float(r[4 * q4]), __uint_as_float(r[4 * q4 + 1]),
+                                    __uint_as_float(r[4 * q4 + 2]), __uint_as_float(r[4 * q4 + 3]));
+          }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh.d_empty[g]);
+        // this slice is there: one arrival per warp on part_bar, then one thread counts it in
+        // global memory (the fences order the partial tile before the count)
+        __threadfence();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh.part_bar);
+        if (warp == 4) {
+          if (!wait_or_abort(&sh.part_bar, dph, &sh, p.status)) goto role_done;
+          if (lane == 0) {
+            __threadfence();
+            atomicAdd(p.tickets + out_tile, 1);
+          }
+        }
+      }
+      dph ^= 1u;
+    }
+    if (SPLIT) {
+      // ---- split K, second half: every CTA has delivered all its partial tiles; now each sums
+      // ---- its share of every output tile it took part in.  An output tile is 32 units of
+      // ---- (32 weight rows, 16 tokens); slice ks takes the units ks, ks + S, ...; a unit is one
+      // ---- warp's work: the S partials are added in slice order (the result does not depend on
+      // ---- timing) and go through the usual epilogue.  Waiting only starts here, after all of
+      // ---- this CTA's own partials are out, so CTAs cannot wait for each other in a circle.
+      const int wi = warp - 4;
+      for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+        int rp, mt, ks, kb0, kb1;
+        tile_coords(tile, rp, mt, ks, kb0, kb1);
+        const int out_tile = mt * n_rp + rp;
+        {
+          const uint32_t* tk = reinterpret_cast<const uint32_t*>(p.tickets + out_tile);
+          uint32_t it = 0, seen = 0;
+          while (true) {
+            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(tk) : "memory");
+            if (seen >= (uint32_t)S || sh.abort_flag) break;
+            if (++it > (1u << 22)) {
+              sh.abort_flag = 1;
+              report_device_error(p.status, QTALE_ERR_TIMEOUT);
+              break;
+            }
+            __nanosleep(64);
+          }
+          if (sh.abort_flag) goto role_done;
+        }
+        const float* tile_part = p.partial + ((size_t)out_tile * S) * (2 * kTileRows * TN);
+        for (int u = ks + S * wi; u < 32; u += S * kDequantWarps) {
+          const int qi = u >> 2, c0 = (u & 3) * kEpiCols;
+          const int g2 = qi >> 2, quad2 = qi & 3;
+          const int nt2 = rp * RT + g2;
+          const int m0 = mt * TW + c0;
+          if (g2 >= RT || nt2 >= p.n_tiles || m0 >= M) continue;  // uniform over the warp
           EpiOperands eo;
           epilogue_fetch_tok<-1>(p, lane, m0, M, eo);
-          epilogue_fetch<-1>(p, lane, nt, quad, m0, M, eo);
-          epilogue_chunk<ACT, -1>(p, stage, lane, nt, quad, m0, M, eo);
+          epilogue_fetch<-1>(p, lane, nt2, quad2, m0, M, eo);
+          splitk_sum_to_stage(tile_part + (size_t)(g2 * kTileRows + quad2 * 32 + lane) * TN + c0, S,
+                              (size_t)2 * kTileRows * TN, stage, lane);
+          __syncwarp();
+          epilogue_chunk<ACT, -1>(p, stage, lane, nt2, quad2, m0, M, eo);
           __syncwarp();
         }
-        tmem_wait_ld();
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&sh.d_empty[g]);
-      dph ^= 1u;
     }
   role_done:;
   }
@@ -1369,7 +1507,7 @@ static int make_tmap_set(TmapSet* set, const void* base, int rows, int cols, int
   return QTALE_OK;
 }
 
-template <int TN, int BITS, int ACT>
+template <int TN, int BITS, int ACT, bool SPLIT = false>
 static int launch_gemm(const TmapSet& tx, const CUtensorMap& tw, const GemmParams& p,
                        cudaStream_t s) {
   using Cfg = GemmCfg<TN, BITS>;
@@ -1377,16 +1515,17 @@ static int launch_gemm(const TmapSet& tx, const CUtensorMap& tw, const GemmParam
   int dev = 0;
   cudaGetDevice(&dev);
   if (dev >= 0 && dev < 64 && !configured[dev]) {
-    if (cudaFuncSetAttribute(wq_gemm_kernel<TN, BITS, ACT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    if (cudaFuncSetAttribute(wq_gemm_kernel<TN, BITS, ACT, SPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)Cfg::kSmemBytes) != cudaSuccess)
       return QTALE_ERR_CUDA;
     configured[dev] = true;
   }
-  const int max_tiles = ((p.M_cap + 31) / 32) * ((p.n_tiles + Cfg::kRowTiles - 1) / Cfg::kRowTiles);
+  const int max_tiles = ((p.M_cap + 31) / 32) * ((p.n_tiles + Cfg::kRowTiles - 1) / Cfg::kRowTiles) *
+                        (p.split_k > 1 ? p.split_k : 1);
   int grid = sm_count();
   if (grid > max_tiles) grid = max_tiles;
   if (grid < 1) grid = 1;
-  wq_gemm_kernel<TN, BITS, ACT><<<grid, kGemmThreads, Cfg::kSmemBytes, s>>>(tx, tw, p);
+  wq_gemm_kernel<TN, BITS, ACT, SPLIT><<<grid, kGemmThreads, Cfg::kSmemBytes, s>>>(tx, tw, p);
   return launch_status(cudaGetLastError());
 }
 
@@ -1510,9 +1649,36 @@ size_t wq_blob_bytes(int N, int K, int bits, int group, int row_mode, WqGeometry
   return q.total;
 }
 
+// Split K for token counts of a decode step (single-CTA tcgen05 kernel, 256 weight rows per
+// tile): the number of K slices that minimises (waves of the grid) x (K blocks per slice + the
+// cost of writing and re-reading a partial tile, about four K blocks).
+static int pick_split_k(int n_rp, int nkb, int sms, size_t ws_bytes) {
+  long best = -1;
+  int best_s = 1;
+  for (int sp = 1; sp <= 8 && sp * 2 <= nkb; ++sp) {
+    if (wq_splitk_ticket_bytes() + (size_t)n_rp * sp * kSplitTileBytes > ws_bytes) break;
+    const long waves = ((long)n_rp * sp + sms - 1) / sms;
+    // in K blocks (about half a microsecond each): per tile of the slowest CTA its K blocks plus
+    // the pipeline refill and the epilogue (4) or the partial tile's write and fence (8); split
+    // only: the second half of the kernel (waiting for the other slices, summing, epilogue: 14)
+    const long cost = waves * ((nkb + sp - 1) / sp + (sp > 1 ? 8 : 4)) + (sp > 1 ? 14 : 0);
+    if (best < 0 || cost < best) { best = cost; best_s = sp; }
+  }
+  return best_s;
+}
+
+size_t wq_splitk_ticket_bytes() { return 4 * 4096; }  // one 4 KB region of counters per linear of a layer
+
+size_t wq_splitk_workspace_bytes() {
+  // tickets + partial tiles for up to sixteen slices of 148 tile groups is more than any layer
+  // needs; 48 MB covers (groups x slices) <= 768
+  return wq_splitk_ticket_bytes() + (size_t)768 * kSplitTileBytes;
+}
+
 int wq_gemm_launch(const void* a, int lda, const int32_t* m_dev, int M_cap,
                    const qtale_wq_weight* w, int act, int epilogue, const qtale_epilogue_args* epi,
-                   void* y, int ldy, cudaStream_t s) {
+                   void* y, int ldy, cudaStream_t s, void* splitk_ws, size_t splitk_bytes,
+                   int splitk_slot) {
   WqGeometry g;
   wq_blob_bytes(w->N, w->K, w->bits, w->group, w->row_mode, &g);
   GemmParams p;
@@ -1551,6 +1717,27 @@ int wq_gemm_launch(const void* a, int lda, const int32_t* m_dev, int M_cap,
     if (act == QTALE_ACT_F16)
       return w->bits == 4 ? launch_pair<4, 1>(px, p, s) : launch_pair<3, 1>(px, p, s);
     return w->bits == 4 ? launch_pair<4, 0>(px, p, s) : launch_pair<3, 0>(px, p, s);
+  }
+  if (M_cap <= kSmallTokens && splitk_ws && g.n_rp <= 1024 && w->bits != 16) {
+    // decode step inside a layer: the tcgen05 kernel with the K dimension split over the SMs
+    TmapSet tx;
+    CUtensorMap tw;
+    memset(&tx, 0, sizeof(tx));
+    memset(&tw, 0, sizeof(tw));
+    const int rc = make_tmap_set(&tx, a, M_cap, w->K, lda, 64, act);
+    if (rc != QTALE_OK) return rc;
+    p.split_k = pick_split_k(g.n_rp, g.nkb, sm_count(), splitk_bytes);
+    p.tickets = static_cast<int*>(splitk_ws) + (splitk_slot & 3) * 1024;
+    p.partial = reinterpret_cast<float*>(static_cast<unsigned char*>(splitk_ws) + wq_splitk_ticket_bytes());
+    if (p.split_k <= 1) {  // enough row tiles for the device: the plain kernel, no partial tiles
+      p.split_k = 1;
+      if (act == QTALE_ACT_F16)
+        return w->bits == 4 ? launch_gemm<64, 4, 1>(tx, tw, p, s) : launch_gemm<64, 3, 1>(tx, tw, p, s);
+      return w->bits == 4 ? launch_gemm<64, 4, 0>(tx, tw, p, s) : launch_gemm<64, 3, 0>(tx, tw, p, s);
+    }
+    if (act == QTALE_ACT_F16)
+      return w->bits == 4 ? launch_gemm<64, 4, 1, true>(tx, tw, p, s) : launch_gemm<64, 3, 1, true>(tx, tw, p, s);
+    return w->bits == 4 ? launch_gemm<64, 4, 0, true>(tx, tw, p, s) : launch_gemm<64, 3, 0, true>(tx, tw, p, s);
   }
   if (M_cap <= kSmallTokens) {
     CUtensorMap tx1;
@@ -1725,9 +1912,11 @@ int qtale_wq_repack(const uint8_t* codes, const uint16_t* scales, const uint16_t
   return QTALE_OK;
 }
 
+size_t qtale_wq_gemm_workspace_bytes(void) { return wq_splitk_workspace_bytes(); }
+
 int qtale_wq_gemm(const void* a, int lda, const int32_t* m_dev, int M_cap, const qtale_wq_weight* w,
                   int act_dtype, int epilogue, const qtale_epilogue_args* epi, void* y, int ldy,
-                  void* stream) {
+                  void* ws, size_t ws_bytes, void* stream) {
   if (!a || !w || !w->packed) return QTALE_ERR_NULL;
   if (act_dtype != QTALE_ACT_BF16 && act_dtype != QTALE_ACT_F16) return QTALE_ERR_MODE;
   if (w->bits != 3 && w->bits != 4) return QTALE_ERR_BITS;
@@ -1755,8 +1944,15 @@ int qtale_wq_gemm(const void* a, int lda, const int32_t* m_dev, int M_cap, const
   if (y && (!aligned16(y) || ldy % 8 != 0)) return QTALE_ERR_ALIGN;
   if (epi && epi->resid && (!aligned16(epi->resid) || epi->ld_resid % 8 != 0)) return QTALE_ERR_ALIGN;
   if (epi && epi->dst && (!aligned16(epi->dst) || epi->ld_dst % 8 != 0)) return QTALE_ERR_ALIGN;
+  if (ws) {
+    if (!aligned16(ws)) return QTALE_ERR_ALIGN;
+    if (ws_bytes < wq_splitk_workspace_bytes()) return QTALE_ERR_WORKSPACE;
+    if (M_cap <= kSmallTokens &&  // the counters of the split-K path start at zero
+        cudaMemsetAsync(ws, 0, 4096, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+      return QTALE_ERR_CUDA;
+  }
   return wq_gemm_launch(a, lda, m_dev, M_cap, w, act_dtype, epilogue, epi, y, ldy,
-                        static_cast<cudaStream_t>(stream));
+                        static_cast<cudaStream_t>(stream), ws, ws_bytes, 0);
 }
 
 }  // extern "C"

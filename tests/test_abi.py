@@ -55,7 +55,7 @@ def test_host_side_argument_validation(api):
     assert L.qtale_scatter_add(None, None, None, None, None, 4, 64, None) == -1
     assert L.qtale_router_select(None, 4, 64, None, 0.0, None, None, None, 1, None, 0, 0.5, 0,
                                  None, None, None, None, None, None, 0, None) == -1
-    assert L.qtale_wq_gemm(None, 64, None, 4, None, 0, 0, None, None, 64, None) == -1
+    assert L.qtale_wq_gemm(None, 64, None, 4, None, 0, 0, None, None, 64, None, 0, None) == -1
     cfg = api.LayerConfig(256, 4, 4, 64, 688, 4, 64, 1e-5, 1e4, 0, 0.5, 1.0, 1)
     assert api.layer_workspace_bytes(cfg, 256, 2) > 256 * 256 * 2
     bad = api.LayerConfig(256, 4, 4, 48, 688, 4, 64, 1e-5, 1e4, 0, 0.5, 1.0, 1)

@@ -299,6 +299,15 @@ def test_wq_gemm_against_oracle(env, M, N, K, bits, group, m_dev, act):
     assert np.abs(y[:mm] - ref_b).max() <= 1e-4 * max(1.0, np.abs(ref_b).max())
     yb = api.to_host_f32(api.wq_gemm(ad, qw, md, api.EPI_STORE_16))
     assert np.array_equal(yb[:mm], round_act(y[:mm], act))
+    if M <= 64:
+        # with a workspace the same product runs with the input dimension split over the SMs
+        # (partial sums added in a fixed order): same tolerance, and bit-identical on a second run
+        ws = torch.full((api.wq_gemm_workspace_bytes(),), 0xFF, dtype=torch.uint8, device=dev)
+        y2 = api.wq_gemm(ad, qw, md, api.EPI_STORE_F32, ws=ws).cpu().numpy()
+        assert not y2[mm:].any()
+        assert np.abs(y2[:mm] - ref_b).max() <= 1e-4 * max(1.0, np.abs(ref_b).max())
+        y3 = api.wq_gemm(ad, qw, md, api.EPI_STORE_F32, ws=ws).cpu().numpy()
+        assert np.array_equal(y2, y3) and api.device_status() == 0
 
 
 @pytest.mark.parametrize("act", [0, 1])

@@ -185,7 +185,7 @@ def test_full_kv_cache_is_reported(env):
     sh = inputs.LayerShape(256, 2, 2, 128, 512, 4, 64)
     B, cap = 3, 16
     case = Case(api, torch, dev, sh, inputs.cu_seqlens_uniform(B, 1), seed=15)
-    kv = api.KvCache(B, cap, sh.kv_dim, dev, act_dtype=1)
+    kv = api.KvCache(B, cap, sh.kv_dim, dev, act_dtype=1, head_dim=sh.head_dim)
     kv.kv_len.copy_(torch.tensor([cap, 3, cap - 1], dtype=torch.int32, device=dev))
     cfg = case.cfg(api.SELECT_THRESHOLD, 1, theta=0.0)          # every sequence executes
     ws = torch.zeros(api.layer_workspace_bytes(cfg, B, B), dtype=torch.uint8, device=dev)
@@ -213,12 +213,12 @@ def test_decode_step_with_executed_only_cache(env, bits, group, Hkv, act):
     cv = np.zeros((B, cap, kvd), np.float32)
     kl = np.zeros(B, np.int32)
     ref, _ = oracle.layer_forward(case.layer, case.x, case.cu, m, cache_k=ck, cache_v=cv, kv_len=kl)
-    kv = api.KvCache(B, cap, kvd, dev, act_dtype=act)
+    kv = api.KvCache(B, cap, kvd, dev, act_dtype=act, head_dim=sh.head_dim)
     cfg = case.cfg(api.SELECT_THRESHOLD, act, theta=0.5)
     out, n, _ = case.gpu(cfg, kv=kv, phase=api.PHASE_PREFILL)
     assert np.array_equal(kv.kv_len.cpu().numpy(), kl)         # bypassed tokens leave no entry
     assert_layer_close(out, ref, strict=True)
-    gk, gv = api.to_host_f32(kv.k), api.to_host_f32(kv.v)
+    gk, gv = api.to_host_f32(kv.k_rows()), api.to_host_f32(kv.v_rows())
     for b in range(B):
         assert np.abs(gk[b, :kl[b]] - ck[b, :kl[b]]).max() <= 4e-2   # 16-bit keys, |k| up to ~5
         assert rel_fro(gk[b, :kl[b]], ck[b, :kl[b]]) <= 5e-3
@@ -267,9 +267,10 @@ def test_decode_step_ragged_cache_lengths(env):
     for b in range(B):
         ck[b, kl[b]:] = 0
         cv[b, kl[b]:] = 0
-    kv = api.KvCache(B, cap, kvd, dev, act_dtype=1)
-    kv.k.copy_(torch.from_numpy(ck).to(dev).to(kv.k.dtype))   # bf16-valued normals are exact in fp16
-    kv.v.copy_(torch.from_numpy(cv).to(dev).to(kv.v.dtype))
+    kv = api.KvCache(B, cap, kvd, dev, act_dtype=1, head_dim=sh.head_dim)
+    shp = (B, cap, kv.n_kv_heads, sh.head_dim)
+    kv.k_view().copy_(torch.from_numpy(ck).to(dev).to(kv.k.dtype).view(shp))   # bf16-valued normals are exact in fp16
+    kv.v_view().copy_(torch.from_numpy(cv).to(dev).to(kv.v.dtype).view(shp))
     kv.kv_len.copy_(torch.from_numpy(kl).to(dev))
     scores = np.full(B, 0.9, np.float32)
     scores[3] = 0.1                                            # one sequence bypasses the layer
@@ -432,7 +433,7 @@ def test_decode_loop_with_diverging_per_layer_caches(env):
     cud = torch.from_numpy(cu).to(dev)
 
     def fresh_caches():
-        return [api.KvCache(B, cap, kvd, dev, act_dtype=1) for _ in range(L)]
+        return [api.KvCache(B, cap, kvd, dev, act_dtype=1, head_dim=sh.head_dim) for _ in range(L)]
 
     # ---- layer by layer, teacher forced: prefill ----
     gc = fresh_caches()
@@ -665,13 +666,14 @@ def test_config3_decode_step_parity(env, cfg_name, ratio):
     kvd = sh.kv_dim
     ck = np.zeros((B, cap, kvd), np.float32)
     cv = np.zeros((B, cap, kvd), np.float32)
-    kv = api.KvCache(B, cap, kvd, dev, act_dtype=1)
+    kv = api.KvCache(B, cap, kvd, dev, act_dtype=1, head_dim=sh.head_dim)
     for b in range(B):
         n = int(kl[b])
         ck[b, :n] = inputs.activations(21, 3000 + b, n, kvd)
         cv[b, :n] = inputs.activations(21, 4000 + b, n, kvd)
-        kv.k[b, :n].copy_(torch.from_numpy(ck[b, :n]).to(dev).to(kv.k.dtype))   # bf16-valued normals
-        kv.v[b, :n].copy_(torch.from_numpy(cv[b, :n]).to(dev).to(kv.v.dtype))   # are exact in fp16
+        shp = (n, kv.n_kv_heads, sh.head_dim)
+        kv.k_view()[b, :n].copy_(torch.from_numpy(ck[b, :n]).to(dev).to(kv.k.dtype).view(shp))   # bf16-valued
+        kv.v_view()[b, :n].copy_(torch.from_numpy(cv[b, :n]).to(dev).to(kv.v.dtype).view(shp))   # normals are exact in fp16
     kv.kv_len.copy_(torch.from_numpy(kl))
     pos0 = kl.copy()
     kl_ref = kl.copy()
@@ -690,7 +692,7 @@ def test_config3_decode_step_parity(env, cfg_name, ratio):
     assert np.array_equal(out[m == 0], case.x[m == 0])
     _assert_c2_close(out, ref, 1, inside=0.999)
     # the appended key / value rows of the compared sequences
-    gk, gv = api.to_host_f32(kv.k), api.to_host_f32(kv.v)
+    gk, gv = api.to_host_f32(kv.k_rows()), api.to_host_f32(kv.v_rows())
     for b in long_seqs:
         if m[b]:
             n = int(kl[b])
