@@ -620,7 +620,8 @@ int router_select_launch(const void* x, int T, int d, const float* w_router, flo
   }
   int grid = sm_count() * cached_per_sm;
   if (grid > kMaxGrid) grid = kMaxGrid;
-  const int want = (T + 31) / 32;
+  // with the scores supplied there is no sweep of x to spread: one CTA per 1024 tokens
+  const int want = scores_override ? (T + 1023) / 1024 : (T + 31) / 32;
   if (grid > want) grid = want;
   int chunk = (T + grid - 1) / grid;
   chunk = (chunk + 1) & ~1;
