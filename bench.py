@@ -48,6 +48,10 @@ WORKLOAD = ("c2: 7B-shaped layer (hidden 4096, 32 heads, FFN 11008), int4 g128, 
 # table), QKV GEMM (+ rotary), attention, O GEMM, RMSNorm, gate/up GEMM (+ SwiGLU), down GEMM
 # (+ residual scatter)
 KERNELS_PER_STEP = 8
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of the four GEMM launches of one step
+# at ratio 0.5 (4096 executed tokens), one ncu capture of the kernels as they stand
+# (profiles/wq_gemm_pair_c2_layer_step.md); None at other ratios.
+GEMM_DRAM_BYTES = 733111296
 ALL_LEGS = ["sweep", "gemm", "bf16", "router", "gather", "decode", "decode_loop", "c4", "c5", "e2e", "cpu"]
 
 
@@ -470,7 +474,9 @@ def run_ours(args):
                         burst=dict(achieved=burst, peak=peaks["bf16_tflops"],
                                    frac=burst / peaks["bf16_tflops"],
                                    note="first region after an idle second, against the burst peak"),
-                        traffic=None,
+                        traffic=GEMM_DRAM_BYTES if abs(ratio - 0.5) < 1e-9 else None,
+                        traffic_unit="bytes per 4 launches (ncu, ratio 0.5)", algorithmic_bytes=int(
+                            2 * k * (8 * sh.d + 4 * qd + 2 * sh.ffn) + accounting.packed_weight_bytes(sh)),
                         ms_per_4_launches=g["ms"], share_of_step=g["ms"] / ms_per_step,
                         executed_tokens=k, clocks=g["clocks"])
         check_status()
