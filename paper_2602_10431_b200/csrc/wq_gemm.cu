@@ -1078,16 +1078,14 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
     const unsigned char* w_stage = w_base + (size_t)set * Cfg::kWStageBytes;
     uint32_t dph = 0;
     uint32_t count = 0;
-    for (int tile = cluster_id; tile < total_tiles; tile += n_clusters) {
-      const int rp = tile % n_rp, mt = tile / n_rp;
-      const int nt = rp * 2 + (int)rank;
-      for (int st = 0; st < n_st; ++st, ++count) {
-        if ((int)(count & 3u) != set) continue;  // ring slot = set
-        const uint32_t ph = (count >> 2) & 1u;
+    // one pipeline step of this set (step `st` of a tile, running number `cnt`): packed weights of
+    // ring slot `set` -> 16-bit values -> tensor memory, then the arrival on the leader's barrier
+    auto dequant_step = [&](int st, uint32_t cnt) -> bool {
+        const uint32_t ph = (cnt >> 2) & 1u;
         const bool two = st * kPairBlocks + 1 < nkb;
         uint32_t cw[kPairBlocks][8];
         uint32_t sz[kPairBlocks];
-        if (!pair_wait(&sh.full_w[set], ph, &sh, p.status)) goto role_done;
+        if (!pair_wait(&sh.full_w[set], ph, &sh, p.status)) return false;
 #pragma unroll
         for (int b = 0; b < kPairBlocks; ++b) {
           const unsigned char* wt = w_stage + (size_t)b * Cfg::kWTileBytes;
@@ -1152,7 +1150,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
         // the first quarter is dequantised before the wait for the free A slot; every store has
         // taken its operands when it returns, so the registers are reused at once
         dequant_half(cw[0], sz[0], 0);
-        if (!pair_wait(&sh.slot_free[set], ph ^ 1u, &sh, p.status)) goto role_done;
+        if (!pair_wait(&sh.slot_free[set], ph ^ 1u, &sh, p.status)) return false;
         tc_fence_after();
         tmem_st_x16(a_taddr0, r);
         dequant_half(cw[0], sz[0], 1);
@@ -1167,6 +1165,30 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive_cluster(ready_leader + 8u * set);
+        return true;
+    };
+    bool prefilled = false;  // this set's first step of the current tile is in tensor memory already
+    for (int tile = cluster_id; tile < total_tiles; tile += n_clusters) {
+      const int rp = tile % n_rp, mt = tile / n_rp;
+      const int nt = rp * 2 + (int)rank;
+      for (int st = 0; st < n_st; ++st, ++count) {
+        if ((int)(count & 3u) != set) continue;  // ring slot = set
+        if (prefilled) {
+          prefilled = false;
+          continue;
+        }
+        if (!dequant_step(st, count)) goto role_done;
+      }
+      // The set's first step of the NEXT tile is dequantised before this tile's epilogue: its ring
+      // slot is free as soon as this tile's last use of it has been multiplied, and the issuer
+      // then finds all four slots ready the moment the accumulator is handed back, instead of
+      // waiting for the dequantisers to restart after the epilogue.
+      if (tile + n_clusters < total_tiles) {
+        const int st0 = (int)(((uint32_t)set - count) & 3u);  // count = running number of the next tile's step 0
+        if (st0 < n_st) {
+          if (!dequant_step(st0, count + (uint32_t)st0)) goto role_done;
+          prefilled = true;
+        }
       }
       // ---- epilogue: set j drains the 16-column chunks j, j + 4, ... of this CTA's accumulator ----
       if (!pair_wait(&sh.d_full, dph, &sh, p.status)) goto role_done;
