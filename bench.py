@@ -52,7 +52,7 @@ KERNELS_PER_STEP = 8
 # at ratio 0.5 (4096 executed tokens), one ncu capture of the kernels as they stand
 # (profiles/wq_gemm_pair_c2_layer_step.md); None at other ratios.
 GEMM_DRAM_BYTES = 733111296
-ALL_LEGS = ["sweep", "gemm", "bf16", "router", "gather", "decode", "decode_loop", "c4", "c5", "e2e", "cpu"]
+ALL_LEGS = ["sweep", "gemm", "bf16", "router", "gather", "scatter", "decode", "decode_loop", "c4", "c5", "e2e", "cpu"]
 
 
 def measured_peaks():
@@ -577,6 +577,29 @@ def run_ours(args):
             us=ms * 1e3, rows="%d of %d, d %d" % (kg, Tg, dg),
             roofline=hbm_roofline("compact_kernel", kg * dg * 4, ms, peaks), clocks=r["clocks"])
         del xg, hn
+        check_status()
+
+    if "scatter" in legs:
+        # standalone residual scatter (the layer path fuses it into the down projection)
+        Ts, ds = 65536, 5120
+        ks = api.topk_count(0.7, Ts)
+        xs = torch.randn(Ts, ds, device=dev, generator=gen).to(torch.bfloat16)
+        xcs = torch.randn(ks, ds, device=dev, generator=gen).to(torch.bfloat16)
+        fs = torch.randn(ks, ds, device=dev, generator=gen) * 1e-3
+        idxs = torch.zeros(Ts, dtype=torch.int32, device=dev)
+        idxs[:ks] = torch.sort(torch.randperm(Ts, device=dev, generator=gen)[:ks])[0].to(torch.int32)
+        ns = torch.tensor([ks], dtype=torch.int32, device=dev)
+        call = lambda: api.scatter_add(xs, xcs, fs, idxs, ns)
+        call()
+        gr = graph_of(torch, call, 5)
+        r = timer.run(lambda i: gr.replay(), 10, 3, 0.25)
+        ms = r["ms"] / 5
+        extra["scatter_add"] = dict(
+            us=ms * 1e3, rows="%d of %d, d %d" % (ks, Ts, ds),
+            roofline=hbm_roofline("scatter_add_kernel", ks * ds * 8, ms, peaks,
+                                  note="bf16 row + fp32 update read, bf16 row written"),
+            clocks=r["clocks"])
+        del xs, xcs, fs
         check_status()
 
     # ---- c3: one decode step of the 7B-shaped layer, 64 sequences with 2048 cached tokens ----

@@ -56,7 +56,7 @@ extern "C" {
 #define QTALE_ERR_NULL (-1)      /* a required pointer is NULL */
 #define QTALE_ERR_ALIGN (-2)     /* pointer or pitch not 16-byte aligned */
 #define QTALE_ERR_SHAPE (-3)     /* unsupported or inconsistent sizes */
-#define QTALE_ERR_BITS (-4)      /* bits not in {3, 4} */
+#define QTALE_ERR_BITS (-4)      /* bits not in {2, 3, 4} */
 #define QTALE_ERR_GROUP (-5)     /* group not in {64, 128} */
 #define QTALE_ERR_WORKSPACE (-6) /* workspace too small */
 #define QTALE_ERR_CAPACITY (-7)  /* a count exceeds the capacity of its buffer */
@@ -238,7 +238,7 @@ int qtale_scatter_add(void* x_inout, const void* xc, const float* f, const int32
 typedef struct {
   const void* packed; /* device copy of the repacked blob */
   int N, K;           /* logical shape */
-  int bits;           /* 3 or 4 */
+  int bits;           /* 2, 3 or 4 */
   int group;          /* 64 or 128 */
   int row_mode;       /* QTALE_WQ_ROWS_* the blob was repacked with */
 } qtale_wq_weight;
@@ -310,7 +310,10 @@ int qtale_wq_gemm(const void* a, int lda, const int32_t* m_dev, int M_cap, const
 
 typedef struct {
   int d, n_heads, n_kv_heads, head_dim, ffn; /* Llama-style decoder layer shape          */
-  int bits, group;                          /* quantisation of the four linears          */
+  int bits, group;                          /* quantisation of the four linears; bits = 0:
+                                               each weight descriptor's own width, so the
+                                               layers of a model may mix 2, 3 and 4 bits
+                                               (mixed precision across layers, App. C)   */
   float rms_eps, rope_theta;                /* RMSNorm epsilon, rotary base               */
   int select_mode;                          /* QTALE_SELECT_*                             */
   float theta;                              /* threshold of Eq. 9 (THRESHOLD)             */

@@ -16,8 +16,10 @@
  * Parts the paper leaves open and that this file fixes (so no external pin
  * exists for them -- "parity unpinned"): the attention / KV treatment of
  * bypassed tokens (they produce no Q, K, V at that layer), RoPE using the
- * original position, the min/max quantiser's rounding, and top-k selection
- * (an extension; the paper controls the ratio through theta only).
+ * original position, the min/max quantiser's rounding, top-k selection
+ * (an extension; the paper controls the ratio through theta only), the ReLU
+ * of the MLP router (Eq. 2 names neither width nor activation), and the
+ * rounding k = floor(ratio n + 0.5) of the theta quantile for a target ratio.
  */
 #include <math.h>
 #include <stdint.h>
@@ -244,10 +246,12 @@ void orc_compact_indices(const uint8_t* mask, int T, const int32_t* cu_seqlens, 
   *n_exec = n;
 }
 
-/* ---- quantised weights (Sec. 4.1: 4-bit / 3-bit, per-group parameters) ---- */
+/* ---- quantised weights (Sec. 4.1: 4-bit / 3-bit, per-group parameters; the mixed
+ * ---- precision appendix interleaves 4-bit and 2-bit layers).  A row of b-bit codes is
+ * ---- a little-endian bit stream: code k occupies bits b k .. b k + b - 1. ---- */
 
 static int row_bytes_for(int K, int bits) {
-  return bits == 4 ? (K + 1) / 2 : (3 * K + 7) / 8;
+  return (bits * K + 7) / 8;
 }
 int orc_row_bytes(int K, int bits) { return row_bytes_for(K, bits); }
 
@@ -256,11 +260,12 @@ static unsigned get_code(const uint8_t* row, int k, int bits) {
     uint8_t b = row[k >> 1];
     return (k & 1) ? (unsigned)(b >> 4) : (unsigned)(b & 0xF);
   }
-  int bit = 3 * k;
-  unsigned lo = row[bit >> 3];
-  unsigned hi = row[(bit >> 3) + ((bit & 7) > 5 ? 1 : 0)];
-  unsigned v = (lo | (hi << 8)) >> (bit & 7);
-  return v & 7u;
+  unsigned v = 0;
+  for (int j = 0; j < bits; ++j) {
+    int bb = bits * k + j;
+    v |= (unsigned)((row[bb >> 3] >> (bb & 7)) & 1u) << j;
+  }
+  return v;
 }
 
 static void put_code(uint8_t* row, int k, int bits, unsigned q) {
@@ -271,9 +276,8 @@ static void put_code(uint8_t* row, int k, int bits, unsigned q) {
       row[k >> 1] = (uint8_t)((row[k >> 1] & 0xF0) | (q & 0xF));
     return;
   }
-  int bit = 3 * k;
-  for (int j = 0; j < 3; ++j) {
-    int bb = bit + j;
+  for (int j = 0; j < bits; ++j) {
+    int bb = bits * k + j;
     uint8_t m = (uint8_t)(1u << (bb & 7));
     if ((q >> j) & 1u)
       row[bb >> 3] |= m;

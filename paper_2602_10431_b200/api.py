@@ -352,8 +352,10 @@ def wq_gemm(a, w: QuantWeight, m_dev=None, epilogue=EPI_STORE_16, y=None, idx=No
 # ---------------------------------------------------------------------------------
 
 def layer_config(sh, select_mode=SELECT_THRESHOLD, theta=0.5, ratio=1.0,
-                 act_dtype=ACT_F16) -> LayerConfig:
-    return LayerConfig(sh.d, sh.n_heads, sh.n_kv_heads, sh.head_dim, sh.ffn, sh.bits, sh.group,
+                 act_dtype=ACT_F16, bits=None) -> LayerConfig:
+    """bits=0: every weight carries its own width (layers of mixed 2/3/4-bit precision)."""
+    return LayerConfig(sh.d, sh.n_heads, sh.n_kv_heads, sh.head_dim, sh.ffn,
+                       sh.bits if bits is None else int(bits), sh.group,
                        sh.rms_eps, sh.rope_theta, int(select_mode), float(theta), float(ratio),
                        int(act_dtype))
 

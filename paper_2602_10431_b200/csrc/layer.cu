@@ -66,7 +66,7 @@ static LayerWs carve(const qtale_layer_config* c, int T, int B, void* base) {
 
 static int check_config(const qtale_layer_config* c) {
   if (!c) return QTALE_ERR_NULL;
-  if (c->bits != 3 && c->bits != 4) return QTALE_ERR_BITS;
+  if (c->bits != 0 && (c->bits < 2 || c->bits > 4)) return QTALE_ERR_BITS;
   if (c->group != 64 && c->group != 128) return QTALE_ERR_GROUP;
   if (c->d < 8 || c->d % 8 || c->n_heads < 1 || c->n_kv_heads < 1 ||
       c->n_heads % c->n_kv_heads || (c->head_dim != 64 && c->head_dim != 128) || c->ffn < 8 ||
@@ -213,7 +213,7 @@ static int check_weights(const qtale_layer_config* c, const qtale_layer_weights*
     return QTALE_ERR_SHAPE;
   const qtale_wq_weight* all[4] = {&w->qkv, &w->o, &w->gate_up, &w->down};
   for (const qtale_wq_weight* q : all) {
-    if (q->bits != c->bits) return QTALE_ERR_BITS;
+    if (c->bits ? q->bits != c->bits : (q->bits < 2 || q->bits > 4)) return QTALE_ERR_BITS;
     if (q->group != c->group) return QTALE_ERR_GROUP;
     if (!aligned16(q->packed)) return QTALE_ERR_ALIGN;
   }

@@ -647,8 +647,10 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
               cw[0] = w0.x; cw[1] = w0.y; cw[2] = w0.z; cw[3] = w0.w;
               cw[4] = w1.x; cw[5] = w1.y; cw[6] = w1.z; cw[7] = w1.w;
             } else {
+              // 3-bit: a 2-bit plane and a 1-bit plane; 2-bit: the 2-bit plane alone
               const uint4 a = reinterpret_cast<const uint4*>(st)[L];
-              const uint2 b = reinterpret_cast<const uint2*>(st + kTileRows * 16)[L];
+              uint2 b = make_uint2(0, 0);
+              if (BITS == 3) b = reinterpret_cast<const uint2*>(st + kTileRows * 16)[L];
               cw[0] = a.x; cw[1] = a.y; cw[2] = a.z; cw[3] = a.w;
               cw[4] = b.x; cw[5] = b.y; cw[6] = 0; cw[7] = 0;
             }
@@ -1098,7 +1100,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
               cw[b][4] = w1.x; cw[b][5] = w1.y; cw[b][6] = w1.z; cw[b][7] = w1.w;
             } else {
               const uint4 a = reinterpret_cast<const uint4*>(wt)[L];
-              const uint2 bb = reinterpret_cast<const uint2*>(wt + kTileRows * 16)[L];
+              uint2 bb = make_uint2(0, 0);
+              if (BITS == 3) bb = reinterpret_cast<const uint2*>(wt + kTileRows * 16)[L];
               cw[b][0] = a.x; cw[b][1] = a.y; cw[b][2] = a.z; cw[b][3] = a.w;
               cw[b][4] = bb.x; cw[b][5] = bb.y; cw[b][6] = 0; cw[b][7] = 0;
             }
@@ -1262,7 +1265,7 @@ struct SmallCfg {
   static constexpr int kQuads = ROWS / 32;
   static constexpr int kXBytes = kSmallTokens * 128;                   // 64 tokens x 64 k
   static constexpr int kCodeA = ROWS * 16;                             // 16 bytes per row
-  static constexpr int kCodeB = BITS == 4 ? ROWS * 16 : ROWS * 8;
+  static constexpr int kCodeB = BITS == 4 ? ROWS * 16 : (BITS == 3 ? ROWS * 8 : 0);  // second code piece
   static constexpr int kSzBytes = ROWS * 4;
   static constexpr int kWBytes = kCodeA + kCodeB + kSzBytes;
   static constexpr int kTileCodeBytes = kTileRows * kKB * BITS / 8;    // code bytes of a full tile block
@@ -1353,7 +1356,8 @@ __global__ void __launch_bounds__(kSmallThreads, 2)
         // int4: two 32-feature parts of 16 bytes per row; int3: a 2-bit plane of 16 and a 1-bit
         // plane of 8 bytes per row; either way the second piece starts 2 KB into the block
         bulk_load(w, blk + slice * Cfg::kCodeA, Cfg::kCodeA, &sh.full[s]);
-        bulk_load(w + Cfg::kCodeA, blk + kTileRows * 16 + slice * Cfg::kCodeB, Cfg::kCodeB, &sh.full[s]);
+        if (Cfg::kCodeB > 0)
+          bulk_load(w + Cfg::kCodeA, blk + kTileRows * 16 + slice * Cfg::kCodeB, Cfg::kCodeB, &sh.full[s]);
         bulk_load(w + Cfg::kCodeA + Cfg::kCodeB, blk + Cfg::kTileCodeBytes + slice * Cfg::kSzBytes,
                   Cfg::kSzBytes, &sh.full[s]);
       }
@@ -1389,7 +1393,8 @@ __global__ void __launch_bounds__(kSmallThreads, 2)
         c[h][4] = b.x; c[h][5] = b.y; c[h][6] = b.z; c[h][7] = b.w;
       } else {
         const uint4 a = reinterpret_cast<const uint4*>(w)[r];
-        const uint2 b = reinterpret_cast<const uint2*>(w + Cfg::kCodeA)[r];
+        uint2 b = make_uint2(0, 0);
+        if (BITS == 3) b = reinterpret_cast<const uint2*>(w + Cfg::kCodeA)[r];
         const uint32_t pa[4] = {a.x, a.y, a.z, a.w};
         const uint32_t pb[2] = {b.x, b.y};
 #pragma unroll
@@ -1651,6 +1656,28 @@ static int launch_small(const CUtensorMap& tx, const GemmParams& p, cudaStream_t
   return launch_small_rows<BITS, ACT, 32>(tx, p, s);
 }
 
+template <int BITS, int ACT>
+static int launch_gemm64(const TmapSet& tx, const CUtensorMap& tw, const GemmParams& p, cudaStream_t s) {
+  return launch_gemm<64, BITS, ACT, false>(tx, tw, p, s);
+}
+template <int BITS, int ACT>
+static int launch_gemm64_split(const TmapSet& tx, const CUtensorMap& tw, const GemmParams& p, cudaStream_t s) {
+  return launch_gemm<64, BITS, ACT, true>(tx, tw, p, s);
+}
+
+// FN<bits, act> ARGS for the weight's bit-width (2, 3, 4) and the activation format
+#define QTALE_BY_BITS_ACT(FN, ARGS)                                              \
+  do {                                                                           \
+    if (act == QTALE_ACT_F16) {                                                  \
+      if (w->bits == 4) return FN<4, 1> ARGS;                                    \
+      if (w->bits == 3) return FN<3, 1> ARGS;                                    \
+      return FN<2, 1> ARGS;                                                      \
+    }                                                                            \
+    if (w->bits == 4) return FN<4, 0> ARGS;                                      \
+    if (w->bits == 3) return FN<3, 0> ARGS;                                      \
+    return FN<2, 0> ARGS;                                                        \
+  } while (0)
+
 // Token counts from which the CTA-pair kernel is used (below, a tile of 256 tokens is mostly padding).
 constexpr int kPairMinTokens = 129;
 
@@ -1736,9 +1763,7 @@ int wq_gemm_launch(const void* a, int lda, const int32_t* m_dev, int M_cap,
     memset(&px, 0, sizeof(px));
     const int rc = make_pair_tmaps(&px, a, M_cap, w->K, lda, act);
     if (rc != QTALE_OK) return rc;
-    if (act == QTALE_ACT_F16)
-      return w->bits == 4 ? launch_pair<4, 1>(px, p, s) : launch_pair<3, 1>(px, p, s);
-    return w->bits == 4 ? launch_pair<4, 0>(px, p, s) : launch_pair<3, 0>(px, p, s);
+    QTALE_BY_BITS_ACT(launch_pair, (px, p, s));
   }
   if (M_cap <= kSmallTokens && splitk_ws && g.n_rp <= 1024 && w->bits != 16) {
     // decode step inside a layer: the tcgen05 kernel with the K dimension split over the SMs
@@ -1753,22 +1778,16 @@ int wq_gemm_launch(const void* a, int lda, const int32_t* m_dev, int M_cap,
     p.partial = reinterpret_cast<float*>(static_cast<unsigned char*>(splitk_ws) + wq_splitk_ticket_bytes());
     if (p.split_k <= 1) {  // enough row tiles for the device: the plain kernel, no partial tiles
       p.split_k = 1;
-      if (act == QTALE_ACT_F16)
-        return w->bits == 4 ? launch_gemm<64, 4, 1>(tx, tw, p, s) : launch_gemm<64, 3, 1>(tx, tw, p, s);
-      return w->bits == 4 ? launch_gemm<64, 4, 0>(tx, tw, p, s) : launch_gemm<64, 3, 0>(tx, tw, p, s);
+      QTALE_BY_BITS_ACT(launch_gemm64, (tx, tw, p, s));
     }
-    if (act == QTALE_ACT_F16)
-      return w->bits == 4 ? launch_gemm<64, 4, 1, true>(tx, tw, p, s) : launch_gemm<64, 3, 1, true>(tx, tw, p, s);
-    return w->bits == 4 ? launch_gemm<64, 4, 0, true>(tx, tw, p, s) : launch_gemm<64, 3, 0, true>(tx, tw, p, s);
+    QTALE_BY_BITS_ACT(launch_gemm64_split, (tx, tw, p, s));
   }
   if (M_cap <= kSmallTokens) {
     CUtensorMap tx1;
     memset(&tx1, 0, sizeof(tx1));
     const int rc = make_tmap_16(&tx1, a, M_cap, w->K, lda, kSmallTokens, act);
     if (rc != QTALE_OK) return rc;
-    if (act == QTALE_ACT_F16)
-      return w->bits == 4 ? launch_small<4, 1>(tx1, p, s) : launch_small<3, 1>(tx1, p, s);
-    return w->bits == 4 ? launch_small<4, 0>(tx1, p, s) : launch_small<3, 0>(tx1, p, s);
+    QTALE_BY_BITS_ACT(launch_small, (tx1, p, s));
   }
   const int tn = pick_tn(M_cap);
   TmapSet tx;
@@ -1777,9 +1796,7 @@ int wq_gemm_launch(const void* a, int lda, const int32_t* m_dev, int M_cap,
   memset(&tw, 0, sizeof(tw));
   int rc = make_tmap_set(&tx, a, M_cap, w->K, lda, tn, act);
   if (rc != QTALE_OK) return rc;
-  if (act == QTALE_ACT_F16)
-    return w->bits == 4 ? dispatch_tn<4, 1>(tx, tw, p, tn, s) : dispatch_tn<3, 1>(tx, tw, p, tn, s);
-  return w->bits == 4 ? dispatch_tn<4, 0>(tx, tw, p, tn, s) : dispatch_tn<3, 0>(tx, tw, p, tn, s);
+  QTALE_BY_BITS_ACT(dispatch_tn, (tx, tw, p, tn, s));
 }
 
 int bf16_gemm_launch(const void* a, int lda, const int32_t* m_dev, int M_cap, const void* w_bf16,
@@ -1812,6 +1829,7 @@ int bf16_gemm_launch(const void* a, int lda, const int32_t* m_dev, int M_cap, co
 
 static inline unsigned canon_code(const uint8_t* row, int k, int bits) {
   if (bits == 4) return (k & 1) ? (row[k >> 1] >> 4) : (row[k >> 1] & 0xF);
+  if (bits == 2) return (row[k >> 2] >> (2 * (k & 3))) & 3u;
   const int bit = 3 * k;
   unsigned v = row[bit >> 3];
   if ((bit & 7) > 5) v |= (unsigned)row[(bit >> 3) + 1] << 8;
@@ -1831,7 +1849,7 @@ extern "C" {
 int qtale_wq_repack(const uint8_t* codes, const uint16_t* scales, const uint16_t* zeros, int N,
                     int K, int bits, int group, int row_mode, void* packed_out, size_t* bytes) {
   if (!bytes) return QTALE_ERR_NULL;
-  if (bits != 3 && bits != 4) return QTALE_ERR_BITS;
+  if (bits < 2 || bits > 4) return QTALE_ERR_BITS;
   if (group != 64 && group != 128) return QTALE_ERR_GROUP;
   if (N < 1 || K < 1) return QTALE_ERR_SHAPE;
   if (row_mode < QTALE_WQ_ROWS_PLAIN || row_mode > QTALE_WQ_ROWS_ROPE128) return QTALE_ERR_MODE;
@@ -1849,7 +1867,7 @@ int qtale_wq_repack(const uint8_t* codes, const uint16_t* scales, const uint16_t
   *bytes = total;
   uint8_t* out = static_cast<uint8_t*>(packed_out);
   memset(out, 0, total);
-  const int row_bytes = bits == 4 ? (K + 1) / 2 : (3 * K + 7) / 8;
+  const int row_bytes = bits == 4 ? (K + 1) / 2 : (bits == 3 ? (3 * K + 7) / 8 : (K + 3) / 4);
   const int ng_in = (K + group - 1) / group;
   const int F = N / 2;
   for (int nt = 0; nt < g.n_tiles; ++nt) {
@@ -1919,14 +1937,16 @@ int qtale_wq_repack(const uint8_t* codes, const uint16_t* scales, const uint16_t
               wv |= (q[8 * (2 * w2 + (f & 1)) + slot_k(f >> 1)] & 3u) << (2 * f);
             a[w2] = wv;
           }
-          uint32_t b0 = 0, b1 = 0;
-          for (int u = 0; u < 8; ++u)
-            for (int i = 0; i < 8; ++i) {
-              const uint32_t hb = (q[8 * u + slot_k(i)] >> 2) & 1u;
-              if (u < 4) b0 |= hb << (4 * i + (u & 3)); else b1 |= hb << (4 * i + (u & 3));
-            }
-          b[0] = b0;
-          b[1] = b1;
+          if (bits == 3) {
+            uint32_t b0 = 0, b1 = 0;
+            for (int u = 0; u < 8; ++u)
+              for (int i = 0; i < 8; ++i) {
+                const uint32_t hb = (q[8 * u + slot_k(i)] >> 2) & 1u;
+                if (u < 4) b0 |= hb << (4 * i + (u & 3)); else b1 |= hb << (4 * i + (u & 3));
+              }
+            b[0] = b0;
+            b[1] = b1;
+          }
         }
       }
     }
@@ -1941,7 +1961,7 @@ int qtale_wq_gemm(const void* a, int lda, const int32_t* m_dev, int M_cap, const
                   void* ws, size_t ws_bytes, void* stream) {
   if (!a || !w || !w->packed) return QTALE_ERR_NULL;
   if (act_dtype != QTALE_ACT_BF16 && act_dtype != QTALE_ACT_F16) return QTALE_ERR_MODE;
-  if (w->bits != 3 && w->bits != 4) return QTALE_ERR_BITS;
+  if (w->bits < 2 || w->bits > 4) return QTALE_ERR_BITS;
   if (w->group != 64 && w->group != 128) return QTALE_ERR_GROUP;
   if (M_cap < 1 || w->N < 1 || w->K < 1 || lda < w->K) return QTALE_ERR_SHAPE;
   if (epilogue < QTALE_EPI_STORE_16 || epilogue > QTALE_EPI_ROPE) return QTALE_ERR_MODE;

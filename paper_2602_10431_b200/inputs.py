@@ -125,7 +125,7 @@ def quantize_groups(w: np.ndarray, bits: int, group: int):
     The last group may be short.  Returns (codes uint8 [N,K], scales fp16 [N,ng],
     zeros fp16 [N,ng]).
     """
-    assert bits in (3, 4)
+    assert bits in (2, 3, 4)
     w = np.ascontiguousarray(w, dtype=np.float32)
     N, K = w.shape
     ng = (K + group - 1) // group
@@ -153,7 +153,8 @@ def pack_codes(codes: np.ndarray, bits: int) -> np.ndarray:
 
     4-bit: two codes per byte, even k in the low nibble.  3-bit: little-endian
     bit stream along K (code k occupies bits 3k .. 3k+2 of the row), 8 codes
-    per 3 bytes.  Rows start on a byte boundary.
+    per 3 bytes.  2-bit: four codes per byte, code k in bits 2 (k % 4) .. + 1 of
+    byte k / 4.  Rows start on a byte boundary.
     """
     codes = np.ascontiguousarray(codes, dtype=np.uint8)
     N, K = codes.shape
@@ -176,7 +177,12 @@ def pack_codes(codes: np.ndarray, bits: int) -> np.ndarray:
         out[:, :, 2] = (word >> 16) & 0xFF
         row_bytes = (3 * K + 7) // 8
         return np.ascontiguousarray(out.reshape(N, -1)[:, :row_bytes])
-    raise ValueError("bits must be 3 or 4")
+    if bits == 2:
+        Kp = (K + 3) // 4 * 4
+        c = np.zeros((N, Kp), dtype=np.uint8)
+        c[:, :K] = codes
+        return (c[:, 0::4] | (c[:, 1::4] << 2) | (c[:, 2::4] << 4) | (c[:, 3::4] << 6)).astype(np.uint8)
+    raise ValueError("bits must be 2, 3 or 4")
 
 
 def quantized_weight(seed: int, sid: int, N: int, K: int, bits: int, group: int, std: float = 0.02):
@@ -187,7 +193,7 @@ def quantized_weight(seed: int, sid: int, N: int, K: int, bits: int, group: int,
     host memory stays bounded.
     """
     ng = (K + group - 1) // group
-    row_bytes = (K + 1) // 2 if bits == 4 else (3 * K + 7) // 8
+    row_bytes = {4: (K + 1) // 2, 3: (3 * K + 7) // 8, 2: (K + 3) // 4}[bits]
     packed = np.empty((N, row_bytes), dtype=np.uint8)
     scales = np.empty((N, ng), dtype=np.float16)
     zeros = np.empty((N, ng), dtype=np.float16)
@@ -244,8 +250,11 @@ CONFIG_SHAPES = {
 }
 
 
-def layer_weights(seed: int, layer: int, sh: LayerShape):
+def layer_weights(seed: int, layer: int, sh: LayerShape, bits: int | None = None):
     """All tensors of one layer: four quantised linears, two norm gains, router.
+
+    `bits` overrides the shape's bit-width for this layer (layer-interleaved
+    mixed precision of the mixed 2&4-bit appendix: even layers 4-bit, odd 2-bit).
 
     Stream ids: layer*16 + {0:qkv, 1:o, 2:gate_up, 3:down, 4:router}.  The QKV
     matrix stacks Wq, Wk, Wv along the output dimension; gate_up stacks the
@@ -255,11 +264,12 @@ def layer_weights(seed: int, layer: int, sh: LayerShape):
     """
     b = layer * 16
     d, F = sh.d, sh.ffn
+    bits = sh.bits if bits is None else bits
     w = {
-        "qkv": quantized_weight(seed, b + 0, sh.q_dim + 2 * sh.kv_dim, d, sh.bits, sh.group),
-        "o": quantized_weight(seed, b + 1, d, sh.q_dim, sh.bits, sh.group),
-        "gate_up": quantized_weight(seed, b + 2, 2 * F, d, sh.bits, sh.group),
-        "down": quantized_weight(seed, b + 3, d, F, sh.bits, sh.group),
+        "qkv": quantized_weight(seed, b + 0, sh.q_dim + 2 * sh.kv_dim, d, bits, sh.group),
+        "o": quantized_weight(seed, b + 1, d, sh.q_dim, bits, sh.group),
+        "gate_up": quantized_weight(seed, b + 2, 2 * F, d, bits, sh.group),
+        "down": quantized_weight(seed, b + 3, d, F, bits, sh.group),
         "gamma1": np.ones(d, dtype=np.float32),
         "gamma2": np.ones(d, dtype=np.float32),
         "router_w": round_bf16((normal(seed, b + 4, d) * 0.02).astype(np.float32)),

@@ -46,6 +46,7 @@ def test_host_side_argument_validation(api):
     L = api.lib()
     n = C.c_size_t(0)
     assert L.qtale_wq_repack(None, None, None, 8, 64, 5, 64, 0, None, C.byref(n)) == -4
+    assert L.qtale_wq_repack(None, None, None, 8, 64, 1, 64, 0, None, C.byref(n)) == -4
     assert L.qtale_wq_repack(None, None, None, 8, 64, 4, 32, 0, None, C.byref(n)) == -5
     assert L.qtale_wq_repack(None, None, None, 0, 64, 4, 64, 0, None, C.byref(n)) == -3
     assert L.qtale_wq_repack(None, None, None, 7, 64, 4, 64, 1, None, C.byref(n)) == -3
@@ -63,7 +64,8 @@ def test_host_side_argument_validation(api):
 
 
 @pytest.mark.parametrize("bits,group,N,K,mode", [(4, 128, 256, 256, 0), (4, 64, 200, 688, 0),
-                                                 (3, 128, 128, 384, 0), (4, 64, 1376, 256, 1)])
+                                                 (3, 128, 128, 384, 0), (4, 64, 1376, 256, 1),
+                                                 (2, 128, 256, 384, 0), (2, 64, 130, 200, 0)])
 def test_repack_blob_size_and_padding(api, bits, group, N, K, mode):
     wq = inputs.quantized_weight(3, 1, N, K, bits, group)
     blob = api.wq_repack(wq["packed"], wq["scales"], wq["zeros"], N, K, bits, group, mode)
@@ -78,6 +80,9 @@ def test_repack_blob_size_and_padding(api, bits, group, N, K, mode):
     if bits == 4 and mode == 0 and K == K_pad and N % 128 == 0:
         chunks = blob.reshape(-1, 4096 + 512)
         assert int(np.unpackbits(chunks[:, :4096]).sum()) == int(np.unpackbits(wq["packed"]).sum())
+    if bits == 2 and K == K_pad and N % 128 == 0:     # the same for the single 2-bit plane
+        chunks = blob.reshape(-1, 2048 + 512)
+        assert int(np.unpackbits(chunks[:, :2048]).sum()) == int(np.unpackbits(wq["packed"]).sum())
     # too-small output buffer is reported, not overrun
     small = np.empty(16, np.uint8)
     nb = C.c_size_t(16)

@@ -272,6 +272,10 @@ GEMM_CASES = [
     (64, 512, 4096, 3, 128, 58),           # decode kernel at the 7B-shaped K: 64 K blocks through the ring
     (64, 256, 11008, 4, 64, 38),           # decode kernel, K of the down projection: 172 K blocks
     (57, 384, 11008, 3, 128, None),        # the same in 3-bit, token count not a multiple of 8
+    (200, 384, 320, 2, 64, 131),           # 2-bit (mixed 2&4-bit layers), single-CTA kernel, ragged tokens
+    (700, 640, 384, 2, 128, 651),          # 2-bit, CTA-pair kernel
+    (64, 9600, 192, 2, 64, 37),            # 2-bit, decode kernel (and split over K with a workspace)
+    (40, 256, 4096, 2, 128, None),         # 2-bit, decode kernel, 64 K blocks
 ]
 
 

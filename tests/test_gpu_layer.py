@@ -294,11 +294,14 @@ def test_decode_step_ragged_cache_lengths(env):
     assert_layer_close(out, ref, strict=True)
 
 
-def test_model_prefill_teacher_forced(env):
+@pytest.mark.parametrize("layer_bits", [None, (4, 2, 4)])
+def test_model_prefill_teacher_forced(env, layer_bits):
     """Stack of layers with one global theta: each layer's selection is checked
     against the oracle's router on the SAME input (the GPU's x_l), the layer output
     against the oracle with the oracle's mask; the one-call model entry point must
-    reproduce the layer-by-layer result bit for bit, and the LM head matches."""
+    reproduce the layer-by-layer result bit for bit, and the LM head matches.
+    With layer_bits the layers alternate 4-bit and 2-bit weights (the mixed 2&4-bit
+    setting) and the configuration leaves the width to each weight."""
     api, torch, dev = env
     sh = inputs.LayerShape(256, 4, 2, 64, 512, 4, 128)
     L, V, B, S = 3, 1000, 3, 90
@@ -307,7 +310,7 @@ def test_model_prefill_teacher_forced(env):
     T = int(cu[-1])
     ws_l, lws = [], []
     for li in range(L):
-        w = inputs.layer_weights(9, li, sh)
+        w = inputs.layer_weights(9, li, sh, bits=layer_bits[li] if layer_bits else None)
         w["router_w"] = inputs.round_bf16((inputs.normal(9, 500 + li, sh.d) * 0.05).astype(np.float32))
         ws_l.append(oracle.DenseLayer(sh, w))
         lws.append(api.LayerWeights(w, dev))
@@ -315,7 +318,7 @@ def test_model_prefill_teacher_forced(env):
     lm_head = inputs.activations(9, 601, V, sh.d, 0.05)
     fgam = (1 + 0.1 * inputs.normal(9, 602, sh.d)).astype(np.float32)
     ids = inputs.integers(9, 603, T, V)
-    cfg = api.layer_config(sh, api.SELECT_THRESHOLD, theta=theta)
+    cfg = api.layer_config(sh, api.SELECT_THRESHOLD, theta=theta, bits=0 if layer_bits else None)
     cud = torch.from_numpy(cu).to(dev)
     # layer by layer, teacher forced
     x = embed[ids]

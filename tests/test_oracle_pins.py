@@ -158,7 +158,8 @@ def test_half_conversion_all_bit_patterns():
             assert L.orc_float_to_half(float(v)) == int(np.float32(v).astype(np.float16).view(np.uint16))
 
 
-@pytest.mark.parametrize("bits,group,K", [(4, 128, 512), (4, 64, 688), (3, 128, 384), (3, 64, 200)])
+@pytest.mark.parametrize("bits,group,K", [(4, 128, 512), (4, 64, 688), (3, 128, 384), (3, 64, 200),
+                                          (2, 128, 384), (2, 64, 203)])
 def test_quantize_roundtrip_and_error_bound(bits, group, K):
     N = 24
     w = (inputs.normal(8, bits * 1000 + K, N * K) * 0.02).astype(np.float32).reshape(N, K)
@@ -183,7 +184,8 @@ def test_quantize_roundtrip_and_error_bound(bits, group, K):
     assert np.all(oracle.dequantize(oracle.pack_codes(c0, bits), s0, z0, K, bits, group) == 0.0)
 
 
-@pytest.mark.parametrize("bits,group,K", [(4, 128, 256), (4, 64, 688), (3, 128, 256), (3, 64, 88)])
+@pytest.mark.parametrize("bits,group,K", [(4, 128, 256), (4, 64, 688), (3, 128, 256), (3, 64, 88),
+                                          (2, 128, 256), (2, 64, 90)])
 def test_input_recipe_matches_oracle_quantiser(bits, group, K):
     N = 16
     w = (inputs.normal(9, K + bits, N * K) * 0.02).astype(np.float32).reshape(N, K)
@@ -202,6 +204,11 @@ def test_packed_layout_hand_example():
     p3 = oracle.pack_codes(codes, 3)
     word = sum(int(c) << (3 * i) for i, c in enumerate(codes[0]))
     assert list(p3[0]) == [(word >> (8 * i)) & 0xFF for i in range(4)]
+    # 2-bit (mixed 2&4-bit appendix): four codes per byte, first code in the low bits
+    c2 = np.array([[0, 1, 2, 3, 3, 0, 1, 0, 2]], np.uint8)
+    p2 = oracle.pack_codes(c2, 2)
+    assert list(p2[0]) == [0b11100100, 0b00010011, 0b00000010]
+    assert np.array_equal(oracle.unpack_codes(p2, 9, 2), c2)
 
 
 def test_model_size_and_bytes_per_weight():
