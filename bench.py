@@ -52,7 +52,7 @@ KERNELS_PER_STEP = 8
 # at ratio 0.5 (4096 executed tokens), one ncu capture of the kernels as they stand
 # (profiles/wq_gemm_pair_c2_layer_step.md); None at other ratios.
 GEMM_DRAM_BYTES = 733111296
-ALL_LEGS = ["sweep", "gemm", "bf16", "router", "gather", "scatter", "decode", "decode_loop", "c4", "c5", "e2e", "cpu"]
+ALL_LEGS = ["sweep", "gemm", "bf16", "router", "gather", "scatter", "attention", "decode", "decode_loop", "c4", "c5", "e2e", "cpu"]
 
 
 def measured_peaks():
@@ -577,6 +577,33 @@ def run_ours(args):
             us=ms * 1e3, rows="%d of %d, d %d" % (kg, Tg, dg),
             roofline=hbm_roofline("compact_kernel", kg * dg * 4, ms, peaks), clocks=r["clocks"])
         del xg, hn
+        check_status()
+
+    if "attention" in legs:
+        # causal attention among the executed tokens alone: 4 sequences of 2048 (ratio 1.0) and of
+        # 1024 (ratio 0.5) executed tokens, 32 heads of 128
+        out = {}
+        H, hd = 32, 128
+        for name, Bq, Sq in (("4x2048", 4, 2048), ("4x1024", 4, 1024), ("16x2048", 16, 2048)):
+            Tq = Bq * Sq
+            qkv = torch.randn(Tq, 3 * H * hd, device=dev, generator=gen).to(torch.float16)
+            ao = torch.empty(Tq, H * hd, dtype=torch.float16, device=dev)
+            cuq = torch.arange(Bq + 1, dtype=torch.int32, device=dev) * Sq
+            call = lambda: api.attention_prefill(qkv, H, H, hd, cuq, api.ACT_F16, ao)
+            call()
+            gr = graph_of(torch, call, 5)
+            r = timer.run(lambda i: gr.replay(), 10, 3, 0.25)
+            ms = r["ms"] / 5
+            fl = accounting.attention_flops([Sq] * Bq, H, hd)
+            tf = fl / (ms * 1e-3) / 1e12
+            out[name] = dict(us=ms * 1e3, tflops=tf, clocks=r["clocks"],
+                             roofline=dict(bound="tensor", kernel="attn_prefill_tc_kernel<128,1>", achieved=tf,
+                                           peak=peaks["bf16_tflops"], unit="TFLOP/s",
+                                           frac=tf / peaks["bf16_tflops"],
+                                           note="causal FLOPs 2*2*S(S+1)/2*H*hd per sequence; the kernel also "
+                                                "computes the masked half of every diagonal tile"))
+            del qkv, ao
+        extra["attention_prefill"] = out
         check_status()
 
     if "scatter" in legs:

@@ -305,6 +305,33 @@ int qtale_wq_gemm(const void* a, int lda, const int32_t* m_dev, int M_cap, const
                   void* ws, size_t ws_bytes, void* stream);
 
 /* ------------------------------------------------------------------------- */
+/* Attention among the executed tokens (Eq. 3: bypassed tokens have no query,   */
+/* key or value at the layer)                                                   */
+/* ------------------------------------------------------------------------- */
+
+/*
+ * Causal softmax attention of a compacted prefill batch: executed token i of a
+ * sequence attends to the executed tokens j <= i of the same sequence, scale
+ * 1/sqrt(head_dim), fp32 softmax, probabilities rounded once to act_dtype.
+ *   qkv [T_cap, ld] act_dtype, device: row i = [n_heads query heads | n_kv_heads
+ *     key heads | n_kv_heads value heads], each head_dim wide, queries and keys
+ *     already rotated; rows in compacted order (sequence by sequence).
+ *   cu_exec [B+1] int32, device: executed rows of sequence b are
+ *     cu_exec[b] .. cu_exec[b+1]-1, non-decreasing, cu_exec[B] <= T_cap.
+ *   out [T_cap, ldo] act_dtype: rows below cu_exec[B] are written (columns
+ *     0 .. n_heads*head_dim-1), the rest left untouched.
+ * Keys and values are read in tiles of 128 rows: the value columns of the rows
+ * from cu_exec[B] to the end of that 128-row tile (as far as T_cap reaches) must
+ * hold finite numbers (their probabilities are zero; the layer path clears them).
+ * head_dim 64 or 128; n_heads a multiple of n_kv_heads; ld, ldo multiples of 8;
+ * qkv and out 16-byte aligned.  Nothing is owned or allocated.
+ * Errors: QTALE_ERR_NULL / _SHAPE / _ALIGN / _MODE before anything is launched.
+ */
+int qtale_attention_prefill(const void* qkv, int ld, int n_heads, int n_kv_heads, int head_dim,
+                            int act_dtype, const int32_t* cu_exec, int B, int T_cap, void* out,
+                            int ldo, void* stream);
+
+/* ------------------------------------------------------------------------- */
 /* Layer and model                                                             */
 /* ------------------------------------------------------------------------- */
 

@@ -111,6 +111,9 @@ def lib():
         L.qtale_wq_gemm.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.POINTER(WqWeight),
                                     C.c_int, C.c_int, C.POINTER(EpilogueArgs), C.c_void_p, C.c_int,
                                     C.c_void_p, C.c_size_t, C.c_void_p]
+        L.qtale_attention_prefill.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
+                                              C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_int,
+                                              C.c_void_p]
         L.qtale_wq_gemm_workspace_bytes.restype = C.c_size_t
         L.qtale_wq_gemm_workspace_bytes.argtypes = []
         L.qtale_layer_workspace_bytes.restype = C.c_size_t
@@ -345,6 +348,23 @@ def wq_gemm(a, w: QuantWeight, m_dev=None, epilogue=EPI_STORE_16, y=None, idx=No
                               ws.numel() * ws.element_size() if ws is not None else 0, _stream()),
           "qtale_wq_gemm")
     return dst if epilogue == EPI_RESID_SCATTER else y
+
+
+# ---------------------------------------------------------------------------------
+# attention
+# ---------------------------------------------------------------------------------
+
+def attention_prefill(qkv, n_heads, n_kv_heads, head_dim, cu_exec, act_dtype=ACT_F16, out=None):
+    """qtale_attention_prefill on a compacted [T_cap, (H + 2 Hkv) hd] tensor of rotated q | k | v."""
+    import torch
+    T_cap = int(qkv.shape[0])
+    if out is None:
+        out = torch.zeros(T_cap, n_heads * head_dim, dtype=qkv.dtype, device=qkv.device)
+    check(lib().qtale_attention_prefill(_ptr(qkv), int(qkv.stride(0)), n_heads, n_kv_heads, head_dim,
+                                        int(act_dtype), _ptr(cu_exec), int(cu_exec.numel()) - 1, T_cap,
+                                        _ptr(out), int(out.stride(0)), _stream()),
+          "qtale_attention_prefill")
+    return out
 
 
 # ---------------------------------------------------------------------------------

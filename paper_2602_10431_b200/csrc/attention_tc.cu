@@ -12,7 +12,7 @@
 //                 in the 16-bit activation format (the A operand of the next MMA);
 //   O += P V      TS MMA with V read straight from its row-major tile (MN-major B
 //                 operand), fp32 output accumulator in tensor memory, rescaled by the
-//                 softmax warps only when a row's running maximum moves.
+//                 softmax warps only when a row's maximum has outgrown the reference by 2^8.
 // Keys and values have rings of their own (three and two tiles) and a producer thread each:
 // a key tile is free as soon as its scores exist, so its successor is loaded three tiles
 // ahead; with one two-stage ring released after P V the load latency (about 1800 cycles) sat
@@ -37,6 +37,7 @@ constexpr int kTcKStages = 3;    // key tiles in flight (the first thing a tile 
 constexpr int kTcVStages = 2;    // value tiles in flight
 constexpr int kTcTile = 128;  // query rows per CTA and keys per tile
 constexpr uint32_t kTcSlices = 1u << 16;  // suspended barrier tests before a wait gives up
+constexpr float kTcMaxSlack = 8.f;        // log2 growth of a row maximum that moves the softmax reference
 
 struct TcShared {
   uint64_t q_full, q_empty, o_empty;
@@ -367,14 +368,19 @@ __global__ void __launch_bounds__(kTcThreads, 1)
         if (lane == 0) mbar_arrive(&sh.max_bar);
         if (!tc_wait(&sh.max_bar, tt & 1u, &sh, p.status)) { alive = false; break; }
         const float row_raw = fmaxf(my_max, sh.row_max[tt & 1][half ^ 1][row]);
-        const float mx = fmaxf(m_run, row_raw * p.scale_log2);
-        const float m_safe = (mx == -INFINITY) ? 0.f : mx;
-        const float corr = ex2_approx(m_run - m_safe);
-        const bool moved = mx > m_run;
-        m_run = mx;
-        l_run *= corr;
+        // The reference maximum only moves when the row's maximum has grown by more than 2^8
+        // (always on the first tile): until then the probabilities are at most 256, which both
+        // 16-bit formats and the fp32 sums hold, and the output accumulator needs no rescaling.
+        const float cand = row_raw * p.scale_log2;
+        const bool moved = cand > m_run + kTcMaxSlack;
+        float corr = 1.f;
+        if (moved) {
+          corr = ex2_approx(m_run - cand);  // 0 on the first tile (m_run = -inf)
+          m_run = cand;
+          l_run *= corr;
+        }
         // probabilities in the 16-bit format, two keys per 32-bit column
-        const float neg_m = -m_safe;
+        const float neg_m = (m_run == -INFINITY) ? 0.f : -m_run;
         float sq[4] = {0.f, 0.f, 0.f, 0.f};
         uint32_t pr[32];
 #pragma unroll
@@ -385,21 +391,22 @@ __global__ void __launch_bounds__(kTcThreads, 1)
           pr[i] = Act16<ACT>::pack(p0, p1);
         }
         l_run += (sq[0] + sq[1]) + (sq[2] + sq[3]);
-        // the previous P V must be complete before O is rescaled or P is overwritten (for the
-        // first tile of an item the output stage of the item before has waited for it)
+        // The previous P V must be complete before O is rescaled.  Every tile waits for it, moved
+        // or not, so that the barrier is never more than one phase ahead of a parity test (by now
+        // that P V, issued a whole softmax earlier, has long finished).
         if (j > 0) {
           if (!tc_wait(&sh.pv_done, (tt - 1) & 1u, &sh, p.status)) { alive = false; break; }
           tc_fence_after();
-          if (__any_sync(0xffffffffu, moved)) {
+        }
+        if (j > 0 && __any_sync(0xffffffffu, moved)) {
 #pragma unroll 1
-            for (int c = 0; c < OC / 32; ++c) {
-              uint32_t r[32];
-              tmem_ld_x32(tmem + lane_addr + O_COL + half * OC + c * 32, r);
-              tmem_wait_ld();
+          for (int c = 0; c < OC / 32; ++c) {
+            uint32_t r[32];
+            tmem_ld_x32(tmem + lane_addr + O_COL + half * OC + c * 32, r);
+            tmem_wait_ld();
 #pragma unroll
-              for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * corr);
-              tmem_st_x32(tmem + lane_addr + O_COL + half * OC + c * 32, r);
-            }
+            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * corr);
+            tmem_st_x32(tmem + lane_addr + O_COL + half * OC + c * 32, r);
           }
         }
         tmem_st_x32(tmem + lane_addr + P_COL + s * 64 + half * 32, pr);
@@ -529,3 +536,19 @@ int launch_attn_prefill(const void* qkv, int ld, int H, int Hkv, int hd, int act
 }
 
 }  // namespace qtale
+
+extern "C" int qtale_attention_prefill(const void* qkv, int ld, int n_heads, int n_kv_heads, int head_dim,
+                                       int act_dtype, const int32_t* cu_exec, int B, int T_cap, void* out,
+                                       int ldo, void* stream) {
+  using namespace qtale;
+  if (act_dtype != QTALE_ACT_BF16 && act_dtype != QTALE_ACT_F16) return QTALE_ERR_MODE;
+  if (!qkv || !cu_exec || !out) return QTALE_ERR_NULL;
+  if (B < 1 || T_cap < 1 || n_heads < 1 || n_kv_heads < 1 || n_heads % n_kv_heads != 0 ||
+      (head_dim != 64 && head_dim != 128))
+    return QTALE_ERR_SHAPE;
+  if (ld < (n_heads + 2 * n_kv_heads) * head_dim || ldo < n_heads * head_dim || ld % 8 != 0 || ldo % 8 != 0)
+    return QTALE_ERR_SHAPE;
+  if (!aligned16(qkv) || !aligned16(out)) return QTALE_ERR_ALIGN;
+  return launch_attn_prefill(qkv, ld, n_heads, n_kv_heads, head_dim, act_dtype, cu_exec, B, T_cap, out, ldo,
+                             static_cast<cudaStream_t>(stream));
+}

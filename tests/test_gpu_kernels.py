@@ -397,6 +397,44 @@ def test_wq_gemm_rotary_epilogue(env, hd, H, Hkv, M, m_dev, act):
     assert np.abs(plain[:mm] - y_ref).max() <= 1e-4 * max(1.0, np.abs(y_ref).max())
 
 
+@pytest.mark.parametrize("hd,H,Hkv,lens", [
+    (128, 4, 2, [300, 1, 0, 128, 257]),      # ragged, an empty sequence, lengths around the tile size
+    (64, 3, 3, [77, 513]),                   # 64-wide heads, five key tiles
+    (128, 2, 1, [1024]),                     # eight query tiles of one sequence
+])
+@pytest.mark.parametrize("act", [0, 1])
+def test_attention_prefill_against_oracle(env, hd, H, Hkv, lens, act):
+    """Stand-alone causal attention among the executed tokens of each sequence (Eq. 3)."""
+    api, torch, dev = env
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    Te = int(cu[-1])
+    T_cap = Te + 70
+    ld = (H + 2 * Hkv) * hd
+    qkv = round_act(inputs.activations(61 + hd, 3, T_cap, ld), act)
+    qkv[Te:, (H + Hkv) * hd:] = 0.0                          # value rows behind the last sequence: finite
+    seq_of = np.repeat(np.arange(len(lens)), lens).astype(np.int32)
+    pos = np.concatenate([np.arange(n) for n in lens]).astype(np.int32)
+    ref = oracle.attention(qkv[:Te, :H * hd], qkv[:Te, H * hd:(H + Hkv) * hd], qkv[:Te, (H + Hkv) * hd:],
+                           H, Hkv, hd, seq_of, pos)
+    out = torch.full((T_cap, H * hd), 7.0, dtype=api.act_torch_dtype(act), device=dev)
+    api.attention_prefill(api.to_device_act(qkv, act, dev), H, Hkv, hd, torch.from_numpy(cu).to(dev), act, out)
+    assert api.device_status() == 0
+    got = api.to_host_f32(out)
+    assert np.all(got[Te:] == 7.0)                           # rows behind the executed ones untouched
+    # probabilities and outputs are rounded once to the 16-bit format: a convex combination of
+    # values moves by at most that rounding of the largest value, plus the output's own rounding
+    vmax = np.abs(qkv[:Te, (H + Hkv) * hd:]).max()
+    assert np.abs(got[:Te] - ref).max() <= 4 * act_eps(act) * vmax
+    assert rel_fro(got[:Te], ref) <= 3 * act_eps(act)
+    # the first token of a sequence sees only itself: its output is its own value row
+    for b, n in enumerate(lens):
+        if n:
+            r = int(cu[b])
+            v = qkv[r, (H + Hkv) * hd:].reshape(Hkv, hd)
+            want = np.repeat(v, H // Hkv, axis=0).reshape(-1)
+            assert np.array_equal(got[r], want)
+
+
 def test_wq_gemm_full_size_sampled(env):
     """7B-sized gate/up projection in the launch configuration the benchmark times
     (8192-token capacity, device-side count): 66 complete output rows, two from every 256-token
