@@ -1,26 +1,27 @@
 // Causal attention among the executed tokens of each sequence (prefill) on the
 // tcgen05 tensor cores (Eq. 3: bypassed tokens have no query, key or value here).
 //
-// A work item is 128 consecutive executed tokens (query rows) of one sequence and one
-// head; the grid is persistent (one CTA per SM walks the items sequence by sequence) and an item
-// streams that sequence's executed keys / values in tiles of 128:
-//   S = Q K^T     SS MMA, Q and K tiles from 128-byte-swizzled shared memory (TMA),
-//                 fp32 scores in tensor memory, double buffered;
-//   softmax       eight warps, two threads per query row (64 keys each; the half-row maxima
-//                 meet through shared memory): running max / sum in the log2 domain (one fma
-//                 and one ex2.approx per score), probabilities written back to tensor memory
-//                 in the 16-bit activation format (the A operand of the next MMA);
-//   O += P V      TS MMA with V read straight from its row-major tile (MN-major B
-//                 operand), fp32 output accumulator in tensor memory, rescaled by the
-//                 softmax warps only when a row's maximum has outgrown the reference by 2^8.
-// Keys and values have rings of their own (three and two tiles) and a producer thread each:
-// a key tile is free as soon as its scores exist, so its successor is loaded three tiles
-// ahead; with one two-stage ring released after P V the load latency (about 1800 cycles) sat
-// in the loop of every tile.  Barrier phases run on across items (tiles are counted per
-// CTA), so the loads and the first Q K^T of the next item overlap the output stage of the
-// current one.
-// Warp roles (352 threads): warp 0 Q / K producer, warp 1 MMA issuer and TMEM allocator,
-// warps 2-9 softmax / correction / output, warp 10 V producer.  Every wait is bounded.
+// A work item is 256 consecutive executed tokens of one sequence and one head, handled as two
+// query tiles A and B of 128 rows that share one stream of key / value tiles (128 keys each).
+// The grid is persistent (one CTA per SM walks the items sequence by sequence).  Per query
+// tile X and key tile j:
+//   S_X = Q_X K^T   SS MMA, Q and K tiles from 128-byte-swizzled shared memory (TMA), fp32
+//                   scores in tensor memory (128 columns per query tile);
+//   softmax         four warps per query tile, one thread per query row: the 128 scores of the
+//                   row in registers, running max / sum in the log2 domain (one fma and one
+//                   ex2.approx per score), probabilities written over the scores' own columns in
+//                   the 16-bit activation format (the A operand of the next MMA);
+//   O_X += P_X V    TS MMA with V read straight from its row-major tile (MN-major B operand),
+//                   fp32 output accumulator in tensor memory, rescaled by the softmax warps only
+//                   when a row's maximum has outgrown the softmax reference by 2^8.
+// Scores, probabilities and outputs of both tiles fill the 512 tensor-memory columns, so a
+// tile's next scores can only be computed once its probabilities have been consumed; the two
+// tiles alternate instead: while the warps of one tile are in their softmax (bound by the
+// special-function unit) the tensor pipe works on P V and Q K^T of the other.  The single
+// issuing thread orders the work A, B, A, B, ...: P_X V (j), then Q_X K^T (j + 1).
+// Tile B of the last item of a sequence may lie wholly behind the sequence: it is skipped.
+// Warp roles (384 threads): warp 0 Q / K producer, warp 1 MMA issuer and TMEM allocator,
+// warp 2 V producer, warps 4-7 softmax of tile A, warps 8-11 of tile B.  Every wait is bounded.
 #include <cuda.h>
 
 #include <string.h>
@@ -32,22 +33,19 @@ namespace qtale {
 
 using namespace ptx;
 
-constexpr int kTcThreads = 352;  // K producer, issuer, eight softmax warps, V producer
-constexpr int kTcKStages = 3;    // key tiles in flight (the first thing a tile needs)
+constexpr int kTcThreads = 384;
+constexpr int kTcKStages = 2;    // key tiles in flight
 constexpr int kTcVStages = 2;    // value tiles in flight
-constexpr int kTcTile = 128;  // query rows per CTA and keys per tile
+constexpr int kTcTile = 128;     // query rows per tile and keys per tile
+constexpr int kTcItemRows = 2 * kTcTile;
 constexpr uint32_t kTcSlices = 1u << 16;  // suspended barrier tests before a wait gives up
 constexpr float kTcMaxSlack = 8.f;        // log2 growth of a row maximum that moves the softmax reference
 
 struct TcShared {
-  uint64_t q_full, q_empty, o_empty;
+  uint64_t q_full, q_empty;
   uint64_t k_full[kTcKStages], k_empty[kTcKStages];
   uint64_t v_full[kTcVStages], v_empty[kTcVStages];
-  uint64_t max_bar, sum_bar;  // the two threads of a query row exchange their half-row maximum / sum
-  float row_max[2][2][kTcTile];  // [tile parity][half][row]
-  float row_sum[2][kTcTile];     // [half][row]
-  uint64_t s_full[2], p_full[2];
-  uint64_t pv_done;
+  uint64_t s_full[2], p_full[2], pv_done[2], o_empty[2];  // per query tile
   uint32_t tmem_base;
   volatile int abort_flag;
 };
@@ -101,32 +99,93 @@ __device__ __forceinline__ uint64_t v_desc(uint32_t smem_addr, int key16) {
   return d;
 }
 
-// Work items of the persistent grid, sequence by sequence; within a sequence by query tile
-// (longest first in even sequences, shortest first in odd ones), each tile for every head.  CTA
-// c takes items c, c + grid, ...  The CTAs running at one time then work on one or two
-// sequences, whose keys and values stay in L2 (with the tiles of all sequences sorted into one
-// list, every sequence's keys were live at once and were re-read from DRAM 3.6 times), and
-// the alternating direction evens out the CTAs' total tile counts.  The cursor only moves forward.
+// Work items of the persistent grid: (sequence, block of 256 query rows, head), a block for every
+// head.  An item's cost grows with its block index (causal attention), and each CTA takes its
+// items in a fixed pattern, so the order of the list decides the balance.  Two orders:
+//  * level order, when the keys and values of the whole call fit the L2 cache: the last blocks of
+//    all sequences first, then the blocks before them, ... (cost descending), dealt to the CTAs
+//    forwards and backwards in alternate rounds, so a CTA that drew the dearest item of one round
+//    draws the cheapest of the next;
+//  * sequence order otherwise: sequence by sequence (longest block first in even sequences,
+//    shortest first in odd ones), dealt round-robin.  The CTAs running at one time then work on
+//    one or two sequences, whose keys and values stay in L2 (with all sequences live at once they
+//    were re-read from DRAM several times).
+// A cursor only moves forward: the k-th item of a CTA has a larger index than its (k-1)-th.
+constexpr long long kTcLevelOrderBytes = 72ll << 20;
+
 struct ItemCursor {
-  int seq;    // sequence being enumerated
+  int seq;    // sequence (sequence order) or level (level order) being enumerated
   int base;   // index of its first item
-  int nt;     // its query tiles (-1: not counted yet)
+  int nt;     // its blocks (sequence order) or sequences (level order); -1: not counted yet
 };
 
-__device__ __forceinline__ int seq_tiles(const TcParams& p, int s) {
-  return (p.cu_exec[s + 1] - p.cu_exec[s] + kTcTile - 1) / kTcTile;
+struct ItemOrder {
+  bool level;      // level order
+  int max_blocks;  // blocks of the longest sequence
+  int n_items;
+};
+
+__device__ __forceinline__ int seq_blocks(const TcParams& p, int s) {
+  return (p.cu_exec[s + 1] - p.cu_exec[s] + kTcItemRows - 1) / kTcItemRows;
 }
 
-// item i (i must not decrease between calls) -> sequence, head, query tile; false past the end
-__device__ __forceinline__ bool item_at(const TcParams& p, ItemCursor& c, int i, int& b, int& h, int& qt) {
+__device__ __forceinline__ ItemOrder item_order(const TcParams& p, int hd) {
+  ItemOrder o;
+  int n_blocks = 0;
+  o.max_blocks = 0;
+  for (int s = 0; s < p.B; ++s) {
+    const int nb = seq_blocks(p, s);
+    n_blocks += nb;
+    o.max_blocks = max(o.max_blocks, nb);
+  }
+  o.n_items = n_blocks * p.H;
+  const long long kv_bytes = (long long)(p.cu_exec[p.B] - p.cu_exec[0]) * (p.H / p.rep) * hd * 4;
+  o.level = kv_bytes <= kTcLevelOrderBytes;
+  return o;
+}
+
+// index of the r-th item of CTA c (grid g)
+__device__ __forceinline__ int item_index(const ItemOrder& o, int r, int c, int g) {
+  return r * g + ((o.level && (r & 1)) ? g - 1 - c : c);
+}
+
+// item i (i must not decrease between calls) -> sequence, head, query block; false past the end
+__device__ __forceinline__ bool item_at(const TcParams& p, const ItemOrder& o, ItemCursor& c, int i, int& b,
+                                        int& h, int& qb) {
+  if (o.level) {
+    while (c.seq < o.max_blocks) {
+      qb = o.max_blocks - 1 - c.seq;
+      if (c.nt < 0) {
+        c.nt = 0;
+        for (int s = 0; s < p.B; ++s) c.nt += seq_blocks(p, s) > qb ? 1 : 0;
+      }
+      const int n = c.nt * p.H;
+      if (i < c.base + n) {
+        const int r = i - c.base;
+        h = r % p.H;
+        int k = r / p.H;  // the k-th sequence that has this block
+        b = 0;
+        for (int s = 0; s < p.B; ++s)
+          if (seq_blocks(p, s) > qb) {
+            if (k == 0) { b = s; break; }
+            --k;
+          }
+        return true;
+      }
+      c.base += n;
+      c.nt = -1;
+      ++c.seq;
+    }
+    return false;
+  }
   while (c.seq < p.B) {
-    if (c.nt < 0) c.nt = seq_tiles(p, c.seq);
+    if (c.nt < 0) c.nt = seq_blocks(p, c.seq);
     const int n = c.nt * p.H;
     if (i < c.base + n) {
       const int r = i - c.base;
       b = c.seq;
       h = r % p.H;
-      qt = (c.seq & 1) ? r / p.H : c.nt - 1 - r / p.H;
+      qb = (c.seq & 1) ? r / p.H : c.nt - 1 - r / p.H;
       return true;
     }
     c.base += n;
@@ -136,36 +195,48 @@ __device__ __forceinline__ bool item_at(const TcParams& p, ItemCursor& c, int i,
   return false;
 }
 
+// What an item asks of the two query tiles
+struct ItemShape {
+  int seq0, len;
+  int jA, jB;   // last key tile of query tile A / B (B = -1 when its rows lie behind the sequence)
+  int nj;       // key tiles the item streams
+};
+
+__device__ __forceinline__ ItemShape item_shape(const TcParams& p, int b, int qb) {
+  ItemShape s;
+  s.seq0 = p.cu_exec[b];
+  s.len = p.cu_exec[b + 1] - s.seq0;
+  s.jA = 2 * qb;
+  s.jB = (qb * kTcItemRows + kTcTile < s.len) ? 2 * qb + 1 : -1;
+  s.nj = (s.jB >= 0 ? s.jB : s.jA) + 1;
+  return s;
+}
+
 template <int HD, int ACT>
 __global__ void __launch_bounds__(kTcThreads, 1)
     attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmap, const TcParams p) {
   constexpr int CH = HD / 64;                       // 16 KB chunks per tile
   constexpr int TILE_BYTES = kTcTile * HD * 2;
-  constexpr int S_COL = 0;                          // two score buffers of 128 columns
-  constexpr int P_COL = 256;                        // two probability buffers of 64 columns
-  constexpr int O_COL = 384;                        // output accumulator, HD columns
+  constexpr int S_COL = 0;                          // scores of tile X: 128 columns at 128 X; its
+                                                    // probabilities reuse the first 64 of them
+  constexpr int O_COL = 256;                        // output accumulator of tile X: HD columns at 256 + 128 X
   extern __shared__ unsigned char smem_dyn[];
   __shared__ TcShared sh;
   unsigned char* base = reinterpret_cast<unsigned char*>(
       (reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~static_cast<uintptr_t>(1023));
-  unsigned char* sQ = base;
-  unsigned char* sK = base + TILE_BYTES;                     // kTcKStages stages
-  unsigned char* sV = base + (1 + kTcKStages) * TILE_BYTES;  // kTcVStages stages
+  unsigned char* sQ = base;                                  // tiles A and B
+  unsigned char* sK = base + 2 * TILE_BYTES;                 // kTcKStages stages
+  unsigned char* sV = base + (2 + kTcKStages) * TILE_BYTES;  // kTcVStages stages
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-  int n_pairs = 0;
-  for (int s = 0; s < p.B; ++s) n_pairs += seq_tiles(p, s);
-  const int n_items = n_pairs * p.H;
+  const ItemOrder order = item_order(p, HD);
+  const int n_items = order.n_items;
   if ((int)blockIdx.x >= n_items) return;  // uniform for the CTA: nothing allocated yet
 
   if (threadIdx.x == 0) {
     mbar_init(&sh.q_full, 1);
     mbar_init(&sh.q_empty, 1);
-    for (int s = 0; s < 2; ++s) {
-      mbar_init(&sh.s_full[s], 1);
-      mbar_init(&sh.p_full[s], 8);
-    }
     for (int s = 0; s < kTcKStages; ++s) {
       mbar_init(&sh.k_full[s], 1);
       mbar_init(&sh.k_empty[s], 1);
@@ -174,10 +245,12 @@ __global__ void __launch_bounds__(kTcThreads, 1)
       mbar_init(&sh.v_full[s], 1);
       mbar_init(&sh.v_empty[s], 1);
     }
-    mbar_init(&sh.max_bar, 8);
-    mbar_init(&sh.sum_bar, 8);
-    mbar_init(&sh.pv_done, 1);
-    mbar_init(&sh.o_empty, 8);
+    for (int x = 0; x < 2; ++x) {
+      mbar_init(&sh.s_full[x], 1);
+      mbar_init(&sh.p_full[x], 4);   // the four softmax warps of the tile
+      mbar_init(&sh.pv_done[x], 1);
+      mbar_init(&sh.o_empty[x], 4);
+    }
     sh.abort_flag = 0;
     fence_barrier_init();
   }
@@ -190,58 +263,64 @@ __global__ void __launch_bounds__(kTcThreads, 1)
   tc_fence_after();
   const uint32_t tmem = sh.tmem_base;
 
-  // every role walks the same item sequence with its own cursor and its own running counters:
-  // t = key tiles so far (ring stage t & 1, phase (t >> 1) & 1), it = items so far
+  // every role walks the same item sequence with its own cursor and its own running counters
+  // (key / value tiles so far pick the ring stage and phase; tiles so far of query tile X the
+  // phase of X's barriers)
   ItemCursor cur;
   cur.seq = 0;
   cur.base = 0;
   cur.nt = -1;
 
   if (warp == 0) {
-    // ------------------------------ TMA producer ------------------------------
+    // ------------------------------ TMA producer: queries and keys ------------------------------
     if (lane == 0) {
       uint32_t t = 0, it = 0;
-      for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++it) {
-        int b, h, qt;
-        if (!item_at(p, cur, item, b, h, qt)) break;
+      for (int rd = 0;; ++rd, ++it) {
+        const int item = item_index(order, rd, blockIdx.x, gridDim.x);
+        int b, h, qb;
+        if (item >= n_items || !item_at(p, order, cur, item, b, h, qb)) break;
+        const ItemShape is = item_shape(p, b, qb);
         const int hk = h / p.rep;
-        const int seq0 = p.cu_exec[b];
+        const int n_q = is.jB >= 0 ? 2 : 1;
         if (!tc_wait(&sh.q_empty, (it & 1u) ^ 1u, &sh, p.status)) break;
-        mbar_arrive_expect_tx(&sh.q_full, TILE_BYTES);
-        for (int c = 0; c < CH; ++c)
-          tma_load_2d(sQ + c * 16384, &tmap, &sh.q_full, h * HD + c * 64, seq0 + qt * kTcTile);
+        mbar_arrive_expect_tx(&sh.q_full, (uint32_t)(n_q * TILE_BYTES));
+        for (int x = 0; x < n_q; ++x)
+          for (int c = 0; c < CH; ++c)
+            tma_load_2d(sQ + x * TILE_BYTES + c * 16384, &tmap, &sh.q_full, h * HD + c * 64,
+                        is.seq0 + qb * kTcItemRows + x * kTcTile);
         bool ok = true;
-        for (int j = 0; j <= qt; ++j, ++t) {
+        for (int j = 0; j < is.nj; ++j, ++t) {
           const int s = t % kTcKStages;
           const uint32_t ph = (t / kTcKStages) & 1u;
           if (!tc_wait(&sh.k_empty[s], ph ^ 1u, &sh, p.status)) { ok = false; break; }
           mbar_arrive_expect_tx(&sh.k_full[s], TILE_BYTES);
           for (int c = 0; c < CH; ++c)
             tma_load_2d(sK + s * TILE_BYTES + c * 16384, &tmap, &sh.k_full[s],
-                        p.k_off + hk * HD + c * 64, seq0 + j * kTcTile);
+                        p.k_off + hk * HD + c * 64, is.seq0 + j * kTcTile);
         }
         if (!ok) break;
       }
     }
-  } else if (warp == 10) {
+  } else if (warp == 2) {
     // ------------------------------ TMA producer of the value tiles ------------------------------
     // (a thread of its own: a full value ring must not hold back the key loads)
     if (lane == 0) {
       uint32_t t = 0;
       bool ok = true;
-      for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
-        int b, h, qt;
-        if (!item_at(p, cur, item, b, h, qt)) break;
+      for (int rd = 0; ok; ++rd) {
+        const int item = item_index(order, rd, blockIdx.x, gridDim.x);
+        int b, h, qb;
+        if (item >= n_items || !item_at(p, order, cur, item, b, h, qb)) break;
+        const ItemShape is = item_shape(p, b, qb);
         const int hk = h / p.rep;
-        const int seq0 = p.cu_exec[b];
-        for (int j = 0; j <= qt; ++j, ++t) {
+        for (int j = 0; j < is.nj; ++j, ++t) {
           const int s = t % kTcVStages;
           const uint32_t ph = (t / kTcVStages) & 1u;
           if (!tc_wait(&sh.v_empty[s], ph ^ 1u, &sh, p.status)) { ok = false; break; }
           mbar_arrive_expect_tx(&sh.v_full[s], TILE_BYTES);
           for (int c = 0; c < CH; ++c)
             tma_load_2d(sV + s * TILE_BYTES + c * 16384, &tmap, &sh.v_full[s],
-                        p.v_off + hk * HD + c * 64, seq0 + j * kTcTile);
+                        p.v_off + hk * HD + c * 64, is.seq0 + j * kTcTile);
         }
       }
     }
@@ -251,123 +330,145 @@ __global__ void __launch_bounds__(kTcThreads, 1)
       constexpr uint32_t idesc_qk = idesc_16bit_f32(128, kTcTile, ACT == 1);
       constexpr uint32_t idesc_pv = idesc_16bit_f32(128, HD, ACT == 1) | (1u << 16);  // B is MN-major
       const uint32_t qa = smem_u32(sQ);
-      auto issue_qk = [&](uint32_t tt) {
-        const int s = tt & 1;
-        const int ks = tt % kTcKStages;
-        if (!tc_wait(&sh.k_full[ks], (tt / kTcKStages) & 1u, &sh, p.status)) return false;
-        tc_fence_after();
+      // scores of query tile x against the key tile in ring stage ks
+      auto issue_qk = [&](int x, int ks) {
         const uint32_t ka = smem_u32(sK + ks * TILE_BYTES);
 #pragma unroll
         for (int kk = 0; kk < HD / 16; ++kk)
-          mma_ss(tmem + S_COL + s * 128, kmajor_desc(qa, kk), kmajor_desc(ka, kk), idesc_qk,
+          mma_ss(tmem + S_COL + x * 128, kmajor_desc(qa + x * TILE_BYTES, kk), kmajor_desc(ka, kk), idesc_qk,
                  kk != 0 ? 1u : 0u);
-        mma_commit(&sh.s_full[s]);
-        mma_commit(&sh.k_empty[ks]);  // the key tile is free as soon as its scores exist
-        return true;
+        mma_commit(&sh.s_full[x]);
       };
-      uint32_t t = 0, it = 0;
-      bool ok = true;
-      for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x, ++it) {
-        int b, h, qt;
-        if (!item_at(p, cur, item, b, h, qt)) break;
-        const int n_kt = qt + 1;
-        if (!tc_wait(&sh.q_full, it & 1u, &sh, p.status)) break;
-        ok = issue_qk(t);
-        if (ok && n_kt == 1) mma_commit(&sh.q_empty);  // the query tile has been read for the last time
-        for (int j = 0; ok && j < n_kt; ++j) {
-          const uint32_t tt = t + j;
-          const int s = tt & 1;
-          const uint32_t ph = (tt >> 1) & 1u;
-          // scores of the next tile are computed while the softmax of this one runs
-          if (j + 1 < n_kt) {
-            ok = issue_qk(tt + 1);
-            if (ok && j + 2 == n_kt) mma_commit(&sh.q_empty);
-          }
-          if (!ok) break;
-          if (!tc_wait(&sh.p_full[s], ph, &sh, p.status)) { ok = false; break; }
-          const int vs = tt % kTcVStages;
-          if (!tc_wait(&sh.v_full[vs], (tt / kTcVStages) & 1u, &sh, p.status)) { ok = false; break; }
-          // the first P V of an item overwrites the accumulator: the previous item's output
-          // must have been read
-          if (j == 0 && !tc_wait(&sh.o_empty, (it & 1u) ^ 1u, &sh, p.status)) { ok = false; break; }
-          tc_fence_after();
-          const uint32_t va = smem_u32(sV + vs * TILE_BYTES);
+      auto issue_pv = [&](int x, int vs, bool first) {
+        const uint32_t va = smem_u32(sV + vs * TILE_BYTES);
 #pragma unroll
-          for (int kk = 0; kk < kTcTile / 16; ++kk)
-            mma_ts(tmem + O_COL, tmem + P_COL + s * 64 + kk * 8, v_desc(va, kk), idesc_pv,
-                   (j | kk) != 0 ? 1u : 0u);
-          mma_commit(&sh.v_empty[vs]);
-          mma_commit(&sh.pv_done);
+        for (int kk = 0; kk < kTcTile / 16; ++kk)
+          mma_ts(tmem + O_COL + x * 128, tmem + S_COL + x * 128 + kk * 8, v_desc(va, kk), idesc_pv,
+                 (first && kk == 0) ? 0u : 1u);
+        mma_commit(&sh.pv_done[x]);
+      };
+      uint32_t tk = 0, tv = 0, it = 0;
+      uint32_t cx[2] = {0, 0};    // tiles so far of query tile x
+      uint32_t itx[2] = {0, 0};   // items so far in which query tile x took part
+      bool ok = true;
+      for (int rd = 0; ok; ++rd, ++it) {
+        const int item = item_index(order, rd, blockIdx.x, gridDim.x);
+        int b, h, qb;
+        if (item >= n_items || !item_at(p, order, cur, item, b, h, qb)) break;
+        const ItemShape is = item_shape(p, b, qb);
+        const bool has_b = is.jB >= 0;
+        if (!tc_wait(&sh.q_full, it & 1u, &sh, p.status)) break;
+        {
+          const int ks = tk % kTcKStages;
+          if (!tc_wait(&sh.k_full[ks], (tk / kTcKStages) & 1u, &sh, p.status)) break;
+          tc_fence_after();
+          issue_qk(0, ks);
+          if (has_b) issue_qk(1, ks);
+          mma_commit(&sh.k_empty[ks]);
+          if (is.nj == 1) mma_commit(&sh.q_empty);  // the query tiles have been read for the last time
         }
-        t += n_kt;
+        for (int j = 0; ok && j < is.nj; ++j) {
+          const int vs = (tv + j) % kTcVStages;
+          const uint32_t vph = ((tv + j) / kTcVStages) & 1u;
+          const int ks1 = (tk + j + 1) % kTcKStages;
+          const uint32_t kph1 = ((tk + j + 1) / kTcKStages) & 1u;
+          // Every barrier this round of (at most) 32 MMAs will need is tested once up front, without
+          // blocking: in the steady state all of them are complete, and the MMAs then follow one
+          // another without a barrier's round trip between the groups, during which the tensor
+          // pipe would drain.  What is not complete yet is waited for where it is needed.
+          bool p_ok[2];
+          p_ok[0] = j <= is.jA && mbar_try_wait(&sh.p_full[0], cx[0] & 1u);
+          p_ok[1] = j <= is.jB && mbar_try_wait(&sh.p_full[1], cx[1] & 1u);
+          bool v_ok = mbar_try_wait(&sh.v_full[vs], vph);
+          bool k_ok = j + 1 < is.nj && mbar_try_wait(&sh.k_full[ks1], kph1);
+#pragma unroll
+          for (int x = 0; x < 2; ++x) {
+            const int jx = x == 0 ? is.jA : is.jB;
+            if (j > jx) continue;
+            // P_x V of this key tile, then the scores of the next one (they overwrite P_x: the
+            // tensor pipe runs the two in issue order)
+            if (!p_ok[x] && !tc_wait(&sh.p_full[x], cx[x] & 1u, &sh, p.status)) { ok = false; break; }
+            // the first P V of an item overwrites the accumulator: the previous item's output
+            // must have been read
+            if (j == 0 && !tc_wait(&sh.o_empty[x], (itx[x] & 1u) ^ 1u, &sh, p.status)) { ok = false; break; }
+            if (!v_ok && !tc_wait(&sh.v_full[vs], vph, &sh, p.status)) { ok = false; break; }
+            v_ok = true;
+            tc_fence_after();
+            issue_pv(x, vs, j == 0);
+            ++cx[x];
+            const bool last_v_user = x == 1 || !(has_b && j <= is.jB);
+            if (last_v_user) mma_commit(&sh.v_empty[vs]);
+            if (j + 1 <= jx) {
+              if (!k_ok && !tc_wait(&sh.k_full[ks1], kph1, &sh, p.status)) { ok = false; break; }
+              k_ok = true;
+              tc_fence_after();
+              issue_qk(x, ks1);
+              const bool last_k_user = x == 1 || !has_b;
+              if (last_k_user) {
+                mma_commit(&sh.k_empty[ks1]);
+                if (j + 2 == is.nj) mma_commit(&sh.q_empty);
+              }
+            }
+          }
+        }
+        tk += is.nj;
+        tv += is.nj;
+        ++itx[0];
+        if (has_b) ++itx[1];
       }
     }
-  } else {
-    // ---------- softmax, correction and output: two threads per query row ----------
-    // Warps 2-5 take keys 0..63 of a tile, warps 6-9 keys 64..127 (the same split of the output
-    // columns at the end); a warp reaches the TMEM lanes 32 (warp % 4) .. + 31.  The two threads
-    // of a row exchange their half-row maximum through shared memory and an mbarrier (bounded
-    // wait, like every other wait here), and their partial sums once per item.
+  } else if (warp >= 4) {
+    // ---------- softmax, correction and output of one query tile: one thread per query row ----------
+    // Warps 4-7 serve tile A, warps 8-11 tile B; a warp reaches the TMEM lanes 32 (warp % 4) .. + 31.
+    const int x = (warp - 4) >> 2;
     const int quad = warp & 3;
-    const int half = (warp - 2) >> 2;
     const int row = quad * 32 + lane;          // TMEM lane = query row of the tile
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
-    constexpr int OC = HD / 2;                 // output columns of this thread
-    uint32_t t = 0, it = 0;
+    const uint32_t s_addr = tmem + lane_addr + S_COL + x * 128;
+    const uint32_t o_addr = tmem + lane_addr + O_COL + x * 128;
+    uint32_t c = 0, itx = 0;   // tiles / items so far of this query tile
     bool alive = true;
-    for (int item = blockIdx.x; alive && item < n_items; item += gridDim.x, ++it) {
-      int b, h, qt;
-      if (!item_at(p, cur, item, b, h, qt)) break;
-      const int seq0 = p.cu_exec[b];
-      const int len = p.cu_exec[b + 1] - seq0;
-      const int q0 = qt * kTcTile;
-      const int n_kt = qt + 1;
-      const int q_row = q0 + row;
-      float m_run = -INFINITY, l_run = 0.f;  // l_run: this thread's half of the row sum
-      for (int j = 0; j < n_kt && alive; ++j) {
-        const uint32_t tt = t + j;
-        const int s = tt & 1;
-        const uint32_t ph = (tt >> 1) & 1u;
-        if (!tc_wait(&sh.s_full[s], ph, &sh, p.status)) { alive = false; break; }
+    for (int rd = 0; alive; ++rd) {
+      const int item = item_index(order, rd, blockIdx.x, gridDim.x);
+      int b, h, qb;
+      if (item >= n_items || !item_at(p, order, cur, item, b, h, qb)) break;
+      const ItemShape is = item_shape(p, b, qb);
+      const int jx = x == 0 ? is.jA : is.jB;
+      if (jx < 0) continue;  // tile B lies behind the sequence
+      const int len = is.len;
+      const int q_row = qb * kTcItemRows + x * kTcTile + row;
+      float m_run = -INFINITY, l_run = 0.f;
+      for (int j = 0; j <= jx && alive; ++j) {
+        if (!tc_wait(&sh.s_full[x], c & 1u, &sh, p.status)) { alive = false; break; }
         tc_fence_after();
-        const uint32_t s_addr = tmem + lane_addr + S_COL + s * 128 + half * 64;
-        const int k0 = j * kTcTile + half * 64;
-        const bool masked = (j == qt) || (j * kTcTile + kTcTile > len);
-        // half a score row (64 keys) in registers, unscaled; the scale (positive) is folded into
-        // the exponent's multiply-add, so an element costs one max, one fma, one ex2, one add
-        float sc[64];
-        {
-          uint32_t r0[32], r1[32];
-          tmem_ld_x32(s_addr, r0);
-          tmem_ld_x32(s_addr + 32, r1);
-          tmem_wait_ld();
+        // the row's 128 scores in registers, unscaled; the scale (positive) is folded into the
+        // exponent's multiply-add, so an element costs one max, one fma, one ex2, one add
+        uint32_t sc[4][32];
+        tmem_ld_x32(s_addr, sc[0]);
+        tmem_ld_x32(s_addr + 32, sc[1]);
+        tmem_ld_x32(s_addr + 64, sc[2]);
+        tmem_ld_x32(s_addr + 96, sc[3]);
+        tmem_wait_ld();
+        if (j == jx || j * kTcTile + kTcTile > len) {
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            sc[i] = __uint_as_float(r0[i]);
-            sc[32 + i] = __uint_as_float(r1[i]);
-          }
-        }
-        if (masked) {
+          for (int cc = 0; cc < 4; ++cc)
 #pragma unroll
-          for (int i = 0; i < 64; ++i) {
-            const int key = k0 + i;
-            if (key > q_row || key >= len) sc[i] = -INFINITY;
-          }
+            for (int i = 0; i < 32; ++i) {
+              const int key = j * kTcTile + cc * 32 + i;
+              if (key > q_row || key >= len) sc[cc][i] = 0xFF800000u;  // -inf
+            }
         }
         float mq[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-        for (int i = 0; i < 64; i += 4) {
-          mq[0] = fmaxf(mq[0], sc[i]);
-          mq[1] = fmaxf(mq[1], sc[i + 1]);
-          mq[2] = fmaxf(mq[2], sc[i + 2]);
-          mq[3] = fmaxf(mq[3], sc[i + 3]);
-        }
-        const float my_max = fmaxf(fmaxf(mq[0], mq[1]), fmaxf(mq[2], mq[3]));
-        sh.row_max[tt & 1][half][row] = my_max;
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&sh.max_bar);
-        if (!tc_wait(&sh.max_bar, tt & 1u, &sh, p.status)) { alive = false; break; }
-        const float row_raw = fmaxf(my_max, sh.row_max[tt & 1][half ^ 1][row]);
+        for (int cc = 0; cc < 4; ++cc)
+#pragma unroll
+          for (int i = 0; i < 32; i += 4) {
+            mq[0] = fmaxf(mq[0], __uint_as_float(sc[cc][i]));
+            mq[1] = fmaxf(mq[1], __uint_as_float(sc[cc][i + 1]));
+            mq[2] = fmaxf(mq[2], __uint_as_float(sc[cc][i + 2]));
+            mq[3] = fmaxf(mq[3], __uint_as_float(sc[cc][i + 3]));
+          }
+        const float row_raw = fmaxf(fmaxf(mq[0], mq[1]), fmaxf(mq[2], mq[3]));
         // The reference maximum only moves when the row's maximum has grown by more than 2^8
         // (always on the first tile): until then the probabilities are at most 256, which both
         // 16-bit formats and the fp32 sums hold, and the output accumulator needs no rescaling.
@@ -379,63 +480,62 @@ __global__ void __launch_bounds__(kTcThreads, 1)
           m_run = cand;
           l_run *= corr;
         }
-        // probabilities in the 16-bit format, two keys per 32-bit column
         const float neg_m = (m_run == -INFINITY) ? 0.f : -m_run;
+        // probabilities in the 16-bit format, two keys per 32-bit column, written over the first
+        // 64 score columns (every score is in registers by now)
         float sq[4] = {0.f, 0.f, 0.f, 0.f};
-        uint32_t pr[32];
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const float p0 = ex2_approx(fmaf(sc[2 * i], p.scale_log2, neg_m));
-          const float p1 = ex2_approx(fmaf(sc[2 * i + 1], p.scale_log2, neg_m));
-          sq[i & 3] += p0 + p1;
-          pr[i] = Act16<ACT>::pack(p0, p1);
+        for (int cc = 0; cc < 4; ++cc) {
+          uint32_t pr[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const float p0 = ex2_approx(fmaf(__uint_as_float(sc[cc][2 * i]), p.scale_log2, neg_m));
+            const float p1 = ex2_approx(fmaf(__uint_as_float(sc[cc][2 * i + 1]), p.scale_log2, neg_m));
+            sq[i & 3] += p0 + p1;
+            pr[i] = Act16<ACT>::pack(p0, p1);
+          }
+          tmem_st_x16(s_addr + cc * 16, pr);
         }
         l_run += (sq[0] + sq[1]) + (sq[2] + sq[3]);
-        // The previous P V must be complete before O is rescaled.  Every tile waits for it, moved
-        // or not, so that the barrier is never more than one phase ahead of a parity test (by now
-        // that P V, issued a whole softmax earlier, has long finished).
+        // The previous P V of this tile was issued before these scores and is complete; the wait
+        // keeps the barrier's phase in step, and the fence orders the rescaling after it.
         if (j > 0) {
-          if (!tc_wait(&sh.pv_done, (tt - 1) & 1u, &sh, p.status)) { alive = false; break; }
+          if (!tc_wait(&sh.pv_done[x], (c - 1) & 1u, &sh, p.status)) { alive = false; break; }
           tc_fence_after();
-        }
-        if (j > 0 && __any_sync(0xffffffffu, moved)) {
+          if (__any_sync(0xffffffffu, moved)) {
 #pragma unroll 1
-          for (int c = 0; c < OC / 32; ++c) {
-            uint32_t r[32];
-            tmem_ld_x32(tmem + lane_addr + O_COL + half * OC + c * 32, r);
-            tmem_wait_ld();
+            for (int cc = 0; cc < HD / 32; ++cc) {
+              uint32_t r[32];
+              tmem_ld_x32(o_addr + cc * 32, r);
+              tmem_wait_ld();
 #pragma unroll
-            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * corr);
-            tmem_st_x32(tmem + lane_addr + O_COL + half * OC + c * 32, r);
+              for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * corr);
+              tmem_st_x32(o_addr + cc * 32, r);
+            }
           }
         }
-        tmem_st_x32(tmem + lane_addr + P_COL + s * 64 + half * 32, pr);
         tmem_wait_st();
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(&sh.p_full[s]);
+        if (lane == 0) mbar_arrive(&sh.p_full[x]);
+        ++c;
       }
       if (!alive) break;
       // output: O / l for the rows that exist; then the accumulator is handed back
-      sh.row_sum[half][row] = l_run;
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&sh.sum_bar);
-      if (!tc_wait(&sh.sum_bar, it & 1u, &sh, p.status)) { alive = false; break; }
-      const float l_tot = l_run + sh.row_sum[half ^ 1][row];
-      if (!tc_wait(&sh.pv_done, (t + n_kt - 1) & 1u, &sh, p.status)) { alive = false; break; }
+      if (!tc_wait(&sh.pv_done[x], (c - 1) & 1u, &sh, p.status)) { alive = false; break; }
       tc_fence_after();
-      const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;
-      unsigned short* out = static_cast<unsigned short*>(p.out) + (size_t)(seq0 + q_row) * p.ldo +
-                            (size_t)h * HD + half * OC;
+      const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+      unsigned short* out = static_cast<unsigned short*>(p.out) + (size_t)(is.seq0 + q_row) * p.ldo +
+                            (size_t)h * HD;
 #pragma unroll 1
-      for (int c = 0; c < OC / 32; ++c) {
+      for (int cc = 0; cc < HD / 32; ++cc) {
         uint32_t r[32];
-        tmem_ld_x32(tmem + lane_addr + O_COL + half * OC + c * 32, r);
+        tmem_ld_x32(o_addr + cc * 32, r);
         tmem_wait_ld();
-        if (c == OC / 32 - 1) {  // every column of this warp's part is in registers
+        if (cc == HD / 32 - 1) {  // every column of this warp's rows is in registers
           tc_fence_before();
           __syncwarp();
-          if (lane == 0) mbar_arrive(&sh.o_empty);
+          if (lane == 0) mbar_arrive(&sh.o_empty[x]);
         }
         if (q_row < len) {
 #pragma unroll
@@ -445,12 +545,13 @@ __global__ void __launch_bounds__(kTcThreads, 1)
             o.y = Act16<ACT>::pack(__uint_as_float(r[8 * i + 2]) * inv, __uint_as_float(r[8 * i + 3]) * inv);
             o.z = Act16<ACT>::pack(__uint_as_float(r[8 * i + 4]) * inv, __uint_as_float(r[8 * i + 5]) * inv);
             o.w = Act16<ACT>::pack(__uint_as_float(r[8 * i + 6]) * inv, __uint_as_float(r[8 * i + 7]) * inv);
-            st_16(out + c * 32 + i * 8, o);
+            st_16(out + cc * 32 + i * 8, o);
           }
         }
       }
-      t += n_kt;
+      ++itx;
     }
+    (void)itx;
   }
 
   tc_fence_before();
@@ -484,7 +585,7 @@ static EncodeTiledFnA encode_fn_a() {
 
 template <int HD, int ACT>
 static int launch_tc(const CUtensorMap& tm, const TcParams& p, int max_tiles, int H, cudaStream_t s) {
-  const size_t smem = (size_t)(1 + kTcKStages + kTcVStages) * kTcTile * HD * 2 + 1024;
+  const size_t smem = (size_t)(2 + kTcKStages + kTcVStages) * kTcTile * HD * 2 + 1024;
   static bool configured[64] = {false};
   int dev = 0;
   cudaGetDevice(&dev);
@@ -494,7 +595,7 @@ static int launch_tc(const CUtensorMap& tm, const TcParams& p, int max_tiles, in
       return QTALE_ERR_CUDA;
     configured[dev] = true;
   }
-  // persistent grid: one CTA per SM walks the (sequence, query tile, head) items
+  // persistent grid: one CTA per SM walks the (sequence, block of 256 query rows, head) items
   (void)max_tiles;
   (void)H;
   attn_prefill_tc_kernel<HD, ACT><<<sm_count(), kTcThreads, smem, s>>>(tm, p);
