@@ -140,6 +140,13 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, Ge
 }
 
 // logical output feature of lane L of tile nt (-1: padding row)
+// feature (inside a tile's block of heads) of element e of the rotary row layout: head e / half,
+// offset e % half, with half = rope_hd / 2 a power of two (no integer division in the epilogues)
+__device__ __forceinline__ int rope_first_half_feature(int e, int rope_hd) {
+  const int half = rope_hd >> 1;
+  return ((e & ~(half - 1)) << 1) + (e & (half - 1));
+}
+
 __device__ __forceinline__ int tile_row_to_n(const GemmParams& p, int nt, int L) {
   if (p.row_mode == QTALE_WQ_ROWS_SWIGLU) {
     const int q = L >> 5, r = L & 31;
@@ -152,7 +159,7 @@ __device__ __forceinline__ int tile_row_to_n(const GemmParams& p, int nt, int L)
     // and their partners half a head further (lanes 16-31)
     const int q = L >> 5, r = L & 31, half = p.rope_hd >> 1;
     const int e = q * 16 + (r & 15);
-    const int n = nt * kTileRows + (e / half) * p.rope_hd + (e % half) + (r < 16 ? 0 : half);
+    const int n = nt * kTileRows + rope_first_half_feature(e, p.rope_hd) + (r < 16 ? 0 : half);
     return n < p.N ? n : -1;
   }
   const int n = nt * kTileRows + L;
@@ -273,10 +280,10 @@ __device__ __forceinline__ void epilogue_fetch(const GemmParams& p, int lane, in
   if (epi == QTALE_EPI_ROPE) {
     const int half = p.rope_hd >> 1;
     const int e0 = quad * 16 + (lane & 1) * 8;
-    const int f_lo = nt * kTileRows + (e0 / half) * p.rope_hd + (e0 % half);
+    const int f_lo = nt * kTileRows + rope_first_half_feature(e0, p.rope_hd);
     const int m = m0 + (lane >> 1);
     if (f_lo < p.N && f_lo < p.rope_limit && m < M) {
-      const uint4* t = reinterpret_cast<const uint4*>(p.rope_cs + (size_t)m * half + (e0 % half));
+      const uint4* t = reinterpret_cast<const uint4*>(p.rope_cs + (size_t)m * half + (e0 & (half - 1)));
 #pragma unroll
       for (int e = 0; e < 4; ++e) o.q[e] = __ldg(t + e);  // (c, s) x 8
     }
@@ -321,8 +328,11 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const float*
     uint32_t w[4];
 #pragma unroll
     for (int e = 0; e < 4; ++e)
-      w[e] = Act16<ACT>::pack(g[2 * e] / (1.f + __expf(-g[2 * e])) * u[2 * e],
-                              g[2 * e + 1] / (1.f + __expf(-g[2 * e + 1])) * u[2 * e + 1]);
+      // SiLU(g) u with the approximate reciprocal (2 ulp, far below the 16-bit rounding that
+      // follows): the exact division is a dozen instructions per value in an epilogue that is
+      // bound by instruction issue
+      w[e] = Act16<ACT>::pack(__fdividef(g[2 * e], 1.f + __expf(-g[2 * e])) * u[2 * e],
+                              __fdividef(g[2 * e + 1], 1.f + __expf(-g[2 * e + 1])) * u[2 * e + 1]);
     st_16(static_cast<unsigned short*>(p.y) + (size_t)m * p.ldy + j0, make_uint4(w[0], w[1], w[2], w[3]));
     return;
   }
@@ -333,7 +343,7 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, const float*
     const int jc = (lane & 1) * 8;
     const int half = p.rope_hd >> 1;
     const int e0 = quad * 16 + jc;
-    const int f_lo = nt * kTileRows + (e0 / half) * p.rope_hd + (e0 % half);
+    const int f_lo = nt * kTileRows + rope_first_half_feature(e0, p.rope_hd);
     const int row = lane >> 1;
     const int m = m0 + row;
     if (f_lo >= p.N || m >= M) return;

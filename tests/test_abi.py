@@ -57,6 +57,15 @@ def test_host_side_argument_validation(api):
     assert L.qtale_router_select(None, 4, 64, None, 0.0, None, None, None, 1, None, 0, 0.5, 0,
                                  None, None, None, None, None, None, 0, None) == -1
     assert L.qtale_wq_gemm(None, 64, None, 4, None, 0, 0, None, None, 64, None, 0, None) == -1
+    assert L.qtale_attention_prefill(None, 384, 1, 1, 128, 1, None, 1, 8, None, 128, None) == -1
+    buf = np.zeros(64, np.uint8)
+    ptr = buf.ctypes.data + (-buf.ctypes.data) % 16
+    # head size, head grouping, row strides and the activation format are checked before any launch
+    assert L.qtale_attention_prefill(ptr, 288, 1, 1, 96, 1, ptr, 1, 8, ptr, 96, None) == -3
+    assert L.qtale_attention_prefill(ptr, 640, 3, 2, 128, 1, ptr, 1, 8, ptr, 384, None) == -3
+    assert L.qtale_attention_prefill(ptr, 380, 1, 1, 128, 1, ptr, 1, 8, ptr, 128, None) == -3
+    assert L.qtale_attention_prefill(ptr, 384, 1, 1, 128, 7, ptr, 1, 8, ptr, 128, None) == api.lib().qtale_attention_prefill(
+        ptr, 384, 1, 1, 128, 9, ptr, 1, 8, ptr, 128, None) != 0
     cfg = api.LayerConfig(256, 4, 4, 64, 688, 4, 64, 1e-5, 1e4, 0, 0.5, 1.0, 1)
     assert api.layer_workspace_bytes(cfg, 256, 2) > 256 * 256 * 2
     bad = api.LayerConfig(256, 4, 4, 48, 688, 4, 64, 1e-5, 1e4, 0, 0.5, 1.0, 1)
