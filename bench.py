@@ -51,7 +51,7 @@ KERNELS_PER_STEP = 8
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of the four GEMM launches of one step
 # at ratio 0.5 (4096 executed tokens), one ncu capture of the kernels as they stand
 # (profiles/wq_gemm_pair_c2_layer_step.md); None at other ratios.
-GEMM_DRAM_BYTES = 728582656
+GEMM_DRAM_BYTES = 729280768
 ALL_LEGS = ["sweep", "gemm", "bf16", "router", "gather", "scatter", "attention", "decode", "decode_loop", "c4", "c5", "e2e", "cpu"]
 
 
