@@ -401,6 +401,8 @@ def test_wq_gemm_rotary_epilogue(env, hd, H, Hkv, M, m_dev, act):
     (128, 4, 2, [300, 1, 0, 128, 257]),      # ragged, an empty sequence, lengths around the tile size
     (64, 3, 3, [77, 513]),                   # 64-wide heads, five key tiles
     (128, 2, 1, [1024]),                     # eight query tiles of one sequence
+    (128, 2, 2, [700, 130, 0, 520, 257]),    # sequences of 3, 1, 0, 3 and 2 blocks of 256 rows: every level of
+                                             # the cost-ordered item list has a different set of sequences
 ])
 @pytest.mark.parametrize("act", [0, 1])
 def test_attention_prefill_against_oracle(env, hd, H, Hkv, lens, act):
