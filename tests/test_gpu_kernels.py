@@ -428,6 +428,10 @@ def test_attention_prefill_against_oracle(env, hd, H, Hkv, lens, act):
     vmax = np.abs(qkv[:Te, (H + Hkv) * hd:]).max()
     assert np.abs(got[:Te] - ref).max() <= 4 * act_eps(act) * vmax
     assert rel_fro(got[:Te], ref) <= 3 * act_eps(act)
+    # a second call on a fresh copy of the input gives the same bits (no dependence on timing)
+    out2 = torch.full((T_cap, H * hd), 7.0, dtype=api.act_torch_dtype(act), device=dev)
+    api.attention_prefill(api.to_device_act(qkv, act, dev), H, Hkv, hd, torch.from_numpy(cu).to(dev), act, out2)
+    assert torch.equal(out, out2)
     # the first token of a sequence sees only itself: its output is its own value row
     for b, n in enumerate(lens):
         if n:
