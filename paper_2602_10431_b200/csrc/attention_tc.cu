@@ -372,7 +372,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
           const uint32_t vph = ((tv + j) / kTcVStages) & 1u;
           const int ks1 = (tk + j + 1) % kTcKStages;
           const uint32_t kph1 = ((tk + j + 1) / kTcKStages) & 1u;
-          // Every barrier this round of (at most) 32 MMAs will need is tested once up front, without
+          // Every barrier this key tile (at most 32 MMAs) will need is tested once up front, without
           // blocking: in the steady state all of them are complete, and the MMAs then follow one
           // another without a barrier's round trip between the groups, during which the tensor
           // pipe would drain.  What is not complete yet is waited for where it is needed.
