@@ -829,6 +829,26 @@ def run_ours(args):
             frac_of_sustained_bf16=fl / (r["ms"] * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
             select="one global theta for all layers (Eq. 9), found on the device for R_avg 0.75",
             clocks=r["clocks"])
+        # (iii) layer-interleaved mixed precision (even layers 4-bit, odd layers 2-bit; the layer
+        # configuration leaves the width to each weight), per-layer top-k 0.75 as in (i)
+        import copy
+        s4b = copy.copy(s4)
+        s4b.bits = 2
+        for li in range(1, L4, 2):
+            layers[li] = timing_layer(torch, api, dev, gen, s4b)
+        mcfg.layer.select_mode = api.SELECT_TOPK
+        mcfg.layer.ratio = 0.75
+        mcfg.layer.bits = 0
+        r = timer.run(mstep, 3, 2, 0.5)
+        check_status()
+        assert per_layer.cpu().tolist() == [k4] * L4
+        fl = L4 * accounting.layer_flops(s4, [S4] * B4, 0.75) + 2.0 * s4.d * V4 * B4
+        extra["c4_model_prefill_mixed_4_2_bit"] = dict(
+            ms_per_step=r["ms"], tokens_per_s=T4 / (r["ms"] * 1e-3), layers=L4, tokens=T4,
+            bits="4, 2, 4, 2, ... by layer", select="per-layer top-k, ratio 0.75",
+            achieved_tflops=fl / (r["ms"] * 1e-3) / 1e12,
+            frac_of_sustained_bf16=fl / (r["ms"] * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
+            clocks=r["clocks"])
         del layers, embed, lm_head, mws, hidden, logits
 
     # ---- c5: 13B-shaped 8-layer stack, 16 x 4096 tokens, per-layer ratios from U[0.4, 1.0],
