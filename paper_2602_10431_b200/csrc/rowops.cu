@@ -45,8 +45,11 @@ __global__ void __launch_bounds__(kGatherThreads)
     }
   }
   int par = 0;
+  // the index of a CTA's next row is fetched one row ahead, so a row's loads do not wait for it
+  int row = (int)blockIdx.x < n ? idx[blockIdx.x] : 0;
   for (int i = blockIdx.x; i < n; i += gridDim.x, par ^= 1) {
-    const uint4* src = x + (size_t)idx[i] * chunks;
+    const uint4* src = x + (size_t)row * chunks;
+    if (i + (int)gridDim.x < n) row = idx[i + gridDim.x];
     if (ex.cs && tid < ex.half) {
       double sn, cn;
       sincos((double)ex.pos[i] * inv_freq, &sn, &cn);
@@ -344,7 +347,7 @@ static int launch_compact_t(const void* x, const int32_t* idx, const int32_t* n_
                             int d, const float* gamma, float eps, void* xc, void* hn,
                             const GatherExtras& ex, cudaStream_t s) {
   const int chunks = d / 8;
-  const int grid = min(cap, row_grid(12));
+  const int grid = min(cap, row_grid(16));
   auto X = static_cast<const uint4*>(x);
   auto XC = static_cast<uint4*>(xc);
   auto HN = static_cast<uint4*>(hn);
